@@ -1,0 +1,50 @@
+"""The pins must notice a broken checker.
+
+Each case plants one plausible mistake in a copy of ``oracle/pg_oracle.c`` (on
+the CPU, never in the CUDA path), points the binding at the copy and runs the
+pin tests in a child process: they have to fail.
+"""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "pg_oracle.c")
+
+MUTATIONS = {
+    "update_not_antisymmetric": ("Xj[(size_t)r * m + cidx] += d;", "Xj[(size_t)r * m + cidx] -= d;"),
+    "weight_dropped": ("double a = w[e] * p[r];", "double a = p[r];"),
+    "left_factor_not_normalised": ("p[r] = ok ? p[r] * inv : 0.0;", "p[r] = ok ? p[r] : 0.0;"),
+    "right_vector_not_refreshed": ("memcpy(c->Q[t] + (size_t)k * m, q, sizeof(double) * (size_t)m);", ";"),
+    "difference_sign_in_transposed_pass": ("Qn[(size_t)k * m + e] = qi[e] - qj[e];",
+                                           "Qn[(size_t)k * m + e] = qi[e] + qj[e];"),
+    "forward_uses_one_endpoint": ("p[r] = pi[r] - pj[r];", "p[r] = pi[r];"),
+    "no_orthogonalisation": ("for (int r = 0; r < n; ++r) p[r] -= a * ph[r];", ";"),
+    "transposed_index": ("for (int cidx = 0; cidx < m; ++cidx) y[cidx] += a[cidx] * vr;",
+                         "for (int cidx = 0; cidx < m; ++cidx) y[cidx] += a[cidx] * v[(r + 1) % n];"),
+    "matching_weight_is_one": ("for (int e = 0; e < E; ++e) w_out[e] = 0.5;",
+                                              "for (int e = 0; e < E; ++e) w_out[e] = 1.0;"),
+    "ring_skips_wraparound": ("edges_out[2 * n + 1] = (i + 1) % N; ++n; }",
+                              "edges_out[2 * n + 1] = (i + 1) % N; if (i + 1 < N) ++n; }"),
+    "philox_round_count": ("round < 10; ++round", "round < 9; ++round"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_pins_catch(name, tmp_path):
+    old, new = MUTATIONS[name]
+    text = open(SRC).read()
+    assert text.count(old) == 1, "mutation anchor must be unique: %r" % old
+    mutated = tmp_path / "pg_oracle_mutated.c"
+    mutated.write_text(text.replace(old, new))
+    env = dict(os.environ)
+    env["PG_ORACLE_SRC"] = str(mutated)
+    env["PG_ORACLE_BUILD"] = str(tmp_path / "build")
+    env["OMP_NUM_THREADS"] = "2"
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
+                        os.path.join(ROOT, "tests", "test_oracle_pins.py")],
+                       cwd=ROOT, env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, timeout=600)
+    assert r.returncode != 0, "pins did not notice mutation %s" % name
+    assert b"failed" in r.stdout

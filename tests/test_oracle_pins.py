@@ -1,0 +1,402 @@
+"""Pins for the fp64 CPU checker: what the paper and the mathematics fix.
+
+None of these compares the checker with itself or with the CUDA path.  Each
+test states which passage of the paper (or which textbook fact) it rests on.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import pg_oracle as po
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden_rows(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+def _fill(o, rng, scale=1.0):
+    xs = []
+    for i in range(o.n_workers):
+        row = []
+        for l, (n, m) in enumerate(o.layer_shapes):
+            x = (rng.standard_normal((n, m)) * scale).astype(np.float32)
+            o.set_params(i, l, x)
+            row.append(x.astype(np.float64))
+        xs.append(row)
+    return xs
+
+
+def _ring_W(N, a):
+    W = np.zeros((N, N), dtype=np.float32)
+    for i in range(N):
+        for j in ((i + 1) % N, (i - 1) % N):
+            if j != i:
+                W[i, j] = a
+    for i in range(N):
+        W[i, i] = 1.0 - W[i].sum()
+    return W
+
+
+# --------------------------------------------------------------------------
+# random numbers and schedules
+# --------------------------------------------------------------------------
+def test_philox_known_answers():
+    """Philox4x32-10 against the published known-answer vectors."""
+    for row in _golden_rows("philox4x32_10_kat.txt"):
+        v = [int(x, 16) for x in row]
+        assert po.philox4x32_10(v[:4], v[4:6]) == tuple(v[6:])
+
+
+def test_init_q_is_standard_normal_and_keyed():
+    """Algorithm 2 initialises every entry from a standard normal."""
+    q = po.init_q(7, 0, 1, 0, 0, 200000).astype(np.float64)
+    assert abs(q.mean()) < 0.01
+    assert abs(q.std() - 1.0) < 0.01
+    assert abs((q ** 3).mean()) < 0.03           # skewness 0
+    assert abs((q ** 4).mean() - 3.0) < 0.08     # kurtosis 3
+    # a prefix of a longer draw is the shorter draw; any key change gives new numbers
+    assert np.array_equal(po.init_q(7, 0, 1, 0, 0, 37), q[:37].astype(np.float32))
+    for other in (po.init_q(8, 0, 1, 0, 0, 64), po.init_q(7, 0, 2, 0, 0, 64),
+                  po.init_q(7, 1, 2, 0, 0, 64), po.init_q(7, 0, 1, 1, 0, 64),
+                  po.init_q(7, 0, 1, 0, 1, 64)):
+        assert not np.array_equal(other, q[:64].astype(np.float32))
+
+
+def test_ring_and_torus_schedules():
+    """Ring: N edges, degree 2.  Torus RxC: 2N edges, degree 4, symmetric."""
+    for N in (3, 4, 8, 16):
+        e = po.schedule(po.RING, N)
+        assert len(e) == N
+        assert np.all(e[:, 0] < e[:, 1])
+        deg = np.bincount(e.ravel(), minlength=N)
+        assert np.all(deg == 2)
+        assert [tuple(x) for x in e] == sorted(set(tuple(x) for x in e))
+        for a, b in e:
+            assert (b - a) % N in (1, N - 1)
+    assert [tuple(x) for x in po.schedule(po.RING, 2)] == [(0, 1)]
+    e = po.schedule(po.TORUS, 64, 8, 8)
+    assert len(e) == 128
+    assert np.all(np.bincount(e.ravel(), minlength=64) == 4)
+    for a, b in e:
+        ra, ca, rb, cb = a // 8, a % 8, b // 8, b % 8
+        assert ((ra == rb and (ca - cb) % 8 in (1, 7)) or (ca == cb and (ra - rb) % 8 in (1, 7)))
+    # a 2x4 torus has doubled vertical links: they are merged
+    e = po.schedule(po.TORUS, 8, 2, 4)
+    assert len(e) == 8 + 4
+    with pytest.raises(ValueError):
+        po.schedule(po.TORUS, 10, 3, 3)
+
+
+def test_matching_schedule():
+    """Time-varying graph: a perfect matching drawn afresh every round."""
+    N = 32
+    seen = set()
+    for t in range(50):
+        e = po.schedule(po.MATCHING, N, seed=5, round_index=t)
+        assert len(e) == N // 2
+        assert sorted(e.ravel().tolist()) == list(range(N))
+        assert np.all(e[:, 0] < e[:, 1])
+        assert list(e[:, 0]) == sorted(e[:, 0])
+        assert np.array_equal(e, po.schedule(po.MATCHING, N, seed=5, round_index=t))
+        seen.add(tuple(map(tuple, e)))
+    assert len(seen) == 50
+    assert not np.array_equal(po.schedule(po.MATCHING, N, seed=6, round_index=0),
+                              po.schedule(po.MATCHING, N, seed=5, round_index=0))
+    with pytest.raises(ValueError):
+        po.schedule(po.MATCHING, 7)
+    # every pair is about equally likely to be matched: N-1 = 31 possible partners
+    hits = np.zeros((8, 8))
+    T = 7000
+    for t in range(T):
+        for a, b in po.schedule(po.MATCHING, 8, seed=11, round_index=t):
+            hits[a, b] += 1
+    freq = hits[np.triu_indices(8, 1)] / T
+    assert np.all(np.abs(freq - 1.0 / 7.0) < 0.02)
+
+
+def test_mixing_weights_satisfy_A4():
+    """Assumption A4: W symmetric, doubly stochastic, non-zero only on edges."""
+    for row in _golden_rows("mixing_presets.txt"):
+        N, a, s = int(row[0]), float(row[1]), float(row[2])
+        assert abs(2 * a + s - 1.0) < 1e-12          # the printed constants are a valid row
+        e = po.schedule(po.RING, N)
+        w = po.edge_weights(po.W_EXPLICIT, N, e, _ring_W(N, a))
+        assert np.allclose(w, a, atol=1e-7)
+    e = po.schedule(po.TORUS, 64, 8, 8)
+    assert np.allclose(po.edge_weights(po.W_METROPOLIS, 64, e), 1.0 / 5.0)
+    assert np.allclose(po.edge_weights(po.W_UNIFORM, 4, po.schedule(po.RING, 4)), 1.0 / 3.0)
+    # a star graph: Metropolis weights 1/(1+max degree of the two ends)
+    star = np.array([[0, 1], [0, 2], [0, 3]], dtype=np.int32)
+    assert np.allclose(po.edge_weights(po.W_METROPOLIS, 4, star), 0.25)
+    bad = _ring_W(4, 1.0 / 3.0)
+    bad[0, 1] = 0.5                                   # not symmetric, row sum off
+    with pytest.raises(ValueError):
+        po.edge_weights(po.W_EXPLICIT, 4, po.schedule(po.RING, 4), bad)
+    bad = _ring_W(4, 1.0 / 3.0)
+    bad[0, 2] = bad[2, 0] = 0.1                       # weight on a non-edge
+    bad[0, 0] -= 0.1
+    bad[2, 2] -= 0.1
+    with pytest.raises(ValueError):
+        po.edge_weights(po.W_EXPLICIT, 4, po.schedule(po.RING, 4), bad)
+
+
+def test_compression_ratios_printed_in_the_paper():
+    """Per-tensor ratios of the ResNet-20 and LSTM parameter tables: one
+    iteration of Algorithm 2 moves (rows + cols)/2 floats on average."""
+    for n, m, printed in _golden_rows("compression_ratios.txt"):
+        n, m, printed = int(n), int(m), int(printed)
+        assert round(po.compression_ratio(n, m, 1, 1)) == printed
+        assert abs(po.compression_ratio(n, m, 1, 4) * 4 - po.compression_ratio(n, m, 1, 1)) < 1e-9
+
+
+# --------------------------------------------------------------------------
+# the gossip round
+# --------------------------------------------------------------------------
+CASES = [
+    dict(kind=po.RING, n_workers=4, layer_shapes=[(9, 7)], rank=1, power_steps=1,
+         weight_rule=po.W_EXPLICIT, W=_ring_W(4, 1.0 / 3.0)),
+    dict(kind=po.RING, n_workers=8, layer_shapes=[(6, 11), (5, 3)], rank=1, power_steps=2,
+         weight_rule=po.W_EXPLICIT, W=_ring_W(8, 0.436)),
+    dict(kind=po.TORUS, n_workers=12, torus_rows=3, torus_cols=4, layer_shapes=[(10, 8)],
+         rank=2, power_steps=2, weight_rule=po.W_METROPOLIS),
+    dict(kind=po.MATCHING, n_workers=6, layer_shapes=[(7, 12), (4, 4)], rank=1, power_steps=1),
+    dict(kind=po.MATCHING, n_workers=6, layer_shapes=[(7, 12)], rank=3, power_steps=2),
+    dict(kind=po.CUSTOM, n_workers=5, custom_edges=[(0, 1), (0, 2), (0, 3), (3, 4)],
+         layer_shapes=[(8, 8)], rank=1, power_steps=1, weight_rule=po.W_METROPOLIS),
+]
+
+
+@pytest.mark.parametrize("case", CASES)
+def test_average_is_conserved_and_distance_never_grows(case):
+    """Lemma 1 (every edge adds to i what it takes from j, so the worker average
+    never moves), and the consensus distance sum_i ||X_i - mean||^2 cannot grow
+    in a step: with projectors Pi_e the update is Delta <- (I - M) Delta with
+    0 <= M = sum_e W_e (e_i-e_j)(e_i-e_j)^T (x) Pi_e <= I - W < 2I."""
+    rng = np.random.default_rng(3)
+    o = po.Oracle(seed=17, **case)
+    _fill(o, rng)
+    avg0 = [o.average(l) for l in range(len(o.layer_shapes))]
+    d_prev = o.consensus_distance()
+    for _ in range(12):
+        o.round()
+        for l in range(len(o.layer_shapes)):
+            scale = np.abs(avg0[l]).max()
+            assert np.abs(o.average(l) - avg0[l]).max() <= 1e-13 * max(scale, 1.0)
+        d = o.consensus_distance()
+        assert d <= d_prev * (1 + 1e-12)
+        d_prev = d
+    assert np.isfinite(d_prev)
+    o.close()
+
+
+def test_rank1_difference_is_removed_exactly():
+    """If X_i - X_j = sigma u v^T, then C_v recovers it exactly (Section 4: with v
+    the top right singular vector C_v(X) is the best rank-1 approximation, here
+    exact): p ~ u, q' = D^T u = sigma v, so the step equals uncompressed gossip on
+    that edge; with W_ij = 1/2 both workers land on their average at once."""
+    rng = np.random.default_rng(5)
+    n, m = 12, 9
+    base = rng.standard_normal((n, m)).astype(np.float32)
+    u = rng.standard_normal((n, 1)).astype(np.float32)
+    v = rng.standard_normal((1, m)).astype(np.float32)
+    # pick entries that are exact in fp32 so that the difference is exactly rank 1
+    base = np.round(base * 64) / 64
+    u = np.round(u * 8) / 8
+    v = np.round(v * 8) / 8
+    x0 = (base + u @ v).astype(np.float32)
+    x1 = base.astype(np.float32)
+    for w_edge in (0.5, 0.3):
+        W = np.array([[1 - w_edge, w_edge], [w_edge, 1 - w_edge]], dtype=np.float32)
+        o = po.Oracle(kind=po.CUSTOM, n_workers=2, custom_edges=[(0, 1)], layer_shapes=[(n, m)],
+                      rank=1, power_steps=1, seed=3, weight_rule=po.W_EXPLICIT, W=W)
+        o.set_params(0, 0, x0)
+        o.set_params(1, 0, x1)
+        o.round()
+        D0 = x0.astype(np.float64) - x1.astype(np.float64)
+        w64 = float(np.float32(w_edge))
+        assert np.allclose(o.get_params(0, 0), x0 - w64 * D0, rtol=0, atol=1e-13)
+        assert np.allclose(o.get_params(1, 0), x1 + w64 * D0, rtol=0, atol=1e-13)
+        if w_edge == 0.5:
+            assert np.allclose(o.get_params(0, 0), o.get_params(1, 0), rtol=0, atol=1e-13)
+        # the stored vector is now D^T p_hat = +- sigma v
+        q = o.get_q(0, 1, 0)[:, 0]
+        sigma = np.linalg.norm(u.astype(np.float64)) * np.linalg.norm(v.astype(np.float64))
+        assert abs(np.linalg.norm(q) - sigma) < 1e-12 * sigma
+        o.close()
+
+
+@pytest.mark.parametrize("rank", [1, 2, 3])
+def test_frozen_difference_converges_to_svd(rank):
+    """Eq. 3: on a difference that does not change the scheme is power iteration,
+    so the warm-started factors converge to the top singular triplets of
+    D = X_0 - X_1 (numpy.linalg.svd), at the rate (sigma_{r+1}/sigma_r)^2 per step.
+    The edge weight 0 freezes X."""
+    rng = np.random.default_rng(11)
+    n, m = 8, 6
+    U, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    V, _ = np.linalg.qr(rng.standard_normal((m, m)))
+    s = np.array([5.0, 3.0, 1.5, 0.6, 0.2, 0.05])
+    D = (U[:, :m] * s) @ V.T
+    x1 = rng.standard_normal((n, m)).astype(np.float32)
+    x0 = (x1 + D).astype(np.float32)
+    Dq = x0.astype(np.float64) - x1.astype(np.float64)          # what the oracle sees
+    Us, ss, Vts = np.linalg.svd(Dq)
+    W = np.eye(2, dtype=np.float32)
+    o = po.Oracle(kind=po.CUSTOM, n_workers=2, custom_edges=[(0, 1)], layer_shapes=[(n, m)],
+                  rank=rank, power_steps=1, seed=9, weight_rule=po.W_EXPLICIT, W=W)
+    o.set_params(0, 0, x0)
+    o.set_params(1, 0, x1)
+    proj_true = Us[:, :rank] @ Us[:, :rank].T
+    errs = []
+    for _ in range(60):
+        o.round()
+        P = o.get_phat(0, 1, 0)
+        errs.append(np.linalg.norm(P @ P.T - proj_true))
+    assert np.array_equal(o.get_params(0, 0), x0.astype(np.float64))   # frozen
+    P = o.get_phat(0, 1, 0)
+    Q = o.get_q(0, 1, 0)
+    assert np.allclose(P.T @ P, np.eye(rank), atol=1e-12)             # orthonormal
+    assert errs[-1] < 1e-9
+    # geometric decay of the subspace error, ratio (s_{r+1}/s_r)^2
+    ratio = (ss[rank] / ss[rank - 1]) ** 2
+    k0, k1 = 6, 12
+    assert errs[k1] / errs[k0] < (ratio ** (k1 - k0)) * 50
+    assert errs[k1] / errs[k0] > (ratio ** (k1 - k0)) / 50
+    # Q = D^T P: its columns converge to sigma_k v_k (up to sign)
+    for k in range(rank):
+        assert abs(np.linalg.norm(Q[:, k]) - ss[k]) < 1e-7 * ss[k]
+        assert abs(abs(Q[:, k] @ Vts[k]) - ss[k]) < 1e-7 * ss[k]
+        assert abs(abs(P[:, k] @ Us[:, k]) - 1.0) < 1e-9
+    # P Q^T is the best rank-r approximation of D (Eckart-Young)
+    best = (Us[:, :rank] * ss[:rank]) @ Vts[:rank]
+    assert np.allclose(P @ Q.T, best, atol=1e-7)
+    o.close()
+
+
+def test_identical_workers_are_a_fixed_point():
+    """Section 4.1: if two workers agree their compressed update is zero, so
+    consensus is a fixed point; nothing becomes NaN and the stored vectors stay."""
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((10, 7)).astype(np.float32)
+    o = po.Oracle(kind=po.RING, n_workers=4, layer_shapes=[(10, 7)], rank=2, power_steps=2,
+                  seed=4, weight_rule=po.W_EXPLICIT, W=_ring_W(4, 1.0 / 3.0))
+    for i in range(4):
+        o.set_params(i, 0, x)
+    q_before = o.get_q(0, 1, 0)
+    o.round(3)
+    for i in range(4):
+        assert np.array_equal(o.get_params(i, 0), x.astype(np.float64))
+    assert np.array_equal(o.get_q(0, 1, 0), q_before)
+    o.close()
+    # only worker 2 differs: after one power step worker 0, whose two edges carry
+    # no difference, has not moved at all
+    o = po.Oracle(kind=po.RING, n_workers=4, layer_shapes=[(10, 7)], rank=2, power_steps=1,
+                  seed=4, weight_rule=po.W_EXPLICIT, W=_ring_W(4, 1.0 / 3.0))
+    for i in range(4):
+        o.set_params(i, 0, x)
+    y = x.copy()
+    y[3, 2] += 1.0
+    o.set_params(2, 0, y)
+    o.round()
+    assert np.array_equal(o.get_params(0, 0), x.astype(np.float64))    # both its edges carry no difference
+    for i in (1, 2, 3):
+        assert np.all(np.isfinite(o.get_params(i, 0)))
+    assert not np.array_equal(o.get_params(1, 0), x.astype(np.float64))
+    o.close()
+
+
+@pytest.mark.parametrize("shape,rank", [((7, 1), 1), ((1, 6), 1), ((3, 5), 3), ((5, 3), 4)])
+@pytest.mark.parametrize("topo", ["ring", "torus", "matching"])
+def test_full_rank_equals_plain_gossip(shape, rank, topo):
+    """With rank >= min(rows, cols) (or a single column / row) the projector
+    Ph Ph^T leaves the difference untouched, so one power step is the gossip term
+    of D-PSGD (Eq. 1): X <- W X.  Checked against numpy's matrix product."""
+    rng = np.random.default_rng(13)
+    n, m = shape
+    if topo == "ring":
+        N = 6
+        W = _ring_W(N, 0.3)
+        o = po.Oracle(kind=po.RING, n_workers=N, layer_shapes=[shape], rank=rank, power_steps=1,
+                      seed=21, weight_rule=po.W_EXPLICIT, W=W)
+        W64 = W.astype(np.float64)
+    elif topo == "torus":
+        N = 12
+        o = po.Oracle(kind=po.TORUS, n_workers=N, torus_rows=3, torus_cols=4, layer_shapes=[shape],
+                      rank=rank, power_steps=1, seed=21, weight_rule=po.W_METROPOLIS)
+        W64 = np.zeros((N, N))
+        for a, b in po.schedule(po.TORUS, N, 3, 4):
+            W64[a, b] = W64[b, a] = 0.2
+        W64 += np.diag(1.0 - W64.sum(1))
+    else:
+        N = 6
+        o = po.Oracle(kind=po.MATCHING, n_workers=N, layer_shapes=[shape], rank=rank,
+                      power_steps=1, seed=21)
+        W64 = np.zeros((N, N))
+        for a, b in po.schedule(po.MATCHING, N, seed=21, round_index=0):
+            W64[a, b] = W64[b, a] = 0.5
+        W64 += np.diag(1.0 - W64.sum(1))
+    xs = _fill(o, rng)
+    X = np.stack([xs[i][0] for i in range(N)])            # N x n x m
+    o.round()
+    expect = np.einsum("ij,jnm->inm", W64, X)
+    got = np.stack([o.get_params(i, 0) for i in range(N)])
+    assert np.allclose(got, expect, rtol=0, atol=1e-12)
+    o.close()
+
+
+def test_one_step_matches_projector_form():
+    """Cross-check of a whole Jacobi step on a ring against the operator form used
+    in the proof of Lemma 2: X_i <- X_i + sum_j W_ij Pi_ij (X_j - X_i) with
+    Pi_ij = p p^T, p = D q / ||D q||  (numpy, left-projector form)."""
+    rng = np.random.default_rng(23)
+    N, n, m = 5, 7, 9
+    W = _ring_W(N, 0.25)
+    o = po.Oracle(kind=po.RING, n_workers=N, layer_shapes=[(n, m)], rank=1, power_steps=1,
+                  seed=31, weight_rule=po.W_EXPLICIT, W=W)
+    xs = _fill(o, rng)
+    X = [xs[i][0] for i in range(N)]
+    edges, w = o.round_schedule()
+    new = [x.copy() for x in X]
+    for (i, j), wij in zip(edges, w):
+        q = po.init_q(31, i, j, 0, 0, m).astype(np.float64)
+        D = X[i] - X[j]
+        p = D @ q
+        p /= np.linalg.norm(p)
+        Pi = np.outer(p, p)
+        new[i] += wij * Pi @ (X[j] - X[i])
+        new[j] += wij * Pi @ (X[i] - X[j])
+    o.round()
+    for i in range(N):
+        assert np.allclose(o.get_params(i, 0), new[i], rtol=0, atol=1e-12)
+    o.close()
+
+
+def test_warm_start_is_kept_per_pair_on_a_time_varying_graph():
+    """A pair that meets again continues from the vector it stored last time, and
+    a pair that has not met yet still has its seed-derived initial vector."""
+    N, m = 4, 5
+    o = po.Oracle(kind=po.MATCHING, n_workers=N, layer_shapes=[(6, m)], rank=1, power_steps=1, seed=77)
+    _fill(o, np.random.default_rng(1))
+    met = {}
+    for t in range(6):
+        edges, _ = o.round_schedule()
+        untouched = [(a, b) for a in range(N) for b in range(a + 1, N)
+                     if (a, b) not in met and (a, b) not in [tuple(e) for e in edges]]
+        o.round()
+        for a, b in untouched:
+            assert np.array_equal(o.get_q(a, b, 0)[:, 0], po.init_q(77, a, b, 0, 0, m).astype(np.float64))
+        for a, b in edges:
+            met[(int(a), int(b))] = o.get_q(a, b, 0).copy()
+        for (a, b), q in met.items():
+            if (a, b) not in [tuple(e) for e in edges]:
+                assert np.array_equal(o.get_q(a, b, 0), q)
+    o.close()
