@@ -1,0 +1,217 @@
+/*
+ * powergossip.h - C ABI of the B200 PowerGossip library.
+ *
+ * PowerGossip (Vogels, Karimireddy, Jaggi, "Practical Low-Rank Communication
+ * Compression in Decentralized Deep Learning"): every pair of neighbouring
+ * workers (i, j) keeps a small warm-started vector and uses power-iteration
+ * steps to build a low-rank approximation of the difference of their
+ * parameter matrices, which replaces the full difference in the gossip
+ * averaging update (Section 4, Eq. 2 and 3, Algorithm 2).
+ *
+ * This library simulates the whole decentralized network on ONE GPU: the
+ * parameter stacks of all workers stay resident in device memory and the
+ * "communication" between the two ends of an edge is an exchange of the small
+ * vectors through device buffers.  All arithmetic of the method runs in CUDA
+ * kernels; there is no CPU fallback.
+ *
+ * Conventions
+ *   - Every call returns a pg_status (PG_OK == 0).  Nothing throws, aborts or
+ *     traps across this boundary.  Out-parameters are written only on success.
+ *   - "host" / "device" is stated for every pointer.  The library allocates no
+ *     device memory: the caller passes one workspace of pg_workspace_bytes()
+ *     bytes (cudaMalloc / torch.empty, 256-byte aligned) which must outlive the
+ *     context.  Host-side tables are owned by the context.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     One context is used from one host thread and one stream at a time.
+ *   - Matrices are dense row-major fp32, rows x cols, on the host side of the
+ *     API; inside the workspace rows are padded to a multiple of 4 floats.
+ *   - Worker ids are 0..n_workers-1.  An edge is stored once, as (i, j), i < j.
+ */
+#ifndef POWERGOSSIP_H_
+#define POWERGOSSIP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(PG_BUILDING_LIBRARY)
+#define PG_API __attribute__((visibility("default")))
+#else
+#define PG_API
+#endif
+
+typedef enum pg_status {
+    PG_OK = 0,
+    PG_ERR_INVALID = 1,    /* bad argument, invalid topology or mixing matrix      */
+    PG_ERR_WORKSPACE = 2,  /* workspace missing, misaligned, too small, not device */
+    PG_ERR_CUDA = 3,       /* a CUDA runtime call failed                           */
+    PG_ERR_STATE = 4,      /* call not allowed in the context's current state      */
+    PG_ERR_TIMEOUT = 5,    /* a bounded device-side wait gave up                   */
+    PG_ERR_NUMERIC = 6     /* a norm was not finite (NaN / Inf in the parameters)  */
+} pg_status;
+
+/* Graph kinds.  The paper's experiments use rings; Assumption A4 (Section 5.1)
+ * allows any undirected connected graph, and Theorem 1 allows the compressors
+ * (hence the graph) to change over time. */
+enum {
+    PG_RING = 0,      /* edges {i, (i+1) mod N}                                       */
+    PG_TORUS = 1,     /* torus_rows x torus_cols grid with wrap-around, id = r*C + c   */
+    PG_MATCHING = 2,  /* time-varying: a perfect matching re-drawn every round (N even) */
+    PG_CUSTOM = 3     /* caller's edge list                                            */
+};
+
+/* How the gossip weight W_ij of an edge is chosen (Assumption A4: W symmetric,
+ * doubly stochastic, non-zero only on edges; the self weight is 1 - row sum). */
+enum {
+    PG_W_UNIFORM = 0,     /* 1 / (max degree + 1)                                  */
+    PG_W_METROPOLIS = 1,  /* 1 / (1 + max(deg_i, deg_j)); 1/2 on a matching        */
+    PG_W_EXPLICIT = 2     /* the N x N matrix passed to pg_create                  */
+};
+
+typedef struct pg_topology {
+    int32_t kind;                 /* PG_RING ... PG_CUSTOM                               */
+    int32_t n_workers;            /* N >= 2                                              */
+    int32_t torus_rows;           /* PG_TORUS only; rows * cols == N                     */
+    int32_t torus_cols;
+    int32_t weight_rule;          /* PG_W_*; ignored for PG_MATCHING (always 1/2)        */
+    int32_t n_custom_edges;       /* PG_CUSTOM only                                      */
+    const int32_t *custom_edges;  /* host, 2*n_custom_edges ints; copied by pg_create    */
+} pg_topology;
+
+typedef struct pg_layer_shape {
+    int32_t rows;  /* output size (output channels for a convolution)               */
+    int32_t cols;  /* input size (input channels x kernel height x kernel width)    */
+} pg_layer_shape;
+
+typedef struct pg_ctx pg_ctx;  /* opaque; host memory owned by the library */
+
+/* Limits of this build. */
+#define PG_MAX_RANK 4          /* columns per edge                                    */
+#define PG_MAX_SLOTS 8         /* (max degree) * rank vectors handled per worker      */
+
+/*
+ * Size in bytes of the device workspace a context with these parameters needs
+ * (parameters of all workers, per-pair vectors, exchange buffers, tables).
+ * `shapes`: host, n_layers entries.  PG_ERR_INVALID for a bad topology, rank
+ * outside 1..PG_MAX_RANK or degree*rank > PG_MAX_SLOTS.
+ */
+PG_API int pg_workspace_bytes(const pg_topology *topo, const pg_layer_shape *shapes, int32_t n_layers,
+                       int32_t rank, size_t *bytes_out);
+
+/*
+ * Build a network (Algorithm 2, initialisation; Assumption A4).
+ *   topo, shapes  host; copied.
+ *   W_host        host, N x N row-major fp32 mixing matrix, required for
+ *                 PG_W_EXPLICIT and ignored otherwise.  Checked against A4:
+ *                 symmetric, off-diagonal entries >= 0 and non-zero only on
+ *                 edges, every row sums to 1 within 1e-5; an edge weight of 0 is
+ *                 accepted only for PG_CUSTOM (it freezes that edge's update).
+ *   rank          columns of every per-edge factor (1 = the paper's Algorithm 2;
+ *                 > 1 orthogonalises instead of normalising, Appendix "Changing
+ *                 rank vs changing # power iterations").
+ *   power_steps   power steps per round; one step = two consecutive iterations
+ *                 of Algorithm 2 (X, then X transposed) followed by the update.
+ *   seed          keys the per-pair standard-normal initial vectors (Philox4x32-10
+ *                 + Box-Muller: entry e of column k of pair (i<j), layer l uses
+ *                 counter (e/4, l, i, j*256+k)) and the per-round matchings.
+ *   dev_workspace device, >= pg_workspace_bytes(), 256-byte aligned, on the
+ *                 current device; zeroed and filled by this call (synchronous).
+ * All parameters start at zero; load them with pg_write_params.
+ */
+PG_API int pg_create(const pg_topology *topo, const float *W_host, const pg_layer_shape *shapes,
+              int32_t n_layers, int32_t rank, int32_t power_steps, uint64_t seed,
+              void *dev_workspace, size_t workspace_bytes, pg_ctx **ctx_out);
+
+/* Free the host side of a context (NULL is accepted).  The workspace stays the
+ * caller's.  Does not synchronise: finish the stream first. */
+PG_API void pg_destroy(pg_ctx *ctx);
+
+/*
+ * Copy one dense rows x cols fp32 matrix from host memory into worker
+ * `worker`'s layer `layer` (Algorithm 1, input X_i^(0)).  Asynchronous on
+ * `stream` when host_src is pinned; host_src must stay valid until the stream
+ * reaches the copy.
+ */
+PG_API int pg_write_params(pg_ctx *ctx, int32_t worker, int32_t layer, const float *host_src, void *stream);
+
+/*
+ * Copy worker `worker`'s layer `layer` to host memory (dense rows x cols fp32),
+ * then wait for `stream` and report the device status word: PG_ERR_NUMERIC if a
+ * non-finite norm was met in any round since the context was created.
+ */
+PG_API int pg_read_params(pg_ctx *ctx, int32_t worker, int32_t layer, float *host_dst, void *stream);
+
+/*
+ * Enqueue one gossip round on `stream` (asynchronous): `power_steps` power
+ * steps on every layer and every edge of this round's graph, each one
+ *     Qh = unit columns of the pair's stored Q        (Algorithm 2, v / ||v||)
+ *     P  = X_i Qh - X_j Qh,  Ph = orthonormalised P   (Eq. 3, odd iteration)
+ *     Q' = X_i^T Ph - X_j^T Ph                        (Eq. 3, even iteration)
+ *     X_i -= W_ij Ph Q'^T,  X_j += W_ij Ph Q'^T,  Q = Q'   (Eq. 2; Lemma 1)
+ * with all edges of a step reading the same pre-update X.  Advances the round
+ * counter.  Host-side errors are returned at once; device-side ones show up in
+ * pg_read_params / pg_device_status.
+ */
+PG_API int pg_round(pg_ctx *ctx, void *stream);
+
+/* Wait for `stream` and return the device status word (PG_OK or PG_ERR_NUMERIC). */
+PG_API int pg_device_status(pg_ctx *ctx, void *stream);
+
+/*
+ * Edge list and weights of round `round` (Assumption A4's graph and W): writes
+ * up to pg_max_edges() pairs (i<j, sorted) to edges_out (host, 2 ints per edge)
+ * and their weights to w_out (host, may be NULL); *n_edges_out = count.
+ */
+PG_API int pg_get_schedule(pg_ctx *ctx, int64_t round, int32_t *edges_out, float *w_out, int32_t *n_edges_out);
+
+/* Upper bound on the number of edges in any round of this context. */
+PG_API int pg_max_edges(pg_ctx *ctx, int32_t *max_edges_out);
+
+/*
+ * Read / overwrite the stored right factor of the unordered pair {i, j} for
+ * one layer (Algorithm 2's v_ij): host buffer of cols*rank floats, column k at
+ * [k*cols, (k+1)*cols).  Synchronous with respect to `stream`.
+ */
+PG_API int pg_read_q(pg_ctx *ctx, int32_t i, int32_t j, int32_t layer, float *host_dst, void *stream);
+PG_API int pg_write_q(pg_ctx *ctx, int32_t i, int32_t j, int32_t layer, const float *host_src, void *stream);
+
+/* Round counter (the index of the next round): read it, or set it when
+ * restoring a checkpoint {all X, all Q, round}. */
+PG_API int pg_get_round(pg_ctx *ctx, int64_t *round_out);
+PG_API int pg_set_round(pg_ctx *ctx, int64_t round);
+
+/*
+ * Context-free, host-only view of the schedule builder: the edge list (i<j,
+ * sorted) and weights that a context with this topology, mixing matrix and seed
+ * uses in round `round` (Assumption A4; for PG_MATCHING a Fisher-Yates shuffle
+ * of 0..N-1 whose draw at position k, from N-1 down to 1, is the low 64 bits of
+ * Philox4x32-10 at counter (k, round_lo, round_hi, 0xFFFFFFFF) modulo k+1, with
+ * consecutive entries paired).  edges_out: host, room for `capacity` pairs;
+ * w_out: host, `capacity` floats, may be NULL.  PG_ERR_INVALID if the topology
+ * or matrix is invalid or `capacity` is too small.  Touches no GPU.
+ */
+PG_API int pg_build_schedule(const pg_topology *topo, const float *W_host, uint64_t seed, int64_t round,
+                             int32_t *edges_out, float *w_out, int32_t capacity, int32_t *n_edges_out);
+
+/*
+ * Host-only: column `col` of the standard-normal vector that pair (i<j) starts
+ * with for layer `layer` (Algorithm 2, initialisation), m floats to host_dst.
+ * This is what pg_create stores; exposed so the seeding can be checked without
+ * a GPU.
+ */
+PG_API int pg_initial_vector(uint64_t seed, int32_t i, int32_t j, int32_t layer, int32_t col, int32_t m,
+                             float *host_dst);
+
+/* Number of kernels this context has launched so far. */
+PG_API int pg_kernel_launches(pg_ctx *ctx, int64_t *count_out);
+
+/* Static string for a status code. */
+PG_API const char *pg_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POWERGOSSIP_H_ */

@@ -446,11 +446,11 @@ static void edge_power_step(const double *Xi, const double *Xj, int n, int m, in
             for (int r = 0; r < n; ++r) p[r] -= a * ph[r];
         }
         double nn = dot(p, p, n);
-        /* a column that is zero, or (for k > 0) whose residual has dropped to
-         * rounding level (norm below 1e-10 of its length before projection: it
-         * was a linear combination of the earlier columns and what is left has
-         * no meaningful direction), contributes nothing and keeps its vector */
-        int ok = (nn > 0.0) && isfinite(nn) && (k == 0 || nn > 1e-20 * pre);
+        /* a column that is zero, or (for k > 0) whose residual has dropped below
+         * 1e-5 of its length before projection (it was, to fp32 working accuracy,
+         * a linear combination of the earlier columns: what is left has no
+         * meaningful direction), contributes nothing and keeps its vector */
+        int ok = (nn > 0.0) && isfinite(nn) && (k == 0 || nn > 1e-10 * pre);
         live[k] = ok;
         double inv = ok ? 1.0 / sqrt(nn) : 0.0;
         for (int r = 0; r < n; ++r) p[r] = ok ? p[r] * inv : 0.0;

@@ -1,0 +1,290 @@
+"""Python binding of the C ABI in ``include/powergossip.h`` (ctypes).
+
+Argument marshalling only: every step of a gossip round runs in the CUDA
+kernels of ``libpowergossip.so``.  PyTorch is used for device memory (the
+workspace tensor), pinned host buffers and streams.  There is no CPU fallback:
+if the library has not been built, loading it raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpowergossip.so")
+
+PG_OK, PG_ERR_INVALID, PG_ERR_WORKSPACE, PG_ERR_CUDA, PG_ERR_STATE, PG_ERR_TIMEOUT, PG_ERR_NUMERIC = range(7)
+PG_RING, PG_TORUS, PG_MATCHING, PG_CUSTOM = 0, 1, 2, 3
+PG_W_UNIFORM, PG_W_METROPOLIS, PG_W_EXPLICIT = 0, 1, 2
+
+EXPORTS = (
+    "pg_workspace_bytes", "pg_create", "pg_destroy", "pg_write_params", "pg_read_params",
+    "pg_round", "pg_device_status", "pg_get_schedule", "pg_max_edges", "pg_read_q", "pg_write_q",
+    "pg_get_round", "pg_set_round", "pg_kernel_launches", "pg_status_string",
+    "pg_build_schedule", "pg_initial_vector",
+)
+
+
+class pg_topology(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("n_workers", ctypes.c_int32),
+                ("torus_rows", ctypes.c_int32), ("torus_cols", ctypes.c_int32),
+                ("weight_rule", ctypes.c_int32), ("n_custom_edges", ctypes.c_int32),
+                ("custom_edges", ctypes.POINTER(ctypes.c_int32))]
+
+
+class pg_layer_shape(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int32), ("cols", ctypes.c_int32)]
+
+
+class PowerGossipError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__("%s: %s (status %d)" % (where, pg_status_string(status), status))
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libpowergossip.so; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("%s is missing: build it with `python -m paper_2008_01425_b200.build` "
+                          "(there is no CPU fallback)" % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64
+    szp = ctypes.POINTER(ctypes.c_size_t)
+    L.pg_workspace_bytes.argtypes = [ctypes.POINTER(pg_topology), ctypes.POINTER(pg_layer_shape), i32, i32, szp]
+    L.pg_create.argtypes = [ctypes.POINTER(pg_topology), vp, ctypes.POINTER(pg_layer_shape), i32, i32, i32,
+                            u64, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    L.pg_destroy.argtypes = [vp]
+    L.pg_destroy.restype = None
+    L.pg_write_params.argtypes = [vp, i32, i32, vp, vp]
+    L.pg_read_params.argtypes = [vp, i32, i32, vp, vp]
+    L.pg_round.argtypes = [vp, vp]
+    L.pg_device_status.argtypes = [vp, vp]
+    L.pg_get_schedule.argtypes = [vp, i64, vp, vp, ctypes.POINTER(i32)]
+    L.pg_max_edges.argtypes = [vp, ctypes.POINTER(i32)]
+    L.pg_read_q.argtypes = [vp, i32, i32, i32, vp, vp]
+    L.pg_write_q.argtypes = [vp, i32, i32, i32, vp, vp]
+    L.pg_get_round.argtypes = [vp, ctypes.POINTER(i64)]
+    L.pg_set_round.argtypes = [vp, i64]
+    L.pg_kernel_launches.argtypes = [vp, ctypes.POINTER(i64)]
+    L.pg_build_schedule.argtypes = [ctypes.POINTER(pg_topology), vp, u64, i64, vp, vp, i32, ctypes.POINTER(i32)]
+    L.pg_initial_vector.argtypes = [u64, i32, i32, i32, i32, i32, vp]
+    L.pg_status_string.argtypes = [ctypes.c_int]
+    L.pg_status_string.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name not in ("pg_destroy", "pg_status_string"):
+            getattr(L, name).restype = ctypes.c_int
+    _lib = L
+    return L
+
+
+def pg_status_string(status: int) -> str:
+    return load_library().pg_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != PG_OK:
+        raise PowerGossipError(status, where)
+
+
+def _topology(kind, n_workers, torus_rows, torus_cols, weight_rule, custom_edges):
+    edges = np.ascontiguousarray(np.asarray(custom_edges, dtype=np.int32).reshape(-1, 2))
+    topo = pg_topology(kind, n_workers, torus_rows, torus_cols, weight_rule, len(edges),
+                       edges.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)) if len(edges) else None)
+    return topo, edges   # keep `edges` alive while `topo` is in use
+
+
+def _shapes(layer_shapes):
+    arr = (pg_layer_shape * len(layer_shapes))()
+    for t, (n, m) in enumerate(layer_shapes):
+        arr[t].rows, arr[t].cols = int(n), int(m)
+    return arr
+
+
+def pg_workspace_bytes(kind: int, n_workers: int, layer_shapes: Sequence[Tuple[int, int]], rank: int,
+                       torus_rows: int = 0, torus_cols: int = 0, weight_rule: int = PG_W_METROPOLIS,
+                       custom_edges: Sequence[Tuple[int, int]] = ()) -> int:
+    topo, _keep = _topology(kind, n_workers, torus_rows, torus_cols, weight_rule, custom_edges)
+    out = ctypes.c_size_t(0)
+    _check(load_library().pg_workspace_bytes(ctypes.byref(topo), _shapes(layer_shapes), len(layer_shapes),
+                                             rank, ctypes.byref(out)), "pg_workspace_bytes")
+    return int(out.value)
+
+
+def pg_build_schedule(kind: int, n_workers: int, seed: int = 0, round_index: int = 0,
+                      torus_rows: int = 0, torus_cols: int = 0, weight_rule: int = PG_W_METROPOLIS,
+                      custom_edges: Sequence[Tuple[int, int]] = (),
+                      W: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Edge list (E, 2) int32 and weights (E,) fp32 of one round; host only, no GPU needed."""
+    topo, keep = _topology(kind, n_workers, torus_rows, torus_cols, weight_rule, custom_edges)
+    cap = max(2 * n_workers, len(keep), 1)
+    edges = np.zeros((cap, 2), dtype=np.int32)
+    w = np.zeros(cap, dtype=np.float32)
+    n = ctypes.c_int32(0)
+    Wf = None if W is None else np.ascontiguousarray(W, dtype=np.float32)
+    _check(load_library().pg_build_schedule(ctypes.byref(topo), None if Wf is None else Wf.ctypes.data,
+                                            seed, round_index, edges.ctypes.data, w.ctypes.data, cap,
+                                            ctypes.byref(n)), "pg_build_schedule")
+    return edges[:n.value].copy(), w[:n.value].copy()
+
+
+def pg_initial_vector(seed: int, i: int, j: int, layer: int, col: int, m: int) -> np.ndarray:
+    """Column `col` of the seeded initial vector of pair (i<j), layer `layer`; host only."""
+    out = np.zeros(m, dtype=np.float32)
+    _check(load_library().pg_initial_vector(seed, i, j, layer, col, m, out.ctypes.data), "pg_initial_vector")
+    return out
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream or None
+    return int(stream.cuda_stream) or None
+
+
+class PowerGossip:
+    """One simulated network on one GPU (thin handle around ``pg_ctx``).
+
+    The workspace is a ``torch.uint8`` tensor on ``device`` that this object
+    keeps alive; every method forwards to the C function of the same name.
+    """
+
+    def __init__(self, kind: int, n_workers: int, layer_shapes: Sequence[Tuple[int, int]],
+                 rank: int = 1, power_steps: int = 1, seed: int = 0,
+                 torus_rows: int = 0, torus_cols: int = 0,
+                 custom_edges: Sequence[Tuple[int, int]] = (),
+                 weight_rule: int = PG_W_METROPOLIS, W: Optional[np.ndarray] = None,
+                 device: str = "cuda:0", workspace=None):
+        import torch
+
+        self._lib = load_library()
+        self._h = None
+        self.n_workers = int(n_workers)
+        self.layer_shapes = [(int(a), int(b)) for a, b in layer_shapes]
+        self.rank = int(rank)
+        self.power_steps = int(power_steps)
+        self.device = torch.device(device)
+        topo, _keep = _topology(kind, n_workers, torus_rows, torus_cols, weight_rule, custom_edges)
+        shapes = _shapes(self.layer_shapes)
+        nbytes = ctypes.c_size_t(0)
+        _check(self._lib.pg_workspace_bytes(ctypes.byref(topo), shapes, len(self.layer_shapes), rank,
+                                            ctypes.byref(nbytes)), "pg_workspace_bytes")
+        self.workspace_bytes = int(nbytes.value)
+        torch.cuda.set_device(self.device)
+        if workspace is None:
+            workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+        self._workspace = workspace
+        base = workspace.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        avail = workspace.numel() - (aligned - base)
+        Wf = None if W is None else np.ascontiguousarray(W, dtype=np.float32)
+        h = ctypes.c_void_p()
+        _check(self._lib.pg_create(ctypes.byref(topo), None if Wf is None else Wf.ctypes.data,
+                                   shapes, len(self.layer_shapes), rank, power_steps, seed,
+                                   ctypes.c_void_p(aligned), avail, ctypes.byref(h)), "pg_create")
+        self._h = h
+
+    # -- lifetime ---------------------------------------------------------
+    def pg_destroy(self) -> None:
+        if self._h is not None:
+            self._lib.pg_destroy(self._h)
+            self._h = None
+
+    close = pg_destroy
+
+    def __del__(self):
+        try:
+            self.pg_destroy()
+        except Exception:
+            pass
+
+    # -- parameters -------------------------------------------------------
+    def pg_write_params(self, worker: int, layer: int, x, stream=None) -> None:
+        """x: numpy array or CPU torch tensor, fp32, dense rows x cols."""
+        ptr, _keep = _host_ptr(x, self.layer_shapes[layer])
+        _check(self._lib.pg_write_params(self._h, worker, layer, ptr, _stream_handle(stream)),
+               "pg_write_params")
+
+    def pg_read_params(self, worker: int, layer: int, out=None, stream=None):
+        if out is None:
+            out = np.empty(self.layer_shapes[layer], dtype=np.float32)
+        ptr, _keep = _host_ptr(out, self.layer_shapes[layer])
+        _check(self._lib.pg_read_params(self._h, worker, layer, ptr, _stream_handle(stream)),
+               "pg_read_params")
+        return out
+
+    def pg_read_q(self, i: int, j: int, layer: int, stream=None) -> np.ndarray:
+        """(cols, rank) array."""
+        m = self.layer_shapes[layer][1]
+        out = np.empty((self.rank, m), dtype=np.float32)
+        _check(self._lib.pg_read_q(self._h, i, j, layer, out.ctypes.data, _stream_handle(stream)), "pg_read_q")
+        return out.T.copy()
+
+    def pg_write_q(self, i: int, j: int, layer: int, q: np.ndarray, stream=None) -> None:
+        m = self.layer_shapes[layer][1]
+        src = np.ascontiguousarray(np.asarray(q, dtype=np.float32).reshape(m, self.rank).T)
+        _check(self._lib.pg_write_q(self._h, i, j, layer, src.ctypes.data, _stream_handle(stream)), "pg_write_q")
+
+    # -- rounds -----------------------------------------------------------
+    def pg_round(self, stream=None) -> None:
+        _check(self._lib.pg_round(self._h, _stream_handle(stream)), "pg_round")
+
+    def pg_device_status(self, stream=None) -> int:
+        return int(self._lib.pg_device_status(self._h, _stream_handle(stream)))
+
+    def pg_get_schedule(self, round_index: int) -> Tuple[np.ndarray, np.ndarray]:
+        cap = ctypes.c_int32(0)
+        _check(self._lib.pg_max_edges(self._h, ctypes.byref(cap)), "pg_max_edges")
+        edges = np.zeros((cap.value, 2), dtype=np.int32)
+        w = np.zeros(cap.value, dtype=np.float32)
+        n = ctypes.c_int32(0)
+        _check(self._lib.pg_get_schedule(self._h, round_index, edges.ctypes.data, w.ctypes.data,
+                                         ctypes.byref(n)), "pg_get_schedule")
+        return edges[:n.value].copy(), w[:n.value].copy()
+
+    def pg_get_round(self) -> int:
+        r = ctypes.c_int64(0)
+        _check(self._lib.pg_get_round(self._h, ctypes.byref(r)), "pg_get_round")
+        return int(r.value)
+
+    def pg_set_round(self, r: int) -> None:
+        _check(self._lib.pg_set_round(self._h, int(r)), "pg_set_round")
+
+    def pg_kernel_launches(self) -> int:
+        r = ctypes.c_int64(0)
+        _check(self._lib.pg_kernel_launches(self._h, ctypes.byref(r)), "pg_kernel_launches")
+        return int(r.value)
+
+    # -- conveniences built only from the calls above ---------------------
+    def write_all(self, params: Sequence[Sequence[np.ndarray]], stream=None) -> None:
+        for i, row in enumerate(params):
+            for l, x in enumerate(row):
+                self.pg_write_params(i, l, x, stream)
+
+    def read_all(self, stream=None) -> List[List[np.ndarray]]:
+        return [[self.pg_read_params(i, l, stream=stream) for l in range(len(self.layer_shapes))]
+                for i in range(self.n_workers)]
+
+
+def _host_ptr(x, shape):
+    """Pointer to a dense fp32 host array (numpy or CPU torch tensor)."""
+    if isinstance(x, np.ndarray):
+        if x.dtype != np.float32 or not x.flags["C_CONTIGUOUS"] or tuple(x.shape) != tuple(shape):
+            raise ValueError("expected a C-contiguous float32 array of shape %r" % (tuple(shape),))
+        return ctypes.c_void_p(x.ctypes.data), x
+    import torch
+
+    if isinstance(x, torch.Tensor):
+        if x.is_cuda or x.dtype != torch.float32 or not x.is_contiguous() or tuple(x.shape) != tuple(shape):
+            raise ValueError("expected a contiguous float32 CPU tensor of shape %r" % (tuple(shape),))
+        return ctypes.c_void_p(x.data_ptr()), x
+    raise TypeError("expected a numpy array or a CPU torch tensor")

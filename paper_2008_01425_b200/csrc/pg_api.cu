@@ -1,0 +1,596 @@
+// Host side of the C ABI declared in include/powergossip.h: argument checks,
+// workspace carve-up, per-round tables and the order in which the kernels of a
+// gossip round are enqueued.  No arithmetic of the method happens here.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <climits>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "powergossip.h"
+#include "pg_device.h"
+#include "pg_schedule.h"
+
+namespace {
+
+using pg::DevState;
+using pg::Edge;
+using pg::LayerGeom;
+using pg::TabLayout;
+using pg::Tile;
+
+constexpr int kTabRing = 4;          // device copies of per-round tables kept alive
+constexpr size_t kAlign = 256;       // every workspace section starts on this boundary
+
+inline long long round_up(long long v, long long a) { return (v + a - 1) / a * a; }
+
+// Byte offsets of the workspace sections.
+struct Layout {
+    std::vector<LayerGeom> layers;
+    long long x_stride = 0, q_stride = 0, y_stride = 0, ph_stride = 0, z_stride = 0;
+    long long n_pairs = 0;
+    int max_edges = 0, max_degree = 0;
+    TabLayout tab{};
+    long long n_row_tiles = 0, n_col_tiles = 0;
+    size_t off_X = 0, off_Q = 0, off_Qinv = 0, off_Y = 0, off_Ph = 0, off_Z = 0, off_live = 0,
+           off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
+    size_t total = 0;
+};
+
+int make_topology(const pg_topology* topo, const float* W_host, pg::Topology& out) {
+    if (!topo || topo->n_workers < 2 || topo->n_workers > 32768) return PG_ERR_INVALID;
+    if (topo->kind < PG_RING || topo->kind > PG_CUSTOM) return PG_ERR_INVALID;
+    out.kind = topo->kind;
+    out.n_workers = topo->n_workers;
+    out.torus_rows = topo->torus_rows;
+    out.torus_cols = topo->torus_cols;
+    out.weight_rule = topo->weight_rule;
+    out.custom.clear();
+    if (topo->kind == PG_CUSTOM) {
+        if (topo->n_custom_edges < 1 || !topo->custom_edges) return PG_ERR_INVALID;
+        for (int e = 0; e < topo->n_custom_edges; ++e) {
+            const int a = topo->custom_edges[2 * e], b = topo->custom_edges[2 * e + 1];
+            if (a < 0 || b < 0 || a >= topo->n_workers || b >= topo->n_workers) return PG_ERR_INVALID;
+            out.custom.push_back(Edge{a, b});
+        }
+        pg::canonicalise(out.custom);
+        if (out.custom.empty()) return PG_ERR_INVALID;
+    }
+    if (topo->kind != PG_MATCHING) {
+        if (topo->weight_rule < PG_W_UNIFORM || topo->weight_rule > PG_W_EXPLICIT) return PG_ERR_INVALID;
+        if (topo->weight_rule == PG_W_EXPLICIT) {
+            if (!W_host) return PG_ERR_INVALID;
+            out.W.assign(W_host, W_host + static_cast<size_t>(topo->n_workers) * topo->n_workers);
+        }
+    }
+    return PG_OK;
+}
+
+int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_layers, int rank,
+                Layout& lay) {
+    if (!shapes || n_layers < 1 || n_layers > 4096) return PG_ERR_INVALID;
+    if (rank < 1 || rank > PG_MAX_RANK) return PG_ERR_INVALID;
+    if (!pg::topology_bounds(topo, &lay.max_edges, &lay.max_degree)) return PG_ERR_INVALID;
+    if (lay.max_degree * rank > PG_MAX_SLOTS) return PG_ERR_INVALID;
+    const int N = topo.n_workers;
+    const int slots = lay.max_degree * rank;
+    lay.n_pairs = topo.kind == PG_MATCHING ? static_cast<long long>(N) * (N - 1) / 2 : lay.max_edges;
+    if (lay.n_pairs > INT_MAX / 2) return PG_ERR_INVALID;
+
+    lay.layers.resize(n_layers);
+    long long x = 0, q = 0, y = 0, ph = 0, z = 0;
+    lay.n_row_tiles = lay.n_col_tiles = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        LayerGeom& g = lay.layers[l];
+        if (shapes[l].rows < 1 || shapes[l].cols < 1) return PG_ERR_INVALID;
+        if (static_cast<long long>(shapes[l].rows) * shapes[l].cols > (1LL << 40)) return PG_ERR_INVALID;
+        g.n = shapes[l].rows;
+        g.m = shapes[l].cols;
+        g.ld = static_cast<int>(round_up(g.m, 4));
+        g.npad = static_cast<int>(round_up(g.n, 4));
+        g.f_rtiles = (g.n + pg::kRowTileRows - 1) / pg::kRowTileRows;
+        g.f_csplit = (g.ld + pg::kRowTileCols - 1) / pg::kRowTileCols;
+        g.f_chunk = static_cast<int>(round_up((g.ld + g.f_csplit - 1) / g.f_csplit, 128));
+        g.f_csplit = (g.ld + g.f_chunk - 1) / g.f_chunk;
+        g.t_rtiles = (g.n + pg::kColTileRows - 1) / pg::kColTileRows;
+        g.t_ctiles = (g.ld + pg::kColTileCols - 1) / pg::kColTileCols;
+        g.x_off = x;
+        g.q_off = q;
+        g.y_off = y;
+        g.ph_off = ph;
+        g.z_off = z;
+        x += round_up(static_cast<long long>(g.n) * g.ld, 64);
+        q += round_up(static_cast<long long>(rank) * g.ld, 64);
+        y += round_up(static_cast<long long>(slots) * g.f_csplit * g.npad, 64);
+        ph += round_up(static_cast<long long>(rank) * g.npad, 64);
+        z += round_up(static_cast<long long>(slots) * g.t_rtiles * g.ld, 64);
+        lay.n_row_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
+        lay.n_col_tiles += static_cast<long long>(N) * g.t_rtiles * g.t_ctiles;
+    }
+    if (lay.n_row_tiles > INT_MAX || lay.n_col_tiles > INT_MAX) return PG_ERR_INVALID;
+    lay.x_stride = x;
+    lay.q_stride = q;
+    lay.y_stride = y;
+    lay.ph_stride = ph;
+    lay.z_stride = z;
+
+    TabLayout& t = lay.tab;
+    t.max_edges = lay.max_edges;
+    t.n_workers = N;
+    t.max_degree = lay.max_degree;
+    int o = 0;
+    t.off_n_edges = o; o += 4;
+    t.off_edge_i = o; o += lay.max_edges;
+    t.off_edge_j = o; o += lay.max_edges;
+    t.off_pair = o; o += lay.max_edges;
+    t.off_w = o; o += lay.max_edges;
+    t.off_slot_i = o; o += lay.max_edges;
+    t.off_slot_j = o; o += lay.max_edges;
+    t.off_degree = o; o += N;
+    t.off_slot_edge = o; o += N * lay.max_degree;
+    t.off_slot_coef = o; o += N * lay.max_degree;
+    t.total_ints = static_cast<int>(round_up(o, 64));
+
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off = static_cast<size_t>(round_up(static_cast<long long>(off + bytes), kAlign));
+        return at;
+    };
+    lay.off_X = take(sizeof(float) * static_cast<size_t>(N) * lay.x_stride);
+    lay.off_Q = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride);
+    lay.off_Qinv = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * n_layers * rank);
+    lay.off_Y = take(sizeof(float) * static_cast<size_t>(N) * lay.y_stride);
+    lay.off_Ph = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * lay.ph_stride);
+    lay.off_Z = take(sizeof(float) * static_cast<size_t>(N) * lay.z_stride);
+    lay.off_live = take(sizeof(int) * static_cast<size_t>(lay.max_edges) * n_layers * rank);
+    lay.off_status = take(sizeof(int) * 64);
+    lay.off_layers = take(sizeof(LayerGeom) * static_cast<size_t>(n_layers));
+    lay.off_tabs = take(sizeof(int) * static_cast<size_t>(kTabRing) * t.total_ints);
+    lay.off_row_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_row_tiles));
+    lay.off_col_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_col_tiles));
+    lay.total = off;
+    return PG_OK;
+}
+
+}  // namespace
+
+struct pg_ctx {
+    pg::Topology topo;
+    pg::PairIndex pairs;
+    Layout lay;
+    DevState st{};
+    uint64_t seed = 0;
+    int rank = 1, power_steps = 1, n_layers = 0;
+    int64_t round = 0;
+    bool y_valid = false;       // Y already holds X Qh for the upcoming round
+    int64_t launches = 0;
+    char* ws = nullptr;
+    int* d_tabs = nullptr;
+    int* h_tabs = nullptr;      // pinned staging, kTabRing tables
+    cudaEvent_t tab_event[kTabRing] = {};
+    int64_t tab_round[kTabRing];
+    bool tab_used[kTabRing];
+    Tile* d_row_tiles = nullptr;
+    Tile* d_col_tiles = nullptr;
+    bool static_graph = true;
+    int device = 0;
+};
+
+namespace {
+
+// Fill the pinned copy of round `round`'s table.
+int fill_table(pg_ctx* c, int64_t round, int* tab) {
+    std::vector<Edge> edges;
+    std::vector<float> w;
+    if (!pg::build_edges(c->topo, c->seed, round, edges)) return PG_ERR_INVALID;
+    if (!pg::edge_weights(c->topo, edges, w)) return PG_ERR_INVALID;
+    if (static_cast<int>(edges.size()) > c->lay.max_edges) return PG_ERR_INVALID;
+    pg::RoundSlots slots;
+    pg::build_slots(c->topo.n_workers, edges, slots);
+    const TabLayout& t = c->lay.tab;
+    std::memset(tab, 0, sizeof(int) * static_cast<size_t>(t.total_ints));
+    tab[t.off_n_edges] = static_cast<int>(edges.size());
+    for (size_t e = 0; e < edges.size(); ++e) {
+        const int64_t pair = c->pairs.of(edges[e].i, edges[e].j);
+        if (pair < 0) return PG_ERR_INVALID;
+        tab[t.off_edge_i + e] = edges[e].i;
+        tab[t.off_edge_j + e] = edges[e].j;
+        tab[t.off_pair + e] = static_cast<int>(pair);
+        std::memcpy(&tab[t.off_w + e], &w[e], sizeof(float));
+        tab[t.off_slot_i + e] = slots.slot_at_i[e];
+        tab[t.off_slot_j + e] = slots.slot_at_j[e];
+    }
+    for (int v = 0; v < c->topo.n_workers; ++v) {
+        if (slots.degree[v] > t.max_degree) return PG_ERR_INVALID;
+        tab[t.off_degree + v] = slots.degree[v];
+        for (int s = 0; s < slots.degree[v]; ++s) {
+            const int e = slots.slot_edge[v][s];
+            const float coef = slots.slot_sign[v][s] * w[e];
+            tab[t.off_slot_edge + v * t.max_degree + s] = e;
+            std::memcpy(&tab[t.off_slot_coef + v * t.max_degree + s], &coef, sizeof(float));
+        }
+    }
+    return PG_OK;
+}
+
+// Device pointer of the table of round `round`, uploading it if needed.
+int ensure_table(pg_ctx* c, int64_t round, cudaStream_t stream, const int** out) {
+    const int64_t key = c->static_graph ? 0 : round;
+    const int slot = static_cast<int>(((key % kTabRing) + kTabRing) % kTabRing);
+    const size_t ints = static_cast<size_t>(c->lay.tab.total_ints);
+    int* dev = c->d_tabs + static_cast<size_t>(slot) * ints;
+    if (c->tab_used[slot] && c->tab_round[slot] == key) {
+        *out = dev;
+        return PG_OK;
+    }
+    int* host = c->h_tabs + static_cast<size_t>(slot) * ints;
+    if (c->tab_used[slot] && cudaEventSynchronize(c->tab_event[slot]) != cudaSuccess) return PG_ERR_CUDA;
+    const int rc = fill_table(c, key, host);
+    if (rc != PG_OK) return rc;
+    if (cudaMemcpyAsync(dev, host, sizeof(int) * ints, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return PG_ERR_CUDA;
+    if (cudaEventRecord(c->tab_event[slot], stream) != cudaSuccess) return PG_ERR_CUDA;
+    c->tab_used[slot] = true;
+    c->tab_round[slot] = key;
+    *out = dev;
+    return PG_OK;
+}
+
+// Kernels and copies go to the device that owns the workspace.
+bool bind_device(const pg_ctx* c) {
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) return false;
+    return cur == c->device || cudaSetDevice(c->device) == cudaSuccess;
+}
+
+int check_worker_layer(const pg_ctx* c, int worker, int layer) {
+    if (!c) return PG_ERR_INVALID;
+    if (worker < 0 || worker >= c->topo.n_workers || layer < 0 || layer >= c->n_layers) return PG_ERR_INVALID;
+    return PG_OK;
+}
+
+int device_status(pg_ctx* c, cudaStream_t stream) {
+    int word = 0;
+    if (cudaMemcpyAsync(&word, c->st.status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return PG_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return PG_ERR_CUDA;
+    if (word & (1 << PG_ERR_TIMEOUT)) return PG_ERR_TIMEOUT;
+    if (word & (1 << PG_ERR_NUMERIC)) return PG_ERR_NUMERIC;
+    return word == 0 ? PG_OK : PG_ERR_STATE;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pg_workspace_bytes(const pg_topology* topo, const pg_layer_shape* shapes, int32_t n_layers,
+                       int32_t rank, size_t* bytes_out) {
+    if (!bytes_out) return PG_ERR_INVALID;
+    pg::Topology t;
+    // the explicit matrix does not change the size: validate the graph only
+    pg_topology probe;
+    if (!topo) return PG_ERR_INVALID;
+    probe = *topo;
+    if (probe.kind != PG_MATCHING && probe.weight_rule == PG_W_EXPLICIT) probe.weight_rule = PG_W_METROPOLIS;
+    int rc = make_topology(&probe, nullptr, t);
+    if (rc != PG_OK) return rc;
+    Layout lay;
+    rc = make_layout(t, shapes, n_layers, rank, lay);
+    if (rc != PG_OK) return rc;
+    *bytes_out = lay.total;
+    return PG_OK;
+}
+
+int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape* shapes,
+              int32_t n_layers, int32_t rank, int32_t power_steps, uint64_t seed,
+              void* dev_workspace, size_t workspace_bytes, pg_ctx** ctx_out) {
+    if (!ctx_out || power_steps < 1) return PG_ERR_INVALID;
+    pg_ctx* c = new (std::nothrow) pg_ctx();
+    if (!c) return PG_ERR_INVALID;
+    int rc = make_topology(topo, W_host, c->topo);
+    if (rc == PG_OK) rc = make_layout(c->topo, shapes, n_layers, rank, c->lay);
+    std::vector<Edge> edges0;
+    std::vector<float> w0;
+    if (rc == PG_OK && !pg::build_edges(c->topo, seed, 0, edges0)) rc = PG_ERR_INVALID;
+    if (rc == PG_OK && !pg::edge_weights(c->topo, edges0, w0)) rc = PG_ERR_INVALID;
+    if (rc == PG_OK) {
+        // workspace: present, aligned, large enough and device memory
+        cudaPointerAttributes attr{};
+        if (!dev_workspace || (reinterpret_cast<uintptr_t>(dev_workspace) % kAlign) != 0 ||
+            workspace_bytes < c->lay.total) {
+            rc = PG_ERR_WORKSPACE;
+        } else if (cudaPointerGetAttributes(&attr, dev_workspace) != cudaSuccess ||
+                   attr.type != cudaMemoryTypeDevice) {
+            cudaGetLastError();
+            rc = PG_ERR_WORKSPACE;
+        } else {
+            c->device = attr.device;
+            if (!bind_device(c)) rc = PG_ERR_CUDA;
+        }
+    }
+    if (rc != PG_OK) {
+        delete c;
+        return rc;
+    }
+    c->seed = seed;
+    c->rank = rank;
+    c->power_steps = power_steps;
+    c->n_layers = n_layers;
+    c->static_graph = c->topo.kind != PG_MATCHING;
+    c->pairs.triangular = !c->static_graph;
+    c->pairs.n_workers = c->topo.n_workers;
+    if (c->static_graph) c->pairs.static_edges = edges0;
+    c->ws = static_cast<char*>(dev_workspace);
+    for (int s = 0; s < kTabRing; ++s) {
+        c->tab_used[s] = false;
+        c->tab_round[s] = -1;
+    }
+
+    const Layout& lay = c->lay;
+    DevState& st = c->st;
+    st.X = reinterpret_cast<float*>(c->ws + lay.off_X);
+    st.Q = reinterpret_cast<float*>(c->ws + lay.off_Q);
+    st.Qinv = reinterpret_cast<float*>(c->ws + lay.off_Qinv);
+    st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
+    st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
+    st.Z = reinterpret_cast<float*>(c->ws + lay.off_Z);
+    st.live = reinterpret_cast<int*>(c->ws + lay.off_live);
+    st.status = reinterpret_cast<int*>(c->ws + lay.off_status);
+    st.layers = reinterpret_cast<const LayerGeom*>(c->ws + lay.off_layers);
+    st.x_stride = lay.x_stride;
+    st.q_stride = lay.q_stride;
+    st.y_stride = lay.y_stride;
+    st.ph_stride = lay.ph_stride;
+    st.z_stride = lay.z_stride;
+    st.n_layers = n_layers;
+    st.rank = rank;
+    st.n_workers = c->topo.n_workers;
+    st.max_degree = lay.max_degree;
+    st.tab = lay.tab;
+    c->d_tabs = reinterpret_cast<int*>(c->ws + lay.off_tabs);
+    c->d_row_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_row_tiles);
+    c->d_col_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_col_tiles);
+
+    bool ok = cudaMemset(c->ws, 0, lay.total) == cudaSuccess;
+    ok = ok && cudaMemcpy(c->ws + lay.off_layers, lay.layers.data(), sizeof(LayerGeom) * n_layers,
+                          cudaMemcpyHostToDevice) == cudaSuccess;
+    // tile lists: worker-major, layers in the caller's order
+    if (ok) {
+        std::vector<Tile> rows, cols;
+        rows.reserve(lay.n_row_tiles);
+        cols.reserve(lay.n_col_tiles);
+        for (int v = 0; v < c->topo.n_workers; ++v)
+            for (int l = 0; l < n_layers; ++l) {
+                const LayerGeom& g = lay.layers[l];
+                for (int rt = 0; rt < g.f_rtiles; ++rt)
+                    for (int ct = 0; ct < g.f_csplit; ++ct) rows.push_back(Tile{v, l, rt, ct});
+                for (int rt = 0; rt < g.t_rtiles; ++rt)
+                    for (int ct = 0; ct < g.t_ctiles; ++ct) cols.push_back(Tile{v, l, rt, ct});
+            }
+        ok = cudaMemcpy(c->d_row_tiles, rows.data(), sizeof(Tile) * rows.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(c->d_col_tiles, cols.data(), sizeof(Tile) * cols.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    }
+    // Algorithm 2, initialisation: one standard-normal vector per pair, layer, column
+    if (ok) {
+        std::vector<Edge> all_pairs;
+        if (c->static_graph) {
+            all_pairs = edges0;
+        } else {
+            for (int a = 0; a < c->topo.n_workers; ++a)
+                for (int b = a + 1; b < c->topo.n_workers; ++b) all_pairs.push_back(Edge{a, b});
+        }
+        std::vector<float> block(static_cast<size_t>(lay.q_stride), 0.0f);
+        for (size_t p = 0; p < all_pairs.size() && ok; ++p) {
+            for (int l = 0; l < n_layers; ++l)
+                for (int k = 0; k < rank; ++k)
+                    pg::init_q_column(seed, all_pairs[p].i, all_pairs[p].j, l, k, lay.layers[l].m,
+                                      block.data() + lay.layers[l].q_off + static_cast<long long>(k) * lay.layers[l].ld);
+            ok = cudaMemcpy(st.Q + static_cast<long long>(p) * lay.q_stride, block.data(),
+                            sizeof(float) * block.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        }
+    }
+    ok = ok && cudaMallocHost(&c->h_tabs, sizeof(int) * static_cast<size_t>(kTabRing) * lay.tab.total_ints) == cudaSuccess;
+    for (int s = 0; s < kTabRing && ok; ++s)
+        ok = cudaEventCreateWithFlags(&c->tab_event[s], cudaEventDisableTiming) == cudaSuccess;
+    if (ok) {
+        ok = pg::launch_column_norms(st, lay.n_pairs, nullptr) == cudaSuccess;
+        c->launches += 1;
+        ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        pg_destroy(c);
+        return PG_ERR_CUDA;
+    }
+    *ctx_out = c;
+    return PG_OK;
+}
+
+void pg_destroy(pg_ctx* c) {
+    if (!c) return;
+    for (int s = 0; s < kTabRing; ++s)
+        if (c->tab_event[s]) cudaEventDestroy(c->tab_event[s]);
+    if (c->h_tabs) cudaFreeHost(c->h_tabs);
+    delete c;
+}
+
+int pg_write_params(pg_ctx* c, int32_t worker, int32_t layer, const float* host_src, void* stream) {
+    int rc = check_worker_layer(c, worker, layer);
+    if (rc != PG_OK || !host_src) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    const LayerGeom& g = c->lay.layers[layer];
+    float* dst = c->st.X + static_cast<long long>(worker) * c->st.x_stride + g.x_off;
+    c->y_valid = false;
+    if (cudaMemcpy2DAsync(dst, sizeof(float) * g.ld, host_src, sizeof(float) * g.m, sizeof(float) * g.m,
+                          g.n, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return PG_ERR_CUDA;
+    return PG_OK;
+}
+
+int pg_read_params(pg_ctx* c, int32_t worker, int32_t layer, float* host_dst, void* stream) {
+    int rc = check_worker_layer(c, worker, layer);
+    if (rc != PG_OK || !host_dst) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    const LayerGeom& g = c->lay.layers[layer];
+    const float* src = c->st.X + static_cast<long long>(worker) * c->st.x_stride + g.x_off;
+    if (cudaMemcpy2DAsync(host_dst, sizeof(float) * g.m, src, sizeof(float) * g.ld, sizeof(float) * g.m,
+                          g.n, cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return PG_ERR_CUDA;
+    return device_status(c, static_cast<cudaStream_t>(stream));
+}
+
+int pg_device_status(pg_ctx* c, void* stream) {
+    if (!c) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    return device_status(c, static_cast<cudaStream_t>(stream));
+}
+
+int pg_round(pg_ctx* c, void* stream_v) {
+    if (!c) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int* tab = nullptr;
+    const int* tab_next = nullptr;
+    int rc = ensure_table(c, c->round, stream, &tab);
+    if (rc == PG_OK) rc = ensure_table(c, c->round + 1, stream, &tab_next);
+    if (rc != PG_OK) return rc;
+    const DevState& st = c->st;
+    const int n_rows = static_cast<int>(c->lay.n_row_tiles), n_cols = static_cast<int>(c->lay.n_col_tiles);
+    bool ok = true;
+    if (!c->y_valid) {
+        ok = ok && pg::launch_forward(st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+        c->launches += 1;
+    }
+    for (int p = 0; p < c->power_steps && ok; ++p) {
+        const int* tab_fwd = (p + 1 < c->power_steps) ? tab : tab_next;
+        ok = ok && pg::launch_edge_left(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+        ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+        ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+        ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+        c->launches += 4;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        c->y_valid = false;
+        return PG_ERR_CUDA;
+    }
+    c->y_valid = true;
+    c->round += 1;
+    return PG_OK;
+}
+
+int pg_max_edges(pg_ctx* c, int32_t* max_edges_out) {
+    if (!c || !max_edges_out) return PG_ERR_INVALID;
+    *max_edges_out = c->lay.max_edges;
+    return PG_OK;
+}
+
+int pg_get_schedule(pg_ctx* c, int64_t round, int32_t* edges_out, float* w_out, int32_t* n_edges_out) {
+    if (!c || !edges_out || !n_edges_out || round < 0) return PG_ERR_INVALID;
+    std::vector<Edge> edges;
+    std::vector<float> w;
+    if (!pg::build_edges(c->topo, c->seed, round, edges)) return PG_ERR_INVALID;
+    if (!pg::edge_weights(c->topo, edges, w)) return PG_ERR_INVALID;
+    for (size_t e = 0; e < edges.size(); ++e) {
+        edges_out[2 * e] = edges[e].i;
+        edges_out[2 * e + 1] = edges[e].j;
+        if (w_out) w_out[e] = w[e];
+    }
+    *n_edges_out = static_cast<int32_t>(edges.size());
+    return PG_OK;
+}
+
+int pg_read_q(pg_ctx* c, int32_t i, int32_t j, int32_t layer, float* host_dst, void* stream_v) {
+    if (!c || !host_dst || layer < 0 || layer >= c->n_layers) return PG_ERR_INVALID;
+    const int64_t pair = c->pairs.of(i, j);
+    if (pair < 0) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const LayerGeom& g = c->lay.layers[layer];
+    const float* src = c->st.Q + pair * c->st.q_stride + g.q_off;
+    if (cudaMemcpy2DAsync(host_dst, sizeof(float) * g.m, src, sizeof(float) * g.ld, sizeof(float) * g.m,
+                          c->rank, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return PG_ERR_CUDA;
+    return cudaStreamSynchronize(stream) == cudaSuccess ? PG_OK : PG_ERR_CUDA;
+}
+
+int pg_write_q(pg_ctx* c, int32_t i, int32_t j, int32_t layer, const float* host_src, void* stream_v) {
+    if (!c || !host_src || layer < 0 || layer >= c->n_layers) return PG_ERR_INVALID;
+    const int64_t pair = c->pairs.of(i, j);
+    if (pair < 0) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const LayerGeom& g = c->lay.layers[layer];
+    float* dst = c->st.Q + pair * c->st.q_stride + g.q_off;
+    c->y_valid = false;
+    if (cudaMemcpy2DAsync(dst, sizeof(float) * g.ld, host_src, sizeof(float) * g.m, sizeof(float) * g.m,
+                          c->rank, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return PG_ERR_CUDA;
+    if (pg::launch_column_norms(c->st, c->lay.n_pairs, stream) != cudaSuccess) return PG_ERR_CUDA;
+    c->launches += 1;
+    return cudaStreamSynchronize(stream) == cudaSuccess ? PG_OK : PG_ERR_CUDA;
+}
+
+int pg_build_schedule(const pg_topology* topo, const float* W_host, uint64_t seed, int64_t round,
+                      int32_t* edges_out, float* w_out, int32_t capacity, int32_t* n_edges_out) {
+    if (!edges_out || !n_edges_out || round < 0) return PG_ERR_INVALID;
+    pg::Topology t;
+    const int rc = make_topology(topo, W_host, t);
+    if (rc != PG_OK) return rc;
+    std::vector<Edge> edges;
+    std::vector<float> w;
+    if (!pg::build_edges(t, seed, round, edges)) return PG_ERR_INVALID;
+    if (!pg::edge_weights(t, edges, w)) return PG_ERR_INVALID;
+    if (static_cast<int64_t>(edges.size()) > capacity) return PG_ERR_INVALID;
+    for (size_t e = 0; e < edges.size(); ++e) {
+        edges_out[2 * e] = edges[e].i;
+        edges_out[2 * e + 1] = edges[e].j;
+        if (w_out) w_out[e] = w[e];
+    }
+    *n_edges_out = static_cast<int32_t>(edges.size());
+    return PG_OK;
+}
+
+int pg_initial_vector(uint64_t seed, int32_t i, int32_t j, int32_t layer, int32_t col, int32_t m,
+                      float* host_dst) {
+    if (!host_dst || i < 0 || j <= i || layer < 0 || col < 0 || col >= 256 || m < 1) return PG_ERR_INVALID;
+    pg::init_q_column(seed, i, j, layer, col, m, host_dst);
+    return PG_OK;
+}
+
+int pg_get_round(pg_ctx* c, int64_t* round_out) {
+    if (!c || !round_out) return PG_ERR_INVALID;
+    *round_out = c->round;
+    return PG_OK;
+}
+
+int pg_set_round(pg_ctx* c, int64_t round) {
+    if (!c || round < 0) return PG_ERR_INVALID;
+    c->round = round;
+    c->y_valid = false;
+    return PG_OK;
+}
+
+int pg_kernel_launches(pg_ctx* c, int64_t* count_out) {
+    if (!c || !count_out) return PG_ERR_INVALID;
+    *count_out = c->launches;
+    return PG_OK;
+}
+
+const char* pg_status_string(int status) {
+    switch (status) {
+        case PG_OK: return "ok";
+        case PG_ERR_INVALID: return "invalid argument, topology or mixing matrix";
+        case PG_ERR_WORKSPACE: return "workspace missing, misaligned, too small or not device memory";
+        case PG_ERR_CUDA: return "a CUDA runtime call failed";
+        case PG_ERR_STATE: return "call not allowed in this state";
+        case PG_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case PG_ERR_NUMERIC: return "a norm was not finite";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,90 @@
+// Device-side data layout of the PowerGossip library and the launchers of its
+// kernels.  Everything lives in the caller's single workspace; offsets are in
+// floats from the start of a section.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace pg {
+
+constexpr int kMaxSlots = 8;   // vectors per worker per sweep: degree * rank
+constexpr int kMaxRank = 4;
+
+// Tiling constants.
+constexpr int kRowTileRows = 64;     // rows of X per CTA in the row-oriented sweeps
+constexpr int kRowTileCols = 2048;   // most columns one CTA reduces over (multiple of 128)
+constexpr int kColTileRows = 256;    // rows of X per CTA in the transposed sweep
+constexpr int kColTileCols = 256;    // columns per CTA in the transposed sweep (64 threads x float4)
+
+// Geometry of one layer (same for every worker).
+struct LayerGeom {
+    int n, m;          // rows, cols of X
+    int ld;            // leading dimension of X in floats: m rounded up to 4
+    int npad;          // n rounded up to 4 (length of n-vectors)
+    int f_rtiles;      // row tiles of the row-oriented sweeps
+    int f_csplit;      // column chunks (partial sums of X q)
+    int f_chunk;       // columns per chunk (multiple of 128)
+    int t_rtiles;      // row tiles of the transposed sweep (partial sums of X^T p)
+    int t_ctiles;      // column tiles of the transposed sweep
+    long long x_off;   // X of this layer inside a worker's parameter block
+    long long q_off;   // Q of this layer inside a pair's block      (rank x ld)
+    long long y_off;   // forward partials inside a worker's block   (slots x f_csplit x npad)
+    long long ph_off;  // P-hat inside an edge's block               (rank x npad)
+    long long z_off;   // transposed partials inside a worker's block (slots x t_rtiles x ld)
+};
+
+// One unit of work of a sweep: a tile of one worker's layer.
+struct Tile {
+    int worker;
+    int layer;
+    int rtile;
+    int ctile;
+};
+
+// Table of one round, in device memory.  Arrays follow the header; their
+// offsets (in ints from the start of the table) are in TabLayout.
+struct TabLayout {
+    int max_edges, n_workers, max_degree;
+    int off_n_edges;     // 1 int
+    int off_edge_i;      // max_edges ints
+    int off_edge_j;      // max_edges ints
+    int off_pair;        // max_edges ints (index into per-pair state; fits int)
+    int off_w;           // max_edges floats
+    int off_slot_i;      // max_edges ints: slot of the edge at its smaller end
+    int off_slot_j;      // max_edges ints: slot at its larger end
+    int off_degree;      // n_workers ints
+    int off_slot_edge;   // n_workers * max_degree ints
+    int off_slot_coef;   // n_workers * max_degree floats: sign * W
+    int total_ints;
+};
+
+// Pointers into the workspace (device) plus sizes; passed to kernels by value.
+struct DevState {
+    float* X;            // [worker][x_stride]
+    float* Q;            // [pair][q_stride]     raw right factors
+    float* Qinv;         // [pair][layer][rank]  1 / column norm (0 for a zero column)
+    float* Y;            // [worker][y_stride]   partial sums of X q
+    float* Ph;           // [edge][ph_stride]    orthonormal left factors of this step
+    float* Z;            // [worker][z_stride]   partial sums of X^T p
+    int* live;           // [edge][layer][rank]  1 if the column took part in this step
+    int* status;         // device status word (bit n set = error code n was raised)
+    const LayerGeom* layers;
+    long long x_stride, q_stride, y_stride, ph_stride, z_stride;
+    int n_layers, rank, n_workers, max_degree;
+    TabLayout tab;
+};
+
+// Launchers (all asynchronous on `stream`; return the cudaError of the launch).
+// `slots` = max_degree * rank of the context.
+cudaError_t launch_forward(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+                           cudaStream_t stream);
+cudaError_t launch_edge_left(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
+cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+                              cudaStream_t stream);
+cudaError_t launch_edge_right(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
+cudaError_t launch_update_forward(const DevState& st, const int* tab_update, const int* tab_forward,
+                                  const Tile* tiles, int n_tiles, cudaStream_t stream);
+cudaError_t launch_column_norms(const DevState& st, long long n_pairs, cudaStream_t stream);
+
+}  // namespace pg

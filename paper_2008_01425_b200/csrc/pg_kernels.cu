@@ -1,0 +1,484 @@
+// CUDA kernels of the PowerGossip power step (sm_100a).
+//
+// One power step of every edge (i<j) and layer (Algorithm 2 of the paper, two
+// consecutive iterations, followed by the gossip update of Eq. 2):
+//   row sweep    Y[w][v]  = X_w Qh_v          for all vectors v of worker w's edges
+//   edge (left)  P = Y[i] - Y[j], orthonormalise -> Ph          (tiny, fp64)
+//   col sweep    Z[w][v]  = X_w^T Ph_v
+//   edge (right) Q' = Z[i] - Z[j]; Q <- Q'; 1/||Q'||            (tiny, fp64)
+//   row sweep    X_w -= sum_v coef_v Ph_v Q'_v^T, and in the same pass the next
+//                step's Y = X_w Qh_next
+// The three sweeps stream X with 16-byte loads; each is bound by HBM bandwidth.
+// Sums over column chunks / row tiles are written as partials and added in a
+// fixed order by the edge kernels, so results are bit-reproducible.
+#include "pg_device.h"
+
+namespace pg {
+namespace {
+
+constexpr int kStatusNumeric = 6;  // PG_ERR_NUMERIC
+
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+    float4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_stream(float* p, const float4& v) {
+    asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y),
+                 "f"(v.z), "f"(v.w)
+                 : "memory");
+}
+
+__device__ __forceinline__ float4 ld_vec(const float* p) {
+    return __ldg(reinterpret_cast<const float4*>(p));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Sum of one double per thread over the whole block, returned to every thread.
+__device__ double block_sum(double v, double* scratch /* >= 33 doubles of shared memory */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nwarps = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();  // scratch may still be read from the previous call
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        double t = lane < nwarps ? scratch[lane] : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0) scratch[32] = t;
+    }
+    __syncthreads();
+    return scratch[32];
+}
+
+// --------------------------------------------------------------------------
+// Row-oriented sweep: optional rank-r update of X, optional forward product.
+// A warp owns RT rows at a time; its lanes walk the columns with float4 loads.
+// --------------------------------------------------------------------------
+template <int S, bool UPDATE, bool FORWARD, int RT>
+__global__ void __launch_bounds__(256)
+row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
+                 const Tile* __restrict__ tiles) {
+    const Tile tile = tiles[blockIdx.x];
+    const LayerGeom g = st.layers[tile.layer];
+    const int w = tile.worker;
+    const int rank = st.rank;
+    float* __restrict__ X = st.X + (long long)w * st.x_stride + g.x_off;
+
+    __shared__ const float* s_uq[S];
+    __shared__ const float* s_up[S];
+    __shared__ float s_uc[S];
+    __shared__ const float* s_fq[S];
+    __shared__ float s_fs[S];
+    __shared__ int s_nu, s_nf;
+
+    if (threadIdx.x < S) {
+        const int v = threadIdx.x;
+        const int slot = v / rank, k = v - slot * rank;
+        if (UPDATE) {
+            const int deg = tab_u[st.tab.off_degree + w];
+            if (slot < deg) {
+                const int e = tab_u[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
+                const int pair = tab_u[st.tab.off_pair + e];
+                s_uq[v] = st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld;
+                s_up[v] = st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad;
+                s_uc[v] = __int_as_float(tab_u[st.tab.off_slot_coef + w * st.tab.max_degree + slot]);
+            }
+            if (v == 0) s_nu = deg * rank;
+        }
+        if (FORWARD) {
+            const int deg = tab_f[st.tab.off_degree + w];
+            if (slot < deg) {
+                const int e = tab_f[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
+                const int pair = tab_f[st.tab.off_pair + e];
+                s_fq[v] = st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld;
+                s_fs[v] = st.Qinv[((long long)pair * st.n_layers + tile.layer) * rank + k];
+            }
+            if (v == 0) s_nf = deg * rank;
+        }
+    }
+    __syncthreads();
+    const int nu = UPDATE ? s_nu : 0;
+    const int nf = FORWARD ? s_nf : 0;
+
+    const int r0 = tile.rtile * kRowTileRows;
+    const int r1 = min(g.n, r0 + kRowTileRows);
+    const int c0 = tile.ctile * g.f_chunk;
+    const int c1 = min(g.ld, c0 + g.f_chunk);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ld = g.ld;
+
+    for (int rb = r0 + warp * RT; rb < r1; rb += 8 * RT) {
+        float a[RT][S];
+        float acc[RT][S];
+        const float* xrow[RT];
+#pragma unroll
+        for (int t = 0; t < RT; ++t) {
+            const int r = min(rb + t, r1 - 1);  // rows past the tile repeat the last one; never stored
+            xrow[t] = X + (long long)r * ld;
+#pragma unroll
+            for (int v = 0; v < S; ++v) {
+                acc[t][v] = 0.0f;
+                a[t][v] = 0.0f;
+                if (UPDATE && v < nu && rb + t < r1) a[t][v] = s_uc[v] * __ldg(s_up[v] + r);
+            }
+        }
+        for (int c = c0 + lane * 4; c < c1; c += 128) {
+            float4 x[RT];
+#pragma unroll
+            for (int t = 0; t < RT; ++t) x[t] = ld_stream(xrow[t] + c);
+            if (UPDATE) {
+#pragma unroll
+                for (int v = 0; v < S; ++v) {
+                    if (v < nu) {
+                        const float4 q = ld_vec(s_uq[v] + c);
+#pragma unroll
+                        for (int t = 0; t < RT; ++t) {
+                            x[t].x = fmaf(-a[t][v], q.x, x[t].x);
+                            x[t].y = fmaf(-a[t][v], q.y, x[t].y);
+                            x[t].z = fmaf(-a[t][v], q.z, x[t].z);
+                            x[t].w = fmaf(-a[t][v], q.w, x[t].w);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < RT; ++t)
+                    if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
+            }
+            if (FORWARD) {
+#pragma unroll
+                for (int v = 0; v < S; ++v) {
+                    if (v < nf) {
+                        const float4 q = ld_vec(s_fq[v] + c);
+#pragma unroll
+                        for (int t = 0; t < RT; ++t) {
+                            acc[t][v] = fmaf(x[t].x, q.x, acc[t][v]);
+                            acc[t][v] = fmaf(x[t].y, q.y, acc[t][v]);
+                            acc[t][v] = fmaf(x[t].z, q.z, acc[t][v]);
+                            acc[t][v] = fmaf(x[t].w, q.w, acc[t][v]);
+                        }
+                    }
+                }
+            }
+        }
+        if (FORWARD) {
+            float* __restrict__ Y = st.Y + (long long)w * st.y_stride + g.y_off;
+#pragma unroll
+            for (int v = 0; v < S; ++v) {
+                if (v < nf) {
+#pragma unroll
+                    for (int t = 0; t < RT; ++t) {
+                        const float s = warp_sum(acc[t][v]);
+                        if (lane == 0 && rb + t < r1)
+                            Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * s_fs[v];
+                    }
+                }
+            }
+        }
+    }
+}
+
+// --------------------------------------------------------------------------
+// Transposed sweep: Z[w][v][c] = sum_r Ph_v[r] X_w[r][c] over one row tile.
+// 64 threads across (a float4 of columns each), 4 row groups down.
+// --------------------------------------------------------------------------
+template <int S>
+__global__ void __launch_bounds__(256)
+col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles) {
+    const Tile tile = tiles[blockIdx.x];
+    const LayerGeom g = st.layers[tile.layer];
+    const int w = tile.worker;
+    const int rank = st.rank;
+    const float* __restrict__ X = st.X + (long long)w * st.x_stride + g.x_off;
+
+    __shared__ float s_p[S][kColTileRows];
+    __shared__ float4 s_red[3][S][64];
+
+    const int r0 = tile.rtile * kColTileRows;
+    const int r1 = min(g.n, r0 + kColTileRows);
+    const int deg = tab[st.tab.off_degree + w];
+    const int nv = deg * rank;
+
+    for (int idx = threadIdx.x; idx < S * kColTileRows; idx += 256) {
+        const int v = idx / kColTileRows, rr = idx - v * kColTileRows;
+        float val = 0.0f;
+        if (v < nv && r0 + rr < r1) {
+            const int slot = v / rank, k = v - slot * rank;
+            const int e = tab[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
+            val = __ldg(st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad + r0 + rr);
+        }
+        s_p[v][rr] = val;
+    }
+    __syncthreads();
+
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+    const int c = tile.ctile * kColTileCols + tx * 4;
+    const int ld = g.ld;
+    float4 acc[S];
+#pragma unroll
+    for (int v = 0; v < S; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    if (c < ld) {
+        const float* xc = X + c;
+        for (int r = r0 + ty; r < r1; r += 16) {
+            float4 x[4];
+            int rr[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                rr[u] = r + 4 * u;                       // rows past r1 read the last row with p = 0
+                x[u] = ld_stream(xc + (long long)min(rr[u], r1 - 1) * ld);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int ro = min(rr[u] - r0, kColTileRows - 1);
+                const bool in = rr[u] < r1;
+#pragma unroll
+                for (int v = 0; v < S; ++v) {
+                    if (v < nv) {
+                        const float p = in ? s_p[v][ro] : 0.0f;
+                        acc[v].x = fmaf(p, x[u].x, acc[v].x);
+                        acc[v].y = fmaf(p, x[u].y, acc[v].y);
+                        acc[v].z = fmaf(p, x[u].z, acc[v].z);
+                        acc[v].w = fmaf(p, x[u].w, acc[v].w);
+                    }
+                }
+            }
+        }
+    }
+    if (ty > 0) {
+#pragma unroll
+        for (int v = 0; v < S; ++v) s_red[ty - 1][v][tx] = acc[v];
+    }
+    __syncthreads();
+    if (ty == 0 && c < ld) {
+        float* __restrict__ Z = st.Z + (long long)w * st.z_stride + g.z_off;
+#pragma unroll
+        for (int v = 0; v < S; ++v) {
+            if (v < nv) {
+                float4 s = acc[v];
+#pragma unroll
+                for (int t = 0; t < 3; ++t) {
+                    const float4 o = s_red[t][v][tx];
+                    s.x += o.x; s.y += o.y; s.z += o.z; s.w += o.w;
+                }
+                *reinterpret_cast<float4*>(Z + ((long long)v * g.t_rtiles + tile.rtile) * ld + c) = s;
+            }
+        }
+    }
+}
+
+// --------------------------------------------------------------------------
+// Edge step, left factor: P = Y[i] - Y[j] (partials added in order, fp64),
+// modified Gram-Schmidt in column order, P-hat stored as fp32.
+// One CTA per (edge, layer).
+// --------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+edge_left_kernel(DevState st, const int* __restrict__ tab) {
+    int* __restrict__ live_out = st.live;
+    __shared__ double scratch[33];
+    const int L = st.n_layers, rank = st.rank;
+    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[l];
+    const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
+    const int pair = tab[st.tab.off_pair + e];
+    const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
+    const float* Yi = st.Y + (long long)wi * st.y_stride + g.y_off;
+    const float* Yj = st.Y + (long long)wj * st.y_stride + g.y_off;
+    float* Ph = st.Ph + (long long)e * st.ph_stride + g.ph_off;
+    double coef[kMaxRank];
+
+    for (int k = 0; k < rank; ++k) {
+        const float* yi = Yi + (long long)(si * rank + k) * g.f_csplit * g.npad;
+        const float* yj = Yj + (long long)(sj * rank + k) * g.f_csplit * g.npad;
+        // the difference of the two endpoints' products, one row at a time
+        auto raw = [&](int r) {
+            double a = 0.0, b = 0.0;
+            for (int cs = 0; cs < g.f_csplit; ++cs) {
+                a += (double)yi[(long long)cs * g.npad + r];
+                b += (double)yj[(long long)cs * g.npad + r];
+            }
+            return a - b;
+        };
+        double part = 0.0;
+        for (int r = threadIdx.x; r < g.n; r += blockDim.x) {
+            const double v = raw(r);
+            part += v * v;
+        }
+        const double pre = block_sum(part, scratch);
+        // project out the earlier columns one after the other (modified Gram-Schmidt)
+        for (int h = 0; h < k; ++h) {
+            part = 0.0;
+            for (int r = threadIdx.x; r < g.n; r += blockDim.x) {
+                double v = raw(r);
+                for (int h2 = 0; h2 < h; ++h2) v -= coef[h2] * (double)Ph[(long long)h2 * g.npad + r];
+                part += v * (double)Ph[(long long)h * g.npad + r];
+            }
+            coef[h] = block_sum(part, scratch);
+        }
+        double nn = pre;
+        if (k > 0) {
+            part = 0.0;
+            for (int r = threadIdx.x; r < g.n; r += blockDim.x) {
+                double v = raw(r);
+                for (int h = 0; h < k; ++h) v -= coef[h] * (double)Ph[(long long)h * g.npad + r];
+                part += v * v;
+            }
+            nn = block_sum(part, scratch);
+        }
+        const bool finite = isfinite(nn);
+        // a residual below 1e-5 of the column's length is rounding noise of the fp32 inputs
+        const bool live = finite && nn > 0.0 && (k == 0 || nn > 1e-10 * pre);
+        const double inv = live ? 1.0 / sqrt(nn) : 0.0;
+        for (int r = threadIdx.x; r < g.npad; r += blockDim.x) {
+            double v = 0.0;
+            if (live && r < g.n) {
+                v = raw(r);
+                for (int h = 0; h < k; ++h) v -= coef[h] * (double)Ph[(long long)h * g.npad + r];
+                v *= inv;
+            }
+            Ph[(long long)k * g.npad + r] = (float)v;
+        }
+        if (threadIdx.x == 0) {
+            live_out[((long long)e * L + l) * rank + k] = live ? 1 : 0;
+            if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
+        }
+        __syncthreads();  // the stored column is read by the next column's projections
+    }
+    (void)pair;
+}
+
+// --------------------------------------------------------------------------
+// Edge step, right factor: Q' = Z[i] - Z[j] (row-tile partials added in order,
+// fp64), stored as the pair's new Q with 1/||Q'||.  Degenerate columns keep
+// their old vector.  One CTA per (edge, layer).
+// --------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+edge_right_kernel(DevState st, const int* __restrict__ tab) {
+    const int* __restrict__ live_in = st.live;
+    __shared__ double scratch[33];
+    const int L = st.n_layers, rank = st.rank;
+    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[l];
+    const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
+    const int pair = tab[st.tab.off_pair + e];
+    const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
+    const float* Zi = st.Z + (long long)wi * st.z_stride + g.z_off;
+    const float* Zj = st.Z + (long long)wj * st.z_stride + g.z_off;
+    float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
+
+    for (int k = 0; k < rank; ++k) {
+        if (!live_in[((long long)e * L + l) * rank + k]) continue;  // uniform over the block
+        const float* zi = Zi + (long long)(si * rank + k) * g.t_rtiles * g.ld;
+        const float* zj = Zj + (long long)(sj * rank + k) * g.t_rtiles * g.ld;
+        double part = 0.0;
+        for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
+            double a = 0.0, b = 0.0;
+            for (int rt = 0; rt < g.t_rtiles; ++rt) {
+                a += (double)zi[(long long)rt * g.ld + c];
+                b += (double)zj[(long long)rt * g.ld + c];
+            }
+            const float q = (float)(a - b);
+            Q[(long long)k * g.ld + c] = q;
+            part += (double)q * (double)q;
+        }
+        const double nn = block_sum(part, scratch);
+        if (threadIdx.x == 0) {
+            st.Qinv[((long long)pair * L + l) * rank + k] = nn > 0.0 ? (float)(1.0 / sqrt(nn)) : 0.0f;
+            if (!isfinite(nn)) atomicOr(st.status, 1 << kStatusNumeric);
+        }
+    }
+}
+
+// 1 / ||column|| of every stored right factor (after initialisation or an
+// external write).  One CTA per (pair, layer).
+__global__ void __launch_bounds__(256)
+column_norms_kernel(DevState st) {
+    __shared__ double scratch[33];
+    const int L = st.n_layers, rank = st.rank;
+    const long long pair = blockIdx.x / L;
+    const int l = blockIdx.x - (int)pair * L;
+    const LayerGeom g = st.layers[l];
+    const float* Q = st.Q + pair * st.q_stride + g.q_off;
+    for (int k = 0; k < rank; ++k) {
+        double part = 0.0;
+        for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
+            const double q = (double)Q[(long long)k * g.ld + c];
+            part += q * q;
+        }
+        const double nn = block_sum(part, scratch);
+        if (threadIdx.x == 0)
+            st.Qinv[(pair * L + l) * rank + k] = nn > 0.0 ? (float)(1.0 / sqrt(nn)) : 0.0f;
+    }
+}
+
+template <bool UPDATE, bool FORWARD>
+cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, const Tile* tiles,
+                       int n_tiles, cudaStream_t stream) {
+    if (n_tiles <= 0) return cudaSuccess;
+    const int slots = st.max_degree * st.rank;
+    if (slots <= 1)
+        row_sweep_kernel<1, UPDATE, FORWARD, 4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+    else if (slots <= 2)
+        row_sweep_kernel<2, UPDATE, FORWARD, 4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+    else if (slots <= 4)
+        row_sweep_kernel<4, UPDATE, FORWARD, 4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+    else
+        row_sweep_kernel<8, UPDATE, FORWARD, 2><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_forward(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+                           cudaStream_t stream) {
+    return launch_row<false, true>(st, tab, tab, tiles, n_tiles, stream);
+}
+
+cudaError_t launch_update_forward(const DevState& st, const int* tab_update, const int* tab_forward,
+                                  const Tile* tiles, int n_tiles, cudaStream_t stream) {
+    return launch_row<true, true>(st, tab_update, tab_forward, tiles, n_tiles, stream);
+}
+
+cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+                              cudaStream_t stream) {
+    if (n_tiles <= 0) return cudaSuccess;
+    const int slots = st.max_degree * st.rank;
+    if (slots <= 1)
+        col_sweep_kernel<1><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+    else if (slots <= 2)
+        col_sweep_kernel<2><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+    else if (slots <= 4)
+        col_sweep_kernel<4><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+    else
+        col_sweep_kernel<8><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_edge_left(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
+    edge_left_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_edge_right(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
+    edge_right_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_column_norms(const DevState& st, long long n_pairs, cudaStream_t stream) {
+    column_norms_kernel<<<(unsigned)(n_pairs * st.n_layers), 256, 0, stream>>>(st);
+    return cudaGetLastError();
+}
+
+}  // namespace pg
