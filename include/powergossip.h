@@ -205,6 +205,25 @@ PG_API int pg_build_schedule(const pg_topology *topo, const float *W_host, uint6
 PG_API int pg_initial_vector(uint64_t seed, int32_t i, int32_t j, int32_t layer, int32_t col, int32_t m,
                              float *host_dst);
 
+/*
+ * Per-kernel device timing (measurement aid; the paper has no counterpart).
+ * While enabled, pg_round brackets every kernel it launches with a pair of CUDA
+ * events on the caller's stream.  pg_timing_read waits for the recorded events,
+ * adds up the elapsed milliseconds and the launch counts per kernel kind into
+ * ms_out / launches_out (host, PG_KERNEL_KINDS entries each, indexed by the
+ * PG_KERNEL_* constants) and forgets them.
+ */
+enum {
+    PG_KERNEL_FORWARD = 0,         /* X q for all incident edges (first round only)     */
+    PG_KERNEL_EDGE_LEFT = 1,       /* difference of the two ends, orthonormalisation    */
+    PG_KERNEL_TRANSPOSED = 2,      /* X^T p-hat                                          */
+    PG_KERNEL_EDGE_RIGHT = 3,      /* difference of the two ends, new stored vector      */
+    PG_KERNEL_UPDATE_FORWARD = 4,  /* rank-r update of X fused with the next X q         */
+    PG_KERNEL_KINDS = 5
+};
+PG_API int pg_timing_enable(pg_ctx *ctx, int32_t on);
+PG_API int pg_timing_read(pg_ctx *ctx, double *ms_out, int64_t *launches_out);
+
 /* Number of kernels this context has launched so far. */
 PG_API int pg_kernel_launches(pg_ctx *ctx, int64_t *count_out);
 

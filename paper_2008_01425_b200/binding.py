@@ -24,8 +24,9 @@ EXPORTS = (
     "pg_workspace_bytes", "pg_create", "pg_destroy", "pg_write_params", "pg_read_params",
     "pg_round", "pg_device_status", "pg_get_schedule", "pg_max_edges", "pg_read_q", "pg_write_q",
     "pg_get_round", "pg_set_round", "pg_kernel_launches", "pg_status_string",
-    "pg_build_schedule", "pg_initial_vector",
+    "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
 )
+KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward")
 
 
 class pg_topology(ctypes.Structure):
@@ -77,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     L.pg_kernel_launches.argtypes = [vp, ctypes.POINTER(i64)]
     L.pg_build_schedule.argtypes = [ctypes.POINTER(pg_topology), vp, u64, i64, vp, vp, i32, ctypes.POINTER(i32)]
     L.pg_initial_vector.argtypes = [u64, i32, i32, i32, i32, i32, vp]
+    L.pg_timing_enable.argtypes = [vp, i32]
+    L.pg_timing_read.argtypes = [vp, vp, vp]
     L.pg_status_string.argtypes = [ctypes.c_int]
     L.pg_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -263,6 +266,16 @@ class PowerGossip:
         r = ctypes.c_int64(0)
         _check(self._lib.pg_kernel_launches(self._h, ctypes.byref(r)), "pg_kernel_launches")
         return int(r.value)
+
+    def pg_timing_enable(self, on: bool) -> None:
+        _check(self._lib.pg_timing_enable(self._h, 1 if on else 0), "pg_timing_enable")
+
+    def pg_timing_read(self):
+        """{kernel kind: (total ms, launches)} since the last read."""
+        ms = np.zeros(len(KERNEL_KINDS), dtype=np.float64)
+        cnt = np.zeros(len(KERNEL_KINDS), dtype=np.int64)
+        _check(self._lib.pg_timing_read(self._h, ms.ctypes.data, cnt.ctypes.data), "pg_timing_read")
+        return {k: (float(ms[t]), int(cnt[t])) for t, k in enumerate(KERNEL_KINDS)}
 
     # -- conveniences built only from the calls above ---------------------
     def write_all(self, params: Sequence[Sequence[np.ndarray]], stream=None) -> None:

@@ -177,6 +177,10 @@ struct pg_ctx {
     Tile* d_col_tiles = nullptr;
     bool static_graph = true;
     int device = 0;
+    // optional per-kernel timing: one event pair per launch while enabled
+    bool timing = false;
+    struct Span { int kind; cudaEvent_t a, b; };
+    std::vector<Span> spans;
 };
 
 namespace {
@@ -238,6 +242,23 @@ int ensure_table(pg_ctx* c, int64_t round, cudaStream_t stream, const int** out)
     *out = dev;
     return PG_OK;
 }
+
+// Brackets one kernel launch with events when timing is on.
+struct Timed {
+    pg_ctx* c;
+    cudaStream_t s;
+    pg_ctx::Span span{};
+    bool on;
+    Timed(pg_ctx* ctx, int kind, cudaStream_t stream) : c(ctx), s(stream), on(ctx->timing) {
+        if (!on) return;
+        span.kind = kind;
+        on = cudaEventCreate(&span.a) == cudaSuccess && cudaEventCreate(&span.b) == cudaSuccess &&
+             cudaEventRecord(span.a, s) == cudaSuccess;
+    }
+    ~Timed() {
+        if (on && cudaEventRecord(span.b, s) == cudaSuccess) c->spans.push_back(span);
+    }
+};
 
 // Kernels and copies go to the device that owns the workspace.
 bool bind_device(const pg_ctx* c) {
@@ -411,6 +432,10 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
 
 void pg_destroy(pg_ctx* c) {
     if (!c) return;
+    for (auto& sp : c->spans) {
+        cudaEventDestroy(sp.a);
+        cudaEventDestroy(sp.b);
+    }
     for (int s = 0; s < kTabRing; ++s)
         if (c->tab_event[s]) cudaEventDestroy(c->tab_event[s]);
     if (c->h_tabs) cudaFreeHost(c->h_tabs);
@@ -461,15 +486,28 @@ int pg_round(pg_ctx* c, void* stream_v) {
     const int n_rows = static_cast<int>(c->lay.n_row_tiles), n_cols = static_cast<int>(c->lay.n_col_tiles);
     bool ok = true;
     if (!c->y_valid) {
+        Timed t(c, PG_KERNEL_FORWARD, stream);
         ok = ok && pg::launch_forward(st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
         c->launches += 1;
     }
     for (int p = 0; p < c->power_steps && ok; ++p) {
         const int* tab_fwd = (p + 1 < c->power_steps) ? tab : tab_next;
-        ok = ok && pg::launch_edge_left(st, tab, c->lay.max_edges, stream) == cudaSuccess;
-        ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
-        ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
-        ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+        {
+            Timed t(c, PG_KERNEL_EDGE_LEFT, stream);
+            ok = ok && pg::launch_edge_left(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+        }
+        {
+            Timed t(c, PG_KERNEL_TRANSPOSED, stream);
+            ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+        }
+        {
+            Timed t(c, PG_KERNEL_EDGE_RIGHT, stream);
+            ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+        }
+        {
+            Timed t(c, PG_KERNEL_UPDATE_FORWARD, stream);
+            ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+        }
         c->launches += 4;
     }
     if (!ok) {
@@ -572,6 +610,35 @@ int pg_set_round(pg_ctx* c, int64_t round) {
     c->round = round;
     c->y_valid = false;
     return PG_OK;
+}
+
+int pg_timing_enable(pg_ctx* c, int32_t on) {
+    if (!c) return PG_ERR_INVALID;
+    c->timing = on != 0;
+    return PG_OK;
+}
+
+int pg_timing_read(pg_ctx* c, double* ms_out, int64_t* launches_out) {
+    if (!c || !ms_out || !launches_out) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    for (int k = 0; k < PG_KERNEL_KINDS; ++k) {
+        ms_out[k] = 0.0;
+        launches_out[k] = 0;
+    }
+    bool ok = true;
+    for (auto& sp : c->spans) {
+        float ms = 0.0f;
+        ok = ok && cudaEventSynchronize(sp.b) == cudaSuccess && cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess;
+        if (ok) {
+            ms_out[sp.kind] += ms;
+            launches_out[sp.kind] += 1;
+        }
+        cudaEventDestroy(sp.a);
+        cudaEventDestroy(sp.b);
+    }
+    c->spans.clear();
+    if (!ok) cudaGetLastError();
+    return ok ? PG_OK : PG_ERR_CUDA;
 }
 
 int pg_kernel_launches(pg_ctx* c, int64_t* count_out) {
