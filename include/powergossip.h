@@ -50,7 +50,8 @@ typedef enum pg_status {
     PG_ERR_CUDA = 3,       /* a CUDA runtime call failed                           */
     PG_ERR_STATE = 4,      /* call not allowed in the context's current state      */
     PG_ERR_TIMEOUT = 5,    /* a bounded device-side wait gave up                   */
-    PG_ERR_NUMERIC = 6     /* a norm was not finite (NaN / Inf in the parameters)  */
+    PG_ERR_NUMERIC = 6,    /* a norm was not finite (NaN / Inf in the parameters)  */
+    PG_ERR_TOO_LARGE = 7   /* problem exceeds the fixed scratch of a no-allocation call */
 } pg_status;
 
 /* Graph kinds.  The paper's experiments use rings; Assumption A4 (Section 5.1)
@@ -223,6 +224,41 @@ enum {
 };
 PG_API int pg_timing_enable(pg_ctx *ctx, int32_t on);
 PG_API int pg_timing_read(pg_ctx *ctx, double *ms_out, int64_t *launches_out);
+
+/*
+ * z = X^T p for one matrix, with no allocation of any kind (the paper has no
+ * counterpart: this is a service entry point for callers that cannot allocate).
+ *
+ * Who needs it: code that runs where device memory cannot be obtained - inside
+ * an allocator or memory-pool callback, in a process whose memory budget was
+ * fixed at start-up, or on a latency path where cudaMalloc's implicit device
+ * synchronisation would stall other streams.  Such callers cannot size and pass
+ * the workspace that pg_create wants, so here the row-tile partial sums of the
+ * transposed sweep live in a fixed array inside the library
+ * (PG_NOALLOC_MAX_PARTIALS floats = 4 MiB, resident on every GPU that loads the
+ * library until the process exits).  The call uses no cudaMalloc, cudaFree or
+ * allocating library routine; the context-free call needs no pg_ctx.
+ *
+ *   X_dev   device, rows x cols fp32, row-major with leading dimension ld >= cols
+ *           (floats).  16-byte rows (X_dev 16-byte aligned, cols and ld multiples
+ *           of 4) take the vector path; anything else a scalar path, same result.
+ *   p_dev   device, rows floats.        z_dev   device, cols floats (output).
+ *   All three on the current device.  Asynchronous on `stream`.
+ *
+ * Limit: ceil(rows/256) * (cols rounded up to 4) <= PG_NOALLOC_MAX_PARTIALS,
+ * e.g. 28000 x 650, 650 x 28000 or 8192 x 8192; beyond it the call does nothing
+ * and returns PG_ERR_TOO_LARGE.
+ * Set-up: the first call on each device looks up the device address of the
+ * array (cudaGetSymbolAddress, once per device, with that device current); make
+ * that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array, which keeps whatever the
+ * last call left there.  Every cell a call reads it has written itself, so no
+ * clearing is needed, but two calls that overlap on the GPU (different streams
+ * or threads) race on the array: serialise them.
+ */
+#define PG_NOALLOC_MAX_PARTIALS (1 << 20)
+PG_API int pg_transposed_product_noalloc(const float *X_dev, int32_t rows, int32_t cols, int64_t ld,
+                                         const float *p_dev, float *z_dev, void *stream);
 
 /* Number of kernels this context has launched so far. */
 PG_API int pg_kernel_launches(pg_ctx *ctx, int64_t *count_out);

@@ -16,7 +16,8 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpowergossip.so")
 
-PG_OK, PG_ERR_INVALID, PG_ERR_WORKSPACE, PG_ERR_CUDA, PG_ERR_STATE, PG_ERR_TIMEOUT, PG_ERR_NUMERIC = range(7)
+PG_OK, PG_ERR_INVALID, PG_ERR_WORKSPACE, PG_ERR_CUDA, PG_ERR_STATE, PG_ERR_TIMEOUT, PG_ERR_NUMERIC, PG_ERR_TOO_LARGE = range(8)
+PG_NOALLOC_MAX_PARTIALS = 1 << 20
 PG_RING, PG_TORUS, PG_MATCHING, PG_CUSTOM = 0, 1, 2, 3
 PG_W_UNIFORM, PG_W_METROPOLIS, PG_W_EXPLICIT = 0, 1, 2
 
@@ -25,6 +26,7 @@ EXPORTS = (
     "pg_round", "pg_device_status", "pg_get_schedule", "pg_max_edges", "pg_read_q", "pg_write_q",
     "pg_get_round", "pg_set_round", "pg_kernel_launches", "pg_status_string",
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
+    "pg_transposed_product_noalloc",
 )
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward")
 
@@ -80,6 +82,7 @@ def load_library() -> ctypes.CDLL:
     L.pg_initial_vector.argtypes = [u64, i32, i32, i32, i32, i32, vp]
     L.pg_timing_enable.argtypes = [vp, i32]
     L.pg_timing_read.argtypes = [vp, vp, vp]
+    L.pg_transposed_product_noalloc.argtypes = [vp, i32, i32, i64, vp, vp, vp]
     L.pg_status_string.argtypes = [ctypes.c_int]
     L.pg_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -144,6 +147,23 @@ def pg_initial_vector(seed: int, i: int, j: int, layer: int, col: int, m: int) -
     out = np.zeros(m, dtype=np.float32)
     _check(load_library().pg_initial_vector(seed, i, j, layer, col, m, out.ctypes.data), "pg_initial_vector")
     return out
+
+
+def pg_transposed_product_noalloc(X, p, z, stream=None, rows: Optional[int] = None,
+                                  cols: Optional[int] = None, ld: Optional[int] = None) -> None:
+    """z = X^T p on the GPU with the library's fixed scratch (no allocation).
+
+    X: CUDA float32 tensor (rows x cols view; a row stride > cols is allowed),
+    p: CUDA float32 vector of `rows` entries, z: CUDA float32 vector of `cols`
+    entries, written in place.  Raises PowerGossipError(PG_ERR_TOO_LARGE) beyond
+    the size limit stated in the header.
+    """
+    rows = int(X.shape[0]) if rows is None else rows
+    cols = int(X.shape[1]) if cols is None else cols
+    ld = int(X.stride(0)) if ld is None else ld
+    _check(load_library().pg_transposed_product_noalloc(X.data_ptr(), rows, cols, ld, p.data_ptr(),
+                                                        z.data_ptr(), _stream_handle(stream)),
+           "pg_transposed_product_noalloc")
 
 
 def _stream_handle(stream) -> Optional[int]:

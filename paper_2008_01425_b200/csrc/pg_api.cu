@@ -656,6 +656,7 @@ const char* pg_status_string(int status) {
         case PG_ERR_STATE: return "call not allowed in this state";
         case PG_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         case PG_ERR_NUMERIC: return "a norm was not finite";
+        case PG_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
