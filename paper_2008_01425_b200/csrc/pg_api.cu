@@ -80,6 +80,12 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     if (lay.n_pairs > INT_MAX / 2) return PG_ERR_INVALID;
 
     lay.layers.resize(n_layers);
+    // aim for about 4096 tiles per sweep, each between 64 KB and 512 KB of X
+    long long total_elems = 0;
+    for (int l = 0; l < n_layers; ++l)
+        if (shapes[l].rows > 0 && shapes[l].cols > 0)
+            total_elems += static_cast<long long>(N) * shapes[l].rows * round_up(shapes[l].cols, 4);
+    const long long tile_elems = std::min<long long>(std::max<long long>(total_elems / 4096, 16 * 1024), 128 * 1024);
     long long x = 0, q = 0, y = 0, ph = 0, z = 0;
     lay.n_row_tiles = lay.n_col_tiles = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -90,11 +96,16 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         g.m = shapes[l].cols;
         g.ld = static_cast<int>(round_up(g.m, 4));
         g.npad = static_cast<int>(round_up(g.n, 4));
-        g.f_rtiles = (g.n + pg::kRowTileRows - 1) / pg::kRowTileRows;
-        g.f_csplit = (g.ld + pg::kRowTileCols - 1) / pg::kRowTileCols;
+        // row sweeps: 32 or 64 rows by up to 2048 columns
+        g.f_rows = tile_elems >= 64 * 1024 ? pg::kRowTileRowsMax : 32;
+        const long long want_cols = std::min<long long>(std::max<long long>(tile_elems / g.f_rows, 128), pg::kRowTileColsMax);
+        g.f_rtiles = (g.n + g.f_rows - 1) / g.f_rows;
+        g.f_csplit = static_cast<int>((g.ld + want_cols - 1) / want_cols);
         g.f_chunk = static_cast<int>(round_up((g.ld + g.f_csplit - 1) / g.f_csplit, 128));
         g.f_csplit = (g.ld + g.f_chunk - 1) / g.f_chunk;
-        g.t_rtiles = (g.n + pg::kColTileRows - 1) / pg::kColTileRows;
+        // transposed sweep: 64, 128 or 256 rows by 256 columns
+        g.t_rows = tile_elems >= 64 * 1024 ? pg::kColTileRowsMax : (tile_elems >= 32 * 1024 ? 128 : 64);
+        g.t_rtiles = (g.n + g.t_rows - 1) / g.t_rows;
         g.t_ctiles = (g.ld + pg::kColTileCols - 1) / pg::kColTileCols;
         g.x_off = x;
         g.q_off = q;

@@ -11,17 +11,21 @@ namespace pg {
 constexpr int kMaxSlots = 8;   // vectors per worker per sweep: degree * rank
 constexpr int kMaxRank = 4;
 
-// Tiling constants.
-constexpr int kRowTileRows = 64;     // rows of X per CTA in the row-oriented sweeps
-constexpr int kRowTileCols = 2048;   // most columns one CTA reduces over (multiple of 128)
-constexpr int kColTileRows = 256;    // rows of X per CTA in the transposed sweep
-constexpr int kColTileCols = 256;    // columns per CTA in the transposed sweep (64 threads x float4)
+// Tiling limits.  The host picks the tile of every layer inside these limits so
+// that each sweep has a few thousand CTAs (several waves on 148 SMs) whatever
+// the size of the stack.
+constexpr int kRowTileRowsMax = 64;    // rows of X per CTA in the row-oriented sweeps (32 or 64)
+constexpr int kRowTileColsMax = 2048;  // most columns one CTA reduces over (multiple of 128)
+constexpr int kColTileRowsMax = 256;   // rows of X per CTA in the transposed sweep (64, 128 or 256)
+constexpr int kColTileCols = 256;      // columns per CTA in the transposed sweep (64 threads x float4)
 
 // Geometry of one layer (same for every worker).
 struct LayerGeom {
     int n, m;          // rows, cols of X
     int ld;            // leading dimension of X in floats: m rounded up to 4
     int npad;          // n rounded up to 4 (length of n-vectors)
+    int f_rows;        // rows per tile of the row-oriented sweeps
+    int t_rows;        // rows per tile of the transposed sweep
     int f_rtiles;      // row tiles of the row-oriented sweeps
     int f_csplit;      // column chunks (partial sums of X q)
     int f_chunk;       // columns per chunk (multiple of 128)

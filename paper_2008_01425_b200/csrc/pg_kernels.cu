@@ -18,6 +18,24 @@ namespace {
 
 constexpr int kStatusNumeric = 6;  // PG_ERR_NUMERIC
 
+// Rows a warp of the row sweep works on at once, per number of vectors S.
+#ifndef PG_RT1
+#define PG_RT1 4
+#endif
+#ifndef PG_RT2
+#define PG_RT2 4
+#endif
+#ifndef PG_RT4
+#define PG_RT4 2
+#endif
+#ifndef PG_RT8
+#define PG_RT8 2
+#endif
+// Resident CTAs per SM the row sweep is compiled for (caps its registers).
+#ifndef PG_ROW_MIN_BLOCKS
+#define PG_ROW_MIN_BLOCKS 4
+#endif
+
 __device__ __forceinline__ float4 ld_stream(const float* p) {
     float4 v;
     asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
@@ -65,8 +83,10 @@ __device__ double block_sum(double v, double* scratch /* >= 33 doubles of shared
 // Row-oriented sweep: optional rank-r update of X, optional forward product.
 // A warp owns RT rows at a time; its lanes walk the columns with float4 loads.
 // --------------------------------------------------------------------------
-template <int S, bool UPDATE, bool FORWARD, int RT>
-__global__ void __launch_bounds__(256)
+// SAME: update and forward use the same vectors (Q' of this step is the next
+// step's q, as on a static graph), so each is loaded once.
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT>
+__global__ void __launch_bounds__(256, PG_ROW_MIN_BLOCKS)
 row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
                  const Tile* __restrict__ tiles) {
     const Tile tile = tiles[blockIdx.x];
@@ -111,8 +131,8 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
     const int nu = UPDATE ? s_nu : 0;
     const int nf = FORWARD ? s_nf : 0;
 
-    const int r0 = tile.rtile * kRowTileRows;
-    const int r1 = min(g.n, r0 + kRowTileRows);
+    const int r0 = tile.rtile * g.f_rows;
+    const int r1 = min(g.n, r0 + g.f_rows);
     const int c0 = tile.ctile * g.f_chunk;
     const int c1 = min(g.ld, c0 + g.f_chunk);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -137,7 +157,38 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
             float4 x[RT];
 #pragma unroll
             for (int t = 0; t < RT; ++t) x[t] = ld_stream(xrow[t] + c);
-            if (UPDATE) {
+            if (UPDATE && SAME) {
+                // slot order: first every correction, then every product, as in the general case
+                float4 q[S];
+#pragma unroll
+                for (int v = 0; v < S; ++v) {
+                    if (v < nu) {
+                        q[v] = ld_vec(s_uq[v] + c);
+#pragma unroll
+                        for (int t = 0; t < RT; ++t) {
+                            x[t].x = fmaf(-a[t][v], q[v].x, x[t].x);
+                            x[t].y = fmaf(-a[t][v], q[v].y, x[t].y);
+                            x[t].z = fmaf(-a[t][v], q[v].z, x[t].z);
+                            x[t].w = fmaf(-a[t][v], q[v].w, x[t].w);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < RT; ++t)
+                    if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
+#pragma unroll
+                for (int v = 0; v < S; ++v) {
+                    if (v < nu) {
+#pragma unroll
+                        for (int t = 0; t < RT; ++t) {
+                            acc[t][v] = fmaf(x[t].x, q[v].x, acc[t][v]);
+                            acc[t][v] = fmaf(x[t].y, q[v].y, acc[t][v]);
+                            acc[t][v] = fmaf(x[t].z, q[v].z, acc[t][v]);
+                            acc[t][v] = fmaf(x[t].w, q[v].w, acc[t][v]);
+                        }
+                    }
+                }
+            } else if (UPDATE) {
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nu) {
@@ -155,7 +206,7 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
                 for (int t = 0; t < RT; ++t)
                     if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
             }
-            if (FORWARD) {
+            if (FORWARD && !(UPDATE && SAME)) {
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nf) {
@@ -201,16 +252,16 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
     const int rank = st.rank;
     const float* __restrict__ X = st.X + (long long)w * st.x_stride + g.x_off;
 
-    __shared__ float s_p[S][kColTileRows];
+    __shared__ float s_p[S][kColTileRowsMax];
     __shared__ float4 s_red[3][S][64];
 
-    const int r0 = tile.rtile * kColTileRows;
-    const int r1 = min(g.n, r0 + kColTileRows);
+    const int r0 = tile.rtile * g.t_rows;
+    const int r1 = min(g.n, r0 + g.t_rows);
     const int deg = tab[st.tab.off_degree + w];
     const int nv = deg * rank;
 
-    for (int idx = threadIdx.x; idx < S * kColTileRows; idx += 256) {
-        const int v = idx / kColTileRows, rr = idx - v * kColTileRows;
+    for (int idx = threadIdx.x; idx < S * kColTileRowsMax; idx += 256) {
+        const int v = idx / kColTileRowsMax, rr = idx - v * kColTileRowsMax;
         float val = 0.0f;
         if (v < nv && r0 + rr < r1) {
             const int slot = v / rank, k = v - slot * rank;
@@ -240,7 +291,7 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int ro = min(rr[u] - r0, kColTileRows - 1);
+                const int ro = min(rr[u] - r0, kColTileRowsMax - 1);
                 const bool in = rr[u] < r1;
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
@@ -423,19 +474,19 @@ column_norms_kernel(DevState st) {
     }
 }
 
-template <bool UPDATE, bool FORWARD>
+template <bool UPDATE, bool FORWARD, bool SAME>
 cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, const Tile* tiles,
                        int n_tiles, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
     const int slots = st.max_degree * st.rank;
     if (slots <= 1)
-        row_sweep_kernel<1, UPDATE, FORWARD, 4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
     else if (slots <= 2)
-        row_sweep_kernel<2, UPDATE, FORWARD, 4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
     else if (slots <= 4)
-        row_sweep_kernel<4, UPDATE, FORWARD, 4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
     else
-        row_sweep_kernel<8, UPDATE, FORWARD, 2><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
     return cudaGetLastError();
 }
 
@@ -443,12 +494,15 @@ cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, c
 
 cudaError_t launch_forward(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
                            cudaStream_t stream) {
-    return launch_row<false, true>(st, tab, tab, tiles, n_tiles, stream);
+    return launch_row<false, true, false>(st, tab, tab, tiles, n_tiles, stream);
 }
 
 cudaError_t launch_update_forward(const DevState& st, const int* tab_update, const int* tab_forward,
                                   const Tile* tiles, int n_tiles, cudaStream_t stream) {
-    return launch_row<true, true>(st, tab_update, tab_forward, tiles, n_tiles, stream);
+    // the same table means the same edges, pairs and vectors for both halves
+    if (tab_update == tab_forward)
+        return launch_row<true, true, true>(st, tab_update, tab_forward, tiles, n_tiles, stream);
+    return launch_row<true, true, false>(st, tab_update, tab_forward, tiles, n_tiles, stream);
 }
 
 cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
