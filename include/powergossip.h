@@ -153,7 +153,10 @@ PG_API int pg_read_params(pg_ctx *ctx, int32_t worker, int32_t layer, float *hos
  *     Q' = X_i^T Ph - X_j^T Ph                        (Eq. 3, even iteration)
  *     X_i -= W_ij Ph Q'^T,  X_j += W_ij Ph Q'^T,  Q = Q'   (Eq. 2; Lemma 1)
  * with all edges of a step reading the same pre-update X.  Advances the round
- * counter.  Host-side errors are returned at once; device-side ones show up in
+ * counter.  On graphs of degree <= 1 at rank 1 (a matching) the correction of a
+ * step is applied to the copy of X in memory by the next step's sweep, or by
+ * pg_read_params / pg_write_params / pg_write_q / pg_set_round, whichever comes
+ * first; every call of this API sees the fully updated X.  Host-side errors are returned at once; device-side ones show up in
  * pg_read_params / pg_device_status.
  */
 PG_API int pg_round(pg_ctx *ctx, void *stream);
@@ -210,9 +213,12 @@ PG_API int pg_initial_vector(uint64_t seed, int32_t i, int32_t j, int32_t layer,
  * Per-kernel device timing (measurement aid; the paper has no counterpart).
  * While enabled, pg_round brackets every kernel it launches with a pair of CUDA
  * events on the caller's stream.  pg_timing_read waits for the recorded events,
- * adds up the elapsed milliseconds and the launch counts per kernel kind into
- * ms_out / launches_out (host, PG_KERNEL_KINDS entries each, indexed by the
- * PG_KERNEL_* constants) and forgets them.
+ * adds up, per kernel kind, the elapsed milliseconds, the launch counts and the
+ * algorithmic bytes of those launches (4 B per parameter of the layers the
+ * launch covers for every time it must read or write X once; 0 for the edge
+ * steps, which touch vectors only) into ms_out / launches_out / bytes_out (host,
+ * PG_KERNEL_KINDS entries each, indexed by the PG_KERNEL_* constants) and
+ * forgets them.
  */
 enum {
     PG_KERNEL_FORWARD = 0,         /* X q for all incident edges (first round only)     */
@@ -220,10 +226,13 @@ enum {
     PG_KERNEL_TRANSPOSED = 2,      /* X^T p-hat                                          */
     PG_KERNEL_EDGE_RIGHT = 3,      /* difference of the two ends, new stored vector      */
     PG_KERNEL_UPDATE_FORWARD = 4,  /* rank-r update of X fused with the next X q         */
-    PG_KERNEL_KINDS = 5
+    PG_KERNEL_PAIR_SWEEP = 5,      /* degree <= 1, rank 1: pending update + X q + X^T p from one read */
+    PG_KERNEL_PAIR_EDGE = 6,       /* its scalar edge step                               */
+    PG_KERNEL_UPDATE_ONLY = 7,     /* applies a pending update before X is read or written */
+    PG_KERNEL_KINDS = 8
 };
 PG_API int pg_timing_enable(pg_ctx *ctx, int32_t on);
-PG_API int pg_timing_read(pg_ctx *ctx, double *ms_out, int64_t *launches_out);
+PG_API int pg_timing_read(pg_ctx *ctx, double *ms_out, int64_t *launches_out, double *bytes_out);
 
 /*
  * z = X^T p for one matrix, with no allocation of any kind (the paper has no

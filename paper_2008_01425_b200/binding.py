@@ -28,7 +28,8 @@ EXPORTS = (
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
     "pg_transposed_product_noalloc",
 )
-KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward")
+KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
+                "pair_sweep", "pair_edge", "update_only")
 
 
 class pg_topology(ctypes.Structure):
@@ -81,7 +82,7 @@ def load_library() -> ctypes.CDLL:
     L.pg_build_schedule.argtypes = [ctypes.POINTER(pg_topology), vp, u64, i64, vp, vp, i32, ctypes.POINTER(i32)]
     L.pg_initial_vector.argtypes = [u64, i32, i32, i32, i32, i32, vp]
     L.pg_timing_enable.argtypes = [vp, i32]
-    L.pg_timing_read.argtypes = [vp, vp, vp]
+    L.pg_timing_read.argtypes = [vp, vp, vp, vp]
     L.pg_transposed_product_noalloc.argtypes = [vp, i32, i32, i64, vp, vp, vp]
     L.pg_status_string.argtypes = [ctypes.c_int]
     L.pg_status_string.restype = ctypes.c_char_p
@@ -291,11 +292,13 @@ class PowerGossip:
         _check(self._lib.pg_timing_enable(self._h, 1 if on else 0), "pg_timing_enable")
 
     def pg_timing_read(self):
-        """{kernel kind: (total ms, launches)} since the last read."""
+        """{kernel kind: (total ms, launches, algorithmic bytes)} since the last read."""
         ms = np.zeros(len(KERNEL_KINDS), dtype=np.float64)
         cnt = np.zeros(len(KERNEL_KINDS), dtype=np.int64)
-        _check(self._lib.pg_timing_read(self._h, ms.ctypes.data, cnt.ctypes.data), "pg_timing_read")
-        return {k: (float(ms[t]), int(cnt[t])) for t, k in enumerate(KERNEL_KINDS)}
+        nbytes = np.zeros(len(KERNEL_KINDS), dtype=np.float64)
+        _check(self._lib.pg_timing_read(self._h, ms.ctypes.data, cnt.ctypes.data, nbytes.ctypes.data),
+               "pg_timing_read")
+        return {k: (float(ms[t]), int(cnt[t]), float(nbytes[t])) for t, k in enumerate(KERNEL_KINDS)}
 
     # -- conveniences built only from the calls above ---------------------
     def write_all(self, params: Sequence[Sequence[np.ndarray]], stream=None) -> None:

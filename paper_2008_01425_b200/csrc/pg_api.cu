@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <climits>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -30,12 +31,15 @@ inline long long round_up(long long v, long long a) { return (v + a - 1) / a * a
 struct Layout {
     std::vector<LayerGeom> layers;
     long long x_stride = 0, q_stride = 0, y_stride = 0, ph_stride = 0, z_stride = 0;
+    long long up_stride = 0, sp_stride = 0;
     long long n_pairs = 0;
+    bool pair_mode = false;        // degree <= 1 and rank 1: thin layers run through the pair sweep
+    long long n_pair_tiles = 0, n_flush_tiles = 0;
     int max_edges = 0, max_degree = 0;
     TabLayout tab{};
     long long n_row_tiles = 0, n_col_tiles = 0;
     size_t off_X = 0, off_Q = 0, off_Qinv = 0, off_Y = 0, off_Ph = 0, off_Z = 0, off_live = 0,
-           off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
+           off_Up = 0, off_Sp = 0, off_pair_tiles = 0, off_flush_tiles = 0, off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
     size_t total = 0;
 };
 
@@ -68,6 +72,13 @@ int make_topology(const pg_topology* topo, const float* W_host, pg::Topology& ou
     return PG_OK;
 }
 
+// The pair sweep can be switched off (PG_DISABLE_PAIR_SWEEP=1 in the environment
+// when the context is created) so that both paths can be compared on one graph.
+bool pair_sweep_allowed() {
+    const char* v = std::getenv("PG_DISABLE_PAIR_SWEEP");
+    return !(v && v[0] == '1');
+}
+
 int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_layers, int rank,
                 Layout& lay) {
     if (!shapes || n_layers < 1 || n_layers > 4096) return PG_ERR_INVALID;
@@ -79,6 +90,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.n_pairs = topo.kind == PG_MATCHING ? static_cast<long long>(N) * (N - 1) / 2 : lay.max_edges;
     if (lay.n_pairs > INT_MAX / 2) return PG_ERR_INVALID;
 
+    lay.pair_mode = lay.max_degree == 1 && rank == 1 && pair_sweep_allowed();
     lay.layers.resize(n_layers);
     // aim for about 4096 tiles per sweep, each between 64 KB and 512 KB of X
     long long total_elems = 0;
@@ -86,8 +98,8 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         if (shapes[l].rows > 0 && shapes[l].cols > 0)
             total_elems += static_cast<long long>(N) * shapes[l].rows * round_up(shapes[l].cols, 4);
     const long long tile_elems = std::min<long long>(std::max<long long>(total_elems / 4096, 16 * 1024), 128 * 1024);
-    long long x = 0, q = 0, y = 0, ph = 0, z = 0;
-    lay.n_row_tiles = lay.n_col_tiles = 0;
+    long long x = 0, q = 0, y = 0, ph = 0, z = 0, up = 0, sp = 0;
+    lay.n_row_tiles = lay.n_col_tiles = lay.n_pair_tiles = lay.n_flush_tiles = 0;
     for (int l = 0; l < n_layers; ++l) {
         LayerGeom& g = lay.layers[l];
         if (shapes[l].rows < 1 || shapes[l].cols < 1) return PG_ERR_INVALID;
@@ -117,9 +129,22 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         y += round_up(static_cast<long long>(slots) * g.f_csplit * g.npad, 64);
         ph += round_up(static_cast<long long>(rank) * g.npad, 64);
         z += round_up(static_cast<long long>(slots) * g.t_rtiles * g.ld, 64);
-        lay.n_row_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
-        lay.n_col_tiles += static_cast<long long>(N) * g.t_rtiles * g.t_ctiles;
+        g.pair_mode = (lay.pair_mode && g.ld <= pg::kPairMaxLd) ? 1 : 0;
+        g.p_rtiles = (g.n + pg::kPairTileRows - 1) / pg::kPairTileRows;
+        g.up_off = up;
+        g.sp_off = sp;
+        if (g.pair_mode) {
+            up += round_up(static_cast<long long>(g.p_rtiles) * g.ld, 64);
+            sp += round_up(g.p_rtiles, 8);
+            lay.n_pair_tiles += static_cast<long long>(lay.max_edges) * g.p_rtiles;
+            lay.n_flush_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
+        } else {
+            lay.n_row_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
+            lay.n_col_tiles += static_cast<long long>(N) * g.t_rtiles * g.t_ctiles;
+        }
     }
+    lay.up_stride = up;
+    lay.sp_stride = sp;
     if (lay.n_row_tiles > INT_MAX || lay.n_col_tiles > INT_MAX) return PG_ERR_INVALID;
     lay.x_stride = x;
     lay.q_stride = q;
@@ -154,7 +179,9 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_Q = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride);
     lay.off_Qinv = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * n_layers * rank);
     lay.off_Y = take(sizeof(float) * static_cast<size_t>(N) * lay.y_stride);
-    lay.off_Ph = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * lay.ph_stride);
+    lay.off_Ph = take(sizeof(float) * 2 * static_cast<size_t>(lay.max_edges) * lay.ph_stride);  // two buffers
+    lay.off_Up = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * lay.up_stride);
+    lay.off_Sp = take(sizeof(double) * static_cast<size_t>(lay.max_edges) * lay.sp_stride);
     lay.off_Z = take(sizeof(float) * static_cast<size_t>(N) * lay.z_stride);
     lay.off_live = take(sizeof(int) * static_cast<size_t>(lay.max_edges) * n_layers * rank);
     lay.off_status = take(sizeof(int) * 64);
@@ -162,6 +189,8 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_tabs = take(sizeof(int) * static_cast<size_t>(kTabRing) * t.total_ints);
     lay.off_row_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_row_tiles));
     lay.off_col_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_col_tiles));
+    lay.off_pair_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_pair_tiles));
+    lay.off_flush_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_flush_tiles));
     lay.total = off;
     return PG_OK;
 }
@@ -177,6 +206,15 @@ struct pg_ctx {
     int rank = 1, power_steps = 1, n_layers = 0;
     int64_t round = 0;
     bool y_valid = false;       // Y already holds X Qh for the upcoming round
+    // pair sweep: the correction of the last step has not been applied to X yet
+    bool pending = false;
+    int64_t pending_key = 0;    // round whose table describes the pending correction
+    int64_t step = 0;           // power steps enqueued so far (selects the P-hat buffer)
+    float* ph_buf[2] = {nullptr, nullptr};
+    Tile* d_pair_tiles = nullptr;
+    Tile* d_flush_tiles = nullptr;
+    struct PairGroup { int nv; int first; int count; double bytes; };
+    std::vector<PairGroup> pair_groups;   // pair tiles grouped by float4 per lane
     int64_t launches = 0;
     char* ws = nullptr;
     int* d_tabs = nullptr;
@@ -190,7 +228,9 @@ struct pg_ctx {
     int device = 0;
     // optional per-kernel timing: one event pair per launch while enabled
     bool timing = false;
-    struct Span { int kind; cudaEvent_t a, b; };
+    struct Span { int kind; double bytes; cudaEvent_t a, b; };
+    double normal_param_bytes = 0.0;   // 4 B x parameters handled by the three-sweep path
+    double pair_param_bytes = 0.0;     // 4 B x parameters handled by the pair sweep
     std::vector<Span> spans;
 };
 
@@ -260,9 +300,11 @@ struct Timed {
     cudaStream_t s;
     pg_ctx::Span span{};
     bool on;
-    Timed(pg_ctx* ctx, int kind, cudaStream_t stream) : c(ctx), s(stream), on(ctx->timing) {
+    // `bytes`: algorithmic bytes of the launch (X read and/or written once)
+    Timed(pg_ctx* ctx, int kind, cudaStream_t stream, double bytes) : c(ctx), s(stream), on(ctx->timing) {
         if (!on) return;
         span.kind = kind;
+        span.bytes = bytes;
         on = cudaEventCreate(&span.a) == cudaSuccess && cudaEventCreate(&span.b) == cudaSuccess &&
              cudaEventRecord(span.a, s) == cudaSuccess;
     }
@@ -276,6 +318,28 @@ bool bind_device(const pg_ctx* c) {
     int cur = -1;
     if (cudaGetDevice(&cur) != cudaSuccess) return false;
     return cur == c->device || cudaSetDevice(c->device) == cudaSuccess;
+}
+
+// Apply the correction the pair sweep left pending, so that X in memory is the
+// live model (needed before X, Q or the round counter are read or overwritten).
+int flush_pending(pg_ctx* c, cudaStream_t stream) {
+    if (!c->pending) return PG_OK;
+    const int* tab_prev = nullptr;
+    const int rc = ensure_table(c, c->pending_key, stream, &tab_prev);
+    if (rc != PG_OK) return rc;
+    DevState st = c->st;
+    st.Ph = c->ph_buf[(c->step + 1) & 1];
+    {
+        Timed t(c, PG_KERNEL_UPDATE_ONLY, stream, 2.0 * c->pair_param_bytes);
+        if (pg::launch_update(st, tab_prev, c->d_flush_tiles, static_cast<int>(c->lay.n_flush_tiles), stream) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            return PG_ERR_CUDA;
+        }
+    }
+    c->launches += 1;
+    c->pending = false;
+    return PG_OK;
 }
 
 int check_worker_layer(const pg_ctx* c, int worker, int layer) {
@@ -352,6 +416,10 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     c->power_steps = power_steps;
     c->n_layers = n_layers;
     c->static_graph = c->topo.kind != PG_MATCHING;
+    for (int l = 0; l < n_layers; ++l) {
+        const double b = 4.0 * c->topo.n_workers * static_cast<double>(c->lay.layers[l].n) * c->lay.layers[l].m;
+        (c->lay.layers[l].pair_mode ? c->pair_param_bytes : c->normal_param_bytes) += b;
+    }
     c->pairs.triangular = !c->static_graph;
     c->pairs.n_workers = c->topo.n_workers;
     if (c->static_graph) c->pairs.static_edges = edges0;
@@ -368,6 +436,15 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.Qinv = reinterpret_cast<float*>(c->ws + lay.off_Qinv);
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
+    st.PhNext = st.Ph + static_cast<long long>(lay.max_edges) * lay.ph_stride;
+    c->ph_buf[0] = st.Ph;
+    c->ph_buf[1] = st.PhNext;
+    st.Up = reinterpret_cast<float*>(c->ws + lay.off_Up);
+    st.Sp = reinterpret_cast<double*>(c->ws + lay.off_Sp);
+    st.up_stride = lay.up_stride;
+    st.sp_stride = lay.sp_stride;
+    c->d_pair_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_pair_tiles);
+    c->d_flush_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_flush_tiles);
     st.Z = reinterpret_cast<float*>(c->ws + lay.off_Z);
     st.live = reinterpret_cast<int*>(c->ws + lay.off_live);
     st.status = reinterpret_cast<int*>(c->ws + lay.off_status);
@@ -389,21 +466,47 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     bool ok = cudaMemset(c->ws, 0, lay.total) == cudaSuccess;
     ok = ok && cudaMemcpy(c->ws + lay.off_layers, lay.layers.data(), sizeof(LayerGeom) * n_layers,
                           cudaMemcpyHostToDevice) == cudaSuccess;
-    // tile lists: worker-major, layers in the caller's order
+    // tile lists: worker-major, layers in the caller's order; layers that run
+    // through the pair sweep get pair tiles (edge, layer, row block), grouped by
+    // the number of float4 a lane holds, and row tiles for flushing a pending
+    // correction
     if (ok) {
-        std::vector<Tile> rows, cols;
+        std::vector<Tile> rows, cols, flush;
         rows.reserve(lay.n_row_tiles);
         cols.reserve(lay.n_col_tiles);
+        flush.reserve(lay.n_flush_tiles);
         for (int v = 0; v < c->topo.n_workers; ++v)
             for (int l = 0; l < n_layers; ++l) {
                 const LayerGeom& g = lay.layers[l];
                 for (int rt = 0; rt < g.f_rtiles; ++rt)
-                    for (int ct = 0; ct < g.f_csplit; ++ct) rows.push_back(Tile{v, l, rt, ct});
+                    for (int ct = 0; ct < g.f_csplit; ++ct)
+                        (g.pair_mode ? flush : rows).push_back(Tile{v, l, rt, ct});
+                if (g.pair_mode) continue;
                 for (int rt = 0; rt < g.t_rtiles; ++rt)
                     for (int ct = 0; ct < g.t_ctiles; ++ct) cols.push_back(Tile{v, l, rt, ct});
             }
-        ok = cudaMemcpy(c->d_row_tiles, rows.data(), sizeof(Tile) * rows.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-        ok = ok && cudaMemcpy(c->d_col_tiles, cols.data(), sizeof(Tile) * cols.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        std::vector<Tile> pairs;
+        pairs.reserve(lay.n_pair_tiles);
+        for (int nv = 1; nv <= pg::kPairMaxLd / 128; ++nv) {
+            const int first = static_cast<int>(pairs.size());
+            for (int l = 0; l < n_layers; ++l) {
+                const LayerGeom& g = lay.layers[l];
+                if (!g.pair_mode || (g.ld + 127) / 128 != nv) continue;
+                for (int e = 0; e < lay.max_edges; ++e)
+                    for (int rt = 0; rt < g.p_rtiles; ++rt) pairs.push_back(Tile{e, l, rt, 0});
+            }
+            const int count = static_cast<int>(pairs.size()) - first;
+            double bytes = 0.0;   // both ends of every edge read once and written once
+            for (int l = 0; l < n_layers; ++l)
+                if (lay.layers[l].pair_mode && (lay.layers[l].ld + 127) / 128 == nv)
+                    bytes += 8.0 * 2.0 * lay.max_edges * static_cast<double>(lay.layers[l].n) * lay.layers[l].m;
+            if (count > 0) c->pair_groups.push_back(pg_ctx::PairGroup{nv, first, count, bytes});
+        }
+        auto put = [](Tile* dst, const std::vector<Tile>& v) {
+            return v.empty() || cudaMemcpy(dst, v.data(), sizeof(Tile) * v.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        };
+        ok = put(c->d_row_tiles, rows) && put(c->d_col_tiles, cols) && put(c->d_pair_tiles, pairs) &&
+             put(c->d_flush_tiles, flush);
     }
     // Algorithm 2, initialisation: one standard-normal vector per pair, layer, column
     if (ok) {
@@ -457,6 +560,8 @@ int pg_write_params(pg_ctx* c, int32_t worker, int32_t layer, const float* host_
     int rc = check_worker_layer(c, worker, layer);
     if (rc != PG_OK || !host_src) return PG_ERR_INVALID;
     if (!bind_device(c)) return PG_ERR_CUDA;
+    rc = flush_pending(c, static_cast<cudaStream_t>(stream));
+    if (rc != PG_OK) return rc;
     const LayerGeom& g = c->lay.layers[layer];
     float* dst = c->st.X + static_cast<long long>(worker) * c->st.x_stride + g.x_off;
     c->y_valid = false;
@@ -470,6 +575,8 @@ int pg_read_params(pg_ctx* c, int32_t worker, int32_t layer, float* host_dst, vo
     int rc = check_worker_layer(c, worker, layer);
     if (rc != PG_OK || !host_dst) return PG_ERR_INVALID;
     if (!bind_device(c)) return PG_ERR_CUDA;
+    rc = flush_pending(c, static_cast<cudaStream_t>(stream));
+    if (rc != PG_OK) return rc;
     const LayerGeom& g = c->lay.layers[layer];
     const float* src = c->st.X + static_cast<long long>(worker) * c->st.x_stride + g.x_off;
     if (cudaMemcpy2DAsync(host_dst, sizeof(float) * g.m, src, sizeof(float) * g.ld, sizeof(float) * g.m,
@@ -493,33 +600,62 @@ int pg_round(pg_ctx* c, void* stream_v) {
     int rc = ensure_table(c, c->round, stream, &tab);
     if (rc == PG_OK) rc = ensure_table(c, c->round + 1, stream, &tab_next);
     if (rc != PG_OK) return rc;
-    const DevState& st = c->st;
     const int n_rows = static_cast<int>(c->lay.n_row_tiles), n_cols = static_cast<int>(c->lay.n_col_tiles);
+    const bool has_pair = c->lay.n_pair_tiles > 0;
     bool ok = true;
-    if (!c->y_valid) {
-        Timed t(c, PG_KERNEL_FORWARD, stream);
-        ok = ok && pg::launch_forward(st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+    if (n_rows > 0 && !c->y_valid) {
+        Timed t(c, PG_KERNEL_FORWARD, stream, c->normal_param_bytes);
+        ok = ok && pg::launch_forward(c->st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
         c->launches += 1;
     }
     for (int p = 0; p < c->power_steps && ok; ++p) {
         const int* tab_fwd = (p + 1 < c->power_steps) ? tab : tab_next;
-        {
-            Timed t(c, PG_KERNEL_EDGE_LEFT, stream);
-            ok = ok && pg::launch_edge_left(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+        float* const ph_cur = c->ph_buf[c->step & 1];        // this step's P-hat
+        float* const ph_prev = c->ph_buf[(c->step + 1) & 1]; // last step's (pending correction)
+        if (n_rows > 0) {
+            DevState st = c->st;
+            st.Ph = ph_cur;
+            {
+                Timed t(c, PG_KERNEL_EDGE_LEFT, stream, 0.0);
+                ok = ok && pg::launch_edge_left(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+            }
+            {
+                Timed t(c, PG_KERNEL_TRANSPOSED, stream, c->normal_param_bytes);
+                ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+            }
+            {
+                Timed t(c, PG_KERNEL_EDGE_RIGHT, stream, 0.0);
+                ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+            }
+            {
+                Timed t(c, PG_KERNEL_UPDATE_FORWARD, stream, 2.0 * c->normal_param_bytes);
+                ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+            }
+            c->launches += 4;
         }
-        {
-            Timed t(c, PG_KERNEL_TRANSPOSED, stream);
-            ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+        if (has_pair && ok) {
+            // one read of both ends of every edge: apply the correction pending from the
+            // last step, form p and this step's share of D^T p; then the scalar edge step
+            const int* tab_prev = tab;
+            if (c->pending) ok = ensure_table(c, c->pending_key, stream, &tab_prev) == PG_OK;
+            DevState st = c->st;
+            st.Ph = ph_prev;
+            st.PhNext = ph_cur;
+            for (const auto& grp : c->pair_groups) {
+                Timed t(c, PG_KERNEL_PAIR_SWEEP, stream, grp.bytes);
+                ok = ok && pg::launch_pair_sweep(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
+                                                 grp.count, grp.nv, stream) == cudaSuccess;
+                c->launches += 1;
+            }
+            {
+                Timed t(c, PG_KERNEL_PAIR_EDGE, stream, 0.0);
+                ok = ok && pg::launch_pair_edge(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+                c->launches += 1;
+            }
+            c->pending = true;
+            c->pending_key = c->static_graph ? 0 : c->round;
         }
-        {
-            Timed t(c, PG_KERNEL_EDGE_RIGHT, stream);
-            ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
-        }
-        {
-            Timed t(c, PG_KERNEL_UPDATE_FORWARD, stream);
-            ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, stream) == cudaSuccess;
-        }
-        c->launches += 4;
+        c->step += 1;
     }
     if (!ok) {
         cudaGetLastError();
@@ -574,6 +710,8 @@ int pg_write_q(pg_ctx* c, int32_t i, int32_t j, int32_t layer, const float* host
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const LayerGeom& g = c->lay.layers[layer];
     float* dst = c->st.Q + pair * c->st.q_stride + g.q_off;
+    const int frc = flush_pending(c, stream);     // the pending correction uses the stored vectors
+    if (frc != PG_OK) return frc;
     c->y_valid = false;
     if (cudaMemcpy2DAsync(dst, sizeof(float) * g.ld, host_src, sizeof(float) * g.m, sizeof(float) * g.m,
                           c->rank, cudaMemcpyHostToDevice, stream) != cudaSuccess)
@@ -618,6 +756,12 @@ int pg_get_round(pg_ctx* c, int64_t* round_out) {
 
 int pg_set_round(pg_ctx* c, int64_t round) {
     if (!c || round < 0) return PG_ERR_INVALID;
+    if (c->pending) {
+        if (!bind_device(c)) return PG_ERR_CUDA;
+        const int rc = flush_pending(c, nullptr);
+        if (rc != PG_OK) return rc;
+        if (cudaStreamSynchronize(nullptr) != cudaSuccess) return PG_ERR_CUDA;
+    }
     c->round = round;
     c->y_valid = false;
     return PG_OK;
@@ -629,12 +773,13 @@ int pg_timing_enable(pg_ctx* c, int32_t on) {
     return PG_OK;
 }
 
-int pg_timing_read(pg_ctx* c, double* ms_out, int64_t* launches_out) {
-    if (!c || !ms_out || !launches_out) return PG_ERR_INVALID;
+int pg_timing_read(pg_ctx* c, double* ms_out, int64_t* launches_out, double* bytes_out) {
+    if (!c || !ms_out || !launches_out || !bytes_out) return PG_ERR_INVALID;
     if (!bind_device(c)) return PG_ERR_CUDA;
     for (int k = 0; k < PG_KERNEL_KINDS; ++k) {
         ms_out[k] = 0.0;
         launches_out[k] = 0;
+        bytes_out[k] = 0.0;
     }
     bool ok = true;
     for (auto& sp : c->spans) {
@@ -643,6 +788,7 @@ int pg_timing_read(pg_ctx* c, double* ms_out, int64_t* launches_out) {
         if (ok) {
             ms_out[sp.kind] += ms;
             launches_out[sp.kind] += 1;
+            bytes_out[sp.kind] += sp.bytes;
         }
         cudaEventDestroy(sp.a);
         cudaEventDestroy(sp.b);

@@ -18,6 +18,8 @@ constexpr int kRowTileRowsMax = 64;    // rows of X per CTA in the row-oriented 
 constexpr int kRowTileColsMax = 2048;  // most columns one CTA reduces over (multiple of 128)
 constexpr int kColTileRowsMax = 256;   // rows of X per CTA in the transposed sweep (64, 128 or 256)
 constexpr int kColTileCols = 256;      // columns per CTA in the transposed sweep (64 threads x float4)
+constexpr int kPairTileRows = 512;     // rows of both matrices per CTA in the pair sweep
+constexpr int kPairMaxLd = 1024;       // widest row a warp of the pair sweep keeps in registers
 
 // Geometry of one layer (same for every worker).
 struct LayerGeom {
@@ -36,6 +38,11 @@ struct LayerGeom {
     long long y_off;   // forward partials inside a worker's block   (slots x f_csplit x npad)
     long long ph_off;  // P-hat inside an edge's block               (rank x npad)
     long long z_off;   // transposed partials inside a worker's block (slots x t_rtiles x ld)
+    // pair sweep (graphs of degree <= 1 at rank 1; rows of at most kPairMaxLd floats)
+    int pair_mode;     // 1 if this layer runs through the pair sweep
+    int p_rtiles;      // row tiles of the pair sweep
+    long long up_off;  // partial sums of D^T p inside an edge's block (p_rtiles x ld)
+    long long sp_off;  // partial sums of ||p||^2 inside an edge's block (p_rtiles doubles)
 };
 
 // One unit of work of a sweep: a tile of one worker's layer.
@@ -71,10 +78,13 @@ struct DevState {
     float* Y;            // [worker][y_stride]   partial sums of X q
     float* Ph;           // [edge][ph_stride]    orthonormal left factors of this step
     float* Z;            // [worker][z_stride]   partial sums of X^T p
+    float* PhNext;       // same shape as Ph: where the pair sweep writes this step's p
+    float* Up;           // [edge][up_stride]    pair sweep: partial sums of D^T p
+    double* Sp;          // [edge][sp_stride]    pair sweep: partial sums of ||p||^2
     int* live;           // [edge][layer][rank]  1 if the column took part in this step
     int* status;         // device status word (bit n set = error code n was raised)
     const LayerGeom* layers;
-    long long x_stride, q_stride, y_stride, ph_stride, z_stride;
+    long long x_stride, q_stride, y_stride, ph_stride, z_stride, up_stride, sp_stride;
     int n_layers, rank, n_workers, max_degree;
     TabLayout tab;
 };
@@ -89,6 +99,11 @@ cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* ti
 cudaError_t launch_edge_right(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_update_forward(const DevState& st, const int* tab_update, const int* tab_forward,
                                   const Tile* tiles, int n_tiles, cudaStream_t stream);
+cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile* tiles, int n_tiles,
+                          cudaStream_t stream);
+cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
+                              const Tile* tiles, int n_tiles, int nv, cudaStream_t stream);
+cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_column_norms(const DevState& st, long long n_pairs, cudaStream_t stream);
 
 }  // namespace pg

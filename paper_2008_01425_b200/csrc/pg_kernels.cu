@@ -341,6 +341,7 @@ edge_left_kernel(DevState st, const int* __restrict__ tab) {
     const int e = blockIdx.x / L, l = blockIdx.x - e * L;
     if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
+    if (g.pair_mode) return;   // handled by the pair sweep's own edge step
     const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
     const int pair = tab[st.tab.off_pair + e];
     const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
@@ -422,6 +423,7 @@ edge_right_kernel(DevState st, const int* __restrict__ tab) {
     const int e = blockIdx.x / L, l = blockIdx.x - e * L;
     if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
+    if (g.pair_mode) return;
     const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
     const int pair = tab[st.tab.off_pair + e];
     const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
@@ -449,6 +451,194 @@ edge_right_kernel(DevState st, const int* __restrict__ tab) {
             st.Qinv[((long long)pair * L + l) * rank + k] = nn > 0.0 ? (float)(1.0 / sqrt(nn)) : 0.0f;
             if (!isfinite(nn)) atomicOr(st.status, 1 << kStatusNumeric);
         }
+    }
+}
+
+// --------------------------------------------------------------------------
+// Pair sweep (graphs of degree <= 1, rank 1).  One CTA owns a block of rows of
+// BOTH ends of an edge (i<j) and reads each row of X_i and X_j once:
+//   - applies the correction that is still pending from the previous step to
+//     each row (each end has its own previous edge) and writes the rows back,
+//   - forms the row of D = X_i - X_j, its product with q-hat:  p_r = D_r . q-hat,
+//   - accumulates u += p_r D_r, i.e. its share of D^T p, and of ||p||^2.
+// The normalisation is a scalar, so it is applied afterwards by the pair edge
+// step:  p-hat = p / ||p||,  Q' = D^T p-hat = u / ||p||.  This is the same power
+// step as the three-sweep path with X read once instead of twice.
+// A warp keeps a whole row (up to 8 float4 per lane) in registers.
+// --------------------------------------------------------------------------
+template <int NV, bool UPDATE>
+__global__ void __launch_bounds__(256, 2)
+pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
+                  const Tile* __restrict__ tiles) {
+    __shared__ __align__(16) float s_q[NV * 128];
+    __shared__ __align__(16) float s_ui[NV * 128];
+    __shared__ __align__(16) float s_uj[NV * 128];
+    __shared__ __align__(16) float s_red[8][NV * 128];
+    __shared__ double s_s[8];
+
+    const Tile tile = tiles[blockIdx.x];
+    const int e = tile.worker;                       // edge index within the current round
+    if (e >= tab_cur[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[tile.layer];
+    const int L = st.n_layers;
+    const int wi = tab_cur[st.tab.off_edge_i + e], wj = tab_cur[st.tab.off_edge_j + e];
+    const int pair = tab_cur[st.tab.off_pair + e];
+    float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
+    float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
+    const int ld = g.ld;
+
+    // this edge's stored vector (unit length after scaling) and, per end, the
+    // factors of the pending correction
+    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float qinv = st.Qinv[(long long)pair * L + tile.layer];
+    const float* ui = q;
+    const float* uj = q;
+    const float* phi = nullptr;
+    const float* phj = nullptr;
+    float coef_i = 0.0f, coef_j = 0.0f;
+    if (UPDATE) {
+        if (tab_prev[st.tab.off_degree + wi] > 0) {
+            const int ep = tab_prev[st.tab.off_slot_edge + wi * st.tab.max_degree];
+            ui = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            phi = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            coef_i = __int_as_float(tab_prev[st.tab.off_slot_coef + wi * st.tab.max_degree]);
+        }
+        if (tab_prev[st.tab.off_degree + wj] > 0) {
+            const int ep = tab_prev[st.tab.off_slot_edge + wj * st.tab.max_degree];
+            uj = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            phj = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            coef_j = __int_as_float(tab_prev[st.tab.off_slot_coef + wj * st.tab.max_degree]);
+        }
+    }
+    for (int idx = threadIdx.x; idx < NV * 128; idx += 256) {
+        const bool in = idx < ld;
+        s_q[idx] = in ? q[idx] * qinv : 0.0f;
+        if (UPDATE) {
+            s_ui[idx] = in ? ui[idx] : 0.0f;
+            s_uj[idx] = in ? uj[idx] : 0.0f;
+        }
+    }
+    __syncthreads();
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = tile.rtile * kPairTileRows;
+    const int r1 = min(g.n, r0 + kPairTileRows);
+    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    float4 u[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float ssum = 0.0f;
+
+    for (int r = r0 + warp; r < r1; r += 8) {
+        float4 xi[NV], xj[NV];
+        float* rowi = Xi + (long long)r * ld;
+        float* rowj = Xj + (long long)r * ld;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int col = (k * 32 + lane) * 4;
+            if (col < ld) {
+                xi[k] = ld_stream(rowi + col);
+                xj[k] = ld_stream(rowj + col);
+            } else {
+                xi[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                xj[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        if (UPDATE) {
+            const float ai = phi ? coef_i * __ldg(phi + r) : 0.0f;
+            const float aj = phj ? coef_j * __ldg(phj + r) : 0.0f;
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int col = (k * 32 + lane) * 4;
+                const float4 vi = *reinterpret_cast<const float4*>(&s_ui[col]);
+                const float4 vj = *reinterpret_cast<const float4*>(&s_uj[col]);
+                xi[k].x = fmaf(-ai, vi.x, xi[k].x); xi[k].y = fmaf(-ai, vi.y, xi[k].y);
+                xi[k].z = fmaf(-ai, vi.z, xi[k].z); xi[k].w = fmaf(-ai, vi.w, xi[k].w);
+                xj[k].x = fmaf(-aj, vj.x, xj[k].x); xj[k].y = fmaf(-aj, vj.y, xj[k].y);
+                xj[k].z = fmaf(-aj, vj.z, xj[k].z); xj[k].w = fmaf(-aj, vj.w, xj[k].w);
+                if (col < ld) {
+                    st_stream(rowi + col, xi[k]);
+                    st_stream(rowj + col, xj[k]);
+                }
+            }
+        }
+        float dot = 0.0f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int col = (k * 32 + lane) * 4;
+            const float4 vq = *reinterpret_cast<const float4*>(&s_q[col]);
+            xi[k].x -= xj[k].x; xi[k].y -= xj[k].y; xi[k].z -= xj[k].z; xi[k].w -= xj[k].w;   // row of D
+            dot = fmaf(xi[k].x, vq.x, dot); dot = fmaf(xi[k].y, vq.y, dot);
+            dot = fmaf(xi[k].z, vq.z, dot); dot = fmaf(xi[k].w, vq.w, dot);
+        }
+        const float p = warp_sum(dot);
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            u[k].x = fmaf(p, xi[k].x, u[k].x); u[k].y = fmaf(p, xi[k].y, u[k].y);
+            u[k].z = fmaf(p, xi[k].z, u[k].z); u[k].w = fmaf(p, xi[k].w, u[k].w);
+        }
+        ssum = fmaf(p, p, ssum);
+        if (lane == 0) Pw[r] = p;
+    }
+#pragma unroll
+    for (int k = 0; k < NV; ++k) *reinterpret_cast<float4*>(&s_red[warp][(k * 32 + lane) * 4]) = u[k];
+    if (lane == 0) s_s[warp] = (double)ssum;
+    __syncthreads();
+    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld;
+    for (int idx = threadIdx.x; idx < ld; idx += 256) {
+        float t = s_red[0][idx];
+#pragma unroll
+        for (int w8 = 1; w8 < 8; ++w8) t += s_red[w8][idx];
+        Up[idx] = t;
+    }
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w8 = 0; w8 < 8; ++w8) t += s_s[w8];
+        st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = t;
+    }
+}
+
+// Pair edge step: ||p||^2 from the tiles' shares, p-hat = p / ||p|| in place,
+// Q' = (sum of the tiles' shares of D^T p) / ||p||, 1 / ||Q'||.  A zero or
+// non-finite norm leaves the stored vector alone and zeroes p-hat.
+// One CTA per (edge, layer).
+__global__ void __launch_bounds__(512)
+pair_edge_kernel(DevState st, const int* __restrict__ tab) {
+    __shared__ double scratch[33];
+    const int L = st.n_layers;
+    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[l];
+    if (!g.pair_mode) return;
+    const int pair = tab[st.tab.off_pair + e];
+    const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
+    double nn = 0.0;
+    for (int t = 0; t < g.p_rtiles; ++t) nn += sp[t];
+    const bool finite = isfinite(nn);
+    const bool live = finite && nn > 0.0;
+    const double inv = live ? 1.0 / sqrt(nn) : 0.0;
+    float* P = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    for (int r = threadIdx.x; r < g.npad; r += blockDim.x)
+        P[r] = (live && r < g.n) ? (float)((double)P[r] * inv) : 0.0f;
+    if (threadIdx.x == 0) {
+        st.live[(long long)e * L + l] = live ? 1 : 0;
+        if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
+    }
+    if (!live) return;   // uniform over the block
+    const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
+    float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    double part = 0.0;
+    for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
+        double a = 0.0;
+        for (int t = 0; t < g.p_rtiles; ++t) a += (double)up[(long long)t * g.ld + c];
+        const float q = (float)(a * inv);
+        Q[c] = q;
+        part += (double)q * (double)q;
+    }
+    const double qq = block_sum(part, scratch);
+    if (threadIdx.x == 0) {
+        st.Qinv[(long long)pair * L + l] = qq > 0.0 ? (float)(1.0 / sqrt(qq)) : 0.0f;
+        if (!isfinite(qq)) atomicOr(st.status, 1 << kStatusNumeric);
     }
 }
 
@@ -503,6 +693,41 @@ cudaError_t launch_update_forward(const DevState& st, const int* tab_update, con
     if (tab_update == tab_forward)
         return launch_row<true, true, true>(st, tab_update, tab_forward, tiles, n_tiles, stream);
     return launch_row<true, true, false>(st, tab_update, tab_forward, tiles, n_tiles, stream);
+}
+
+cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile* tiles, int n_tiles,
+                          cudaStream_t stream) {
+    return launch_row<true, false, false>(st, tab_update, tab_update, tiles, n_tiles, stream);
+}
+
+template <bool UPDATE>
+static cudaError_t launch_pair(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
+                               int n_tiles, int nv, cudaStream_t stream) {
+    switch (nv) {
+        case 1: pair_sweep_kernel<1, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        case 2: pair_sweep_kernel<2, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        case 3: pair_sweep_kernel<3, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        case 4: pair_sweep_kernel<4, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        case 5: pair_sweep_kernel<5, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        case 6: pair_sweep_kernel<6, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        case 7: pair_sweep_kernel<7, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        default: pair_sweep_kernel<8, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+    }
+    return cudaGetLastError();
+}
+
+// `tiles` must list tiles of layers with the same number of float4 per lane
+// (ceil(ld / 128)); the host launches one group per value.
+cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
+                              const Tile* tiles, int n_tiles, int nv, cudaStream_t stream) {
+    if (n_tiles <= 0) return cudaSuccess;
+    return apply_pending ? launch_pair<true>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
+                         : launch_pair<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+}
+
+cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
+    pair_edge_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
