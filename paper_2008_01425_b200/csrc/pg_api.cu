@@ -5,6 +5,7 @@
 
 #include <algorithm>
 #include <climits>
+#include <cmath>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -38,6 +39,7 @@ struct Layout {
     int max_edges = 0, max_degree = 0;
     TabLayout tab{};
     long long n_row_tiles = 0, n_col_tiles = 0;
+    size_t off_Qn2 = 0;
     size_t off_X = 0, off_Q = 0, off_Qinv = 0, off_Y = 0, off_Ph = 0, off_Z = 0, off_live = 0,
            off_Up = 0, off_Sp = 0, off_pair_tiles = 0, off_flush_tiles = 0, off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
     size_t total = 0;
@@ -79,8 +81,30 @@ bool pair_sweep_allowed() {
     return !(v && v[0] == '1');
 }
 
+// Rows per cluster tile of a wide pair-sweep layer: with `resident` clusters
+// running at once, split every edge's rows into S equal parts so that the
+// max_edges * S tiles fill whole waves as nearly as possible.
+int wide_tile_rows(int n, int max_edges, int resident) {
+    if (resident <= 0) return pg::kPairWideRows;
+    int best_s = 1;
+    double best_eff = 0.0;
+    for (int s = 1; s <= pg::kPairWideMaxTiles && s * 8 <= std::max(n, 8); ++s) {
+        const double waves = static_cast<double>(max_edges) * s / resident;
+        const double eff = waves / std::ceil(waves);
+        if (eff > best_eff + 1e-9) {
+            best_eff = eff;
+            best_s = s;
+        }
+    }
+    const int rows = (n + best_s - 1) / best_s;
+    return (rows + pg::kPairWideStep - 1) / pg::kPairWideStep * pg::kPairWideStep;
+}
+
+// query_device: ask the current device how many clusters of the wide pair sweep
+// fit at once and shape its tiles accordingly.  Section sizes do not depend on
+// the answer, so a sizing pass without a device gives the same total.
 int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_layers, int rank,
-                Layout& lay) {
+                Layout& lay, bool query_device = false) {
     if (!shapes || n_layers < 1 || n_layers > 4096) return PG_ERR_INVALID;
     if (rank < 1 || rank > PG_MAX_RANK) return PG_ERR_INVALID;
     if (!pg::topology_bounds(topo, &lay.max_edges, &lay.max_degree)) return PG_ERR_INVALID;
@@ -129,14 +153,26 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         y += round_up(static_cast<long long>(slots) * g.f_csplit * g.npad, 64);
         ph += round_up(static_cast<long long>(rank) * g.npad, 64);
         z += round_up(static_cast<long long>(slots) * g.t_rtiles * g.ld, 64);
-        g.pair_mode = (lay.pair_mode && g.ld <= pg::kPairMaxLd) ? 1 : 0;
-        g.p_rtiles = (g.n + pg::kPairTileRows - 1) / pg::kPairTileRows;
+        g.pair_mode = !lay.pair_mode ? 0 : (g.ld <= pg::kPairMaxLd ? 1 : (g.ld <= pg::kPairWideMaxLd ? 2 : 0));
+        g.p_slice = static_cast<int>(round_up((g.ld + pg::kPairCluster - 1) / pg::kPairCluster, 4));
+        g.p_rows = pg::kPairTileRows;
+        if (g.pair_mode == 2) {
+            const int resident = query_device
+                ? pg::pair_wide_resident_clusters((g.p_slice / 4 + 255) / 256, g.p_slice) : 0;
+            g.p_rows = wide_tile_rows(g.n, lay.max_edges, resident);
+            if ((g.n + g.p_rows - 1) / g.p_rows > pg::kPairWideMaxTiles)
+                g.p_rows = static_cast<int>(round_up((g.n + pg::kPairWideMaxTiles - 1) / pg::kPairWideMaxTiles,
+                                                     pg::kPairWideStep));
+        }
+        g.p_rtiles = (g.n + g.p_rows - 1) / g.p_rows;
         g.up_off = up;
         g.sp_off = sp;
-        if (g.pair_mode) {
-            up += round_up(static_cast<long long>(g.p_rtiles) * g.ld, 64);
-            sp += round_up(g.p_rtiles, 8);
-            lay.n_pair_tiles += static_cast<long long>(lay.max_edges) * g.p_rtiles;
+        if (g.pair_mode != 0) {
+            // wide layers: room for any tile count the device query may choose
+            const int max_tiles = g.pair_mode == 2 ? pg::kPairWideMaxTiles : g.p_rtiles;
+            up += round_up(static_cast<long long>(max_tiles) * g.ld, 64);
+            sp += round_up(max_tiles, 8);
+            lay.n_pair_tiles += static_cast<long long>(lay.max_edges) * max_tiles;
             lay.n_flush_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
         } else {
             lay.n_row_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
@@ -178,6 +214,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_X = take(sizeof(float) * static_cast<size_t>(N) * lay.x_stride);
     lay.off_Q = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride);
     lay.off_Qinv = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * n_layers * rank);
+    lay.off_Qn2 = take(sizeof(double) * static_cast<size_t>(lay.n_pairs) * n_layers * pg::kEdgeChunks);
     lay.off_Y = take(sizeof(float) * static_cast<size_t>(N) * lay.y_stride);
     lay.off_Ph = take(sizeof(float) * 2 * static_cast<size_t>(lay.max_edges) * lay.ph_stride);  // two buffers
     lay.off_Up = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * lay.up_stride);
@@ -213,7 +250,7 @@ struct pg_ctx {
     float* ph_buf[2] = {nullptr, nullptr};
     Tile* d_pair_tiles = nullptr;
     Tile* d_flush_tiles = nullptr;
-    struct PairGroup { int nv; int first; int count; double bytes; };
+    struct PairGroup { int mode; int nv; int slice; int first; int count; double bytes; };
     std::vector<PairGroup> pair_groups;   // pair tiles grouped by float4 per lane
     int64_t launches = 0;
     char* ws = nullptr;
@@ -407,6 +444,12 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
             if (!bind_device(c)) rc = PG_ERR_CUDA;
         }
     }
+    if (rc == PG_OK) {
+        // same sections and sizes as the sizing pass; tile shapes tuned to this device
+        const size_t need = c->lay.total;
+        rc = make_layout(c->topo, shapes, n_layers, rank, c->lay, true);
+        if (rc == PG_OK && c->lay.total != need) rc = PG_ERR_STATE;
+    }
     if (rc != PG_OK) {
         delete c;
         return rc;
@@ -434,6 +477,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.X = reinterpret_cast<float*>(c->ws + lay.off_X);
     st.Q = reinterpret_cast<float*>(c->ws + lay.off_Q);
     st.Qinv = reinterpret_cast<float*>(c->ws + lay.off_Qinv);
+    st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
     st.PhNext = st.Ph + static_cast<long long>(lay.max_edges) * lay.ph_stride;
@@ -487,20 +531,36 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
             }
         std::vector<Tile> pairs;
         pairs.reserve(lay.n_pair_tiles);
-        for (int nv = 1; nv <= pg::kPairMaxLd / 128; ++nv) {
+        // one launch per group of layers that share the kernel instantiation
+        auto group_of = [&](const LayerGeom& g, int* nv, int* slice) {
+            if (g.pair_mode == 1) {
+                *nv = (g.ld + 127) / 128;
+                *slice = 0;
+            } else {
+                *nv = (g.p_slice / 4 + 255) / 256;
+                *slice = g.p_slice;
+            }
+        };
+        std::vector<char> done(n_layers, 0);
+        for (int l0 = 0; l0 < n_layers; ++l0) {
+            if (!lay.layers[l0].pair_mode || done[l0]) continue;
+            int nv0 = 0, slice0 = 0;
+            group_of(lay.layers[l0], &nv0, &slice0);
             const int first = static_cast<int>(pairs.size());
-            for (int l = 0; l < n_layers; ++l) {
+            double bytes = 0.0;   // both ends of every edge read once and written once
+            for (int l = l0; l < n_layers; ++l) {
                 const LayerGeom& g = lay.layers[l];
-                if (!g.pair_mode || (g.ld + 127) / 128 != nv) continue;
+                int nv = 0, slice = 0;
+                if (!g.pair_mode || done[l] || g.pair_mode != lay.layers[l0].pair_mode) continue;
+                group_of(g, &nv, &slice);
+                if (nv != nv0 || slice != slice0) continue;
+                done[l] = 1;
                 for (int e = 0; e < lay.max_edges; ++e)
                     for (int rt = 0; rt < g.p_rtiles; ++rt) pairs.push_back(Tile{e, l, rt, 0});
+                bytes += 8.0 * 2.0 * lay.max_edges * static_cast<double>(g.n) * g.m;
             }
             const int count = static_cast<int>(pairs.size()) - first;
-            double bytes = 0.0;   // both ends of every edge read once and written once
-            for (int l = 0; l < n_layers; ++l)
-                if (lay.layers[l].pair_mode && (lay.layers[l].ld + 127) / 128 == nv)
-                    bytes += 8.0 * 2.0 * lay.max_edges * static_cast<double>(lay.layers[l].n) * lay.layers[l].m;
-            if (count > 0) c->pair_groups.push_back(pg_ctx::PairGroup{nv, first, count, bytes});
+            c->pair_groups.push_back(pg_ctx::PairGroup{lay.layers[l0].pair_mode, nv0, slice0, first, count, bytes});
         }
         auto put = [](Tile* dst, const std::vector<Tile>& v) {
             return v.empty() || cudaMemcpy(dst, v.data(), sizeof(Tile) * v.size(), cudaMemcpyHostToDevice) == cudaSuccess;
@@ -643,8 +703,12 @@ int pg_round(pg_ctx* c, void* stream_v) {
             st.PhNext = ph_cur;
             for (const auto& grp : c->pair_groups) {
                 Timed t(c, PG_KERNEL_PAIR_SWEEP, stream, grp.bytes);
-                ok = ok && pg::launch_pair_sweep(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
-                                                 grp.count, grp.nv, stream) == cudaSuccess;
+                if (grp.mode == 1)
+                    ok = ok && pg::launch_pair_sweep(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
+                                                     grp.count, grp.nv, stream) == cudaSuccess;
+                else
+                    ok = ok && pg::launch_pair_sweep_wide(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
+                                                          grp.count, grp.nv, grp.slice, stream) == cudaSuccess;
                 c->launches += 1;
             }
             {

@@ -20,6 +20,12 @@ constexpr int kColTileRowsMax = 256;   // rows of X per CTA in the transposed sw
 constexpr int kColTileCols = 256;      // columns per CTA in the transposed sweep (64 threads x float4)
 constexpr int kPairTileRows = 512;     // rows of both matrices per CTA in the pair sweep
 constexpr int kPairMaxLd = 1024;       // widest row a warp of the pair sweep keeps in registers
+constexpr int kPairCluster = 8;        // CTAs that share a row of a wider layer (thread-block cluster)
+constexpr int kPairWideRows = 32;      // rows per cluster tile of a wider layer when residency is unknown
+constexpr int kPairWideMaxTiles = 32;  // most row tiles per (edge, wide layer); sizes the partial-sum buffer
+constexpr int kPairWideStep = 2;       // rows a cluster handles between two barriers
+constexpr int kPairWideMaxLd = 8 * 256 * 4 * kPairCluster;  // widest row the cluster variant covers
+constexpr int kEdgeChunks = 32;        // CTAs that share the pair edge step of one (edge, layer)
 
 // Geometry of one layer (same for every worker).
 struct LayerGeom {
@@ -39,8 +45,10 @@ struct LayerGeom {
     long long ph_off;  // P-hat inside an edge's block               (rank x npad)
     long long z_off;   // transposed partials inside a worker's block (slots x t_rtiles x ld)
     // pair sweep (graphs of degree <= 1 at rank 1; rows of at most kPairMaxLd floats)
-    int pair_mode;     // 1 if this layer runs through the pair sweep
+    int pair_mode;     // 0: three sweeps; 1: pair sweep, row per warp; 2: pair sweep, row per cluster
+    int p_rows;        // rows per tile of the pair sweep
     int p_rtiles;      // row tiles of the pair sweep
+    int p_slice;       // mode 2: columns per CTA of the cluster (multiple of 4)
     long long up_off;  // partial sums of D^T p inside an edge's block (p_rtiles x ld)
     long long sp_off;  // partial sums of ||p||^2 inside an edge's block (p_rtiles doubles)
 };
@@ -75,6 +83,7 @@ struct DevState {
     float* X;            // [worker][x_stride]
     float* Q;            // [pair][q_stride]     raw right factors
     float* Qinv;         // [pair][layer][rank]  1 / column norm (0 for a zero column)
+    double* Qn2;         // [pair][layer][kEdgeChunks]  pair sweep layers: shares of ||Q||^2
     float* Y;            // [worker][y_stride]   partial sums of X q
     float* Ph;           // [edge][ph_stride]    orthonormal left factors of this step
     float* Z;            // [worker][z_stride]   partial sums of X^T p
@@ -103,6 +112,11 @@ cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile*
                           cudaStream_t stream);
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
                               const Tile* tiles, int n_tiles, int nv, cudaStream_t stream);
+cudaError_t launch_pair_sweep_wide(const DevState& st, const int* tab_prev, const int* tab_cur,
+                                   bool apply_pending, const Tile* tiles, int n_tiles, int nv, int slice,
+                                   cudaStream_t stream);
+// Clusters of the wide pair sweep that can be resident at once (0 if unknown).
+int pair_wide_resident_clusters(int nv, int slice);
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_column_norms(const DevState& st, long long n_pairs, cudaStream_t stream);
 

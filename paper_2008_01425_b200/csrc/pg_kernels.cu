@@ -11,6 +11,8 @@
 // The three sweeps stream X with 16-byte loads; each is bound by HBM bandwidth.
 // Sums over column chunks / row tiles are written as partials and added in a
 // fixed order by the edge kernels, so results are bit-reproducible.
+#include <cooperative_groups.h>
+
 #include "pg_device.h"
 
 namespace pg {
@@ -454,6 +456,15 @@ edge_right_kernel(DevState st, const int* __restrict__ tab) {
     }
 }
 
+// 1 / ||Q|| of a pair-sweep layer from the shares the pair edge step left.
+__device__ __forceinline__ float pair_qinv(const DevState& st, int pair, int layer) {
+    const double* n2 = st.Qn2 + ((long long)pair * st.n_layers + layer) * kEdgeChunks;
+    double t = 0.0;
+#pragma unroll
+    for (int k = 0; k < kEdgeChunks; ++k) t += n2[k];
+    return t > 0.0 ? (float)(1.0 / sqrt(t)) : 0.0f;
+}
+
 // --------------------------------------------------------------------------
 // Pair sweep (graphs of degree <= 1, rank 1).  One CTA owns a block of rows of
 // BOTH ends of an edge (i<j) and reads each row of X_i and X_j once:
@@ -480,7 +491,6 @@ pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __re
     const int e = tile.worker;                       // edge index within the current round
     if (e >= tab_cur[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[tile.layer];
-    const int L = st.n_layers;
     const int wi = tab_cur[st.tab.off_edge_i + e], wj = tab_cur[st.tab.off_edge_j + e];
     const int pair = tab_cur[st.tab.off_pair + e];
     float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
@@ -490,7 +500,7 @@ pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __re
     // this edge's stored vector (unit length after scaling) and, per end, the
     // factors of the pending correction
     const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
-    const float qinv = st.Qinv[(long long)pair * L + tile.layer];
+    const float qinv = pair_qinv(st, pair, tile.layer);
     const float* ui = q;
     const float* uj = q;
     const float* phi = nullptr;
@@ -521,8 +531,8 @@ pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __re
     __syncthreads();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int r0 = tile.rtile * kPairTileRows;
-    const int r1 = min(g.n, r0 + kPairTileRows);
+    const int r0 = tile.rtile * g.p_rows;
+    const int r1 = min(g.n, r0 + g.p_rows);
     float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
     float4 u[NV];
 #pragma unroll
@@ -598,46 +608,240 @@ pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __re
     }
 }
 
+// --------------------------------------------------------------------------
+// Pair sweep for rows too long for one warp: a cluster of kPairCluster CTAs
+// shares every row.  CTA `rank` owns the columns [rank*slice, (rank+1)*slice):
+// it keeps that slice of the three vectors in shared memory for the whole tile
+// and its slice of the rows in flight in registers.  The row products
+// p_r = D_r . q-hat need all columns, so every CTA writes its share into the
+// shared memory of all CTAs of the cluster (distributed shared memory) and a
+// cluster barrier makes them visible; the shares are added in rank order, so
+// every CTA gets the same bits.  Each thread then adds p_r D_r to the columns it
+// owns: no reduction is needed for u.  The barrier is split (arrive ... wait)
+// and the loads of the next rows are issued in between.
+// --------------------------------------------------------------------------
+template <int NVW, bool UPDATE>
+__global__ void __cluster_dims__(kPairCluster, 1, 1) __launch_bounds__(256, 2)
+pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
+                       const Tile* __restrict__ tiles, int slice_pad) {
+    namespace cg = cooperative_groups;
+    extern __shared__ __align__(16) float s_vec[];               // q-hat, u_i, u_j slices
+    __shared__ float s_share[2][kPairCluster][kPairWideStep];    // [parity][rank][row]
+    __shared__ float s_warp[8][kPairWideStep];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+
+    const Tile tile = tiles[blockIdx.x / kPairCluster];
+    const int e = tile.worker;
+    if (e >= tab_cur[st.tab.off_n_edges]) return;                // the same for the whole cluster
+    const LayerGeom g = st.layers[tile.layer];
+    const int wi = tab_cur[st.tab.off_edge_i + e], wj = tab_cur[st.tab.off_edge_j + e];
+    const int pair = tab_cur[st.tab.off_pair + e];
+    float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
+    float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
+    const int ld = g.ld;
+    const int c_begin = rank * g.p_slice;
+    const int c_end = min(ld, c_begin + g.p_slice);
+
+    float* s_q = s_vec;
+    float* s_ui = s_vec + slice_pad;
+    float* s_uj = s_vec + 2 * slice_pad;
+    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float qinv = pair_qinv(st, pair, tile.layer);
+    const float* ui = q;
+    const float* uj = q;
+    const float* phi = nullptr;
+    const float* phj = nullptr;
+    float coef_i = 0.0f, coef_j = 0.0f;
+    if (UPDATE) {
+        if (tab_prev[st.tab.off_degree + wi] > 0) {
+            const int ep = tab_prev[st.tab.off_slot_edge + wi * st.tab.max_degree];
+            ui = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            phi = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            coef_i = __int_as_float(tab_prev[st.tab.off_slot_coef + wi * st.tab.max_degree]);
+        }
+        if (tab_prev[st.tab.off_degree + wj] > 0) {
+            const int ep = tab_prev[st.tab.off_slot_edge + wj * st.tab.max_degree];
+            uj = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            phj = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            coef_j = __int_as_float(tab_prev[st.tab.off_slot_coef + wj * st.tab.max_degree]);
+        }
+    }
+    for (int idx = threadIdx.x; idx < slice_pad; idx += 256) {
+        const int col = c_begin + idx;
+        const bool in = col < c_end;
+        s_q[idx] = in ? q[col] * qinv : 0.0f;
+        if (UPDATE) {
+            s_ui[idx] = in ? ui[col] : 0.0f;
+            s_uj[idx] = in ? uj[col] : 0.0f;
+        }
+    }
+    __syncthreads();
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = tile.rtile * g.p_rows;
+    const int r1 = min(g.n, r0 + g.p_rows);
+    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    constexpr int RS = kPairWideStep;
+    float4 u[NVW];
+#pragma unroll
+    for (int k = 0; k < NVW; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float ssum = 0.0f;
+
+    // rows r .. r+RS-1 of both ends, this CTA's slice; rows past the tile read as zero
+    float4 xi[RS][NVW], xj[RS][NVW];
+    auto load_rows = [&](int r) {
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            const bool in_row = r + t < r1;
+            const long long base = (long long)(in_row ? r + t : r1 - 1) * ld + c_begin;
+#pragma unroll
+            for (int k = 0; k < NVW; ++k) {
+                const int off = (k * 256 + threadIdx.x) * 4;
+                if (in_row && c_begin + off < c_end) {
+                    xi[t][k] = ld_stream(Xi + base + off);
+                    xj[t][k] = ld_stream(Xj + base + off);
+                } else {
+                    xi[t][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    xj[t][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+    };
+    load_rows(r0);
+    int it = 0;
+    for (int r = r0; r < r1; r += RS, ++it) {
+        float4 d[RS][NVW];        // this CTA's slice of RS rows of D
+        float dot[RS];
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            dot[t] = 0.0f;
+            const bool in_row = r + t < r1;
+            const long long base = (long long)(in_row ? r + t : r1 - 1) * ld + c_begin;
+            float ai = 0.0f, aj = 0.0f;
+            if (UPDATE && in_row) {
+                ai = phi ? coef_i * __ldg(phi + r + t) : 0.0f;
+                aj = phj ? coef_j * __ldg(phj + r + t) : 0.0f;
+            }
+#pragma unroll
+            for (int k = 0; k < NVW; ++k) {
+                const int off = (k * 256 + threadIdx.x) * 4;
+                const bool in = in_row && c_begin + off < c_end;
+                if (UPDATE && in) {
+                    const float4 vi = *reinterpret_cast<const float4*>(&s_ui[off]);
+                    const float4 vj = *reinterpret_cast<const float4*>(&s_uj[off]);
+                    xi[t][k].x = fmaf(-ai, vi.x, xi[t][k].x); xi[t][k].y = fmaf(-ai, vi.y, xi[t][k].y);
+                    xi[t][k].z = fmaf(-ai, vi.z, xi[t][k].z); xi[t][k].w = fmaf(-ai, vi.w, xi[t][k].w);
+                    xj[t][k].x = fmaf(-aj, vj.x, xj[t][k].x); xj[t][k].y = fmaf(-aj, vj.y, xj[t][k].y);
+                    xj[t][k].z = fmaf(-aj, vj.z, xj[t][k].z); xj[t][k].w = fmaf(-aj, vj.w, xj[t][k].w);
+                    st_stream(Xi + base + off, xi[t][k]);
+                    st_stream(Xj + base + off, xj[t][k]);
+                }
+                d[t][k].x = xi[t][k].x - xj[t][k].x; d[t][k].y = xi[t][k].y - xj[t][k].y;
+                d[t][k].z = xi[t][k].z - xj[t][k].z; d[t][k].w = xi[t][k].w - xj[t][k].w;
+                if (in) {
+                    const float4 vq = *reinterpret_cast<const float4*>(&s_q[off]);
+                    dot[t] = fmaf(d[t][k].x, vq.x, dot[t]); dot[t] = fmaf(d[t][k].y, vq.y, dot[t]);
+                    dot[t] = fmaf(d[t][k].z, vq.z, dot[t]); dot[t] = fmaf(d[t][k].w, vq.w, dot[t]);
+                }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            dot[t] = warp_sum(dot[t]);
+            if (lane == 0) s_warp[warp][t] = dot[t];
+        }
+        __syncthreads();
+        if (threadIdx.x < RS * kPairCluster) {
+            // thread (dst, t): this CTA's share of row t goes to CTA dst of the cluster
+            const int dst = threadIdx.x / RS, t = threadIdx.x % RS;
+            float share = 0.0f;
+#pragma unroll
+            for (int w8 = 0; w8 < 8; ++w8) share += s_warp[w8][t];
+            *cluster.map_shared_rank(&s_share[it & 1][rank][t], dst) = share;
+        }
+        // split cluster barrier: announce the shares, start the next rows' loads while the
+        // other CTAs catch up, then wait until all shares of these rows have landed
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        if (r + RS < r1) load_rows(r + RS);
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            float p = 0.0f;
+#pragma unroll
+            for (int rk = 0; rk < kPairCluster; ++rk) p += s_share[it & 1][rk][t];
+#pragma unroll
+            for (int k = 0; k < NVW; ++k) {
+                u[k].x = fmaf(p, d[t][k].x, u[k].x); u[k].y = fmaf(p, d[t][k].y, u[k].y);
+                u[k].z = fmaf(p, d[t][k].z, u[k].z); u[k].w = fmaf(p, d[t][k].w, u[k].w);
+            }
+            ssum = fmaf(p, p, ssum);
+            if (rank == 0 && threadIdx.x == 0 && r + t < r1) Pw[r + t] = p;
+        }
+    }
+    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld + c_begin;
+#pragma unroll
+    for (int k = 0; k < NVW; ++k) {
+        const int off = (k * 256 + threadIdx.x) * 4;
+        if (c_begin + off < c_end) *reinterpret_cast<float4*>(Up + off) = u[k];
+    }
+    if (rank == 0 && threadIdx.x == 0)
+        st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = (double)ssum;
+    cluster.sync();              // nobody leaves while a peer could still address its shared memory
+}
+
 // Pair edge step: ||p||^2 from the tiles' shares, p-hat = p / ||p|| in place,
-// Q' = (sum of the tiles' shares of D^T p) / ||p||, 1 / ||Q'||.  A zero or
-// non-finite norm leaves the stored vector alone and zeroes p-hat.
-// One CTA per (edge, layer).
-__global__ void __launch_bounds__(512)
+// Q' = (sum of the tiles' shares of D^T p) / ||p||, and the shares of ||Q'||^2
+// (the sweep that uses Q' next adds them up).  A zero or non-finite norm leaves
+// the stored vector alone and zeroes p-hat.  kEdgeChunks CTAs per (edge, layer),
+// each taking a slice of the rows and of the columns.
+__global__ void __launch_bounds__(256)
 pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     __shared__ double scratch[33];
     const int L = st.n_layers;
-    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
+    const int chunk = blockIdx.x % kEdgeChunks;
+    const int el = blockIdx.x / kEdgeChunks;
+    const int e = el / L, l = el - e * L;
     if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
     if (!g.pair_mode) return;
     const int pair = tab[st.tab.off_pair + e];
     const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
-    double nn = 0.0;
-    for (int t = 0; t < g.p_rtiles; ++t) nn += sp[t];
+    double part = 0.0;
+    for (int t = threadIdx.x; t < g.p_rtiles; t += blockDim.x) part += sp[t];
+    const double nn = block_sum(part, scratch);      // same order, hence same bits, in every chunk
     const bool finite = isfinite(nn);
     const bool live = finite && nn > 0.0;
     const double inv = live ? 1.0 / sqrt(nn) : 0.0;
     float* P = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
-    for (int r = threadIdx.x; r < g.npad; r += blockDim.x)
+    const int rw = (g.npad + kEdgeChunks - 1) / kEdgeChunks;
+    for (int r = chunk * rw + threadIdx.x; r < min(g.npad, (chunk + 1) * rw); r += blockDim.x)
         P[r] = (live && r < g.n) ? (float)((double)P[r] * inv) : 0.0f;
-    if (threadIdx.x == 0) {
+    if (chunk == 0 && threadIdx.x == 0) {
         st.live[(long long)e * L + l] = live ? 1 : 0;
         if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
     }
     if (!live) return;   // uniform over the block
     const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
     float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
-    double part = 0.0;
-    for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
+    const int cw = (g.m + kEdgeChunks - 1) / kEdgeChunks;
+    part = 0.0;
+    for (int c = chunk * cw + threadIdx.x; c < min(g.m, (chunk + 1) * cw); c += blockDim.x) {
         double a = 0.0;
-        for (int t = 0; t < g.p_rtiles; ++t) a += (double)up[(long long)t * g.ld + c];
+        for (int t = 0; t < g.p_rtiles; t += 8) {        // eight independent loads, added in tile order
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = t + j < g.p_rtiles ? up[(long long)(t + j) * g.ld + c] : 0.0f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a += (double)v[j];
+        }
         const float q = (float)(a * inv);
         Q[c] = q;
         part += (double)q * (double)q;
     }
     const double qq = block_sum(part, scratch);
     if (threadIdx.x == 0) {
-        st.Qinv[(long long)pair * L + l] = qq > 0.0 ? (float)(1.0 / sqrt(qq)) : 0.0f;
+        st.Qn2[((long long)pair * L + l) * kEdgeChunks + chunk] = qq;
         if (!isfinite(qq)) atomicOr(st.status, 1 << kStatusNumeric);
     }
 }
@@ -659,8 +863,14 @@ column_norms_kernel(DevState st) {
             part += q * q;
         }
         const double nn = block_sum(part, scratch);
-        if (threadIdx.x == 0)
+        if (threadIdx.x == 0) {
             st.Qinv[(pair * L + l) * rank + k] = nn > 0.0 ? (float)(1.0 / sqrt(nn)) : 0.0f;
+            if (k == 0) {   // the pair sweep reads the squared norm as kEdgeChunks shares
+                double* n2 = st.Qn2 + (pair * L + l) * kEdgeChunks;
+                n2[0] = nn;
+                for (int t = 1; t < kEdgeChunks; ++t) n2[t] = 0.0;
+            }
+        }
     }
 }
 
@@ -725,8 +935,88 @@ cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int
                          : launch_pair<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
 }
 
+template <int NVW>
+static cudaError_t launch_wide(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd,
+                               const Tile* tiles, int n_tiles, int slice_pad, cudaStream_t stream) {
+    const size_t smem = sizeof(float) * 3 * static_cast<size_t>(slice_pad);
+    const dim3 grid(static_cast<unsigned>(n_tiles) * kPairCluster);
+    cudaError_t rc = cudaSuccess;
+    if (upd) {
+        if (smem > 48 * 1024)
+            rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (rc != cudaSuccess) return rc;
+        pair_sweep_wide_kernel<NVW, true><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
+    } else {
+        if (smem > 48 * 1024)
+            rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (rc != cudaSuccess) return rc;
+        pair_sweep_wide_kernel<NVW, false><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
+    }
+    return cudaGetLastError();
+}
+
+// `tiles`: cluster tiles of layers with the same float4 count per thread `nv` and
+// the same slice width `slice` (columns per CTA).
+cudaError_t launch_pair_sweep_wide(const DevState& st, const int* tab_prev, const int* tab_cur,
+                                   bool apply_pending, const Tile* tiles, int n_tiles, int nv, int slice,
+                                   cudaStream_t stream) {
+    if (n_tiles <= 0) return cudaSuccess;
+    const int slice_pad = (slice + 3) / 4 * 4;
+    switch (nv) {
+        case 1: return launch_wide<1>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        case 2: return launch_wide<2>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        case 3: return launch_wide<3>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        case 4: return launch_wide<4>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        case 5: return launch_wide<5>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        case 6: return launch_wide<6>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        case 7: return launch_wide<7>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        default: return launch_wide<8>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+    }
+}
+
+template <int NVW>
+static int resident_clusters(int slice_pad) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kPairCluster * 1024);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = sizeof(float) * 3 * static_cast<size_t>(slice_pad);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kPairCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cfg.dynamicSmemBytes > 48 * 1024 &&
+        cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)cfg.dynamicSmemBytes) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (cudaOccupancyMaxActiveClusters(&n, pair_sweep_wide_kernel<NVW, true>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
+int pair_wide_resident_clusters(int nv, int slice) {
+    const int slice_pad = (slice + 3) / 4 * 4;
+    switch (nv) {
+        case 1: return resident_clusters<1>(slice_pad);
+        case 2: return resident_clusters<2>(slice_pad);
+        case 3: return resident_clusters<3>(slice_pad);
+        case 4: return resident_clusters<4>(slice_pad);
+        case 5: return resident_clusters<5>(slice_pad);
+        case 6: return resident_clusters<6>(slice_pad);
+        case 7: return resident_clusters<7>(slice_pad);
+        default: return resident_clusters<8>(slice_pad);
+    }
+}
+
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
-    pair_edge_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    pair_edge_kernel<<<max_edges * st.n_layers * kEdgeChunks, 256, 0, stream>>>(st, tab);
     return cudaGetLastError();
 }
 
