@@ -23,7 +23,13 @@ constexpr int kPairMaxLd = 1024;       // widest row a warp of the pair sweep ke
 constexpr int kPairCluster = 8;        // CTAs that share a row of a wider layer (thread-block cluster)
 constexpr int kPairWideRows = 32;      // rows per cluster tile of a wider layer when residency is unknown
 constexpr int kPairWideMaxTiles = 32;  // most row tiles per (edge, wide layer); sizes the partial-sum buffer
-constexpr int kPairWideStep = 2;       // rows a cluster handles between two barriers
+#ifndef PG_WIDE_STEP
+#define PG_WIDE_STEP 1
+#endif
+#ifndef PG_WIDE_MIN_BLOCKS
+#define PG_WIDE_MIN_BLOCKS 3
+#endif
+constexpr int kPairWideStep = PG_WIDE_STEP;  // rows a cluster handles between two barriers
 constexpr int kPairWideMaxLd = 8 * 256 * 4 * kPairCluster;  // widest row the cluster variant covers
 constexpr int kEdgeChunks = 32;        // CTAs that share the pair edge step of one (edge, layer)
 

@@ -621,7 +621,7 @@ pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __re
 // and the loads of the next rows are issued in between.
 // --------------------------------------------------------------------------
 template <int NVW, bool UPDATE>
-__global__ void __cluster_dims__(kPairCluster, 1, 1) __launch_bounds__(256, 2)
+__global__ void __cluster_dims__(kPairCluster, 1, 1) __launch_bounds__(256, PG_WIDE_MIN_BLOCKS)
 pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles, int slice_pad) {
     namespace cg = cooperative_groups;
