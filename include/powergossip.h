@@ -161,6 +161,27 @@ PG_API int pg_read_params(pg_ctx *ctx, int32_t worker, int32_t layer, float *hos
  */
 PG_API int pg_round(pg_ctx *ctx, void *stream);
 
+/*
+ * Enqueue `n_rounds` rounds (same result as calling pg_round that many times).
+ * When the graph is static and the whole stack is small enough to stay in L2
+ * (at most 64 MiB of parameters, degree > 1 or rank > 1), all rounds run in ONE
+ * cooperative kernel launch whose phases are separated by a grid barrier; the
+ * barrier waits are bounded, and a wait that runs out ends the launch and sets
+ * PG_ERR_TIMEOUT in the device status word.  Otherwise the rounds are enqueued
+ * one by one.  Per-kernel timing (pg_timing_enable) forces the latter.
+ */
+PG_API int pg_rounds(pg_ctx *ctx, int32_t n_rounds, void *stream);
+
+/*
+ * Self-test of the bounded grid barrier (the paper has no counterpart): launches
+ * a few CTAs on a barrier that expects one arrival more than will come.  Every
+ * CTA must give up after about a millisecond; the call waits for `stream` and
+ * returns PG_ERR_TIMEOUT when that happened (the expected outcome), PG_OK if the
+ * wait was not reported.  The status word keeps the time-out bit afterwards:
+ * use a context of its own.
+ */
+PG_API int pg_selftest_barrier_timeout(pg_ctx *ctx, void *stream);
+
 /* Wait for `stream` and return the device status word (PG_OK or PG_ERR_NUMERIC). */
 PG_API int pg_device_status(pg_ctx *ctx, void *stream);
 

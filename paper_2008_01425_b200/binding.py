@@ -26,7 +26,7 @@ EXPORTS = (
     "pg_round", "pg_device_status", "pg_get_schedule", "pg_max_edges", "pg_read_q", "pg_write_q",
     "pg_get_round", "pg_set_round", "pg_kernel_launches", "pg_status_string",
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
-    "pg_transposed_product_noalloc",
+    "pg_transposed_product_noalloc", "pg_rounds", "pg_selftest_barrier_timeout",
 )
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
                 "pair_sweep", "pair_edge", "update_only")
@@ -72,6 +72,8 @@ def load_library() -> ctypes.CDLL:
     L.pg_read_params.argtypes = [vp, i32, i32, vp, vp]
     L.pg_round.argtypes = [vp, vp]
     L.pg_device_status.argtypes = [vp, vp]
+    L.pg_rounds.argtypes = [vp, i32, vp]
+    L.pg_selftest_barrier_timeout.argtypes = [vp, vp]
     L.pg_get_schedule.argtypes = [vp, i64, vp, vp, ctypes.POINTER(i32)]
     L.pg_max_edges.argtypes = [vp, ctypes.POINTER(i32)]
     L.pg_read_q.argtypes = [vp, i32, i32, i32, vp, vp]
@@ -261,6 +263,12 @@ class PowerGossip:
     # -- rounds -----------------------------------------------------------
     def pg_round(self, stream=None) -> None:
         _check(self._lib.pg_round(self._h, _stream_handle(stream)), "pg_round")
+
+    def pg_rounds(self, n_rounds: int, stream=None) -> None:
+        _check(self._lib.pg_rounds(self._h, int(n_rounds), _stream_handle(stream)), "pg_rounds")
+
+    def pg_selftest_barrier_timeout(self, stream=None) -> int:
+        return int(self._lib.pg_selftest_barrier_timeout(self._h, _stream_handle(stream)))
 
     def pg_device_status(self, stream=None) -> int:
         return int(self._lib.pg_device_status(self._h, _stream_handle(stream)))

@@ -221,7 +221,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_Sp = take(sizeof(double) * static_cast<size_t>(lay.max_edges) * lay.sp_stride);
     lay.off_Z = take(sizeof(float) * static_cast<size_t>(N) * lay.z_stride);
     lay.off_live = take(sizeof(int) * static_cast<size_t>(lay.max_edges) * n_layers * rank);
-    lay.off_status = take(sizeof(int) * 64);
+    lay.off_status = take(sizeof(int) * 64);   // [0] status word, [16..17] grid barrier of the persistent kernel
     lay.off_layers = take(sizeof(LayerGeom) * static_cast<size_t>(n_layers));
     lay.off_tabs = take(sizeof(int) * static_cast<size_t>(kTabRing) * t.total_ints);
     lay.off_row_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_row_tiles));
@@ -262,6 +262,7 @@ struct pg_ctx {
     Tile* d_row_tiles = nullptr;
     Tile* d_col_tiles = nullptr;
     bool static_graph = true;
+    bool coop_ok = false;       // the device supports cooperative launches
     int device = 0;
     // optional per-kernel timing: one event pair per launch while enabled
     bool timing = false;
@@ -459,6 +460,10 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     c->power_steps = power_steps;
     c->n_layers = n_layers;
     c->static_graph = c->topo.kind != PG_MATCHING;
+    {
+        int coop = 0;
+        c->coop_ok = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) == cudaSuccess && coop != 0;
+    }
     for (int l = 0; l < n_layers; ++l) {
         const double b = 4.0 * c->topo.n_workers * static_cast<double>(c->lay.layers[l].n) * c->lay.layers[l].m;
         (c->lay.layers[l].pair_mode ? c->pair_param_bytes : c->normal_param_bytes) += b;
@@ -729,6 +734,57 @@ int pg_round(pg_ctx* c, void* stream_v) {
     c->y_valid = true;
     c->round += 1;
     return PG_OK;
+}
+
+int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
+    if (!c || n_rounds < 0) return PG_ERR_INVALID;
+    if (n_rounds == 0) return PG_OK;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    // One cooperative launch when the graph is static, no layer uses the pair sweep and the
+    // whole stack stays in L2; otherwise the rounds are enqueued one by one.
+    const double x_bytes = c->normal_param_bytes;
+    const bool persistent = c->static_graph && c->lay.n_pair_tiles == 0 && c->coop_ok &&
+                            x_bytes <= 64.0 * 1024 * 1024 && !c->timing;
+    if (!persistent) {
+        for (int r = 0; r < n_rounds; ++r) {
+            const int rc = pg_round(c, stream_v);
+            if (rc != PG_OK) return rc;
+        }
+        return PG_OK;
+    }
+    const int* tab = nullptr;
+    int rc = ensure_table(c, c->round, stream, &tab);
+    if (rc != PG_OK) return rc;
+    DevState st = c->st;
+    st.Ph = c->ph_buf[0];
+    const long long steps = static_cast<long long>(n_rounds) * c->power_steps;
+    if (steps > INT_MAX) return PG_ERR_INVALID;
+    int* bar = c->st.status + 16;
+    if (pg::launch_persistent(st, tab, c->d_row_tiles, static_cast<int>(c->lay.n_row_tiles), c->d_col_tiles,
+                              static_cast<int>(c->lay.n_col_tiles), static_cast<int>(steps), !c->y_valid, bar,
+                              stream) != cudaSuccess) {
+        cudaGetLastError();
+        c->y_valid = false;
+        return PG_ERR_CUDA;
+    }
+    c->launches += 1;
+    c->y_valid = true;
+    c->step += steps;
+    c->round += n_rounds;
+    return PG_OK;
+}
+
+int pg_selftest_barrier_timeout(pg_ctx* c, void* stream_v) {
+    if (!c) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    if (pg::launch_barrier_timeout_probe(c->st.status + 16, c->st.status, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return PG_ERR_CUDA;
+    }
+    c->launches += 1;
+    return device_status(c, stream);
 }
 
 int pg_max_edges(pg_ctx* c, int32_t* max_edges_out) {

@@ -124,6 +124,11 @@ cudaError_t launch_pair_sweep_wide(const DevState& st, const int* tab_prev, cons
 // Clusters of the wide pair sweep that can be resident at once (0 if unknown).
 int pair_wide_resident_clusters(int nv, int slice);
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
+// One cooperative launch for `n_steps` power steps of a static graph (small stacks).
+cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* row_tiles, int n_rows,
+                              const Tile* col_tiles, int n_cols, int n_steps, bool forward_first, int* bar,
+                              cudaStream_t stream);
+cudaError_t launch_barrier_timeout_probe(int* bar, int* status, cudaStream_t stream);
 cudaError_t launch_column_norms(const DevState& st, long long n_pairs, cudaStream_t stream);
 
 }  // namespace pg

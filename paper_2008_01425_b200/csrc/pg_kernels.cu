@@ -19,6 +19,7 @@ namespace pg {
 namespace {
 
 constexpr int kStatusNumeric = 6;  // PG_ERR_NUMERIC
+constexpr long long kBarrierSpinLimit = 1LL << 23;   // polls before a grid barrier gives up (a few seconds)
 
 // Rows a warp of the row sweep works on at once, per number of vectors S.
 #ifndef PG_RT1
@@ -52,8 +53,26 @@ __device__ __forceinline__ void st_stream(float* p, const float4& v) {
                  : "memory");
 }
 
+// Vector / scalar loads of data that other CTAs produce.  In the multi-launch
+// path a kernel boundary separates producer and consumer, so the read-only
+// (L1-cached) path is fine.  COH = true is for the persistent kernel, where
+// producer and consumer run in the same launch: those loads go past L1.
+template <bool COH>
 __device__ __forceinline__ float4 ld_vec(const float* p) {
-    return __ldg(reinterpret_cast<const float4*>(p));
+    return COH ? __ldcg(reinterpret_cast<const float4*>(p)) : __ldg(reinterpret_cast<const float4*>(p));
+}
+template <bool COH>
+__device__ __forceinline__ float ld_f(const float* p) {
+    return COH ? __ldcg(p) : __ldg(p);
+}
+// Data the running kernel itself wrote earlier (never the read-only path).
+template <bool COH>
+__device__ __forceinline__ float ld_own(const float* p) {
+    return COH ? __ldcg(p) : *p;
+}
+template <bool COH>
+__device__ __forceinline__ int ld_i(const int* p) {
+    return COH ? __ldcg(p) : *p;
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -87,22 +106,24 @@ __device__ double block_sum(double v, double* scratch /* >= 33 doubles of shared
 // --------------------------------------------------------------------------
 // SAME: update and forward use the same vectors (Q' of this step is the next
 // step's q, as on a static graph), so each is loaded once.
-template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT>
-__global__ void __launch_bounds__(256, PG_ROW_MIN_BLOCKS)
-row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
-                 const Tile* __restrict__ tiles) {
-    const Tile tile = tiles[blockIdx.x];
+template <int S>
+struct RowShared {
+    const float* uq[S];
+    const float* up[S];
+    float uc[S];
+    const float* fq[S];
+    float fs[S];
+    int nu, nf;
+};
+
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH>
+__device__ __forceinline__ void row_tile(const DevState& st, const int* __restrict__ tab_u,
+                                         const int* __restrict__ tab_f, const Tile tile,
+                                         RowShared<S>& sh) {
     const LayerGeom g = st.layers[tile.layer];
     const int w = tile.worker;
     const int rank = st.rank;
     float* __restrict__ X = st.X + (long long)w * st.x_stride + g.x_off;
-
-    __shared__ const float* s_uq[S];
-    __shared__ const float* s_up[S];
-    __shared__ float s_uc[S];
-    __shared__ const float* s_fq[S];
-    __shared__ float s_fs[S];
-    __shared__ int s_nu, s_nf;
 
     if (threadIdx.x < S) {
         const int v = threadIdx.x;
@@ -112,26 +133,26 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
             if (slot < deg) {
                 const int e = tab_u[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
                 const int pair = tab_u[st.tab.off_pair + e];
-                s_uq[v] = st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld;
-                s_up[v] = st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad;
-                s_uc[v] = __int_as_float(tab_u[st.tab.off_slot_coef + w * st.tab.max_degree + slot]);
+                sh.uq[v] = st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld;
+                sh.up[v] = st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad;
+                sh.uc[v] = __int_as_float(tab_u[st.tab.off_slot_coef + w * st.tab.max_degree + slot]);
             }
-            if (v == 0) s_nu = deg * rank;
+            if (v == 0) sh.nu = deg * rank;
         }
         if (FORWARD) {
             const int deg = tab_f[st.tab.off_degree + w];
             if (slot < deg) {
                 const int e = tab_f[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
                 const int pair = tab_f[st.tab.off_pair + e];
-                s_fq[v] = st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld;
-                s_fs[v] = st.Qinv[((long long)pair * st.n_layers + tile.layer) * rank + k];
+                sh.fq[v] = st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld;
+                sh.fs[v] = ld_f<COH>(&st.Qinv[((long long)pair * st.n_layers + tile.layer) * rank + k]);
             }
-            if (v == 0) s_nf = deg * rank;
+            if (v == 0) sh.nf = deg * rank;
         }
     }
     __syncthreads();
-    const int nu = UPDATE ? s_nu : 0;
-    const int nf = FORWARD ? s_nf : 0;
+    const int nu = UPDATE ? sh.nu : 0;
+    const int nf = FORWARD ? sh.nf : 0;
 
     const int r0 = tile.rtile * g.f_rows;
     const int r1 = min(g.n, r0 + g.f_rows);
@@ -152,7 +173,7 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
             for (int v = 0; v < S; ++v) {
                 acc[t][v] = 0.0f;
                 a[t][v] = 0.0f;
-                if (UPDATE && v < nu && rb + t < r1) a[t][v] = s_uc[v] * __ldg(s_up[v] + r);
+                if (UPDATE && v < nu && rb + t < r1) a[t][v] = sh.uc[v] * ld_f<COH>(sh.up[v] + r);
             }
         }
         for (int c = c0 + lane * 4; c < c1; c += 128) {
@@ -165,7 +186,7 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nu) {
-                        q[v] = ld_vec(s_uq[v] + c);
+                        q[v] = ld_vec<COH>(sh.uq[v] + c);
 #pragma unroll
                         for (int t = 0; t < RT; ++t) {
                             x[t].x = fmaf(-a[t][v], q[v].x, x[t].x);
@@ -194,7 +215,7 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nu) {
-                        const float4 q = ld_vec(s_uq[v] + c);
+                        const float4 q = ld_vec<COH>(sh.uq[v] + c);
 #pragma unroll
                         for (int t = 0; t < RT; ++t) {
                             x[t].x = fmaf(-a[t][v], q.x, x[t].x);
@@ -212,7 +233,7 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nf) {
-                        const float4 q = ld_vec(s_fq[v] + c);
+                        const float4 q = ld_vec<COH>(sh.fq[v] + c);
 #pragma unroll
                         for (int t = 0; t < RT; ++t) {
                             acc[t][v] = fmaf(x[t].x, q.x, acc[t][v]);
@@ -233,7 +254,7 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
                     for (int t = 0; t < RT; ++t) {
                         const float s = warp_sum(acc[t][v]);
                         if (lane == 0 && rb + t < r1)
-                            Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * s_fs[v];
+                            Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * sh.fs[v];
                     }
                 }
             }
@@ -241,21 +262,32 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
     }
 }
 
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT>
+__global__ void __launch_bounds__(256, PG_ROW_MIN_BLOCKS)
+row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
+                 const Tile* __restrict__ tiles) {
+    __shared__ RowShared<S> sh;
+    row_tile<S, UPDATE, FORWARD, SAME, RT, false>(st, tab_u, tab_f, tiles[blockIdx.x], sh);
+}
+
 // --------------------------------------------------------------------------
 // Transposed sweep: Z[w][v][c] = sum_r Ph_v[r] X_w[r][c] over one row tile.
 // 64 threads across (a float4 of columns each), 4 row groups down.
 // --------------------------------------------------------------------------
 template <int S>
-__global__ void __launch_bounds__(256)
-col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles) {
-    const Tile tile = tiles[blockIdx.x];
+struct ColShared {
+    float p[S][kColTileRowsMax];
+    float4 red[3][S][64];
+};
+
+template <int S, bool COH>
+__device__ __forceinline__ void col_tile(const DevState& st, const int* __restrict__ tab, const Tile tile,
+                                         ColShared<S>& sh) {
     const LayerGeom g = st.layers[tile.layer];
     const int w = tile.worker;
     const int rank = st.rank;
     const float* __restrict__ X = st.X + (long long)w * st.x_stride + g.x_off;
 
-    __shared__ float s_p[S][kColTileRowsMax];
-    __shared__ float4 s_red[3][S][64];
 
     const int r0 = tile.rtile * g.t_rows;
     const int r1 = min(g.n, r0 + g.t_rows);
@@ -268,9 +300,9 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
         if (v < nv && r0 + rr < r1) {
             const int slot = v / rank, k = v - slot * rank;
             const int e = tab[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
-            val = __ldg(st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad + r0 + rr);
+            val = ld_f<COH>(st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad + r0 + rr);
         }
-        s_p[v][rr] = val;
+        sh.p[v][rr] = val;
     }
     __syncthreads();
 
@@ -298,7 +330,7 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nv) {
-                        const float p = in ? s_p[v][ro] : 0.0f;
+                        const float p = in ? sh.p[v][ro] : 0.0f;
                         acc[v].x = fmaf(p, x[u].x, acc[v].x);
                         acc[v].y = fmaf(p, x[u].y, acc[v].y);
                         acc[v].z = fmaf(p, x[u].z, acc[v].z);
@@ -310,7 +342,7 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
     }
     if (ty > 0) {
 #pragma unroll
-        for (int v = 0; v < S; ++v) s_red[ty - 1][v][tx] = acc[v];
+        for (int v = 0; v < S; ++v) sh.red[ty - 1][v][tx] = acc[v];
     }
     __syncthreads();
     if (ty == 0 && c < ld) {
@@ -321,7 +353,7 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
                 float4 s = acc[v];
 #pragma unroll
                 for (int t = 0; t < 3; ++t) {
-                    const float4 o = s_red[t][v][tx];
+                    const float4 o = sh.red[t][v][tx];
                     s.x += o.x; s.y += o.y; s.z += o.z; s.w += o.w;
                 }
                 *reinterpret_cast<float4*>(Z + ((long long)v * g.t_rtiles + tile.rtile) * ld + c) = s;
@@ -330,18 +362,23 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
     }
 }
 
+template <int S>
+__global__ void __launch_bounds__(256)
+col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles) {
+    __shared__ ColShared<S> sh;
+    col_tile<S, false>(st, tab, tiles[blockIdx.x], sh);
+}
+
 // --------------------------------------------------------------------------
 // Edge step, left factor: P = Y[i] - Y[j] (partials added in order, fp64),
 // modified Gram-Schmidt in column order, P-hat stored as fp32.
 // One CTA per (edge, layer).
 // --------------------------------------------------------------------------
-__global__ void __launch_bounds__(512)
-edge_left_kernel(DevState st, const int* __restrict__ tab) {
-    int* __restrict__ live_out = st.live;
-    __shared__ double scratch[33];
+template <bool COH>
+__device__ __forceinline__ void edge_left_step(const DevState& st, const int* __restrict__ tab, int e, int l,
+                                               double* scratch) {
+    int* live_out = st.live;
     const int L = st.n_layers, rank = st.rank;
-    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
-    if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
     if (g.pair_mode) return;   // handled by the pair sweep's own edge step
     const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
@@ -359,8 +396,8 @@ edge_left_kernel(DevState st, const int* __restrict__ tab) {
         auto raw = [&](int r) {
             double a = 0.0, b = 0.0;
             for (int cs = 0; cs < g.f_csplit; ++cs) {
-                a += (double)yi[(long long)cs * g.npad + r];
-                b += (double)yj[(long long)cs * g.npad + r];
+                a += (double)ld_f<COH>(yi + (long long)cs * g.npad + r);
+                b += (double)ld_f<COH>(yj + (long long)cs * g.npad + r);
             }
             return a - b;
         };
@@ -375,8 +412,8 @@ edge_left_kernel(DevState st, const int* __restrict__ tab) {
             part = 0.0;
             for (int r = threadIdx.x; r < g.n; r += blockDim.x) {
                 double v = raw(r);
-                for (int h2 = 0; h2 < h; ++h2) v -= coef[h2] * (double)Ph[(long long)h2 * g.npad + r];
-                part += v * (double)Ph[(long long)h * g.npad + r];
+                for (int h2 = 0; h2 < h; ++h2) v -= coef[h2] * (double)ld_own<COH>(Ph + (long long)h2 * g.npad + r);
+                part += v * (double)ld_own<COH>(Ph + (long long)h * g.npad + r);
             }
             coef[h] = block_sum(part, scratch);
         }
@@ -385,7 +422,7 @@ edge_left_kernel(DevState st, const int* __restrict__ tab) {
             part = 0.0;
             for (int r = threadIdx.x; r < g.n; r += blockDim.x) {
                 double v = raw(r);
-                for (int h = 0; h < k; ++h) v -= coef[h] * (double)Ph[(long long)h * g.npad + r];
+                for (int h = 0; h < k; ++h) v -= coef[h] * (double)ld_own<COH>(Ph + (long long)h * g.npad + r);
                 part += v * v;
             }
             nn = block_sum(part, scratch);
@@ -398,7 +435,7 @@ edge_left_kernel(DevState st, const int* __restrict__ tab) {
             double v = 0.0;
             if (live && r < g.n) {
                 v = raw(r);
-                for (int h = 0; h < k; ++h) v -= coef[h] * (double)Ph[(long long)h * g.npad + r];
+                for (int h = 0; h < k; ++h) v -= coef[h] * (double)ld_own<COH>(Ph + (long long)h * g.npad + r);
                 v *= inv;
             }
             Ph[(long long)k * g.npad + r] = (float)v;
@@ -412,18 +449,24 @@ edge_left_kernel(DevState st, const int* __restrict__ tab) {
     (void)pair;
 }
 
+__global__ void __launch_bounds__(512)
+edge_left_kernel(DevState st, const int* __restrict__ tab) {
+    __shared__ double scratch[33];
+    const int e = blockIdx.x / st.n_layers, l = blockIdx.x - e * st.n_layers;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    edge_left_step<false>(st, tab, e, l, scratch);
+}
+
 // --------------------------------------------------------------------------
 // Edge step, right factor: Q' = Z[i] - Z[j] (row-tile partials added in order,
 // fp64), stored as the pair's new Q with 1/||Q'||.  Degenerate columns keep
 // their old vector.  One CTA per (edge, layer).
 // --------------------------------------------------------------------------
-__global__ void __launch_bounds__(512)
-edge_right_kernel(DevState st, const int* __restrict__ tab) {
-    const int* __restrict__ live_in = st.live;
-    __shared__ double scratch[33];
+template <bool COH>
+__device__ __forceinline__ void edge_right_step(const DevState& st, const int* __restrict__ tab, int e, int l,
+                                                double* scratch) {
+    const int* live_in = st.live;
     const int L = st.n_layers, rank = st.rank;
-    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
-    if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
     if (g.pair_mode) return;
     const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
@@ -434,15 +477,24 @@ edge_right_kernel(DevState st, const int* __restrict__ tab) {
     float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
 
     for (int k = 0; k < rank; ++k) {
-        if (!live_in[((long long)e * L + l) * rank + k]) continue;  // uniform over the block
+        if (!ld_i<COH>(&live_in[((long long)e * L + l) * rank + k])) continue;  // uniform over the block
         const float* zi = Zi + (long long)(si * rank + k) * g.t_rtiles * g.ld;
         const float* zj = Zj + (long long)(sj * rank + k) * g.t_rtiles * g.ld;
         double part = 0.0;
         for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
             double a = 0.0, b = 0.0;
-            for (int rt = 0; rt < g.t_rtiles; ++rt) {
-                a += (double)zi[(long long)rt * g.ld + c];
-                b += (double)zj[(long long)rt * g.ld + c];
+            for (int rt = 0; rt < g.t_rtiles; rt += 4) {     // eight independent loads, added in tile order
+                float va[4], vb[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    va[t] = rt + t < g.t_rtiles ? ld_f<COH>(zi + (long long)(rt + t) * g.ld + c) : 0.0f;
+                    vb[t] = rt + t < g.t_rtiles ? ld_f<COH>(zj + (long long)(rt + t) * g.ld + c) : 0.0f;
+                }
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    a += (double)va[t];
+                    b += (double)vb[t];
+                }
             }
             const float q = (float)(a - b);
             Q[(long long)k * g.ld + c] = q;
@@ -454,6 +506,14 @@ edge_right_kernel(DevState st, const int* __restrict__ tab) {
             if (!isfinite(nn)) atomicOr(st.status, 1 << kStatusNumeric);
         }
     }
+}
+
+__global__ void __launch_bounds__(512)
+edge_right_kernel(DevState st, const int* __restrict__ tab) {
+    __shared__ double scratch[33];
+    const int e = blockIdx.x / st.n_layers, l = blockIdx.x - e * st.n_layers;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    edge_right_step<false>(st, tab, e, l, scratch);
 }
 
 // 1 / ||Q|| of a pair-sweep layer from the shares the pair edge step left.
@@ -874,6 +934,92 @@ column_norms_kernel(DevState st) {
     }
 }
 
+// --------------------------------------------------------------------------
+// Persistent rounds for small stacks (everything stays in L2): one cooperative
+// launch runs any number of power steps.  The four phases of a step are
+// separated by a grid barrier instead of a kernel boundary.  The barrier is a
+// counter plus a generation word in global memory; a CTA that waits gives up
+// after `spin_limit` polls, raises the time-out bit of the status word and
+// leaves, so a launch can never hang the device.
+// --------------------------------------------------------------------------
+constexpr int kStatusTimeout = 5;  // PG_ERR_TIMEOUT
+
+__device__ bool grid_barrier(int* bar, int expected_blocks, int* status, long long spin_limit, int* s_ok) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ok = 1;
+        __threadfence();                                  // this CTA's results are out before it is counted
+        volatile int* gen_word = bar + 1;
+        const int gen = *gen_word;
+        if (atomicAdd(&bar[0], 1) == expected_blocks - 1) {
+            atomicExch(&bar[0], 0);
+            __threadfence();
+            atomicAdd(&bar[1], 1);                        // release the others
+        } else {
+            long long spins = 0;
+            while (*gen_word == gen) {                    // bounded: a few seconds at most
+                if (++spins > spin_limit) {
+                    atomicOr(status, 1 << kStatusTimeout);
+                    ok = 0;
+                    break;
+                }
+            }
+        }
+        __threadfence();
+        *s_ok = ok;
+    }
+    __syncthreads();
+    return *s_ok != 0;
+}
+
+template <int S, int RT>
+__global__ void __launch_bounds__(256, 2)
+persistent_rounds_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ row_tiles,
+                         int n_rows, const Tile* __restrict__ col_tiles, int n_cols, int n_steps,
+                         int forward_first, int* bar, int expected_blocks, long long spin_limit) {
+    constexpr size_t kBytes = sizeof(ColShared<S>) > sizeof(RowShared<S>) ? sizeof(ColShared<S>) : sizeof(RowShared<S>);
+    __shared__ __align__(16) unsigned char s_raw[kBytes];
+    __shared__ double scratch[33];
+    __shared__ int s_ok;
+    RowShared<S>& rsh = *reinterpret_cast<RowShared<S>*>(s_raw);
+    ColShared<S>& csh = *reinterpret_cast<ColShared<S>*>(s_raw);
+    const int nb = gridDim.x;
+    const int L = st.n_layers;
+    const int n_items = tab[st.tab.off_n_edges] * L;
+
+    if (forward_first) {
+        for (int t = blockIdx.x; t < n_rows; t += nb) {
+            row_tile<S, false, true, false, RT, true>(st, tab, tab, row_tiles[t], rsh);
+            __syncthreads();
+        }
+        if (!grid_barrier(bar, expected_blocks, st.status, spin_limit, &s_ok)) return;
+    }
+    for (int step = 0; step < n_steps; ++step) {
+        for (int it = blockIdx.x; it < n_items; it += nb) edge_left_step<true>(st, tab, it / L, it % L, scratch);
+        if (!grid_barrier(bar, expected_blocks, st.status, spin_limit, &s_ok)) return;
+        for (int t = blockIdx.x; t < n_cols; t += nb) {
+            col_tile<S, true>(st, tab, col_tiles[t], csh);
+            __syncthreads();
+        }
+        if (!grid_barrier(bar, expected_blocks, st.status, spin_limit, &s_ok)) return;
+        for (int it = blockIdx.x; it < n_items; it += nb) edge_right_step<true>(st, tab, it / L, it % L, scratch);
+        if (!grid_barrier(bar, expected_blocks, st.status, spin_limit, &s_ok)) return;
+        for (int t = blockIdx.x; t < n_rows; t += nb) {
+            row_tile<S, true, true, true, RT, true>(st, tab, tab, row_tiles[t], rsh);
+            __syncthreads();
+        }
+        if (step + 1 < n_steps && !grid_barrier(bar, expected_blocks, st.status, spin_limit, &s_ok)) return;
+    }
+}
+
+// A barrier that one arrival too few will reach: every CTA must give up after
+// `spin_limit` polls and report the time-out instead of hanging.
+__global__ void __launch_bounds__(64)
+barrier_timeout_probe_kernel(int* bar, int* status, long long spin_limit) {
+    __shared__ int s_ok;
+    grid_barrier(bar, (int)gridDim.x + 1, status, spin_limit, &s_ok);
+}
+
 template <bool UPDATE, bool FORWARD, bool SAME>
 cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, const Tile* tiles,
                        int n_tiles, cudaStream_t stream) {
@@ -1042,6 +1188,49 @@ cudaError_t launch_edge_left(const DevState& st, const int* tab, int max_edges, 
 
 cudaError_t launch_edge_right(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
     edge_right_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    return cudaGetLastError();
+}
+
+template <int S, int RT>
+static cudaError_t launch_persistent_t(const DevState& st, const int* tab, const Tile* row_tiles, int n_rows,
+                                       const Tile* col_tiles, int n_cols, int n_steps, bool forward_first,
+                                       int* bar, int max_blocks, cudaStream_t stream) {
+    int per_sm = 0, dev = 0, sms = 0;
+    cudaError_t rc = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, persistent_rounds_kernel<S, RT>, 256, 0);
+    if (rc == cudaSuccess) rc = cudaGetDevice(&dev);
+    if (rc == cudaSuccess) rc = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (rc != cudaSuccess) return rc;
+    int grid = per_sm * sms;                       // all CTAs resident at once: the barrier needs that
+    if (grid > max_blocks) grid = max_blocks;
+    if (grid < 1) return cudaErrorInvalidConfiguration;
+    rc = cudaMemsetAsync(bar, 0, 2 * sizeof(int), stream);
+    if (rc != cudaSuccess) return rc;
+    DevState st_copy = st;
+    int fwd = forward_first ? 1 : 0, expected = grid;
+    long long limit = kBarrierSpinLimit;
+    void* args[] = {&st_copy, &tab, &row_tiles, &n_rows, &col_tiles, &n_cols, &n_steps, &fwd, &bar, &expected, &limit};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(persistent_rounds_kernel<S, RT>), dim3(grid),
+                                       dim3(256), args, 0, stream);
+}
+
+cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* row_tiles, int n_rows,
+                              const Tile* col_tiles, int n_cols, int n_steps, bool forward_first, int* bar,
+                              cudaStream_t stream) {
+    const int slots = st.max_degree * st.rank;
+    const int max_blocks = n_rows > n_cols ? n_rows : n_cols;
+    if (slots <= 1)
+        return launch_persistent_t<1, PG_RT1>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+    if (slots <= 2)
+        return launch_persistent_t<2, PG_RT2>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+    if (slots <= 4)
+        return launch_persistent_t<4, PG_RT4>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+    return launch_persistent_t<8, PG_RT8>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+}
+
+cudaError_t launch_barrier_timeout_probe(int* bar, int* status, cudaStream_t stream) {
+    cudaError_t rc = cudaMemsetAsync(bar, 0, 2 * sizeof(int), stream);
+    if (rc != cudaSuccess) return rc;
+    barrier_timeout_probe_kernel<<<4, 64, 0, stream>>>(bar, status, 20000);   // a few milliseconds of polling
     return cudaGetLastError();
 }
 

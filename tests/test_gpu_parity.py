@@ -271,3 +271,60 @@ def test_initial_vectors_on_device_are_the_seeded_ones():
         for k in range(2):
             assert np.array_equal(q[:, k], po.init_q(w.seed, i, j, 0, k, 70))
     net.close()
+
+
+# ---- one cooperative launch for many rounds (small stacks) --------------------
+PERSISTENT_CASES = [
+    wl.tiny_ring(),
+    wl.resnet20_ring8().replace(rounds=12),
+    wl.shrink(wl.torus8x8(2), [(200, 136)], 6),
+    wl.shrink(wl.vgg16_ring16(2), [(max(n // 8, 3), max(m // 8, 5)) for n, m in wl.VGG16_SHAPES], 5),
+]
+
+
+@pytest.mark.parametrize("w", PERSISTENT_CASES, ids=lambda w: w.name)
+def test_pg_rounds_equals_repeated_pg_round_bit_for_bit(w):
+    """pg_rounds(n) runs the same arithmetic in the same order as n calls of pg_round."""
+    a, b = common.network_for(w), common.network_for(w)
+    common.load_both(w, None, a)
+    common.load_both(w, None, b)
+    for _ in range(w.rounds):
+        a.pg_round()
+    b.pg_rounds(3)                 # starts with the stand-alone forward product
+    b.pg_rounds(w.rounds - 3)      # continues from the cached one
+    assert a.pg_get_round() == b.pg_get_round() == w.rounds
+    assert a.pg_device_status() == 0 and b.pg_device_status() == 0
+    for i in range(w.n_workers):
+        for l in range(len(w.layer_shapes)):
+            assert np.array_equal(a.pg_read_params(i, l), b.pg_read_params(i, l))
+    e = a.pg_get_schedule(0)[0][0]
+    assert np.array_equal(a.pg_read_q(int(e[0]), int(e[1]), 0), b.pg_read_q(int(e[0]), int(e[1]), 0))
+    a.close()
+    b.close()
+
+
+def test_pg_rounds_against_the_checker():
+    w = wl.tiny_ring()
+    oracle, net = common.oracle_for(w), common.network_for(w)
+    common.load_both(w, oracle, net)
+    net.pg_rounds(w.rounds)
+    oracle.round(w.rounds)
+    err, where = common.max_relative_error(w, oracle, net)
+    assert err <= REL_TOL, (err, where)
+    net.close()
+    oracle.close()
+
+
+def test_grid_barrier_gives_up_instead_of_hanging():
+    """A barrier that can never complete must time out, report it and leave the GPU usable."""
+    from paper_2008_01425_b200 import binding as pg
+
+    w = wl.tiny_ring()
+    net = common.network_for(w)
+    assert net.pg_selftest_barrier_timeout() == pg.PG_ERR_TIMEOUT
+    net.close()
+    other = common.network_for(w)          # the device still works
+    common.load_both(w, None, other)
+    other.pg_rounds(2)
+    assert other.pg_device_status() == pg.PG_OK
+    other.close()
