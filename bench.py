@@ -130,6 +130,25 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------
+# replicas: every rank runs its own network; the job's time is the slowest rank's
+# ----------------------------------------------------------------------------
+def max_over_ranks(ms_local: float, dist, device) -> float:
+    """Largest device time over all ranks (identity without a process group)."""
+    if dist is None:
+        return float(ms_local)
+    import torch
+
+    t = torch.tensor([ms_local], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, steps: int, ms_total: float) -> float:
+    """Rounds per second of all replicas together: world x steps over the slowest rank's time."""
+    return world * steps / (ms_total / 1e3)
+
+
+# ----------------------------------------------------------------------------
 # the CPU checker as a timed baseline (bounded sample)
 # ----------------------------------------------------------------------------
 def time_oracle_sample(w, sample_workers: int, rounds: int, warmup: int = 1):
@@ -290,12 +309,9 @@ def main():
     kernel_times = net.pg_timing_read()
     status = net.pg_device_status(stream)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([ms_total], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, device)
     ms_step = ms_total / args.steps
-    value = world * args.steps / (ms_total / 1e3)
+    value = whole_job_rate(world, args.steps, ms_total)
 
     # ---- end to end through the C ABI with host buffers -------------------------
     e2e_steps = max(1, args.e2e_steps)
@@ -311,11 +327,8 @@ def main():
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * e2e_steps / (ms_e2e / 1e3)
+    ms_e2e = max_over_ranks(ms_e2e, dist, device)
+    e2e_value = whole_job_rate(world, e2e_steps, ms_e2e)
     finite = bool(torch.isfinite(back[: min(total, 1 << 22)]).all())
 
     if rank != 0:
