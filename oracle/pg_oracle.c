@@ -251,6 +251,8 @@ typedef struct pgo_ctx {
     double **Q;          /* Q[pair*L + l]: rank columns of length cols, NULL until first met */
     double **Ph;         /* last orthonormal left factor of the pair: rank columns of length rows */
     int max_edges;
+    int half_step;       /* 1: Algorithm 2 read literally, one mat-vec per iteration */
+    int64_t iteration;   /* half-step mode: Algorithm 2's counter k (shared: all pairs move in lockstep) */
 } pgo_ctx;
 
 static size_t pair_index(int N, int i, int j)  /* i < j, over all N(N-1)/2 pairs */
@@ -317,7 +319,10 @@ static double *q_of(pgo_ctx *c, int i, int j, int l)   /* i < j; drawn on first 
     if (c->Q[t] == NULL) {
         int m = c->cols[l];
         float *tmp = (float *)malloc(sizeof(float) * (size_t)m);
-        c->Q[t] = (double *)malloc(sizeof(double) * (size_t)m * (size_t)c->rank);
+        /* in half-step mode the vector alternates between R^cols and R^rows: room for both */
+        size_t room = (size_t)m * (size_t)c->rank;
+        if (c->half_step && (size_t)c->rows[l] > room) room = (size_t)c->rows[l];
+        c->Q[t] = (double *)calloc(room, sizeof(double));
         for (int k = 0; k < c->rank; ++k) {
             pgo_init_q(c->seed, i, j, l, k, m, tmp);
             for (int e = 0; e < m; ++e) c->Q[t][(size_t)k * m + e] = (double)tmp[e];
@@ -465,10 +470,110 @@ static void edge_power_step(const double *Xi, const double *Xj, int n, int m, in
     free(qh); free(pi); free(pj); free(qi); free(qj);
 }
 
+/* ------------------------------------------------------------------------- */
+/* Algorithm 2 read literally ("half-step mode").                             */
+/*                                                                           */
+/* Every iteration is ONE mat-vec and ONE gossip update with that iteration's */
+/* approximation; `power_steps` is the algorithm's s, the iterations per      */
+/* round.  With D = X_i - X_j (i < j), counter k:                             */
+/*   k odd : vh = v/||v|| in R^cols;  p = X_i vh - X_j vh;                     */
+/*           X_i -= W p vh^T,  X_j += W p vh^T;   v <- p      (now in R^rows) */
+/*   k even: the same with X transposed: vh in R^rows;  q = X_i^T vh - X_j^T vh */
+/*           X_i -= W vh q^T,  X_j += W vh q^T;   v <- q      (now in R^cols) */
+/* One iteration moves (rows+cols)/2 floats per edge direction on average,    */
+/* which is what the paper's per-tensor compression ratios count.  Rank 1 and */
+/* static graphs only (all pairs share k).  A zero vector normalises to zero  */
+/* (0/||0|| := 0), so an edge whose ends agree exactly stays silent.          */
+/* ------------------------------------------------------------------------- */
+int pgo_set_half_step(pgo_ctx *c, int on)
+{
+    if (!c) return -1;
+    if (on && (c->rank != 1 || c->kind == PGO_MATCHING || c->round != 0)) return -1;
+    c->half_step = on ? 1 : 0;
+    c->iteration = 0;
+    return 0;
+}
+
+/* current vector of the pair: rows entries after an odd iteration, cols after an
+ * even one (or before the first); returns its length, or -1 */
+int pgo_get_vector(pgo_ctx *c, int i, int j, int l, double *dst)
+{
+    if (!c || i == j || i < 0 || j < 0 || i >= c->N || j >= c->N || l < 0 || l >= c->L) return -1;
+    int a = i < j ? i : j, b = i < j ? j : i;
+    int len = (c->half_step && (c->iteration % 2 == 1)) ? c->rows[l] : c->cols[l];
+    memcpy(dst, q_of(c, a, b, l), sizeof(double) * (size_t)len);
+    return len;
+}
+
+static int half_step_round(pgo_ctx *c)
+{
+    int *edges = (int *)malloc(sizeof(int) * 2 * (size_t)c->max_edges);
+    double *w = (double *)malloc(sizeof(double) * (size_t)c->max_edges);
+    int E = pgo_round_schedule(c, c->round, edges, w);
+    if (E < 0) { free(edges); free(w); return -1; }
+    for (int e = 0; e < E; ++e)
+        for (int l = 0; l < c->L; ++l) (void)q_of(c, edges[2 * e], edges[2 * e + 1], l);
+    double **out = (double **)calloc((size_t)E * (size_t)c->L, sizeof(double *));
+    double **vh = (double **)calloc((size_t)E * (size_t)c->L, sizeof(double *));
+    for (int it = 0; it < c->power_steps; ++it) {
+        c->iteration += 1;
+        const int odd = (int)(c->iteration % 2);
+        /* every edge forms its vector from the same pre-update X */
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+        for (int l = 0; l < c->L; ++l)
+            for (int e = 0; e < E; ++e) {
+                int i = edges[2 * e], j = edges[2 * e + 1];
+                int n = c->rows[l], m = c->cols[l];
+                int len_in = odd ? m : n, len_out = odd ? n : m;
+                size_t t = pair_index(c->N, i, j) * (size_t)c->L + (size_t)l;
+                size_t u = (size_t)e * (size_t)c->L + (size_t)l;
+                const double *v = c->Q[t];
+                double nv = sqrt(dot(v, v, len_in));
+                vh[u] = (double *)malloc(sizeof(double) * (size_t)len_in);
+                for (int a = 0; a < len_in; ++a) vh[u][a] = (nv > 0.0 && isfinite(nv)) ? v[a] / nv : 0.0;
+                double *pi = (double *)malloc(sizeof(double) * (size_t)len_out);
+                double *pj = (double *)malloc(sizeof(double) * (size_t)len_out);
+                const double *Xi = c->X[(size_t)i * c->L + l], *Xj = c->X[(size_t)j * c->L + l];
+                if (odd) { matvec(Xi, n, m, vh[u], pi); matvec(Xj, n, m, vh[u], pj); }
+                else     { matvec_t(Xi, n, m, vh[u], pi); matvec_t(Xj, n, m, vh[u], pj); }
+                for (int a = 0; a < len_out; ++a) pi[a] -= pj[a];
+                out[u] = pi;
+                free(pj);
+            }
+        /* the update of this iteration, then the vector moves to the other space */
+        for (int l = 0; l < c->L; ++l) {
+            int n = c->rows[l], m = c->cols[l];
+            for (int e = 0; e < E; ++e) {
+                int i = edges[2 * e], j = edges[2 * e + 1];
+                size_t t = pair_index(c->N, i, j) * (size_t)c->L + (size_t)l;
+                size_t u = (size_t)e * (size_t)c->L + (size_t)l;
+                double *Xi = c->X[(size_t)i * c->L + l], *Xj = c->X[(size_t)j * c->L + l];
+                const double *left = odd ? out[u] : vh[u];     /* length rows */
+                const double *right = odd ? vh[u] : out[u];    /* length cols */
+                for (int r = 0; r < n; ++r) {
+                    double a = w[e] * left[r];
+                    for (int cidx = 0; cidx < m; ++cidx) {
+                        double d = a * right[cidx];
+                        Xi[(size_t)r * m + cidx] = Xi[(size_t)r * m + cidx] - d;   /* what i loses ... */
+                        Xj[(size_t)r * m + cidx] = Xj[(size_t)r * m + cidx] + d;   /* ... j gains */
+                    }
+                }
+                memcpy(c->Q[t], out[u], sizeof(double) * (size_t)(odd ? n : m));
+                free(out[u]); free(vh[u]);
+                out[u] = vh[u] = NULL;
+            }
+        }
+    }
+    free(out); free(vh); free(edges); free(w);
+    c->round += 1;
+    return 0;
+}
+
 /* One gossip round = power_steps power steps on every layer and every edge of
  * this round's graph.  Returns 0, or -1 on an invalid schedule. */
 int pgo_round(pgo_ctx *c)
 {
+    if (c->half_step) return half_step_round(c);
     int *edges = (int *)malloc(sizeof(int) * 2 * (size_t)c->max_edges);
     double *w = (double *)malloc(sizeof(double) * (size_t)c->max_edges);
     int E = pgo_round_schedule(c, c->round, edges, w);

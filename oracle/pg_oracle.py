@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
         L.pgo_average.restype = c_int
         L.pgo_compression_ratio.argtypes = [c_int, c_int, c_int, c_int]
         L.pgo_compression_ratio.restype = c_dbl
+        L.pgo_set_half_step.argtypes = [vp, c_int]
+        L.pgo_set_half_step.restype = c_int
+        L.pgo_get_vector.argtypes = [vp, c_int, c_int, c_int, vp]
+        L.pgo_get_vector.restype = c_int
         L.pgo_num_threads.argtypes = []
         L.pgo_num_threads.restype = c_int
         _lib = L
@@ -198,6 +202,20 @@ class Oracle:
         if lib().pgo_get_phat(self._h, i, j, layer, _ptr(out)) != 0:
             raise KeyError("pair has not been an edge yet")
         return out.T.copy()
+
+    def set_half_step(self, on: bool = True) -> None:
+        """Algorithm 2 read literally: one mat-vec and one update per iteration;
+        `power_steps` then counts iterations per round.  Rank 1, static graphs."""
+        if lib().pgo_set_half_step(self._h, int(on)) != 0:
+            raise ValueError("half-step mode needs rank 1, a static graph and round 0")
+
+    def get_vector(self, i: int, j: int, layer: int) -> np.ndarray:
+        """The pair's current vector (rows entries after an odd iteration, else cols)."""
+        n, m = self.layer_shapes[layer]
+        out = np.zeros(max(n, m), dtype=np.float64)
+        k = lib().pgo_get_vector(self._h, i, j, layer, _ptr(out))
+        assert k > 0
+        return out[:k].copy()
 
     @property
     def round_index(self) -> int:

@@ -29,6 +29,16 @@ MUTATIONS = {
     "ring_skips_wraparound": ("edges_out[2 * n + 1] = (i + 1) % N; ++n; }",
                               "edges_out[2 * n + 1] = (i + 1) % N; if (i + 1 < N) ++n; }"),
     "philox_round_count": ("round < 10; ++round", "round < 9; ++round"),
+    # Algorithm 2 read literally (half-step mode)
+    "half_step_parity_swapped": ("const int odd = (int)(c->iteration % 2);",
+                                 "const int odd = (int)(c->iteration % 2 == 0);"),
+    "half_step_vector_not_normalised": ("vh[u][a] = (nv > 0.0 && isfinite(nv)) ? v[a] / nv : 0.0;",
+                                        "vh[u][a] = v[a];"),
+    "half_step_vector_not_moved": ("memcpy(c->Q[t], out[u], sizeof(double) * (size_t)(odd ? n : m));", ";"),
+    "half_step_update_not_antisymmetric": ("Xj[(size_t)r * m + cidx] = Xj[(size_t)r * m + cidx] + d;",
+                                           "Xj[(size_t)r * m + cidx] = Xj[(size_t)r * m + cidx] - d;"),
+    "half_step_transposed_operand": ("else     { matvec_t(Xi, n, m, vh[u], pi); matvec_t(Xj, n, m, vh[u], pj); }",
+                                     "else     { matvec_t(Xi, n, m, vh[u], pi); matvec_t(Xi, n, m, vh[u], pj); }"),
 }
 
 

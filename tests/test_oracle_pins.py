@@ -400,3 +400,178 @@ def test_warm_start_is_kept_per_pair_on_a_time_varying_graph():
             if (a, b) not in [tuple(e) for e in edges]:
                 assert np.array_equal(o.get_q(a, b, 0), q)
     o.close()
+
+
+# --------------------------------------------------------------------------
+# Algorithm 2 read literally: one mat-vec and one update per iteration
+# --------------------------------------------------------------------------
+def _pair(n, m, w_edge, iterations, seed=3):
+    W = np.array([[1 - w_edge, w_edge], [w_edge, 1 - w_edge]], dtype=np.float32)
+    o = po.Oracle(kind=po.CUSTOM, n_workers=2, custom_edges=[(0, 1)], layer_shapes=[(n, m)], rank=1,
+                  power_steps=iterations, seed=seed, weight_rule=po.W_EXPLICIT, W=W)
+    o.set_half_step()
+    return o
+
+
+def test_half_step_mode_needs_rank_one_and_a_static_graph():
+    o = po.Oracle(kind=po.RING, n_workers=4, layer_shapes=[(5, 4)], rank=2, power_steps=1, seed=1,
+                  weight_rule=po.W_UNIFORM)
+    with pytest.raises(ValueError):
+        o.set_half_step()
+    o = po.Oracle(kind=po.MATCHING, n_workers=4, layer_shapes=[(5, 4)], rank=1, power_steps=1, seed=1)
+    with pytest.raises(ValueError):
+        o.set_half_step()
+
+
+@pytest.mark.parametrize("case", [CASES[0], CASES[1], CASES[5],
+                                  dict(kind=po.TORUS, n_workers=12, torus_rows=3, torus_cols=4,
+                                       layer_shapes=[(10, 8)], rank=1, power_steps=3,
+                                       weight_rule=po.W_METROPOLIS)])
+def test_half_step_average_conserved_and_distance_never_grows(case):
+    """Lemma 1 holds for every iteration's update; a projection along a unit vector on
+    either side is still a projector, so the consensus distance cannot grow."""
+    rng = np.random.default_rng(4)
+    o = po.Oracle(seed=19, **case)
+    o.set_half_step()
+    _fill(o, rng)
+    avg0 = [o.average(l) for l in range(len(o.layer_shapes))]
+    d_prev = o.consensus_distance()
+    for _ in range(10):
+        o.round()
+        for l in range(len(o.layer_shapes)):
+            assert np.abs(o.average(l) - avg0[l]).max() <= 1e-13 * max(np.abs(avg0[l]).max(), 1.0)
+        d = o.consensus_distance()
+        assert d <= d_prev * (1 + 1e-12)
+        d_prev = d
+    o.close()
+
+
+def test_half_step_vector_alternates_between_the_two_spaces():
+    """After an odd iteration the pair's vector lives in R^rows, after an even one in
+    R^cols (Algorithm 2's comment), so an iteration moves (rows+cols)/2 floats on
+    average: the count behind the printed per-tensor compression ratios."""
+    n, m = 64, 576
+    o = _pair(n, m, 0.25, 1)
+    _fill(o, np.random.default_rng(0))
+    lengths = []
+    for _ in range(6):
+        o.round()
+        lengths.append(len(o.get_vector(0, 1, 0)))
+    assert lengths == [n, m, n, m, n, m]
+    assert round(n * m / np.mean(lengths)) == 115            # the ResNet-20 table prints 115/r
+    o.close()
+
+
+def test_half_step_removes_a_rank_one_difference_in_two_iterations():
+    """D = sigma u v^T: the odd iteration leaves a difference that is still u times a
+    row vector and makes the stored vector parallel to u; the even iteration's
+    approximation vh vh^T D is then exact, so with W = 1/2 both ends meet at their
+    average after two iterations."""
+    rng = np.random.default_rng(6)
+    n, m = 9, 7
+    base = np.round(rng.standard_normal((n, m)) * 64) / 64
+    u = np.round(rng.standard_normal((n, 1)) * 8) / 8
+    v = np.round(rng.standard_normal((1, m)) * 8) / 8
+    x0, x1 = (base + u @ v).astype(np.float32), base.astype(np.float32)
+    o = _pair(n, m, 0.5, 2)
+    o.set_params(0, 0, x0)
+    o.set_params(1, 0, x1)
+    o.round()
+    mean = (x0.astype(np.float64) + x1.astype(np.float64)) / 2
+    assert np.allclose(o.get_params(0, 0), mean, rtol=0, atol=1e-13)
+    assert np.allclose(o.get_params(1, 0), mean, rtol=0, atol=1e-13)
+    # after ONE iteration they have not met yet (unless v happens to be parallel to the seed vector)
+    o2 = _pair(n, m, 0.5, 1)
+    o2.set_params(0, 0, x0)
+    o2.set_params(1, 0, x1)
+    o2.round()
+    assert not np.allclose(o2.get_params(0, 0), mean, rtol=0, atol=1e-6)
+    o.close()
+    o2.close()
+
+
+def test_half_step_on_a_frozen_difference_is_power_iteration():
+    """Eq. 3 with D fixed (edge weight 0): the stored vector converges to sigma_1 u_1 after odd
+    iterations and sigma_1 v_1 after even ones (numpy.linalg.svd)."""
+    rng = np.random.default_rng(12)
+    n, m = 8, 6
+    U, _ = np.linalg.qr(rng.standard_normal((n, n)))
+    V, _ = np.linalg.qr(rng.standard_normal((m, m)))
+    sv = np.array([4.0, 2.0, 1.0, 0.5, 0.2, 0.1])
+    x1 = rng.standard_normal((n, m)).astype(np.float32)
+    x0 = (x1 + (U[:, :m] * sv) @ V.T).astype(np.float32)
+    D = x0.astype(np.float64) - x1.astype(np.float64)
+    Us, ss, Vts = np.linalg.svd(D)
+    o = _pair(n, m, 0.0, 1)
+    o.set_params(0, 0, x0)
+    o.set_params(1, 0, x1)
+    for it in range(1, 61):
+        o.round()
+    vec = o.get_vector(0, 1, 0)                 # 60 iterations: even, so in R^cols
+    assert len(vec) == m
+    assert abs(np.linalg.norm(vec) - ss[0]) < 1e-8 * ss[0]
+    assert abs(abs(vec @ Vts[0]) - ss[0]) < 1e-8 * ss[0]
+    o.round()
+    vec = o.get_vector(0, 1, 0)                 # odd: in R^rows
+    assert len(vec) == n
+    assert abs(abs(vec @ Us[:, 0]) - ss[0]) < 1e-8 * ss[0]
+    assert np.array_equal(o.get_params(0, 0), x0.astype(np.float64))
+    o.close()
+
+
+def test_half_step_first_iteration_on_single_column_layers_is_plain_gossip():
+    """For an n x 1 tensor the first (odd) iteration projects on a 1-vector, which
+    reproduces every difference exactly: one uncompressed gossip step X <- W X
+    (Eq. 1's averaging term), on a ring with all edges acting at once."""
+    rng = np.random.default_rng(14)
+    N, n = 6, 7
+    W = _ring_W(N, 0.3)
+    o = po.Oracle(kind=po.RING, n_workers=N, layer_shapes=[(n, 1)], rank=1, power_steps=1,
+                  seed=23, weight_rule=po.W_EXPLICIT, W=W)
+    o.set_half_step()
+    xs = _fill(o, rng)
+    X = np.stack([xs[i][0] for i in range(N)])
+    o.round()
+    expect = np.einsum("ij,jnm->inm", W.astype(np.float64), X)
+    got = np.stack([o.get_params(i, 0) for i in range(N)])
+    assert np.allclose(got, expect, rtol=0, atol=1e-12)
+    o.close()
+
+
+@pytest.mark.parametrize("shape", [(7, 1), (1, 7)])
+@pytest.mark.parametrize("iterations", [2, 3, 4])
+def test_half_step_isolated_pair_single_column_or_row(shape, iterations):
+    """Two workers, an n x 1 (or 1 x m) tensor: the difference keeps its direction, so
+    every iteration whose unit vector lives in the 1-dimensional space is exact and
+    the others project a vector on itself: the difference shrinks by (1 - 2W) per
+    exact iteration.  n x 1: all iterations exact.  1 x m: the first (odd) one
+    projects the row on the seed direction, all later ones are exact."""
+    rng = np.random.default_rng(15)
+    wgt = 0.3
+    o = _pair(shape[0], shape[1], wgt, iterations)
+    xs = _fill(o, rng)
+    D0 = xs[0][0] - xs[1][0]
+    o.round()
+    D = o.get_params(0, 0) - o.get_params(1, 0)
+    w64 = float(np.float32(wgt))
+    if shape[1] == 1:
+        assert np.allclose(D, (1 - 2 * w64) ** iterations * D0, rtol=0, atol=1e-13)
+    else:
+        q = po.init_q(3, 0, 1, 0, 0, shape[1]).astype(np.float64)
+        q /= np.linalg.norm(q)
+        D1 = D0 - 2 * w64 * (D0 @ q)[:, None] * q[None, :]          # after the first iteration
+        assert np.allclose(D, (1 - 2 * w64) ** (iterations - 1) * D1, rtol=0, atol=1e-13)
+    o.close()
+
+
+def test_half_step_identical_workers_stay_put():
+    x = np.random.default_rng(2).standard_normal((6, 5)).astype(np.float32)
+    o = po.Oracle(kind=po.RING, n_workers=4, layer_shapes=[(6, 5)], rank=1, power_steps=3, seed=4,
+                  weight_rule=po.W_UNIFORM)
+    o.set_half_step()
+    for i in range(4):
+        o.set_params(i, 0, x)
+    o.round(2)
+    for i in range(4):
+        assert np.array_equal(o.get_params(i, 0), x.astype(np.float64))
+    o.close()
