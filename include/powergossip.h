@@ -162,6 +162,23 @@ PG_API int pg_read_params(pg_ctx *ctx, int32_t worker, int32_t layer, float *hos
 PG_API int pg_round(pg_ctx *ctx, void *stream);
 
 /*
+ * Algorithm 2 read literally ("half-step mode"): every iteration is ONE
+ * mat-vec and one gossip update with that iteration's approximation, and the
+ * stored vector alternates between R^cols and R^rows:
+ *   k odd :  vh = v/||v||;  p = X_i vh - X_j vh;  X_i -= W p vh^T, X_j += W p vh^T;  v <- p
+ *   k even:  the same with X transposed:  q = X_i^T vh - X_j^T vh;
+ *            X_i -= W vh q^T, X_j += W vh q^T;  v <- q
+ * `power_steps` then counts iterations per round (the algorithm's s), and one
+ * iteration moves (rows+cols)/2 floats per edge direction on average, the count
+ * behind the per-tensor compression ratios of the paper's parameter tables.  A
+ * zero vector normalises to zero.  Call before the first round.  Needs rank 1
+ * and a static graph of degree >= 2 (PG_ERR_INVALID otherwise; PG_ERR_STATE once
+ * rounds have run).  In this mode pg_read_q / pg_write_q are only meaningful
+ * after an even number of iterations, when the vector is back in R^cols.
+ */
+PG_API int pg_set_half_step(pg_ctx *ctx, int32_t on);
+
+/*
  * Enqueue `n_rounds` rounds (same result as calling pg_round that many times).
  * When the graph is static and the whole stack is small enough to stay in L2
  * (at most 64 MiB of parameters, degree > 1 or rank > 1), all rounds run in ONE

@@ -39,7 +39,7 @@ struct Layout {
     int max_edges = 0, max_degree = 0;
     TabLayout tab{};
     long long n_row_tiles = 0, n_col_tiles = 0;
-    size_t off_Qn2 = 0;
+    size_t off_Qn2 = 0, off_Pn = 0;
     size_t off_X = 0, off_Q = 0, off_Qinv = 0, off_Y = 0, off_Ph = 0, off_Z = 0, off_live = 0,
            off_Up = 0, off_Sp = 0, off_pair_tiles = 0, off_flush_tiles = 0, off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
     size_t total = 0;
@@ -215,6 +215,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_Q = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride);
     lay.off_Qinv = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * n_layers * rank);
     lay.off_Qn2 = take(sizeof(double) * static_cast<size_t>(lay.n_pairs) * n_layers * pg::kEdgeChunks);
+    lay.off_Pn = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * n_layers);
     lay.off_Y = take(sizeof(float) * static_cast<size_t>(N) * lay.y_stride);
     lay.off_Ph = take(sizeof(float) * 2 * static_cast<size_t>(lay.max_edges) * lay.ph_stride);  // two buffers
     lay.off_Up = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * lay.up_stride);
@@ -261,6 +262,10 @@ struct pg_ctx {
     bool tab_used[kTabRing];
     Tile* d_row_tiles = nullptr;
     Tile* d_col_tiles = nullptr;
+    // Algorithm 2 read literally: one mat-vec and one update per iteration
+    bool half_step = false;
+    int64_t iteration = 0;      // Algorithm 2's counter k
+    bool half_pending = false;  // an odd iteration's update has not been applied to X yet
     bool static_graph = true;
     bool coop_ok = false;       // the device supports cooperative launches
     int device = 0;
@@ -361,6 +366,24 @@ bool bind_device(const pg_ctx* c) {
 // Apply the correction the pair sweep left pending, so that X in memory is the
 // live model (needed before X, Q or the round counter are read or overwritten).
 int flush_pending(pg_ctx* c, cudaStream_t stream) {
+    if (c->half_pending) {
+        // the odd iteration's update p q-hat^T, with the scaled coefficients
+        const int* tab = nullptr;
+        const int rc = ensure_table(c, c->round, stream, &tab);
+        if (rc != PG_OK) return rc;
+        DevState st = c->st;
+        st.Ph = c->ph_buf[0];
+        st.half_odd = 1;
+        Timed t(c, PG_KERNEL_UPDATE_ONLY, stream, 2.0 * c->normal_param_bytes);
+        if (pg::launch_update(st, tab, c->d_row_tiles, static_cast<int>(c->lay.n_row_tiles), stream) != cudaSuccess) {
+            cudaGetLastError();
+            return PG_ERR_CUDA;
+        }
+        c->launches += 1;
+        c->half_pending = false;
+        c->y_valid = false;
+        return PG_OK;
+    }
     if (!c->pending) return PG_OK;
     const int* tab_prev = nullptr;
     const int rc = ensure_table(c, c->pending_key, stream, &tab_prev);
@@ -483,6 +506,8 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.Q = reinterpret_cast<float*>(c->ws + lay.off_Q);
     st.Qinv = reinterpret_cast<float*>(c->ws + lay.off_Qinv);
     st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
+    st.Pn = reinterpret_cast<float*>(c->ws + lay.off_Pn);
+    st.half_odd = 0;
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
     st.PhNext = st.Ph + static_cast<long long>(lay.max_edges) * lay.ph_stride;
@@ -668,6 +693,56 @@ int pg_round(pg_ctx* c, void* stream_v) {
     const int n_rows = static_cast<int>(c->lay.n_row_tiles), n_cols = static_cast<int>(c->lay.n_col_tiles);
     const bool has_pair = c->lay.n_pair_tiles > 0;
     bool ok = true;
+    if (c->half_step) {
+        // `power_steps` iterations of Algorithm 2.  Odd: X q-hat -> p; its update stays
+        // pending and is applied by the even iteration's transposed sweep.  Even:
+        // X^T p-hat -> q; its update is fused with the next odd iteration's X q-hat.
+        DevState st = c->st;
+        st.Ph = c->ph_buf[0];
+        for (int it = 0; it < c->power_steps && ok; ++it) {
+            c->iteration += 1;
+            if (c->iteration % 2 == 1) {
+                if (!c->y_valid) {
+                    Timed t(c, PG_KERNEL_FORWARD, stream, c->normal_param_bytes);
+                    ok = ok && pg::launch_forward(st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+                    c->launches += 1;
+                }
+                {
+                    Timed t(c, PG_KERNEL_EDGE_LEFT, stream, 0.0);
+                    ok = ok && pg::launch_edge_odd(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+                }
+                c->launches += 1;
+                c->half_pending = true;
+                c->y_valid = false;
+            } else {
+                if (c->half_pending) {
+                    Timed t(c, PG_KERNEL_TRANSPOSED, stream, 2.0 * c->normal_param_bytes);
+                    ok = ok && pg::launch_transposed_update(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+                } else {
+                    Timed t(c, PG_KERNEL_TRANSPOSED, stream, c->normal_param_bytes);
+                    ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+                }
+                c->half_pending = false;
+                {
+                    Timed t(c, PG_KERNEL_EDGE_RIGHT, stream, 0.0);
+                    ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+                }
+                {
+                    Timed t(c, PG_KERNEL_UPDATE_FORWARD, stream, 2.0 * c->normal_param_bytes);
+                    ok = ok && pg::launch_update_forward(st, tab, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+                }
+                c->launches += 3;
+                c->y_valid = true;
+            }
+        }
+        if (!ok) {
+            cudaGetLastError();
+            c->y_valid = false;
+            return PG_ERR_CUDA;
+        }
+        c->round += 1;
+        return PG_OK;
+    }
     if (n_rows > 0 && !c->y_valid) {
         Timed t(c, PG_KERNEL_FORWARD, stream, c->normal_param_bytes);
         ok = ok && pg::launch_forward(c->st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
@@ -736,6 +811,15 @@ int pg_round(pg_ctx* c, void* stream_v) {
     return PG_OK;
 }
 
+int pg_set_half_step(pg_ctx* c, int32_t on) {
+    if (!c) return PG_ERR_INVALID;
+    if (c->round != 0 || c->pending || c->y_valid) return PG_ERR_STATE;
+    if (on && (c->rank != 1 || !c->static_graph || c->lay.n_pair_tiles > 0)) return PG_ERR_INVALID;
+    c->half_step = on != 0;
+    c->iteration = 0;
+    return PG_OK;
+}
+
 int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
     if (!c || n_rounds < 0) return PG_ERR_INVALID;
     if (n_rounds == 0) return PG_OK;
@@ -744,7 +828,7 @@ int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
     // One cooperative launch when the graph is static, no layer uses the pair sweep and the
     // whole stack stays in L2; otherwise the rounds are enqueued one by one.
     const double x_bytes = c->normal_param_bytes;
-    const bool persistent = c->static_graph && c->lay.n_pair_tiles == 0 && c->coop_ok &&
+    const bool persistent = c->static_graph && !c->half_step && c->lay.n_pair_tiles == 0 && c->coop_ok &&
                             x_bytes <= 64.0 * 1024 * 1024 && !c->timing;
     if (!persistent) {
         for (int r = 0; r < n_rounds; ++r) {

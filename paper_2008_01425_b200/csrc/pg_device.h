@@ -96,6 +96,9 @@ struct DevState {
     float* PhNext;       // same shape as Ph: where the pair sweep writes this step's p
     float* Up;           // [edge][up_stride]    pair sweep: partial sums of D^T p
     double* Sp;          // [edge][sp_stride]    pair sweep: partial sums of ||p||^2
+    float* Pn;           // [edge][layer]  half-step mode: ||p|| of the last odd iteration
+    int half_odd;        // half-step mode: the update being applied is an odd iteration's,
+                         // p q-hat^T = (||p|| / ||q||) p-hat q^T: scale the coefficients accordingly
     int* live;           // [edge][layer][rank]  1 if the column took part in this step
     int* status;         // device status word (bit n set = error code n was raised)
     const LayerGeom* layers;
@@ -114,6 +117,10 @@ cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* ti
 cudaError_t launch_edge_right(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_update_forward(const DevState& st, const int* tab_update, const int* tab_forward,
                                   const Tile* tiles, int n_tiles, cudaStream_t stream);
+// half-step mode
+cudaError_t launch_edge_odd(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
+cudaError_t launch_transposed_update(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+                                     cudaStream_t stream);
 cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile* tiles, int n_tiles,
                           cudaStream_t stream);
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,

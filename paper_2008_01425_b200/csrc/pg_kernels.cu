@@ -136,6 +136,9 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                 sh.uq[v] = st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld;
                 sh.up[v] = st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad;
                 sh.uc[v] = __int_as_float(tab_u[st.tab.off_slot_coef + w * st.tab.max_degree + slot]);
+                if (st.half_odd)   // odd iteration of Algorithm 2: the update is p q-hat^T
+                    sh.uc[v] *= ld_f<COH>(&st.Pn[(long long)e * st.n_layers + tile.layer]) *
+                                ld_f<COH>(&st.Qinv[((long long)pair * st.n_layers + tile.layer) * rank + k]);
             }
             if (v == 0) sh.nu = deg * rank;
         }
@@ -277,10 +280,14 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
 template <int S>
 struct ColShared {
     float p[S][kColTileRowsMax];
+    float a[S][kColTileRowsMax];   // UPDATE: coefficient of the pending correction per row
     float4 red[3][S][64];
 };
 
-template <int S, bool COH>
+// UPDATE (half-step mode): the pending correction of the odd iteration,
+// X_w -= sum_v a_v[r] Q_v[c], is applied to the tile on its way through and the
+// product is taken with the corrected values.
+template <int S, bool COH, bool UPDATE>
 __device__ __forceinline__ void col_tile(const DevState& st, const int* __restrict__ tab, const Tile tile,
                                          ColShared<S>& sh) {
     const LayerGeom g = st.layers[tile.layer];
@@ -301,6 +308,15 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
             const int slot = v / rank, k = v - slot * rank;
             const int e = tab[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
             val = ld_f<COH>(st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad + r0 + rr);
+            if (UPDATE) {
+                const int pair = tab[st.tab.off_pair + e];
+                const float coef = __int_as_float(tab[st.tab.off_slot_coef + w * st.tab.max_degree + slot]) *
+                                   ld_f<COH>(&st.Pn[(long long)e * st.n_layers + tile.layer]) *
+                                   ld_f<COH>(&st.Qinv[((long long)pair * st.n_layers + tile.layer) * rank + k]);
+                sh.a[v][rr] = coef * val;
+            }
+        } else if (UPDATE) {
+            sh.a[v][rr] = 0.0f;
         }
         sh.p[v][rr] = val;
     }
@@ -313,6 +329,19 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
 #pragma unroll
     for (int v = 0; v < S; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
 
+    float4 qv[S];
+    if (UPDATE && c < ld) {
+#pragma unroll
+        for (int v = 0; v < S; ++v) {
+            qv[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (v < nv) {
+                const int slot = v / rank, k = v - slot * rank;
+                const int e = tab[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
+                const int pair = tab[st.tab.off_pair + e];
+                qv[v] = ld_vec<COH>(st.Q + (long long)pair * st.q_stride + g.q_off + (long long)k * g.ld + c);
+            }
+        }
+    }
     if (c < ld) {
         const float* xc = X + c;
         for (int r = r0 + ty; r < r1; r += 16) {
@@ -327,6 +356,17 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
             for (int u = 0; u < 4; ++u) {
                 const int ro = min(rr[u] - r0, kColTileRowsMax - 1);
                 const bool in = rr[u] < r1;
+                if (UPDATE && in) {
+#pragma unroll
+                    for (int v = 0; v < S; ++v) {
+                        if (v < nv) {
+                            const float a = sh.a[v][ro];
+                            x[u].x = fmaf(-a, qv[v].x, x[u].x); x[u].y = fmaf(-a, qv[v].y, x[u].y);
+                            x[u].z = fmaf(-a, qv[v].z, x[u].z); x[u].w = fmaf(-a, qv[v].w, x[u].w);
+                        }
+                    }
+                    st_stream(const_cast<float*>(xc) + (long long)rr[u] * ld, x[u]);
+                }
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nv) {
@@ -362,11 +402,53 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
     }
 }
 
-template <int S>
+template <int S, bool UPDATE>
 __global__ void __launch_bounds__(256)
 col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles) {
     __shared__ ColShared<S> sh;
-    col_tile<S, false>(st, tab, tiles[blockIdx.x], sh);
+    col_tile<S, false, UPDATE>(st, tab, tiles[blockIdx.x], sh);
+}
+
+// Half-step mode, odd iteration: p = Y[i] - Y[j] (fp64 sums of the partials),
+// P-hat = p / ||p|| as fp32 and ||p|| kept beside it, so that the update
+// p q-hat^T and the next iteration's unit vector both come from P-hat.  A zero or
+// non-finite p gives P-hat = 0 (the edge falls silent).  One CTA per (edge, layer).
+__global__ void __launch_bounds__(512)
+edge_odd_kernel(DevState st, const int* __restrict__ tab) {
+    __shared__ double scratch[33];
+    const int L = st.n_layers;
+    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[l];
+    const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
+    const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
+    const float* yi = st.Y + (long long)wi * st.y_stride + g.y_off + (long long)si * g.f_csplit * g.npad;
+    const float* yj = st.Y + (long long)wj * st.y_stride + g.y_off + (long long)sj * g.f_csplit * g.npad;
+    float* Ph = st.Ph + (long long)e * st.ph_stride + g.ph_off;
+    auto raw = [&](int r) {
+        double a = 0.0, b = 0.0;
+        for (int cs = 0; cs < g.f_csplit; ++cs) {
+            a += (double)yi[(long long)cs * g.npad + r];
+            b += (double)yj[(long long)cs * g.npad + r];
+        }
+        return a - b;
+    };
+    double part = 0.0;
+    for (int r = threadIdx.x; r < g.n; r += blockDim.x) {
+        const double v = raw(r);
+        part += v * v;
+    }
+    const double nn = block_sum(part, scratch);
+    const bool finite = isfinite(nn);
+    const bool live = finite && nn > 0.0;
+    const double inv = live ? 1.0 / sqrt(nn) : 0.0;
+    for (int r = threadIdx.x; r < g.npad; r += blockDim.x)
+        Ph[r] = (live && r < g.n) ? (float)(raw(r) * inv) : 0.0f;
+    if (threadIdx.x == 0) {
+        st.Pn[(long long)e * L + l] = live ? (float)sqrt(nn) : 0.0f;
+        st.live[(long long)e * L + l] = 1;     // the even iteration always stores its vector, zero included
+        if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
+    }
 }
 
 // --------------------------------------------------------------------------
@@ -998,7 +1080,7 @@ persistent_rounds_kernel(DevState st, const int* __restrict__ tab, const Tile* _
         for (int it = blockIdx.x; it < n_items; it += nb) edge_left_step<true>(st, tab, it / L, it % L, scratch);
         if (!grid_barrier(bar, expected_blocks, st.status, spin_limit, &s_ok)) return;
         for (int t = blockIdx.x; t < n_cols; t += nb) {
-            col_tile<S, true>(st, tab, col_tiles[t], csh);
+            col_tile<S, true, false>(st, tab, col_tiles[t], csh);
             __syncthreads();
         }
         if (!grid_barrier(bar, expected_blocks, st.status, spin_limit, &s_ok)) return;
@@ -1166,18 +1248,34 @@ cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, 
     return cudaGetLastError();
 }
 
-cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+template <bool UPDATE>
+static cudaError_t launch_col(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
                               cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
     const int slots = st.max_degree * st.rank;
     if (slots <= 1)
-        col_sweep_kernel<1><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        col_sweep_kernel<1, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
     else if (slots <= 2)
-        col_sweep_kernel<2><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        col_sweep_kernel<2, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
     else if (slots <= 4)
-        col_sweep_kernel<4><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        col_sweep_kernel<4, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
     else
-        col_sweep_kernel<8><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        col_sweep_kernel<8, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+                              cudaStream_t stream) {
+    return launch_col<false>(st, tab, tiles, n_tiles, stream);
+}
+
+cudaError_t launch_transposed_update(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
+                                     cudaStream_t stream) {
+    return launch_col<true>(st, tab, tiles, n_tiles, stream);
+}
+
+cudaError_t launch_edge_odd(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
+    edge_odd_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
     return cudaGetLastError();
 }
 

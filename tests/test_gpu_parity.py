@@ -328,3 +328,73 @@ def test_grid_barrier_gives_up_instead_of_hanging():
     other.pg_rounds(2)
     assert other.pg_device_status() == pg.PG_OK
     other.close()
+
+
+# ---- Algorithm 2 read literally (half-step mode) ------------------------------
+def _run_half(w, rounds, rebase_every=None, check_every=1):
+    """Half-step mode on both sides.  `power_steps` counts iterations per round.  Re-basing
+    (checker state -> fp32 -> both sides) only happens after an even number of iterations,
+    when the pair vectors are back in R^cols and can be written through pg_write_q."""
+    from paper_2008_01425_b200 import binding as pg
+
+    oracle, net = common.oracle_for(w), common.network_for(w)
+    oracle.set_half_step()
+    common.load_both(w, oracle, net)
+    net.pg_set_half_step()
+    avg0 = [common.initial_average(w, l) for l in range(len(w.layer_shapes))]
+    pairs = set((int(a), int(b)) for a, b in oracle.round_schedule(0)[0])
+    for t in range(1, rounds + 1):
+        net.pg_round()
+        oracle.round()
+        if t % check_every == 0 or t == rounds:
+            err, where = common.max_relative_error(w, oracle, net)     # reading X flushes a pending update
+            assert err <= REL_TOL, "round %d: relative error %.3e at %r" % (t, err, where)
+        if rebase_every and t % rebase_every == 0 and t < rounds:
+            assert (t * w.power_steps) % 2 == 0
+            common.rebase(w, oracle, net, pairs)
+    assert net.pg_device_status() == pg.PG_OK
+    _check_average(w, net, avg0)
+    net.close()
+    oracle.close()
+
+
+def test_half_step_tiny_ring_free_running():
+    _run_half(wl.tiny_ring(), 20, check_every=1)       # a read after every odd iteration: the flush path
+
+
+def test_half_step_tiny_ring_few_reads():
+    _run_half(wl.tiny_ring(), 20, check_every=20)      # pending updates consumed by the transposed sweep
+
+
+def test_half_step_resnet20_two_iterations_rebased():
+    _run_half(wl.resnet20_ring8().replace(power_steps=2), 30, rebase_every=4, check_every=2)
+
+
+def test_half_step_torus_small_three_iterations_rebased():
+    w = wl.shrink(wl.torus8x8(3), [(200, 136)], 12)
+    _run_half(w, 12, rebase_every=2, check_every=1)
+
+
+@pytest.mark.parametrize("iterations", [1, 2])
+def test_half_step_ragged_shapes(iterations):
+    w = wl.Workload("half_edge", 9, 4, wl.RING, 0, 0, wl.W_EXPLICIT, 0.3,
+                    ((67, 131), (5, 3), (9, 1), (1, 9), (300, 7)), 1, iterations, 6, 77, "normal1")
+    _run_half(w, 6, rebase_every=2)
+
+
+def test_half_step_mode_is_refused_where_it_does_not_apply():
+    from paper_2008_01425_b200 import binding as pg
+
+    for w in (wl.tiny_ring().replace(rank=2), wl.shrink(wl.lstm_matching32(), [(30, 20)], 1).replace(n_workers=4)):
+        net = common.network_for(w)
+        with pytest.raises(pg.PowerGossipError) as e:
+            net.pg_set_half_step()
+        assert e.value.status == pg.PG_ERR_INVALID
+        net.close()
+    net = common.network_for(wl.tiny_ring())
+    common.load_both(wl.tiny_ring(), None, net)
+    net.pg_round()
+    with pytest.raises(pg.PowerGossipError) as e:
+        net.pg_set_half_step()
+    assert e.value.status == pg.PG_ERR_STATE
+    net.close()
