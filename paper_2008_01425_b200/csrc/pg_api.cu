@@ -116,12 +116,13 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
 
     lay.pair_mode = lay.max_degree == 1 && rank == 1 && pair_sweep_allowed();
     lay.layers.resize(n_layers);
-    // aim for about 4096 tiles per sweep, each between 64 KB and 512 KB of X
+    // aim for about 4096 tiles per sweep, each between 128 KB and 512 KB of X
     long long total_elems = 0;
     for (int l = 0; l < n_layers; ++l)
         if (shapes[l].rows > 0 && shapes[l].cols > 0)
             total_elems += static_cast<long long>(N) * shapes[l].rows * round_up(shapes[l].cols, 4);
-    const long long tile_elems = std::min<long long>(std::max<long long>(total_elems / 4096, 16 * 1024), 128 * 1024);
+    long long tile_elems = std::min<long long>(std::max<long long>(total_elems / 4096, 32 * 1024), 128 * 1024);
+    if (const char* v = std::getenv("PG_TILE_ELEMS")) tile_elems = std::max(4096LL, std::atoll(v));   // tuning aid
     long long x = 0, q = 0, y = 0, ph = 0, z = 0, up = 0, sp = 0;
     lay.n_row_tiles = lay.n_col_tiles = lay.n_pair_tiles = lay.n_flush_tiles = 0;
     for (int l = 0; l < n_layers; ++l) {

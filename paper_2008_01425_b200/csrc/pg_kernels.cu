@@ -565,18 +565,9 @@ __device__ __forceinline__ void edge_right_step(const DevState& st, const int* _
         double part = 0.0;
         for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
             double a = 0.0, b = 0.0;
-            for (int rt = 0; rt < g.t_rtiles; rt += 4) {     // eight independent loads, added in tile order
-                float va[4], vb[4];
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    va[t] = rt + t < g.t_rtiles ? ld_f<COH>(zi + (long long)(rt + t) * g.ld + c) : 0.0f;
-                    vb[t] = rt + t < g.t_rtiles ? ld_f<COH>(zj + (long long)(rt + t) * g.ld + c) : 0.0f;
-                }
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    a += (double)va[t];
-                    b += (double)vb[t];
-                }
+            for (int rt = 0; rt < g.t_rtiles; ++rt) {        // added in tile order
+                a += (double)ld_own<COH>(zi + (long long)rt * g.ld + c);
+                b += (double)ld_own<COH>(zj + (long long)rt * g.ld + c);
             }
             const float q = (float)(a - b);
             Q[(long long)k * g.ld + c] = q;
