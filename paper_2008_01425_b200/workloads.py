@@ -118,9 +118,17 @@ def lstm_matching32() -> Workload:
                     LSTM_SHAPES, 1, 1, 20, 1005, "uniform0.1")
 
 
+def consensus_ring8(iterations_per_round: int = 1, rounds: int = 400) -> Workload:
+    """The paper's consensus experiment (Appendix "Experimental settings", table
+    "Experimental settings for Consensus"): 8 workers in a ring, one 100 x 100
+    standard-normal matrix each, W = 0.436 / 0.128."""
+    return Workload("consensus_ring8_100x100", 6, 8, RING, 0, 0, W_EXPLICIT, 0.436,
+                    ((100, 100),), 1, iterations_per_round, rounds, 1006, "normal1")
+
+
 def all_workloads() -> List[Workload]:
     return [tiny_ring(), resnet20_ring8(), torus8x8(1), torus8x8(2), torus8x8(4),
-            vgg16_ring16(1), vgg16_ring16(2), lstm_matching32()]
+            vgg16_ring16(1), vgg16_ring16(2), lstm_matching32(), consensus_ring8()]
 
 
 def by_name(name: str) -> Workload:
