@@ -146,6 +146,21 @@ PG_API int pg_write_params(pg_ctx *ctx, int32_t worker, int32_t layer, const flo
 PG_API int pg_read_params(pg_ctx *ctx, int32_t worker, int32_t layer, float *host_dst, void *stream);
 
 /*
+ * Device view of worker `worker`'s layer `layer` for local updates between
+ * rounds - Algorithm 1's  - eta G  term: the caller subtracts its scaled
+ * gradient in place with its own kernels.  *dev_ptr_out points at rows x cols
+ * fp32 values with leading dimension *ld_out floats (cols rounded up to 4; the
+ * padding columns must stay zero).  Any correction still pending is applied
+ * first (enqueued on `stream`), and the cached forward product is dropped, so
+ * the next pg_round starts from whatever the caller leaves there.  Work on the
+ * view must be ordered after this call and before the next pg_round on the same
+ * stream.  The pointer stays valid for the life of the workspace, but call this
+ * again after every round before touching X.
+ */
+PG_API int pg_params_device(pg_ctx *ctx, int32_t worker, int32_t layer, void *stream, float **dev_ptr_out,
+                            int64_t *ld_out);
+
+/*
  * Enqueue one gossip round on `stream` (asynchronous): `power_steps` power
  * steps on every layer and every edge of this round's graph, each one
  *     Qh = unit columns of the pair's stored Q        (Algorithm 2, v / ||v||)

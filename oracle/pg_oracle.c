@@ -341,6 +341,16 @@ int pgo_set_params(pgo_ctx *c, int i, int l, const float *src)
     return 0;
 }
 
+/* Algorithm 1's local term: X_i <- X_i + delta (the caller passes -eta * G). */
+int pgo_add_params(pgo_ctx *c, int i, int l, const double *delta)
+{
+    if (!c || i < 0 || i >= c->N || l < 0 || l >= c->L) return -1;
+    size_t cnt = (size_t)c->rows[l] * (size_t)c->cols[l];
+    double *x = c->X[(size_t)i * c->L + l];
+    for (size_t t = 0; t < cnt; ++t) x[t] += delta[t];
+    return 0;
+}
+
 int pgo_get_params(pgo_ctx *c, int i, int l, double *dst)
 {
     if (!c || i < 0 || i >= c->N || l < 0 || l >= c->L) return -1;

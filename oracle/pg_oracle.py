@@ -60,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.pgo_destroy.restype = None
         L.pgo_set_params.argtypes = [vp, c_int, c_int, vp]
         L.pgo_set_params.restype = c_int
+        L.pgo_add_params.argtypes = [vp, c_int, c_int, vp]
+        L.pgo_add_params.restype = c_int
         L.pgo_get_params.argtypes = [vp, c_int, c_int, vp]
         L.pgo_get_params.restype = c_int
         for f in (L.pgo_get_q, L.pgo_set_q, L.pgo_get_phat):
@@ -176,6 +178,12 @@ class Oracle:
         x = np.ascontiguousarray(x, dtype=np.float32)
         assert x.shape == self.layer_shapes[layer]
         assert lib().pgo_set_params(self._h, worker, layer, _ptr(x)) == 0
+
+    def add_params(self, worker: int, layer: int, delta: np.ndarray) -> None:
+        """X_worker[layer] += delta in fp64 (Algorithm 1's -eta*G term)."""
+        d = np.ascontiguousarray(delta, dtype=np.float64)
+        assert d.shape == self.layer_shapes[layer]
+        assert lib().pgo_add_params(self._h, worker, layer, _ptr(d)) == 0
 
     def get_params(self, worker: int, layer: int) -> np.ndarray:
         out = np.zeros(self.layer_shapes[layer], dtype=np.float64)

@@ -27,7 +27,7 @@ EXPORTS = (
     "pg_get_round", "pg_set_round", "pg_kernel_launches", "pg_status_string",
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
     "pg_transposed_product_noalloc", "pg_rounds", "pg_selftest_barrier_timeout",
-    "pg_set_half_step",
+    "pg_set_half_step", "pg_params_device",
 )
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
                 "pair_sweep", "pair_edge", "update_only")
@@ -72,6 +72,7 @@ def load_library() -> ctypes.CDLL:
     L.pg_write_params.argtypes = [vp, i32, i32, vp, vp]
     L.pg_read_params.argtypes = [vp, i32, i32, vp, vp]
     L.pg_round.argtypes = [vp, vp]
+    L.pg_params_device.argtypes = [vp, i32, i32, vp, ctypes.POINTER(vp), ctypes.POINTER(i64)]
     L.pg_device_status.argtypes = [vp, vp]
     L.pg_rounds.argtypes = [vp, i32, vp]
     L.pg_set_half_step.argtypes = [vp, i32]
@@ -249,6 +250,20 @@ class PowerGossip:
         _check(self._lib.pg_read_params(self._h, worker, layer, ptr, _stream_handle(stream)),
                "pg_read_params")
         return out
+
+    def pg_params_device(self, worker: int, layer: int, stream=None):
+        """(rows x cols) torch view of the worker's matrix in the workspace (row stride = the
+        padded leading dimension), for in-place local updates such as  X -= eta * G."""
+        import torch
+
+        ptr, ld = ctypes.c_void_p(), ctypes.c_int64(0)
+        _check(self._lib.pg_params_device(self._h, worker, layer, _stream_handle(stream), ctypes.byref(ptr),
+                                          ctypes.byref(ld)), "pg_params_device")
+        n, m = self.layer_shapes[layer]
+        offset = (ptr.value - self._workspace.data_ptr()) // 4
+        flat = self._workspace.view(torch.float32) if self._workspace.data_ptr() % 4 == 0 else None
+        assert flat is not None
+        return torch.as_strided(flat, (n, m), (int(ld.value), 1), storage_offset=int(offset))
 
     def pg_read_q(self, i: int, j: int, layer: int, stream=None) -> np.ndarray:
         """(cols, rank) array."""

@@ -676,6 +676,20 @@ int pg_read_params(pg_ctx* c, int32_t worker, int32_t layer, float* host_dst, vo
     return device_status(c, static_cast<cudaStream_t>(stream));
 }
 
+int pg_params_device(pg_ctx* c, int32_t worker, int32_t layer, void* stream, float** dev_ptr_out,
+                     int64_t* ld_out) {
+    int rc = check_worker_layer(c, worker, layer);
+    if (rc != PG_OK || !dev_ptr_out || !ld_out) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    rc = flush_pending(c, static_cast<cudaStream_t>(stream));
+    if (rc != PG_OK) return rc;
+    const LayerGeom& g = c->lay.layers[layer];
+    *dev_ptr_out = c->st.X + static_cast<long long>(worker) * c->st.x_stride + g.x_off;
+    *ld_out = g.ld;
+    c->y_valid = false;     // the caller is about to change X
+    return PG_OK;
+}
+
 int pg_device_status(pg_ctx* c, void* stream) {
     if (!c) return PG_ERR_INVALID;
     if (!bind_device(c)) return PG_ERR_CUDA;

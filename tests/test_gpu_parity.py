@@ -398,3 +398,30 @@ def test_half_step_mode_is_refused_where_it_does_not_apply():
         net.pg_set_half_step()
     assert e.value.status == pg.PG_ERR_STATE
     net.close()
+
+
+# ---- Algorithm 1: a local gradient term between gossip rounds ----------------
+@pytest.mark.parametrize("w", [wl.tiny_ring(), wl.shrink(wl.lstm_matching32(), [(130, 70), (70, 1300)], 6).replace(n_workers=8)],
+                         ids=lambda w: w.name)
+def test_local_gradient_steps_between_rounds(w):
+    """X_i <- X_i + gossip - eta G with a synthetic per-worker G, applied by the caller
+    in place through pg_params_device (torch) and by add_params on the checker."""
+    import torch
+
+    oracle, net = common.oracle_for(w), common.network_for(w)
+    common.load_both(w, oracle, net)
+    eta = 0.05
+    for t in range(6):
+        net.pg_round()
+        oracle.round()
+        for i in range(w.n_workers):
+            for l, (n, m) in enumerate(w.layer_shapes):
+                g = np.random.default_rng([t, i, l]).standard_normal((n, m)).astype(np.float32)
+                view = net.pg_params_device(i, l)
+                assert tuple(view.shape) == (n, m)
+                view -= eta * torch.from_numpy(g).to(view.device)
+                oracle.add_params(i, l, -(np.float64(np.float32(eta)) * g.astype(np.float64)))
+        err, where = common.max_relative_error(w, oracle, net)
+        assert err <= REL_TOL, (t, err, where)
+    net.close()
+    oracle.close()
