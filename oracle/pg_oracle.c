@@ -252,6 +252,8 @@ typedef struct pgo_ctx {
     double **Ph;         /* last orthonormal left factor of the pair: rank columns of length rows */
     int max_edges;
     int half_step;       /* 1: Algorithm 2 read literally, one mat-vec per iteration */
+    int random_proj;     /* 0: power iteration; 1: random right projections R_k; 2: random left projections */
+    int64_t step;        /* random projections: steps taken so far (keys the directions) */
     int64_t iteration;   /* half-step mode: Algorithm 2's counter k (shared: all pairs move in lockstep) */
 } pgo_ctx;
 
@@ -579,11 +581,116 @@ static int half_step_round(pgo_ctx *c)
     return 0;
 }
 
+/* ------------------------------------------------------------------------- */
+/* Random-projection compressors (Section 5.1, the examples after A5).        */
+/*   right:  R_k(X) = (X U) U^T,  U a uniformly drawn orthonormal cols x k      */
+/*   left :  L_k(X) = V (V^T X),  V a uniformly drawn orthonormal rows x k      */
+/* A fresh direction set per edge, layer and step; nothing is warm-started.    */
+/* Directions: entry e of column c for pair (i<j), layer l, step t is the same  */
+/* Philox/Box-Muller normal as the initial vectors, with the key               */
+/* (seed_lo ^ low32(t+1), seed_hi ^ high32(t+1) ^ 0x52503031), rounded to fp32; */
+/* the columns are then orthonormalised (modified Gram-Schmidt, same dependent- */
+/* column rule as the power step), which makes them uniform on the Stiefel      */
+/* manifold.  delta of A5 is k/cols (right) or k/rows (left).                   */
+/* ------------------------------------------------------------------------- */
+int pgo_set_random_projection(pgo_ctx *c, int mode)
+{
+    if (!c || mode < 0 || mode > 2 || c->round != 0 || c->half_step) return -1;
+    c->random_proj = mode;
+    c->step = 0;
+    return 0;
+}
+
+/* the orthonormal directions of one (pair, layer, step): len x rank, column-major, fp64 */
+void pgo_random_directions(uint64_t seed, int64_t step, int i, int j, int layer, int len, int rank, double *out)
+{
+    uint64_t t1 = (uint64_t)step + 1u;
+    uint64_t key = seed ^ (t1 & 0xFFFFFFFFu) ^ (((t1 >> 32) ^ 0x52503031u) << 32);
+    float *tmp = (float *)malloc(sizeof(float) * (size_t)len);
+    for (int k = 0; k < rank; ++k) {
+        double *u = out + (size_t)k * len;
+        pgo_init_q(key, i, j, layer, k, len, tmp);
+        for (int e = 0; e < len; ++e) u[e] = (double)tmp[e];
+        double pre = dot(u, u, len);
+        for (int h = 0; h < k; ++h) {
+            const double *uh = out + (size_t)h * len;
+            double a = dot(uh, u, len);
+            for (int e = 0; e < len; ++e) u[e] -= a * uh[e];
+        }
+        double nn = dot(u, u, len);
+        int ok = (nn > 0.0) && isfinite(nn) && (k == 0 || nn > 1e-10 * pre);
+        double inv = ok ? 1.0 / sqrt(nn) : 0.0;
+        for (int e = 0; e < len; ++e) u[e] = ok ? u[e] * inv : 0.0;
+    }
+    free(tmp);
+}
+
+static int random_projection_round(pgo_ctx *c)
+{
+    int *edges = (int *)malloc(sizeof(int) * 2 * (size_t)c->max_edges);
+    double *w = (double *)malloc(sizeof(double) * (size_t)c->max_edges);
+    int E = pgo_round_schedule(c, c->round, edges, w);
+    if (E < 0) { free(edges); free(w); return -1; }
+    const int rank = c->rank, right = c->random_proj == 1;
+    double **dirs = (double **)calloc((size_t)E * (size_t)c->L, sizeof(double *));
+    double **prod = (double **)calloc((size_t)E * (size_t)c->L, sizeof(double *));
+    for (int step = 0; step < c->power_steps; ++step) {
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+        for (int l = 0; l < c->L; ++l)
+            for (int e = 0; e < E; ++e) {
+                int i = edges[2 * e], j = edges[2 * e + 1];
+                int n = c->rows[l], m = c->cols[l];
+                int len_in = right ? m : n, len_out = right ? n : m;
+                size_t u = (size_t)e * (size_t)c->L + (size_t)l;
+                dirs[u] = (double *)malloc(sizeof(double) * (size_t)len_in * (size_t)rank);
+                prod[u] = (double *)malloc(sizeof(double) * (size_t)len_out * (size_t)rank);
+                pgo_random_directions(c->seed, c->step, i, j, l, len_in, rank, dirs[u]);
+                double *tmp = (double *)malloc(sizeof(double) * (size_t)len_out);
+                const double *Xi = c->X[(size_t)i * c->L + l], *Xj = c->X[(size_t)j * c->L + l];
+                for (int k = 0; k < rank; ++k) {
+                    double *o = prod[u] + (size_t)k * len_out;
+                    const double *d = dirs[u] + (size_t)k * len_in;
+                    if (right) { matvec(Xi, n, m, d, o); matvec(Xj, n, m, d, tmp); }
+                    else       { matvec_t(Xi, n, m, d, o); matvec_t(Xj, n, m, d, tmp); }
+                    for (int a = 0; a < len_out; ++a) o[a] -= tmp[a];
+                }
+                free(tmp);
+            }
+        for (int l = 0; l < c->L; ++l) {
+            int n = c->rows[l], m = c->cols[l];
+            for (int e = 0; e < E; ++e) {
+                int i = edges[2 * e], j = edges[2 * e + 1];
+                size_t u = (size_t)e * (size_t)c->L + (size_t)l;
+                double *Xi = c->X[(size_t)i * c->L + l], *Xj = c->X[(size_t)j * c->L + l];
+                for (int k = 0; k < rank; ++k) {
+                    const double *left = right ? prod[u] + (size_t)k * n : dirs[u] + (size_t)k * n;
+                    const double *rightv = right ? dirs[u] + (size_t)k * m : prod[u] + (size_t)k * m;
+                    for (int r = 0; r < n; ++r) {
+                        double a = w[e] * left[r];
+                        for (int cidx = 0; cidx < m; ++cidx) {
+                            double d = a * rightv[cidx];
+                            Xi[(size_t)r * m + cidx] = Xi[(size_t)r * m + cidx] - d;   /* taken from i ...   */
+                            Xj[(size_t)r * m + cidx] = d + Xj[(size_t)r * m + cidx];   /* ... and given to j */
+                        }
+                    }
+                }
+                free(dirs[u]); free(prod[u]);
+                dirs[u] = prod[u] = NULL;
+            }
+        }
+        c->step += 1;
+    }
+    free(dirs); free(prod); free(edges); free(w);
+    c->round += 1;
+    return 0;
+}
+
 /* One gossip round = power_steps power steps on every layer and every edge of
  * this round's graph.  Returns 0, or -1 on an invalid schedule. */
 int pgo_round(pgo_ctx *c)
 {
     if (c->half_step) return half_step_round(c);
+    if (c->random_proj) return random_projection_round(c);
     int *edges = (int *)malloc(sizeof(int) * 2 * (size_t)c->max_edges);
     double *w = (double *)malloc(sizeof(double) * (size_t)c->max_edges);
     int E = pgo_round_schedule(c, c->round, edges, w);

@@ -81,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.pgo_average.restype = c_int
         L.pgo_compression_ratio.argtypes = [c_int, c_int, c_int, c_int]
         L.pgo_compression_ratio.restype = c_dbl
+        L.pgo_set_random_projection.argtypes = [vp, c_int]
+        L.pgo_set_random_projection.restype = c_int
+        L.pgo_random_directions.argtypes = [c_u64, c_i64, c_int, c_int, c_int, c_int, c_int, vp]
+        L.pgo_random_directions.restype = None
         L.pgo_set_half_step.argtypes = [vp, c_int]
         L.pgo_set_half_step.restype = c_int
         L.pgo_get_vector.argtypes = [vp, c_int, c_int, c_int, vp]
@@ -142,6 +146,16 @@ def compression_ratio(n: int, m: int, rank: int = 1, iterations: int = 1) -> flo
 
 def num_threads() -> int:
     return int(lib().pgo_num_threads())
+
+
+RANDOM_RIGHT, RANDOM_LEFT = 1, 2
+
+
+def random_directions(seed: int, step: int, i: int, j: int, layer: int, length: int, rank: int) -> np.ndarray:
+    """(length, rank) orthonormal directions of one pair, layer and step."""
+    out = np.zeros((rank, length), dtype=np.float64)
+    lib().pgo_random_directions(seed, step, i, j, layer, length, rank, _ptr(out))
+    return out.T.copy()
 
 
 class Oracle:
@@ -210,6 +224,12 @@ class Oracle:
         if lib().pgo_get_phat(self._h, i, j, layer, _ptr(out)) != 0:
             raise KeyError("pair has not been an edge yet")
         return out.T.copy()
+
+    def set_random_projection(self, mode: int) -> None:
+        """RANDOM_RIGHT: C(X) = (X U) U^T;  RANDOM_LEFT: C(X) = V (V^T X); fresh orthonormal
+        directions per edge, layer and step (0 switches back to power iteration)."""
+        if lib().pgo_set_random_projection(self._h, int(mode)) != 0:
+            raise ValueError("random projections must be chosen before the first round")
 
     def set_half_step(self, on: bool = True) -> None:
         """Algorithm 2 read literally: one mat-vec and one update per iteration;

@@ -37,6 +37,13 @@ MUTATIONS = {
     "half_step_vector_not_moved": ("memcpy(c->Q[t], out[u], sizeof(double) * (size_t)(odd ? n : m));", ";"),
     "half_step_update_not_antisymmetric": ("Xj[(size_t)r * m + cidx] = Xj[(size_t)r * m + cidx] + d;",
                                            "Xj[(size_t)r * m + cidx] = Xj[(size_t)r * m + cidx] - d;"),
+    # random-projection compressors
+    "random_directions_not_fresh": ("pgo_random_directions(c->seed, c->step, i, j, l, len_in, rank, dirs[u]);",
+                                    "pgo_random_directions(c->seed, 0, i, j, l, len_in, rank, dirs[u]);"),
+    "random_directions_not_orthogonalised": ("for (int e = 0; e < len; ++e) u[e] -= a * uh[e];", ";"),
+    "random_projection_left_uses_forward_product": (
+        "else       { matvec_t(Xi, n, m, d, o); matvec_t(Xj, n, m, d, tmp); }",
+        "else       { matvec_t(Xi, n, m, d, o); matvec_t(Xi, n, m, d, tmp); }"),
     "half_step_transposed_operand": ("else     { matvec_t(Xi, n, m, vh[u], pi); matvec_t(Xj, n, m, vh[u], pj); }",
                                      "else     { matvec_t(Xi, n, m, vh[u], pi); matvec_t(Xi, n, m, vh[u], pj); }"),
 }

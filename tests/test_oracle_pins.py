@@ -575,3 +575,132 @@ def test_half_step_identical_workers_stay_put():
     for i in range(4):
         assert np.array_equal(o.get_params(i, 0), x.astype(np.float64))
     o.close()
+
+
+# --------------------------------------------------------------------------
+# random-projection compressors (Section 5.1): R_k(X) = (X U) U^T,  L_k(X) = V (V^T X)
+# --------------------------------------------------------------------------
+def test_random_directions_are_orthonormal_keyed_and_uniform():
+    """u ~ uniform on the sphere means E[u u^T] = I/len, and for k orthonormal columns
+    E[U U^T] = (k/len) I: the delta of assumption A5."""
+    U = po.random_directions(9, 0, 0, 1, 0, 40, 4)
+    assert np.allclose(U.T @ U, np.eye(4), atol=1e-12)
+    assert np.array_equal(U, po.random_directions(9, 0, 0, 1, 0, 40, 4))
+    for other in (po.random_directions(9, 1, 0, 1, 0, 40, 4), po.random_directions(10, 0, 0, 1, 0, 40, 4),
+                  po.random_directions(9, 0, 0, 2, 0, 40, 4), po.random_directions(9, 0, 0, 1, 1, 40, 4)):
+        assert np.abs(other - U).max() > 0.05
+    for k in (1, 2):
+        acc = np.zeros((6, 6))
+        T = 6000
+        for t in range(T):
+            V = po.random_directions(3, t, 0, 1, 0, 6, k)
+            acc += V @ V.T
+        assert np.abs(acc / T - (k / 6.0) * np.eye(6)).max() < 0.02
+    # more columns than dimensions: the surplus columns are dropped
+    V = po.random_directions(3, 0, 0, 1, 0, 2, 4)
+    assert np.allclose(V[:, :2].T @ V[:, :2], np.eye(2), atol=1e-12) and np.all(V[:, 2:] == 0)
+
+
+@pytest.mark.parametrize("mode", [po.RANDOM_RIGHT, po.RANDOM_LEFT])
+@pytest.mark.parametrize("case", [CASES[1], CASES[2], CASES[3]])
+def test_random_projection_average_conserved_and_distance_never_grows(mode, case):
+    rng = np.random.default_rng(8)
+    o = po.Oracle(seed=29, **case)
+    o.set_random_projection(mode)
+    _fill(o, rng)
+    avg0 = [o.average(l) for l in range(len(o.layer_shapes))]
+    d_prev = o.consensus_distance()
+    for _ in range(8):
+        o.round()
+        for l in range(len(o.layer_shapes)):
+            assert np.abs(o.average(l) - avg0[l]).max() <= 1e-13 * max(np.abs(avg0[l]).max(), 1.0)
+        d = o.consensus_distance()
+        assert d <= d_prev * (1 + 1e-12)
+        d_prev = d
+    o.close()
+
+
+@pytest.mark.parametrize("mode,shape,rank", [(po.RANDOM_RIGHT, (7, 3), 3), (po.RANDOM_RIGHT, (5, 1), 1),
+                                             (po.RANDOM_LEFT, (3, 7), 3), (po.RANDOM_LEFT, (2, 9), 4)])
+def test_random_projection_with_a_full_basis_is_plain_gossip(mode, shape, rank):
+    """k = cols (right) or k = rows (left): U U^T = I, so the step is X <- W X (Eq. 1)."""
+    rng = np.random.default_rng(16)
+    N = 6
+    W = _ring_W(N, 0.3)
+    o = po.Oracle(kind=po.RING, n_workers=N, layer_shapes=[shape], rank=rank, power_steps=1, seed=33,
+                  weight_rule=po.W_EXPLICIT, W=W)
+    o.set_random_projection(mode)
+    xs = _fill(o, rng)
+    X = np.stack([xs[i][0] for i in range(N)])
+    o.round()
+    expect = np.einsum("ij,jnm->inm", W.astype(np.float64), X)
+    got = np.stack([o.get_params(i, 0) for i in range(N)])
+    assert np.allclose(got, expect, rtol=0, atol=1e-12)
+    o.close()
+
+
+@pytest.mark.parametrize("mode", [po.RANDOM_RIGHT, po.RANDOM_LEFT])
+def test_random_projection_one_step_is_the_projector_update(mode):
+    """Eq. (compressed consensus): X_i += sum_j W_ij (C(X_j) - C(X_i)) with the step's own directions."""
+    rng = np.random.default_rng(21)
+    N, n, m, k = 5, 7, 9, 2
+    W = _ring_W(N, 0.25)
+    o = po.Oracle(kind=po.RING, n_workers=N, layer_shapes=[(n, m)], rank=k, power_steps=1, seed=41,
+                  weight_rule=po.W_EXPLICIT, W=W)
+    o.set_random_projection(mode)
+    xs = _fill(o, rng)
+    X = [xs[i][0] for i in range(N)]
+    edges, w = o.round_schedule()
+    new = [x.copy() for x in X]
+    for (i, j), wij in zip(edges, w):
+        if mode == po.RANDOM_RIGHT:
+            U = po.random_directions(41, 0, i, j, 0, m, k)
+            C = lambda A: (A @ U) @ U.T
+        else:
+            V = po.random_directions(41, 0, i, j, 0, n, k)
+            C = lambda A: V @ (V.T @ A)
+        new[i] += wij * (C(X[j]) - C(X[i]))
+        new[j] += wij * (C(X[i]) - C(X[j]))
+    o.round()
+    for i in range(N):
+        assert np.allclose(o.get_params(i, 0), new[i], rtol=0, atol=1e-12)
+    o.close()
+
+
+def test_random_projection_directions_are_fresh_every_step():
+    """An isolated pair with W = 1/2 loses the component of D along u entirely at every
+    step; with fresh directions E||D||^2 shrinks by (1 - 1/cols) per step, so D vanishes."""
+    o = _pair(5, 6, 0.5, 1)
+    o.set_half_step(False)
+    o.set_random_projection(po.RANDOM_RIGHT)
+    xs = _fill(o, np.random.default_rng(3))
+    d0 = np.linalg.norm(xs[0][0] - xs[1][0])
+    o.round(250)
+    assert np.linalg.norm(o.get_params(0, 0) - o.get_params(1, 0)) < 1e-6 * d0
+    o.close()
+
+
+def test_theorem_1_contraction_in_expectation():
+    """Theorem 1: E sum_i ||X_i - mean||^2 shrinks by at least (1 - rho delta) per step,
+    rho = 1 - lambda_2(W)^2, delta = k/cols for R_k.  Averaged over 400 direction seeds."""
+    rng = np.random.default_rng(31)
+    N, n, m, k = 6, 4, 6, 1
+    W = _ring_W(N, 0.3)
+    lam = np.sort(np.abs(np.linalg.eigvalsh(W.astype(np.float64))))[::-1]
+    rho, delta = 1.0 - lam[1] ** 2, k / m
+    X = [(rng.standard_normal((n, m))).astype(np.float32) for _ in range(N)]
+    ratios = []
+    for seed in range(400):
+        o = po.Oracle(kind=po.RING, n_workers=N, layer_shapes=[(n, m)], rank=k, power_steps=1, seed=seed,
+                      weight_rule=po.W_EXPLICIT, W=W)
+        o.set_random_projection(po.RANDOM_RIGHT)
+        for i in range(N):
+            o.set_params(i, 0, X[i])
+        d0 = o.consensus_distance()
+        o.round()
+        ratios.append(o.consensus_distance() / d0)
+        o.close()
+    ratios = np.array(ratios)
+    sem = ratios.std() / np.sqrt(len(ratios))
+    assert ratios.mean() <= (1.0 - rho * delta) + 3 * sem
+    assert ratios.mean() < 1.0 - 0.5 * rho * delta        # and it does contract
