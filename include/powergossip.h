@@ -194,6 +194,23 @@ PG_API int pg_round(pg_ctx *ctx, void *stream);
 PG_API int pg_set_half_step(pg_ctx *ctx, int32_t on);
 
 /*
+ * Random-projection compressors instead of power iteration (Section 5.1, the
+ * examples after Assumption A5; the paper's comparison "random projections vs
+ * power iteration"):
+ *   PG_RANDOM_RIGHT  C(X) = (X U) U^T,  U uniformly drawn orthonormal cols x rank   (delta = rank/cols)
+ *   PG_RANDOM_LEFT   C(X) = V (V^T X),  V uniformly drawn orthonormal rows x rank   (delta = rank/rows)
+ * Fresh directions for every edge, layer and power step, nothing warm-started:
+ * Philox4x32-10 / Box-Muller normals as for the initial vectors, under the key
+ * (seed_lo ^ low32(t+1), seed_hi ^ high32(t+1) ^ 0x52503031) for step t, then
+ * Gram-Schmidt.  The stored per-pair vectors are overwritten by the directions.
+ * Call before the first round; not available on graphs of degree <= 1 at rank 1
+ * (PG_ERR_INVALID), nor together with half-step mode.  A step costs one read of X
+ * for the product and one read + write for the update (12 B per parameter).
+ */
+enum { PG_POWER_ITERATION = 0, PG_RANDOM_RIGHT = 1, PG_RANDOM_LEFT = 2 };
+PG_API int pg_set_random_projection(pg_ctx *ctx, int32_t mode);
+
+/*
  * Enqueue `n_rounds` rounds (same result as calling pg_round that many times).
  * When the graph is static and the whole stack is small enough to stay in L2
  * (at most 64 MiB of parameters, degree > 1 or rank > 1), all rounds run in ONE

@@ -27,8 +27,9 @@ EXPORTS = (
     "pg_get_round", "pg_set_round", "pg_kernel_launches", "pg_status_string",
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
     "pg_transposed_product_noalloc", "pg_rounds", "pg_selftest_barrier_timeout",
-    "pg_set_half_step", "pg_params_device",
+    "pg_set_half_step", "pg_params_device", "pg_set_random_projection",
 )
+PG_POWER_ITERATION, PG_RANDOM_RIGHT, PG_RANDOM_LEFT = 0, 1, 2
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
                 "pair_sweep", "pair_edge", "update_only")
 
@@ -76,6 +77,7 @@ def load_library() -> ctypes.CDLL:
     L.pg_device_status.argtypes = [vp, vp]
     L.pg_rounds.argtypes = [vp, i32, vp]
     L.pg_set_half_step.argtypes = [vp, i32]
+    L.pg_set_random_projection.argtypes = [vp, i32]
     L.pg_selftest_barrier_timeout.argtypes = [vp, vp]
     L.pg_get_schedule.argtypes = [vp, i64, vp, vp, ctypes.POINTER(i32)]
     L.pg_max_edges.argtypes = [vp, ctypes.POINTER(i32)]
@@ -283,6 +285,9 @@ class PowerGossip:
 
     def pg_set_half_step(self, on: bool = True) -> None:
         _check(self._lib.pg_set_half_step(self._h, 1 if on else 0), "pg_set_half_step")
+
+    def pg_set_random_projection(self, mode: int) -> None:
+        _check(self._lib.pg_set_random_projection(self._h, int(mode)), "pg_set_random_projection")
 
     def pg_rounds(self, n_rounds: int, stream=None) -> None:
         _check(self._lib.pg_rounds(self._h, int(n_rounds), _stream_handle(stream)), "pg_rounds")

@@ -267,6 +267,7 @@ struct pg_ctx {
     bool half_step = false;
     int64_t iteration = 0;      // Algorithm 2's counter k
     bool half_pending = false;  // an odd iteration's update has not been applied to X yet
+    int random_proj = 0;        // 0 power iteration, 1 random right projections, 2 random left projections
     bool static_graph = true;
     bool coop_ok = false;       // the device supports cooperative launches
     int device = 0;
@@ -708,6 +709,49 @@ int pg_round(pg_ctx* c, void* stream_v) {
     const int n_rows = static_cast<int>(c->lay.n_row_tiles), n_cols = static_cast<int>(c->lay.n_col_tiles);
     const bool has_pair = c->lay.n_pair_tiles > 0;
     bool ok = true;
+    if (c->random_proj) {
+        // fresh orthonormal directions, one product, the raw difference, the update
+        DevState st = c->st;
+        st.Ph = c->ph_buf[0];
+        for (int p = 0; p < c->power_steps && ok; ++p) {
+            const uint64_t t1 = static_cast<uint64_t>(c->step) + 1u;
+            const uint64_t key = c->seed ^ (t1 & 0xFFFFFFFFu) ^ (((t1 >> 32) ^ 0x52503031u) << 32);
+            const unsigned klo = static_cast<unsigned>(key), khi = static_cast<unsigned>(key >> 32);
+            {
+                Timed t(c, PG_KERNEL_EDGE_LEFT, stream, 0.0);
+                ok = ok && pg::launch_random_directions(st, tab, c->lay.max_edges, klo, khi,
+                                                        c->random_proj == 1 ? 0 : 1, stream) == cudaSuccess;
+            }
+            if (c->random_proj == 1) {
+                {
+                    Timed t(c, PG_KERNEL_FORWARD, stream, c->normal_param_bytes);
+                    ok = ok && pg::launch_forward(st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+                }
+                Timed t(c, PG_KERNEL_EDGE_RIGHT, stream, 0.0);
+                ok = ok && pg::launch_edge_raw(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+            } else {
+                {
+                    Timed t(c, PG_KERNEL_TRANSPOSED, stream, c->normal_param_bytes);
+                    ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+                }
+                Timed t(c, PG_KERNEL_EDGE_RIGHT, stream, 0.0);
+                ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+            }
+            {
+                Timed t(c, PG_KERNEL_UPDATE_ONLY, stream, 2.0 * c->normal_param_bytes);
+                ok = ok && pg::launch_update(st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+            }
+            c->launches += 4;
+            c->step += 1;
+        }
+        c->y_valid = false;
+        if (!ok) {
+            cudaGetLastError();
+            return PG_ERR_CUDA;
+        }
+        c->round += 1;
+        return PG_OK;
+    }
     if (c->half_step) {
         // `power_steps` iterations of Algorithm 2.  Odd: X q-hat -> p; its update stays
         // pending and is applied by the even iteration's transposed sweep.  Even:
@@ -829,9 +873,17 @@ int pg_round(pg_ctx* c, void* stream_v) {
 int pg_set_half_step(pg_ctx* c, int32_t on) {
     if (!c) return PG_ERR_INVALID;
     if (c->round != 0 || c->pending || c->y_valid) return PG_ERR_STATE;
-    if (on && (c->rank != 1 || !c->static_graph || c->lay.n_pair_tiles > 0)) return PG_ERR_INVALID;
+    if (on && (c->rank != 1 || !c->static_graph || c->lay.n_pair_tiles > 0 || c->random_proj)) return PG_ERR_INVALID;
     c->half_step = on != 0;
     c->iteration = 0;
+    return PG_OK;
+}
+
+int pg_set_random_projection(pg_ctx* c, int32_t mode) {
+    if (!c || mode < 0 || mode > 2) return PG_ERR_INVALID;
+    if (c->round != 0 || c->pending || c->y_valid || c->half_step) return PG_ERR_STATE;
+    if (mode != 0 && c->lay.n_pair_tiles > 0) return PG_ERR_INVALID;
+    c->random_proj = mode;
     return PG_OK;
 }
 
@@ -843,7 +895,7 @@ int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
     // One cooperative launch when the graph is static, no layer uses the pair sweep and the
     // whole stack stays in L2; otherwise the rounds are enqueued one by one.
     const double x_bytes = c->normal_param_bytes;
-    const bool persistent = c->static_graph && !c->half_step && c->lay.n_pair_tiles == 0 && c->coop_ok &&
+    const bool persistent = c->static_graph && !c->half_step && !c->random_proj && c->lay.n_pair_tiles == 0 && c->coop_ok &&
                             x_bytes <= 64.0 * 1024 * 1024 && !c->timing;
     if (!persistent) {
         for (int r = 0; r < n_rounds; ++r) {

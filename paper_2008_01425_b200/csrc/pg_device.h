@@ -121,6 +121,11 @@ cudaError_t launch_update_forward(const DevState& st, const int* tab_update, con
 cudaError_t launch_edge_odd(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_transposed_update(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
                                      cudaStream_t stream);
+// random-projection compressors: fresh orthonormal directions per (edge, layer) into Q
+// (side 0, length cols) or P-hat (side 1, length rows); raw difference of the forward products
+cudaError_t launch_random_directions(const DevState& st, const int* tab, int max_edges, unsigned key_lo,
+                                     unsigned key_hi, int side, cudaStream_t stream);
+cudaError_t launch_edge_raw(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile* tiles, int n_tiles,
                           cudaStream_t stream);
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,

@@ -589,6 +589,120 @@ edge_right_kernel(DevState st, const int* __restrict__ tab) {
     edge_right_step<false>(st, tab, e, l, scratch);
 }
 
+// --------------------------------------------------------------------------
+// Random-projection compressors (Section 5.1 of the paper): fresh directions.
+// Philox4x32-10 (Salmon et al., SC'11) and Box-Muller in fp64, the same stream
+// as the seeded initial vectors but under the step's key; entry e of column k of
+// pair (i<j), layer l uses counter (e/4, l, i, j*256+k).  The rank columns are
+// then orthonormalised (modified Gram-Schmidt in fp64 against the stored fp32
+// columns, same dependent-column rule as the power step).
+// side 0: directions in R^cols, written to the pair's Q with 1/norm = 1;
+// side 1: directions in R^rows, written to the edge's P-hat.
+// One CTA per (edge, layer).
+// --------------------------------------------------------------------------
+__device__ __forceinline__ void philox4x32_10(unsigned c0, unsigned c1, unsigned c2, unsigned c3,
+                                              unsigned k0, unsigned k1, unsigned out[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const unsigned hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const unsigned hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        const unsigned n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+__global__ void __launch_bounds__(256)
+random_directions_kernel(DevState st, const int* __restrict__ tab, unsigned key_lo, unsigned key_hi, int side) {
+    __shared__ double scratch[33];
+    const int L = st.n_layers, rank = st.rank;
+    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[l];
+    const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
+    const int pair = tab[st.tab.off_pair + e];
+    const int len = side == 0 ? g.m : g.n;
+    const int stride = side == 0 ? g.ld : g.npad;
+    float* dst = side == 0 ? st.Q + (long long)pair * st.q_stride + g.q_off
+                           : st.Ph + (long long)e * st.ph_stride + g.ph_off;
+    double coef[kMaxRank];
+    for (int k = 0; k < rank; ++k) {
+        float* col = dst + (long long)k * stride;
+        for (int b = threadIdx.x; 4 * b < stride; b += blockDim.x) {
+            unsigned x[4];
+            philox4x32_10((unsigned)b, (unsigned)l, (unsigned)wi, (unsigned)wj * 256u + (unsigned)k, key_lo, key_hi, x);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const double u1 = ((double)x[2 * h] + 0.5) * (1.0 / 4294967296.0);
+                const double u2 = ((double)x[2 * h + 1] + 0.5) * (1.0 / 4294967296.0);
+                const double radius = sqrt(-2.0 * log(u1));
+                const double angle = 6.283185307179586476925286766559 * u2;
+                const int e0 = 4 * b + 2 * h;
+                if (e0 < stride) col[e0] = e0 < len ? (float)(radius * cos(angle)) : 0.0f;
+                if (e0 + 1 < stride) col[e0 + 1] = e0 + 1 < len ? (float)(radius * sin(angle)) : 0.0f;
+            }
+        }
+        __syncthreads();
+        auto resid = [&](int r, int upto) {
+            double v = (double)col[r];
+            for (int h = 0; h < upto; ++h) v -= coef[h] * (double)dst[(long long)h * stride + r];
+            return v;
+        };
+        double part = 0.0;
+        for (int r = threadIdx.x; r < len; r += blockDim.x) part += (double)col[r] * (double)col[r];
+        const double pre = block_sum(part, scratch);
+        for (int h = 0; h < k; ++h) {
+            part = 0.0;
+            for (int r = threadIdx.x; r < len; r += blockDim.x) part += resid(r, h) * (double)dst[(long long)h * stride + r];
+            coef[h] = block_sum(part, scratch);
+        }
+        part = 0.0;
+        for (int r = threadIdx.x; r < len; r += blockDim.x) {
+            const double v = resid(r, k);
+            part += v * v;
+        }
+        const double nn = block_sum(part, scratch);
+        const bool live = isfinite(nn) && nn > 0.0 && (k == 0 || nn > 1e-10 * pre);
+        const double inv = live ? 1.0 / sqrt(nn) : 0.0;
+        for (int r = threadIdx.x; r < len; r += blockDim.x) col[r] = live ? (float)(resid(r, k) * inv) : 0.0f;
+        if (threadIdx.x == 0) {
+            if (side == 0) st.Qinv[((long long)pair * L + l) * rank + k] = live ? 1.0f : 0.0f;
+            st.live[((long long)e * L + l) * rank + k] = 1;
+        }
+        __syncthreads();
+    }
+}
+
+// P = Y[i] - Y[j], unnormalised (the directions are orthonormal already): the
+// left factor of the random right projection's update (X_i U - X_j U) U^T.
+__global__ void __launch_bounds__(256)
+edge_raw_kernel(DevState st, const int* __restrict__ tab) {
+    const int L = st.n_layers, rank = st.rank;
+    const int e = blockIdx.x / L, l = blockIdx.x - e * L;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[l];
+    const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
+    const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
+    const float* Yi = st.Y + (long long)wi * st.y_stride + g.y_off;
+    const float* Yj = st.Y + (long long)wj * st.y_stride + g.y_off;
+    float* Ph = st.Ph + (long long)e * st.ph_stride + g.ph_off;
+    for (int k = 0; k < rank; ++k) {
+        const float* yi = Yi + (long long)(si * rank + k) * g.f_csplit * g.npad;
+        const float* yj = Yj + (long long)(sj * rank + k) * g.f_csplit * g.npad;
+        for (int r = threadIdx.x; r < g.npad; r += blockDim.x) {
+            double a = 0.0, b = 0.0;
+            if (r < g.n)
+                for (int cs = 0; cs < g.f_csplit; ++cs) {
+                    a += (double)yi[(long long)cs * g.npad + r];
+                    b += (double)yj[(long long)cs * g.npad + r];
+                }
+            Ph[(long long)k * g.npad + r] = (float)(a - b);
+        }
+    }
+}
+
 // 1 / ||Q|| of a pair-sweep layer from the shares the pair edge step left.
 __device__ __forceinline__ float pair_qinv(const DevState& st, int pair, int layer) {
     const double* n2 = st.Qn2 + ((long long)pair * st.n_layers + layer) * kEdgeChunks;
@@ -1263,6 +1377,17 @@ cudaError_t launch_transposed(const DevState& st, const int* tab, const Tile* ti
 cudaError_t launch_transposed_update(const DevState& st, const int* tab, const Tile* tiles, int n_tiles,
                                      cudaStream_t stream) {
     return launch_col<true>(st, tab, tiles, n_tiles, stream);
+}
+
+cudaError_t launch_random_directions(const DevState& st, const int* tab, int max_edges, unsigned key_lo,
+                                     unsigned key_hi, int side, cudaStream_t stream) {
+    random_directions_kernel<<<max_edges * st.n_layers, 256, 0, stream>>>(st, tab, key_lo, key_hi, side);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_edge_raw(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
+    edge_raw_kernel<<<max_edges * st.n_layers, 256, 0, stream>>>(st, tab);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_edge_odd(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {

@@ -425,3 +425,49 @@ def test_local_gradient_steps_between_rounds(w):
         assert err <= REL_TOL, (t, err, where)
     net.close()
     oracle.close()
+
+
+# ---- random-projection compressors (Section 5.1) ------------------------------
+RANDOM_CASES = [
+    wl.tiny_ring().replace(rounds=30),
+    wl.tiny_ring().replace(rounds=10, rank=4, power_steps=2),
+    wl.resnet20_ring8().replace(rounds=20),
+    wl.shrink(wl.torus8x8(2), [(200, 136)], 20).replace(rank=2),
+    wl.Workload("rand_edge", 9, 4, wl.RING, 0, 0, wl.W_EXPLICIT, 0.3,
+                ((67, 131), (5, 3), (9, 1), (1, 9), (3, 2500)), 2, 1, 8, 77, "normal1"),
+]
+
+
+@pytest.mark.parametrize("mode", [1, 2], ids=["right", "left"])
+@pytest.mark.parametrize("w", RANDOM_CASES, ids=lambda w: "%s_r%d" % (w.name, w.rank))
+def test_random_projection_compressors(w, mode):
+    """The update is linear in X for given directions, so a free-running comparison over all
+    rounds is meaningful here (no warm-started state, no chaos)."""
+    from paper_2008_01425_b200 import binding as pg
+
+    oracle, net = common.oracle_for(w), common.network_for(w)
+    oracle.set_random_projection(mode)
+    common.load_both(w, oracle, net)
+    net.pg_set_random_projection(mode)
+    avg0 = [common.initial_average(w, l) for l in range(len(w.layer_shapes))]
+    for _ in range(w.rounds):
+        net.pg_round()
+    oracle.round(w.rounds)
+    err, where = common.max_relative_error(w, oracle, net)
+    assert err <= REL_TOL, (err, where)
+    assert net.pg_device_status() == pg.PG_OK
+    _check_average(w, net, avg0)
+    d_ref, d_gpu = oracle.consensus_distance(), common.gpu_consensus_distance(w, net)
+    assert abs(d_gpu - d_ref) <= 1e-3 * d_ref
+    net.close()
+    oracle.close()
+
+
+def test_random_projection_is_refused_on_a_matching():
+    from paper_2008_01425_b200 import binding as pg
+
+    net = common.network_for(wl.shrink(wl.lstm_matching32(), [(30, 20)], 1).replace(n_workers=4))
+    with pytest.raises(pg.PowerGossipError) as e:
+        net.pg_set_random_projection(pg.PG_RANDOM_RIGHT)
+    assert e.value.status == pg.PG_ERR_INVALID
+    net.close()
