@@ -156,7 +156,10 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         z += round_up(static_cast<long long>(slots) * g.t_rtiles * g.ld, 64);
         g.pair_mode = !lay.pair_mode ? 0 : (g.ld <= pg::kPairMaxLd ? 1 : (g.ld <= pg::kPairWideMaxLd ? 2 : 0));
         g.p_slice = static_cast<int>(round_up((g.ld + pg::kPairCluster - 1) / pg::kPairCluster, 4));
-        g.p_rows = pg::kPairTileRows;
+        {   // equal tiles of at most kPairTileRows rows (a multiple of 8: one row per warp and stage)
+            const int parts = (g.n + pg::kPairTileRows - 1) / pg::kPairTileRows;
+            g.p_rows = static_cast<int>(round_up((g.n + parts - 1) / parts, 8));
+        }
         if (g.pair_mode == 2) {
             const int resident = query_device
                 ? pg::pair_wide_resident_clusters((g.p_slice / 4 + 255) / 256, g.p_slice) : 0;
@@ -510,6 +513,11 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
     st.Pn = reinterpret_cast<float*>(c->ws + lay.off_Pn);
     st.half_odd = 0;
+    {
+        // PG_PAIR_BULK=0 selects the register-fed variant of the row-per-warp pair sweep
+        const char* v = std::getenv("PG_PAIR_BULK");
+        st.pair_bulk = (v && v[0] == '0') ? 0 : 1;
+    }
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
     st.PhNext = st.Ph + static_cast<long long>(lay.max_edges) * lay.ph_stride;

@@ -97,6 +97,7 @@ struct DevState {
     float* Up;           // [edge][up_stride]    pair sweep: partial sums of D^T p
     double* Sp;          // [edge][sp_stride]    pair sweep: partial sums of ||p||^2
     float* Pn;           // [edge][layer]  half-step mode: ||p|| of the last odd iteration
+    int pair_bulk;       // row-per-warp pair sweep fed by bulk asynchronous copies (TMA)
     int half_odd;        // half-step mode: the update being applied is an odd iteration's,
                          // p q-hat^T = (||p|| / ||q||) p-hat q^T: scale the coefficients accordingly
     int* live;           // [edge][layer][rank]  1 if the column took part in this step

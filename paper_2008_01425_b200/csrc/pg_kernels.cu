@@ -19,6 +19,7 @@ namespace pg {
 namespace {
 
 constexpr int kStatusNumeric = 6;  // PG_ERR_NUMERIC
+constexpr int kStatusTimeout = 5;  // PG_ERR_TIMEOUT
 constexpr long long kBarrierSpinLimit = 1LL << 23;   // polls before a grid barrier gives up (a few seconds)
 
 // Rows a warp of the row sweep works on at once, per number of vectors S.
@@ -856,6 +857,246 @@ pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __re
 }
 
 // --------------------------------------------------------------------------
+// Pair sweep, row-per-warp variant fed by bulk asynchronous copies (TMA).
+// The rows of a tile are contiguous in memory (full rows, padded leading
+// dimension), so one thread moves kBulkRows rows of X_i and of X_j into shared
+// memory with two cp.async.bulk copies per stage; an mbarrier per stage counts
+// the bytes.  kBulkStages stages are in flight, so the loads of the next stages
+// never wait for registers or for the arithmetic of the current one.  Every
+// warp then works on one row of the stage out of shared memory exactly as the
+// register variant does, and writes the corrected rows straight to global
+// memory.  All mbarrier waits are bounded: a wait that runs out raises the
+// time-out bit of the status word and the CTA leaves after waiting (bounded
+// again) for the copies it still has in flight.
+// --------------------------------------------------------------------------
+constexpr int kBulkRows = 8;      // rows per stage = warps per CTA
+#ifndef PG_BULK_STAGES
+#define PG_BULK_STAGES 3
+#endif
+#ifndef PG_BULK_MIN_BLOCKS
+#define PG_BULK_MIN_BLOCKS 1
+#endif
+constexpr int kBulkStages = PG_BULK_STAGES;
+constexpr int kBulkSpinLimit = 1 << 24;
+
+__device__ __forceinline__ unsigned smem_addr(const void* p) {
+    return static_cast<unsigned>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// bytes and both addresses must be multiples of 16
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, unsigned bytes,
+                                          unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// waits for phase `parity` of `bar`; false if it gave up (or another thread did)
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity, volatile int* abort_flag,
+                                                  int* status) {
+    for (int spin = 0; spin < kBulkSpinLimit; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicOr(status, 1 << kStatusTimeout);
+    return false;
+}
+
+template <int NV, bool UPDATE>
+__global__ void __launch_bounds__(256, PG_BULK_MIN_BLOCKS)
+pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
+                       const Tile* __restrict__ tiles) {
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    __shared__ __align__(16) float s_q[NV * 128];
+    __shared__ __align__(16) float s_ui[NV * 128];
+    __shared__ __align__(16) float s_uj[NV * 128];
+    __shared__ __align__(8) unsigned long long s_full[kBulkStages];
+    __shared__ double s_s[8];
+    __shared__ int s_abort;
+
+    const Tile tile = tiles[blockIdx.x];
+    const int e = tile.worker;
+    if (e >= tab_cur[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[tile.layer];
+    const int wi = tab_cur[st.tab.off_edge_i + e], wj = tab_cur[st.tab.off_edge_j + e];
+    const int pair = tab_cur[st.tab.off_pair + e];
+    float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
+    float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
+    const int ld = g.ld;
+    const unsigned row_bytes = (unsigned)ld * 4u;                 // multiple of 16: ld is a multiple of 4
+    float* s_stage = reinterpret_cast<float*>(s_dyn);             // [stage][matrix][row][ld]
+
+    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float qinv = pair_qinv(st, pair, tile.layer);
+    const float* ui = q;
+    const float* uj = q;
+    const float* phi = nullptr;
+    const float* phj = nullptr;
+    float coef_i = 0.0f, coef_j = 0.0f;
+    if (UPDATE) {
+        if (tab_prev[st.tab.off_degree + wi] > 0) {
+            const int ep = tab_prev[st.tab.off_slot_edge + wi * st.tab.max_degree];
+            ui = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            phi = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            coef_i = __int_as_float(tab_prev[st.tab.off_slot_coef + wi * st.tab.max_degree]);
+        }
+        if (tab_prev[st.tab.off_degree + wj] > 0) {
+            const int ep = tab_prev[st.tab.off_slot_edge + wj * st.tab.max_degree];
+            uj = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            phj = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            coef_j = __int_as_float(tab_prev[st.tab.off_slot_coef + wj * st.tab.max_degree]);
+        }
+    }
+    const int r0 = tile.rtile * g.p_rows;
+    const int r1 = min(g.n, r0 + g.p_rows);
+    const int n_stages = (r1 - r0 + kBulkRows - 1) / kBulkRows;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s2 = 0; s2 < kBulkStages; ++s2) mbar_init(&s_full[s2], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int idx = threadIdx.x; idx < NV * 128; idx += 256) {
+        const bool in = idx < ld;
+        s_q[idx] = in ? q[idx] * qinv : 0.0f;
+        if (UPDATE) {
+            s_ui[idx] = in ? ui[idx] : 0.0f;
+            s_uj[idx] = in ? uj[idx] : 0.0f;
+        }
+    }
+    __syncthreads();
+
+    // stage `sidx` covers rows r0 + sidx*kBulkRows ...; both slabs are contiguous in global memory
+    auto issue = [&](int sidx) {
+        const int slot = sidx % kBulkStages;
+        const int row = r0 + sidx * kBulkRows;
+        const unsigned bytes = (unsigned)min(kBulkRows, r1 - row) * row_bytes;
+        float* dst = s_stage + (size_t)slot * 2 * kBulkRows * ld;
+        mbar_expect_tx(&s_full[slot], 2 * bytes);
+        bulk_load(dst, Xi + (long long)row * ld, bytes, &s_full[slot]);
+        bulk_load(dst + (size_t)kBulkRows * ld, Xj + (long long)row * ld, bytes, &s_full[slot]);
+    };
+    int issued = 0;
+    if (threadIdx.x == 0)
+        for (; issued < kBulkStages - 1 && issued < n_stages; ++issued) issue(issued);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    float4 u[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float ssum = 0.0f;
+    bool ok = true;
+
+    for (int it = 0; it < n_stages; ++it) {
+        const int slot = it % kBulkStages;
+        if (threadIdx.x == 0 && it + kBulkStages - 1 < n_stages) {
+            issue(it + kBulkStages - 1);      // its slot was read for the last time before the barrier below
+            issued = it + kBulkStages;
+        }
+        const bool mine = mbar_wait_bounded(&s_full[slot], (unsigned)((it / kBulkStages) & 1), &s_abort, st.status);
+        ok = __syncthreads_and(mine) != 0;        // either every thread goes on or all leave together
+        if (!ok) break;
+        const int r = r0 + it * kBulkRows + warp;
+        if (r < r1) {
+            const float* si = s_stage + (size_t)slot * 2 * kBulkRows * ld + (size_t)warp * ld;
+            const float* sj = si + (size_t)kBulkRows * ld;
+            float4 xi[NV], xj[NV];
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int col = (k * 32 + lane) * 4;
+                if (col < ld) {
+                    xi[k] = *reinterpret_cast<const float4*>(si + col);
+                    xj[k] = *reinterpret_cast<const float4*>(sj + col);
+                } else {
+                    xi[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    xj[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+            if (UPDATE) {
+                const float ai = phi ? coef_i * __ldg(phi + r) : 0.0f;
+                const float aj = phj ? coef_j * __ldg(phj + r) : 0.0f;
+                float* rowi = Xi + (long long)r * ld;
+                float* rowj = Xj + (long long)r * ld;
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    const int col = (k * 32 + lane) * 4;
+                    const float4 vi = *reinterpret_cast<const float4*>(&s_ui[col]);
+                    const float4 vj = *reinterpret_cast<const float4*>(&s_uj[col]);
+                    xi[k].x = fmaf(-ai, vi.x, xi[k].x); xi[k].y = fmaf(-ai, vi.y, xi[k].y);
+                    xi[k].z = fmaf(-ai, vi.z, xi[k].z); xi[k].w = fmaf(-ai, vi.w, xi[k].w);
+                    xj[k].x = fmaf(-aj, vj.x, xj[k].x); xj[k].y = fmaf(-aj, vj.y, xj[k].y);
+                    xj[k].z = fmaf(-aj, vj.z, xj[k].z); xj[k].w = fmaf(-aj, vj.w, xj[k].w);
+                    if (col < ld) {
+                        st_stream(rowi + col, xi[k]);
+                        st_stream(rowj + col, xj[k]);
+                    }
+                }
+            }
+            float dot = 0.0f;
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int col = (k * 32 + lane) * 4;
+                const float4 vq = *reinterpret_cast<const float4*>(&s_q[col]);
+                xi[k].x -= xj[k].x; xi[k].y -= xj[k].y; xi[k].z -= xj[k].z; xi[k].w -= xj[k].w;
+                dot = fmaf(xi[k].x, vq.x, dot); dot = fmaf(xi[k].y, vq.y, dot);
+                dot = fmaf(xi[k].z, vq.z, dot); dot = fmaf(xi[k].w, vq.w, dot);
+            }
+            const float p = warp_sum(dot);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                u[k].x = fmaf(p, xi[k].x, u[k].x); u[k].y = fmaf(p, xi[k].y, u[k].y);
+                u[k].z = fmaf(p, xi[k].z, u[k].z); u[k].w = fmaf(p, xi[k].w, u[k].w);
+            }
+            ssum = fmaf(p, p, ssum);
+            if (lane == 0) Pw[r] = p;
+        }
+        __syncthreads();          // every warp is done with this slot before it is filled again
+    }
+    if (!ok) {
+        // leave only after the copies still in flight have landed (bounded)
+        if (threadIdx.x == 0)
+            for (int sidx = 0; sidx < issued; ++sidx) {
+                const int slot = sidx % kBulkStages;
+                for (int spin = 0; spin < kBulkSpinLimit; ++spin)
+                    if (mbar_try_wait(&s_full[slot], (unsigned)((sidx / kBulkStages) & 1))) break;
+            }
+        return;
+    }
+    // the stage buffers are free now: reduce u across the warps through them
+    float* s_red = s_stage;                                  // [8][NV*128]
+#pragma unroll
+    for (int k = 0; k < NV; ++k) *reinterpret_cast<float4*>(&s_red[warp * NV * 128 + (k * 32 + lane) * 4]) = u[k];
+    if (lane == 0) s_s[warp] = (double)ssum;
+    __syncthreads();
+    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld;
+    for (int idx = threadIdx.x; idx < ld; idx += 256) {
+        float t = s_red[idx];
+#pragma unroll
+        for (int w8 = 1; w8 < 8; ++w8) t += s_red[w8 * NV * 128 + idx];
+        Up[idx] = t;
+    }
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w8 = 0; w8 < 8; ++w8) t += s_s[w8];
+        st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = t;
+    }
+}
+
+// --------------------------------------------------------------------------
 // Pair sweep for rows too long for one warp: a cluster of kPairCluster CTAs
 // shares every row.  CTA `rank` owns the columns [rank*slice, (rank+1)*slice):
 // it keeps that slice of the three vectors in shared memory for the whole tile
@@ -1129,7 +1370,6 @@ column_norms_kernel(DevState st) {
 // after `spin_limit` polls, raises the time-out bit of the status word and
 // leaves, so a launch can never hang the device.
 // --------------------------------------------------------------------------
-constexpr int kStatusTimeout = 5;  // PG_ERR_TIMEOUT
 
 __device__ bool grid_barrier(int* bar, int expected_blocks, int* status, long long spin_limit, int* s_ok) {
     __syncthreads();
@@ -1243,6 +1483,36 @@ cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile*
     return launch_row<true, false, false>(st, tab_update, tab_update, tiles, n_tiles, stream);
 }
 
+template <int NV, bool UPDATE>
+static cudaError_t launch_pair_bulk_t(const DevState& st, const int* tab_prev, const int* tab_cur,
+                                      const Tile* tiles, int n_tiles, int max_ld, cudaStream_t stream) {
+    // stage buffers; they also hold the 8 x NV*128 floats of the final reduction
+    size_t smem = sizeof(float) * (size_t)kBulkStages * 2 * kBulkRows * max_ld;
+    const size_t red = sizeof(float) * 8 * NV * 128;
+    if (smem < red) smem = red;
+    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (rc != cudaSuccess) return rc;
+    pair_sweep_bulk_kernel<NV, UPDATE><<<n_tiles, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles);
+    return cudaGetLastError();
+}
+
+template <bool UPDATE>
+static cudaError_t launch_pair_bulk(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
+                                    int n_tiles, int nv, cudaStream_t stream) {
+    const int max_ld = nv * 128;
+    switch (nv) {
+        case 1: return launch_pair_bulk_t<1, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 2: return launch_pair_bulk_t<2, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 3: return launch_pair_bulk_t<3, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 4: return launch_pair_bulk_t<4, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 5: return launch_pair_bulk_t<5, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 6: return launch_pair_bulk_t<6, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 7: return launch_pair_bulk_t<7, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        default: return launch_pair_bulk_t<8, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+    }
+}
+
 template <bool UPDATE>
 static cudaError_t launch_pair(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
                                int n_tiles, int nv, cudaStream_t stream) {
@@ -1264,6 +1534,9 @@ static cudaError_t launch_pair(const DevState& st, const int* tab_prev, const in
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
                               const Tile* tiles, int n_tiles, int nv, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
+    if (st.pair_bulk)
+        return apply_pending ? launch_pair_bulk<true>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
+                             : launch_pair_bulk<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
     return apply_pending ? launch_pair<true>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
                          : launch_pair<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
 }
