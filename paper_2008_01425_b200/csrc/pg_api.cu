@@ -103,6 +103,12 @@ int wide_tile_rows(int n, int max_edges, int resident) {
 // query_device: ask the current device how many clusters of the wide pair sweep
 // fit at once and shape its tiles accordingly.  Section sizes do not depend on
 // the answer, so a sizing pass without a device gives the same total.
+// PG_PAIR_BULK=0 in the environment selects the register-fed pair sweeps.
+bool pair_bulk_wanted() {
+    const char* v = std::getenv("PG_PAIR_BULK");
+    return !(v && v[0] == '0');
+}
+
 int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_layers, int rank,
                 Layout& lay, bool query_device = false) {
     if (!shapes || n_layers < 1 || n_layers > 4096) return PG_ERR_INVALID;
@@ -513,11 +519,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
     st.Pn = reinterpret_cast<float*>(c->ws + lay.off_Pn);
     st.half_odd = 0;
-    {
-        // PG_PAIR_BULK=0 selects the register-fed variant of the row-per-warp pair sweep
-        const char* v = std::getenv("PG_PAIR_BULK");
-        st.pair_bulk = (v && v[0] == '0') ? 0 : 1;
-    }
+    st.pair_bulk = pair_bulk_wanted() ? 1 : 0;
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
     st.PhNext = st.Ph + static_cast<long long>(lay.max_edges) * lay.ph_stride;

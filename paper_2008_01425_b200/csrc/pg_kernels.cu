@@ -1541,24 +1541,25 @@ cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int
                          : launch_pair<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
 }
 
+template <int NVW, bool UPDATE>
+static cudaError_t launch_wide_t(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
+                                 int n_tiles, int slice_pad, cudaStream_t stream) {
+    const dim3 grid(static_cast<unsigned>(n_tiles) * kPairCluster);
+    const size_t smem = sizeof(float) * 3 * static_cast<size_t>(slice_pad);
+    if (smem > 48 * 1024) {
+        cudaError_t rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, UPDATE>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (rc != cudaSuccess) return rc;
+    }
+    pair_sweep_wide_kernel<NVW, UPDATE><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
+    return cudaGetLastError();
+}
+
 template <int NVW>
 static cudaError_t launch_wide(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd,
                                const Tile* tiles, int n_tiles, int slice_pad, cudaStream_t stream) {
-    const size_t smem = sizeof(float) * 3 * static_cast<size_t>(slice_pad);
-    const dim3 grid(static_cast<unsigned>(n_tiles) * kPairCluster);
-    cudaError_t rc = cudaSuccess;
-    if (upd) {
-        if (smem > 48 * 1024)
-            rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (rc != cudaSuccess) return rc;
-        pair_sweep_wide_kernel<NVW, true><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
-    } else {
-        if (smem > 48 * 1024)
-            rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (rc != cudaSuccess) return rc;
-        pair_sweep_wide_kernel<NVW, false><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
-    }
-    return cudaGetLastError();
+    return upd ? launch_wide_t<NVW, true>(st, tab_prev, tab_cur, tiles, n_tiles, slice_pad, stream)
+               : launch_wide_t<NVW, false>(st, tab_prev, tab_cur, tiles, n_tiles, slice_pad, stream);
 }
 
 // `tiles`: cluster tiles of layers with the same float4 count per thread `nv` and
@@ -1594,13 +1595,12 @@ static int resident_clusters(int slice_pad) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cfg.dynamicSmemBytes > 48 * 1024 &&
-        cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)cfg.dynamicSmemBytes) != cudaSuccess) {
-        cudaGetLastError();
-        return 0;
-    }
-    if (cudaOccupancyMaxActiveClusters(&n, pair_sweep_wide_kernel<NVW, true>, &cfg) != cudaSuccess) {
+    cudaError_t rc = cudaSuccess;
+    if (cfg.dynamicSmemBytes > 48 * 1024)
+        rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)cfg.dynamicSmemBytes);
+    if (rc == cudaSuccess) rc = cudaOccupancyMaxActiveClusters(&n, pair_sweep_wide_kernel<NVW, true>, &cfg);
+    if (rc != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
