@@ -1114,8 +1114,10 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                        const Tile* __restrict__ tiles, int slice_pad) {
     namespace cg = cooperative_groups;
     extern __shared__ __align__(16) float s_vec[];               // q-hat, u_i, u_j slices
-    __shared__ float s_share[2][kPairCluster][kPairWideStep];    // [parity][rank][row]
+    __shared__ __align__(16) float s_share[2][kPairCluster][kPairWideStep];    // [parity][rank][row]
     __shared__ float s_warp[8][kPairWideStep];
+    __shared__ __align__(8) unsigned long long s_arrived[2];     // one mbarrier per parity: counts the shares' bytes
+    __shared__ int s_gave_up;
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
 
@@ -1155,6 +1157,12 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
             coef_j = __int_as_float(tab_prev[st.tab.off_slot_coef + wj * st.tab.max_degree]);
         }
     }
+    if (threadIdx.x == 0) {
+        s_gave_up = 0;
+        mbar_init(&s_arrived[0], 1);
+        mbar_init(&s_arrived[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     for (int idx = threadIdx.x; idx < slice_pad; idx += 256) {
         const int col = c_begin + idx;
         const bool in = col < c_end;
@@ -1164,7 +1172,7 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
             s_uj[idx] = in ? uj[col] : 0.0f;
         }
     }
-    __syncthreads();
+    cluster.sync();      // every CTA's mbarriers exist before a peer signals them
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r0 = tile.rtile * g.p_rows;
@@ -1240,19 +1248,27 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
             if (lane == 0) s_warp[warp][t] = dot[t];
         }
         __syncthreads();
+        // Data-flow exchange instead of a cluster-wide barrier: this CTA expects the
+        // RS floats of every rank on its own mbarrier of this parity, and sends its share
+        // to every rank (itself included) with a store that completes the receiver's count.
+        if (threadIdx.x == 0) mbar_expect_tx(&s_arrived[it & 1], (unsigned)(kPairCluster * RS * sizeof(float)));
         if (threadIdx.x < RS * kPairCluster) {
-            // thread (dst, t): this CTA's share of row t goes to CTA dst of the cluster
             const int dst = threadIdx.x / RS, t = threadIdx.x % RS;
             float share = 0.0f;
 #pragma unroll
             for (int w8 = 0; w8 < 8; ++w8) share += s_warp[w8][t];
-            *cluster.map_shared_rank(&s_share[it & 1][rank][t], dst) = share;
+            unsigned remote_data, remote_bar;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote_data)
+                         : "r"(smem_addr(&s_share[it & 1][rank][t])), "r"(dst));
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote_bar)
+                         : "r"(smem_addr(&s_arrived[it & 1])), "r"(dst));
+            asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                         ::"r"(remote_data), "r"(__float_as_uint(share)), "r"(remote_bar) : "memory");
         }
-        // split cluster barrier: announce the shares, start the next rows' loads while the
-        // other CTAs catch up, then wait until all shares of these rows have landed
-        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-        if (r + RS < r1) load_rows(r + RS);
-        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (r + RS < r1) load_rows(r + RS);      // the next rows' loads are in flight during the wait
+        // bounded wait; a CTA that gives up keeps going (its peers still need its shares)
+        if (!s_gave_up)
+            mbar_wait_bounded(&s_arrived[it & 1], (unsigned)((it >> 1) & 1), &s_gave_up, st.status);
 #pragma unroll
         for (int t = 0; t < RS; ++t) {
             float p = 0.0f;
