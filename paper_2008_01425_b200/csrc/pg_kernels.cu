@@ -1329,19 +1329,41 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
     float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
     const int cw = (g.m + kEdgeChunks - 1) / kEdgeChunks;
+    const int c_lo = chunk * cw, c_hi = min(g.m, (chunk + 1) * cw);
     part = 0.0;
-    for (int c = chunk * cw + threadIdx.x; c < min(g.m, (chunk + 1) * cw); c += blockDim.x) {
+    if (cw <= 32) {
+        // few columns, many tiles: 8 thread groups each add every 8th tile's share, then the
+        // groups are added in order (a fixed order, so the result is reproducible)
+        __shared__ double s_grp[8][32];
+        const int col = threadIdx.x & 31, grp = threadIdx.x >> 5;
+        const int c = c_lo + col;
         double a = 0.0;
-        for (int t = 0; t < g.p_rtiles; t += 8) {        // eight independent loads, added in tile order
-            float v[8];
+        if (c < c_hi)
+            for (int t = grp; t < g.p_rtiles; t += 8) a += (double)up[(long long)t * g.ld + c];
+        s_grp[grp][col] = a;
+        __syncthreads();
+        if (grp == 0 && c < c_hi) {
+            double tot = 0.0;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = t + j < g.p_rtiles ? up[(long long)(t + j) * g.ld + c] : 0.0f;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) a += (double)v[j];
+            for (int k = 0; k < 8; ++k) tot += s_grp[k][col];
+            const float q = (float)(tot * inv);
+            Q[c] = q;
+            part = (double)q * (double)q;
         }
-        const float q = (float)(a * inv);
-        Q[c] = q;
-        part += (double)q * (double)q;
+    } else {
+        for (int c = c_lo + threadIdx.x; c < c_hi; c += blockDim.x) {
+            double a = 0.0;
+            for (int t = 0; t < g.p_rtiles; t += 8) {        // eight independent loads, added in tile order
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = t + j < g.p_rtiles ? up[(long long)(t + j) * g.ld + c] : 0.0f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) a += (double)v[j];
+            }
+            const float q = (float)(a * inv);
+            Q[c] = q;
+            part += (double)q * (double)q;
+        }
     }
     const double qq = block_sum(part, scratch);
     if (threadIdx.x == 0) {
