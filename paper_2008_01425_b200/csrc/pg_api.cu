@@ -604,6 +604,9 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
             const int count = static_cast<int>(pairs.size()) - first;
             c->pair_groups.push_back(pg_ctx::PairGroup{lay.layers[l0].pair_mode, nv0, slice0, first, count, bytes});
         }
+        // serpentine: the transposed sweep walks the stack in the opposite direction to the row
+        // sweeps that run before and after it, so each sweep starts on what is still in L2
+        if (!std::getenv("PG_NO_SERPENTINE")) std::reverse(cols.begin(), cols.end());
         auto put = [](Tile* dst, const std::vector<Tile>& v) {
             return v.empty() || cudaMemcpy(dst, v.data(), sizeof(Tile) * v.size(), cudaMemcpyHostToDevice) == cudaSuccess;
         };
