@@ -95,8 +95,9 @@ typedef struct pg_ctx pg_ctx;  /* opaque; host memory owned by the library */
 
 /*
  * Size in bytes of the device workspace a context with these parameters needs
- * (parameters of all workers, per-pair vectors, exchange buffers, tables).
- * `shapes`: host, n_layers entries.  PG_ERR_INVALID for a bad topology, rank
+ * (parameters of all workers, per-pair vectors, exchange buffers, tables; on a
+ * static graph of degree 2 at rank 1 a second copy of the parameters, see
+ * pg_round).  `shapes`: host, n_layers entries.  PG_ERR_INVALID for a bad topology, rank
  * outside 1..PG_MAX_RANK or degree*rank > PG_MAX_SLOTS.
  */
 PG_API int pg_workspace_bytes(const pg_topology *topo, const pg_layer_shape *shapes, int32_t n_layers,
@@ -168,10 +169,19 @@ PG_API int pg_params_device(pg_ctx *ctx, int32_t worker, int32_t layer, void *st
  *     Q' = X_i^T Ph - X_j^T Ph                        (Eq. 3, even iteration)
  *     X_i -= W_ij Ph Q'^T,  X_j += W_ij Ph Q'^T,  Q = Q'   (Eq. 2; Lemma 1)
  * with all edges of a step reading the same pre-update X.  Advances the round
- * counter.  On graphs of degree <= 1 at rank 1 (a matching) the correction of a
- * step is applied to the copy of X in memory by the next step's sweep, or by
- * pg_read_params / pg_write_params / pg_write_q / pg_set_round, whichever comes
- * first; every call of this API sees the fully updated X.  Host-side errors are returned at once; device-side ones show up in
+ * counter.  At rank 1, on a matching and on static graphs of degree <= 2 without
+ * isolated workers (rings, paths), layers may run through the "pair sweep": one
+ * read of both ends of an edge gives p = D q-hat and D^T p, and the correction
+ * of a step is applied to the copy of X in memory by the next step's sweep, or
+ * by pg_read_params / pg_write_params / pg_params_device / pg_write_q /
+ * pg_set_round, whichever comes first; every call of this API sees the fully
+ * updated X.  On degree 2 a row has two readers, so the sweep writes corrected
+ * rows to a second copy of the stack and the copies swap roles every step; the
+ * calls above always leave the result in the copy pg_params_device points to.
+ * There, all layers take the pair sweep when the stack is at most 48 MiB, else
+ * only layers of at least 256 rows and 2^20 elements.  PG_DISABLE_PAIR_SWEEP=1
+ * in the environment at creation selects the general three-sweep path.
+ * Host-side errors are returned at once; device-side ones show up in
  * pg_read_params / pg_device_status.
  */
 PG_API int pg_round(pg_ctx *ctx, void *stream);
@@ -187,8 +197,8 @@ PG_API int pg_round(pg_ctx *ctx, void *stream);
  * iteration moves (rows+cols)/2 floats per edge direction on average, the count
  * behind the per-tensor compression ratios of the paper's parameter tables.  A
  * zero vector normalises to zero.  Call before the first round.  Needs rank 1
- * and a static graph of degree >= 2 (PG_ERR_INVALID otherwise; PG_ERR_STATE once
- * rounds have run).  In this mode pg_read_q / pg_write_q are only meaningful
+ * and a static graph (PG_ERR_INVALID otherwise; PG_ERR_STATE once rounds have
+ * run).  Moves every layer to the three-sweep path for the life of the context.  In this mode pg_read_q / pg_write_q are only meaningful
  * after an even number of iterations, when the vector is back in R^cols.
  */
 PG_API int pg_set_half_step(pg_ctx *ctx, int32_t on);
@@ -203,8 +213,9 @@ PG_API int pg_set_half_step(pg_ctx *ctx, int32_t on);
  * Philox4x32-10 / Box-Muller normals as for the initial vectors, under the key
  * (seed_lo ^ low32(t+1), seed_hi ^ high32(t+1) ^ 0x52503031) for step t, then
  * Gram-Schmidt.  The stored per-pair vectors are overwritten by the directions.
- * Call before the first round; not available on graphs of degree <= 1 at rank 1
- * (PG_ERR_INVALID), nor together with half-step mode.  A step costs one read of X
+ * Call before the first round; not available on PG_MATCHING (PG_ERR_INVALID),
+ * nor together with half-step mode.  Moves every layer to the three-sweep path
+ * for the life of the context.  A step costs one read of X
  * for the product and one read + write for the update (12 B per parameter).
  */
 enum { PG_POWER_ITERATION = 0, PG_RANDOM_RIGHT = 1, PG_RANDOM_LEFT = 2 };
@@ -213,7 +224,7 @@ PG_API int pg_set_random_projection(pg_ctx *ctx, int32_t mode);
 /*
  * Enqueue `n_rounds` rounds (same result as calling pg_round that many times).
  * When the graph is static and the whole stack is small enough to stay in L2
- * (at most 64 MiB of parameters, degree > 1 or rank > 1), all rounds run in ONE
+ * (at most 64 MiB of parameters, no layer on the pair sweep), all rounds run in ONE
  * cooperative kernel launch whose phases are separated by a grid barrier; the
  * barrier waits are bounded, and a wait that runs out ends the launch and sets
  * PG_ERR_TIMEOUT in the device status word.  Otherwise the rounds are enqueued
@@ -296,7 +307,7 @@ enum {
     PG_KERNEL_TRANSPOSED = 2,      /* X^T p-hat                                          */
     PG_KERNEL_EDGE_RIGHT = 3,      /* difference of the two ends, new stored vector      */
     PG_KERNEL_UPDATE_FORWARD = 4,  /* rank-r update of X fused with the next X q         */
-    PG_KERNEL_PAIR_SWEEP = 5,      /* degree <= 1, rank 1: pending update + X q + X^T p from one read */
+    PG_KERNEL_PAIR_SWEEP = 5,      /* rank 1, degree <= 2: pending update + X q + X^T p from one read */
     PG_KERNEL_PAIR_EDGE = 6,       /* its scalar edge step                               */
     PG_KERNEL_UPDATE_ONLY = 7,     /* applies a pending update before X is read or written */
     PG_KERNEL_KINDS = 8

@@ -34,12 +34,16 @@ struct Layout {
     long long x_stride = 0, q_stride = 0, y_stride = 0, ph_stride = 0, z_stride = 0;
     long long up_stride = 0, sp_stride = 0;
     long long n_pairs = 0;
-    bool pair_mode = false;        // degree <= 1 and rank 1: thin layers run through the pair sweep
+    bool pair_mode = false;        // rank 1 and degree <= 2: layers run through the pair sweep
+    int pend_slots = 1;            // corrections that can be pending at a worker in pair mode (its degree)
+    bool two_copies = false;       // pair mode on a graph of degree 2: the sweep writes to a second copy of X
     long long n_pair_tiles = 0, n_flush_tiles = 0;
+    long long row_tile_cap = 0, col_tile_cap = 0;   // room for the lists with every layer on the three-sweep path
+    long long n_pair_tiles_cap = 0, n_flush_tiles_cap = 0;
     int max_edges = 0, max_degree = 0;
     TabLayout tab{};
     long long n_row_tiles = 0, n_col_tiles = 0;
-    size_t off_Qn2 = 0, off_Pn = 0;
+    size_t off_Qn2 = 0, off_Pn = 0, off_edge_tab = 0;
     size_t off_X = 0, off_Q = 0, off_Qinv = 0, off_Y = 0, off_Ph = 0, off_Z = 0, off_live = 0,
            off_Up = 0, off_Sp = 0, off_pair_tiles = 0, off_flush_tiles = 0, off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
     size_t total = 0;
@@ -120,7 +124,32 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.n_pairs = topo.kind == PG_MATCHING ? static_cast<long long>(N) * (N - 1) / 2 : lay.max_edges;
     if (lay.n_pairs > INT_MAX / 2) return PG_ERR_INVALID;
 
-    lay.pair_mode = lay.max_degree == 1 && rank == 1 && pair_sweep_allowed();
+    // The pair sweep reads both ends of an edge in one pass.  On a perfect matching a
+    // row has one reader, so it is corrected in place.  On a static graph of degree 2
+    // with no isolated worker (a ring, a path) a row has up to two readers: the edge in
+    // the worker's slot 0 writes the corrected row to a second copy of X, which becomes
+    // the current one after the sweep.
+    lay.pair_mode = false;
+    lay.pend_slots = 1;
+    lay.two_copies = false;
+    if (rank == 1 && pair_sweep_allowed()) {
+        if (lay.max_degree == 1) {
+            lay.pair_mode = true;
+        } else if (lay.max_degree == 2 && topo.kind != PG_MATCHING && pair_bulk_wanted()) {
+            std::vector<Edge> edges;
+            if (!pg::build_edges(topo, 0, 0, edges)) return PG_ERR_INVALID;
+            std::vector<int> degree(N, 0);
+            for (const Edge& ed : edges) {
+                degree[ed.i] += 1;
+                degree[ed.j] += 1;
+            }
+            if (*std::min_element(degree.begin(), degree.end()) >= 1) {
+                lay.pair_mode = true;
+                lay.pend_slots = 2;
+                lay.two_copies = true;
+            }
+        }
+    }
     lay.layers.resize(n_layers);
     // aim for about 4096 tiles per sweep, each between 128 KB and 512 KB of X
     long long total_elems = 0;
@@ -129,8 +158,10 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
             total_elems += static_cast<long long>(N) * shapes[l].rows * round_up(shapes[l].cols, 4);
     long long tile_elems = std::min<long long>(std::max<long long>(total_elems / 4096, 32 * 1024), 128 * 1024);
     if (const char* v = std::getenv("PG_TILE_ELEMS")) tile_elems = std::max(4096LL, std::atoll(v));   // tuning aid
+    const bool small_stack = total_elems * 4 <= 48LL * 1024 * 1024;
     long long x = 0, q = 0, y = 0, ph = 0, z = 0, up = 0, sp = 0;
     lay.n_row_tiles = lay.n_col_tiles = lay.n_pair_tiles = lay.n_flush_tiles = 0;
+    lay.row_tile_cap = lay.col_tile_cap = 0;
     for (int l = 0; l < n_layers; ++l) {
         LayerGeom& g = lay.layers[l];
         if (shapes[l].rows < 1 || shapes[l].cols < 1) return PG_ERR_INVALID;
@@ -160,23 +191,44 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         y += round_up(static_cast<long long>(slots) * g.f_csplit * g.npad, 64);
         ph += round_up(static_cast<long long>(rank) * g.npad, 64);
         z += round_up(static_cast<long long>(slots) * g.t_rtiles * g.ld, 64);
-        g.pair_mode = !lay.pair_mode ? 0 : (g.ld <= pg::kPairMaxLd ? 1 : (g.ld <= pg::kPairWideMaxLd ? 2 : 0));
+        // a row per warp up to kPairMaxLd floats, per CTA up to kPairMidMaxLd, per cluster beyond
+        g.pair_mode = !lay.pair_mode ? 0
+                      : g.ld <= pg::kPairMaxLd ? 1
+                      : g.ld <= pg::kPairMidMaxLd ? 3
+                      : g.ld <= pg::kPairWideMaxLd ? 2 : 0;
+        // With two readers per row the pair sweep pays off in two regimes: a stack small
+        // enough to live in L2, where it halves the launches of a step, and layers large
+        // enough to keep every SM busy for many rows.  Other layers take the three sweeps.
+        if (lay.two_copies && !small_stack && !(g.n >= 256 && static_cast<long long>(g.n) * g.ld >= (1LL << 20)))
+            g.pair_mode = 0;
         g.p_slice = static_cast<int>(round_up((g.ld + pg::kPairCluster - 1) / pg::kPairCluster, 4));
-        {   // equal tiles of at most kPairTileRows rows (a multiple of 8: one row per warp and stage)
-            const int parts = (g.n + pg::kPairTileRows - 1) / pg::kPairTileRows;
+        {   // equal tiles of at most kPairTileRows rows (a multiple of 8: one row per warp and stage);
+            // on graphs of degree 2 short matrices are cut finer, down to 16 rows, so that a layer gives
+            // about two CTAs per SM
+            const int by_height = (g.n + pg::kPairTileRows - 1) / pg::kPairTileRows;
+            const int by_count = std::min((296 + lay.max_edges - 1) / lay.max_edges, std::max(g.n / 16, 1));
+            // (on a matching every layer of the stack shares one launch, which has tiles enough)
+            const int parts = lay.two_copies ? std::max(by_height, by_count) : by_height;
             g.p_rows = static_cast<int>(round_up((g.n + parts - 1) / parts, 8));
         }
         if (g.pair_mode == 2) {
             const int resident = query_device
-                ? pg::pair_wide_resident_clusters((g.p_slice / 4 + 255) / 256, g.p_slice) : 0;
+                ? pg::pair_wide_resident_clusters((g.p_slice / 4 + 255) / 256, g.p_slice, lay.pend_slots) : 0;
             g.p_rows = wide_tile_rows(g.n, lay.max_edges, resident);
             if ((g.n + g.p_rows - 1) / g.p_rows > pg::kPairWideMaxTiles)
                 g.p_rows = static_cast<int>(round_up((g.n + pg::kPairWideMaxTiles - 1) / pg::kPairWideMaxTiles,
                                                      pg::kPairWideStep));
         }
         g.p_rtiles = (g.n + g.p_rows - 1) / g.p_rows;
+        {   // pair edge step: about 2048 partial sums or rows per CTA
+            const int max_tiles = g.pair_mode == 2 ? pg::kPairWideMaxTiles : g.p_rtiles;
+            const long long work = static_cast<long long>(max_tiles) * g.ld + g.npad;
+            g.e_chunks = static_cast<int>(std::min<long long>(std::max<long long>((work + 2047) / 2048, 1), pg::kEdgeChunks));
+        }
         g.up_off = up;
         g.sp_off = sp;
+        lay.row_tile_cap += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
+        lay.col_tile_cap += static_cast<long long>(N) * g.t_rtiles * g.t_ctiles;
         if (g.pair_mode != 0) {
             // wide layers: room for any tile count the device query may choose
             const int max_tiles = g.pair_mode == 2 ? pg::kPairWideMaxTiles : g.p_rtiles;
@@ -191,7 +243,9 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     }
     lay.up_stride = up;
     lay.sp_stride = sp;
-    if (lay.n_row_tiles > INT_MAX || lay.n_col_tiles > INT_MAX) return PG_ERR_INVALID;
+    lay.n_pair_tiles_cap = lay.n_pair_tiles;
+    lay.n_flush_tiles_cap = lay.n_flush_tiles;
+    if (lay.row_tile_cap > INT_MAX || lay.col_tile_cap > INT_MAX) return PG_ERR_INVALID;
     lay.x_stride = x;
     lay.q_stride = q;
     lay.y_stride = y;
@@ -221,7 +275,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         off = static_cast<size_t>(round_up(static_cast<long long>(off + bytes), kAlign));
         return at;
     };
-    lay.off_X = take(sizeof(float) * static_cast<size_t>(N) * lay.x_stride);
+    lay.off_X = take(sizeof(float) * static_cast<size_t>(N) * lay.x_stride * (lay.two_copies ? 2 : 1));
     lay.off_Q = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride);
     lay.off_Qinv = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * n_layers * rank);
     lay.off_Qn2 = take(sizeof(double) * static_cast<size_t>(lay.n_pairs) * n_layers * pg::kEdgeChunks);
@@ -234,11 +288,12 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_live = take(sizeof(int) * static_cast<size_t>(lay.max_edges) * n_layers * rank);
     lay.off_status = take(sizeof(int) * 64);   // [0] status word, [16..17] grid barrier of the persistent kernel
     lay.off_layers = take(sizeof(LayerGeom) * static_cast<size_t>(n_layers));
+    lay.off_edge_tab = take(sizeof(int) * 2 * static_cast<size_t>(n_layers) * pg::kEdgeChunks);
     lay.off_tabs = take(sizeof(int) * static_cast<size_t>(kTabRing) * t.total_ints);
-    lay.off_row_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_row_tiles));
-    lay.off_col_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_col_tiles));
-    lay.off_pair_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_pair_tiles));
-    lay.off_flush_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_flush_tiles));
+    lay.off_row_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.row_tile_cap));
+    lay.off_col_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.col_tile_cap));
+    lay.off_pair_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_pair_tiles_cap));
+    lay.off_flush_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_flush_tiles_cap));
     lay.total = off;
     return PG_OK;
 }
@@ -257,10 +312,12 @@ struct pg_ctx {
     // pair sweep: the correction of the last step has not been applied to X yet
     bool pending = false;
     int64_t pending_key = 0;    // round whose table describes the pending correction
+    int xbuf = 0;               // which copy of X is current (always 0 unless a correction is pending)
     int64_t step = 0;           // power steps enqueued so far (selects the P-hat buffer)
     float* ph_buf[2] = {nullptr, nullptr};
     Tile* d_pair_tiles = nullptr;
     Tile* d_flush_tiles = nullptr;
+    // slice: widest per-CTA column slice (mode 2) or widest padded row (mode 3) in the group
     struct PairGroup { int mode; int nv; int slice; int first; int count; double bytes; };
     std::vector<PairGroup> pair_groups;   // pair tiles grouped by float4 per lane
     int64_t launches = 0;
@@ -401,6 +458,9 @@ int flush_pending(pg_ctx* c, cudaStream_t stream) {
     if (rc != PG_OK) return rc;
     DevState st = c->st;
     st.Ph = c->ph_buf[(c->step + 1) & 1];
+    // the corrected stack always lands in the first copy of X, the one the caller sees
+    st.X = c->st.X + c->xbuf * static_cast<long long>(c->topo.n_workers) * c->lay.x_stride;
+    st.Xw = c->st.X;
     {
         Timed t(c, PG_KERNEL_UPDATE_ONLY, stream, 2.0 * c->pair_param_bytes);
         if (pg::launch_update(st, tab_prev, c->d_flush_tiles, static_cast<int>(c->lay.n_flush_tiles), stream) !=
@@ -411,7 +471,142 @@ int flush_pending(pg_ctx* c, cudaStream_t stream) {
     }
     c->launches += 1;
     c->pending = false;
+    c->xbuf = 0;
     return PG_OK;
+}
+
+// Build and upload the tile lists for the current assignment of layers to paths
+// (LayerGeom::pair_mode) and refresh the counts and byte totals that go with them.
+// Row and column tiles: worker-major, layers in the caller's order.  Layers on the
+// pair sweep get pair tiles, grouped by kernel instantiation, and row tiles for
+// flushing a pending correction.
+bool upload_tile_lists(pg_ctx* c) {
+    Layout& lay = c->lay;
+    const int n_layers = c->n_layers;
+    const int N = c->topo.n_workers;
+    std::vector<Tile> rows, cols, flush, pairs;
+    c->pair_groups.clear();
+    c->normal_param_bytes = c->pair_param_bytes = 0.0;
+    for (int l = 0; l < n_layers; ++l) {
+        const double b = 4.0 * N * static_cast<double>(lay.layers[l].n) * lay.layers[l].m;
+        (lay.layers[l].pair_mode ? c->pair_param_bytes : c->normal_param_bytes) += b;
+    }
+    for (int v = 0; v < N; ++v)
+        for (int l = 0; l < n_layers; ++l) {
+            const LayerGeom& g = lay.layers[l];
+            for (int rt = 0; rt < g.f_rtiles; ++rt)
+                for (int ct = 0; ct < g.f_csplit; ++ct)
+                    (g.pair_mode ? flush : rows).push_back(Tile{v, l, rt, ct});
+            if (g.pair_mode) continue;
+            for (int rt = 0; rt < g.t_rtiles; ++rt)
+                for (int ct = 0; ct < g.t_ctiles; ++ct) cols.push_back(Tile{v, l, rt, ct});
+        }
+    // one launch per group of layers that share the kernel instantiation
+    auto group_of = [&](const LayerGeom& g, int* nv, int* slice) {
+        if (g.pair_mode == 1) {
+            *nv = (g.ld + 127) / 128;
+            *slice = 0;
+        } else if (g.pair_mode == 3) {
+            *nv = (g.ld + 1023) / 1024;
+            *slice = g.ld;
+        } else {
+            *nv = (g.p_slice / 4 + 255) / 256;
+            *slice = g.p_slice;
+        }
+    };
+    std::vector<char> done(n_layers, 0);
+    for (int l0 = 0; l0 < n_layers; ++l0) {
+        if (!lay.layers[l0].pair_mode || done[l0]) continue;
+        int nv0 = 0, slice0 = 0;
+        group_of(lay.layers[l0], &nv0, &slice0);
+        const int first = static_cast<int>(pairs.size());
+        double bytes = 0.0;   // every worker's rows read from memory once and written once
+        for (int l = l0; l < n_layers; ++l) {
+            const LayerGeom& g = lay.layers[l];
+            int nv = 0, slice = 0;
+            if (!g.pair_mode || done[l] || g.pair_mode != lay.layers[l0].pair_mode) continue;
+            group_of(g, &nv, &slice);
+            if (nv != nv0) continue;
+            slice0 = std::max(slice0, slice);     // sizes the shared-memory vectors of the launch
+            done[l] = 1;
+            if (lay.two_copies) {
+                // the readers of a row block run next to each other, so the second one finds it in L2
+                for (int rt = 0; rt < g.p_rtiles; ++rt)
+                    for (int e = 0; e < lay.max_edges; ++e) pairs.push_back(Tile{e, l, rt, 0});
+            } else {
+                for (int e = 0; e < lay.max_edges; ++e)
+                    for (int rt = 0; rt < g.p_rtiles; ++rt) pairs.push_back(Tile{e, l, rt, 0});
+            }
+            bytes += 8.0 * N * static_cast<double>(g.n) * g.m;
+        }
+        const int count = static_cast<int>(pairs.size()) - first;
+        c->pair_groups.push_back(pg_ctx::PairGroup{lay.layers[l0].pair_mode, nv0, slice0, first, count, bytes});
+    }
+    // a group with fewer than two tiles per SM joins the next group of its kind with longer rows
+    // (the kernels take any row up to their template's width): fewer, fuller launches
+    {
+        std::vector<pg_ctx::PairGroup>& gr = c->pair_groups;
+        std::stable_sort(gr.begin(), gr.end(), [](const pg_ctx::PairGroup& a, const pg_ctx::PairGroup& b) {
+            return a.mode != b.mode ? a.mode < b.mode : a.nv < b.nv;
+        });
+        std::vector<Tile> merged;
+        std::vector<pg_ctx::PairGroup> out;
+        merged.reserve(pairs.size());
+        for (size_t i = 0; i < gr.size(); ++i) {
+            pg_ctx::PairGroup cur = gr[i];
+            const int first = static_cast<int>(merged.size());
+            merged.insert(merged.end(), pairs.begin() + cur.first, pairs.begin() + cur.first + cur.count);
+            while (cur.mode != 2 && cur.count < 296 && i + 1 < gr.size() && gr[i + 1].mode == cur.mode) {
+                const pg_ctx::PairGroup& nx = gr[++i];
+                merged.insert(merged.end(), pairs.begin() + nx.first, pairs.begin() + nx.first + nx.count);
+                cur.nv = nx.nv;
+                cur.slice = std::max(cur.slice, nx.slice);
+                cur.count += nx.count;
+                cur.bytes += nx.bytes;
+            }
+            cur.first = first;
+            out.push_back(cur);
+        }
+        pairs.swap(merged);
+        gr.swap(out);
+    }
+    // serpentine: the transposed sweep walks the stack in the opposite direction to the row
+    // sweeps that run before and after it, so each sweep starts on what is still in L2
+    if (!std::getenv("PG_NO_SERPENTINE")) std::reverse(cols.begin(), cols.end());
+    if (static_cast<long long>(rows.size()) > lay.row_tile_cap || static_cast<long long>(cols.size()) > lay.col_tile_cap ||
+        static_cast<long long>(pairs.size()) > lay.n_pair_tiles_cap || static_cast<long long>(flush.size()) > lay.n_flush_tiles_cap)
+        return false;
+    lay.n_row_tiles = static_cast<long long>(rows.size());
+    lay.n_col_tiles = static_cast<long long>(cols.size());
+    lay.n_pair_tiles = static_cast<long long>(pairs.size());
+    lay.n_flush_tiles = static_cast<long long>(flush.size());
+    auto put = [](Tile* dst, const std::vector<Tile>& v) {
+        return v.empty() || cudaMemcpy(dst, v.data(), sizeof(Tile) * v.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    };
+    // the CTAs of the pair edge step of one edge: (layer, chunk)
+    std::vector<int> edge_tab;
+    for (int l = 0; l < n_layers; ++l)
+        if (lay.layers[l].pair_mode)
+            for (int ch = 0; ch < lay.layers[l].e_chunks; ++ch) {
+                edge_tab.push_back(l);
+                edge_tab.push_back(ch);
+            }
+    c->st.e_total = static_cast<int>(edge_tab.size() / 2);
+    if (!edge_tab.empty() && cudaMemcpy(c->ws + lay.off_edge_tab, edge_tab.data(), sizeof(int) * edge_tab.size(),
+                                        cudaMemcpyHostToDevice) != cudaSuccess)
+        return false;
+    return cudaMemcpy(c->ws + lay.off_layers, lay.layers.data(), sizeof(LayerGeom) * n_layers, cudaMemcpyHostToDevice) ==
+               cudaSuccess &&
+           put(c->d_row_tiles, rows) && put(c->d_col_tiles, cols) && put(c->d_pair_tiles, pairs) &&
+           put(c->d_flush_tiles, flush);
+}
+
+// Move every layer to the three-sweep path (the modes that have no pair-sweep form
+// need it).  Only before the first round, with nothing pending.
+bool leave_pair_mode(pg_ctx* c) {
+    if (c->lay.n_pair_tiles == 0) return true;
+    for (LayerGeom& g : c->lay.layers) g.pair_mode = 0;
+    return upload_tile_lists(c);
 }
 
 int check_worker_layer(const pg_ctx* c, int worker, int layer) {
@@ -498,10 +693,6 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
         int coop = 0;
         c->coop_ok = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) == cudaSuccess && coop != 0;
     }
-    for (int l = 0; l < n_layers; ++l) {
-        const double b = 4.0 * c->topo.n_workers * static_cast<double>(c->lay.layers[l].n) * c->lay.layers[l].m;
-        (c->lay.layers[l].pair_mode ? c->pair_param_bytes : c->normal_param_bytes) += b;
-    }
     c->pairs.triangular = !c->static_graph;
     c->pairs.n_workers = c->topo.n_workers;
     if (c->static_graph) c->pairs.static_edges = edges0;
@@ -514,6 +705,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     const Layout& lay = c->lay;
     DevState& st = c->st;
     st.X = reinterpret_cast<float*>(c->ws + lay.off_X);
+    st.Xw = st.X;
     st.Q = reinterpret_cast<float*>(c->ws + lay.off_Q);
     st.Qinv = reinterpret_cast<float*>(c->ws + lay.off_Qinv);
     st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
@@ -535,6 +727,8 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.live = reinterpret_cast<int*>(c->ws + lay.off_live);
     st.status = reinterpret_cast<int*>(c->ws + lay.off_status);
     st.layers = reinterpret_cast<const LayerGeom*>(c->ws + lay.off_layers);
+    st.edge_tab = reinterpret_cast<const int*>(c->ws + lay.off_edge_tab);
+    st.e_total = 0;
     st.x_stride = lay.x_stride;
     st.q_stride = lay.q_stride;
     st.y_stride = lay.y_stride;
@@ -550,69 +744,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     c->d_col_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_col_tiles);
 
     bool ok = cudaMemset(c->ws, 0, lay.total) == cudaSuccess;
-    ok = ok && cudaMemcpy(c->ws + lay.off_layers, lay.layers.data(), sizeof(LayerGeom) * n_layers,
-                          cudaMemcpyHostToDevice) == cudaSuccess;
-    // tile lists: worker-major, layers in the caller's order; layers that run
-    // through the pair sweep get pair tiles (edge, layer, row block), grouped by
-    // the number of float4 a lane holds, and row tiles for flushing a pending
-    // correction
-    if (ok) {
-        std::vector<Tile> rows, cols, flush;
-        rows.reserve(lay.n_row_tiles);
-        cols.reserve(lay.n_col_tiles);
-        flush.reserve(lay.n_flush_tiles);
-        for (int v = 0; v < c->topo.n_workers; ++v)
-            for (int l = 0; l < n_layers; ++l) {
-                const LayerGeom& g = lay.layers[l];
-                for (int rt = 0; rt < g.f_rtiles; ++rt)
-                    for (int ct = 0; ct < g.f_csplit; ++ct)
-                        (g.pair_mode ? flush : rows).push_back(Tile{v, l, rt, ct});
-                if (g.pair_mode) continue;
-                for (int rt = 0; rt < g.t_rtiles; ++rt)
-                    for (int ct = 0; ct < g.t_ctiles; ++ct) cols.push_back(Tile{v, l, rt, ct});
-            }
-        std::vector<Tile> pairs;
-        pairs.reserve(lay.n_pair_tiles);
-        // one launch per group of layers that share the kernel instantiation
-        auto group_of = [&](const LayerGeom& g, int* nv, int* slice) {
-            if (g.pair_mode == 1) {
-                *nv = (g.ld + 127) / 128;
-                *slice = 0;
-            } else {
-                *nv = (g.p_slice / 4 + 255) / 256;
-                *slice = g.p_slice;
-            }
-        };
-        std::vector<char> done(n_layers, 0);
-        for (int l0 = 0; l0 < n_layers; ++l0) {
-            if (!lay.layers[l0].pair_mode || done[l0]) continue;
-            int nv0 = 0, slice0 = 0;
-            group_of(lay.layers[l0], &nv0, &slice0);
-            const int first = static_cast<int>(pairs.size());
-            double bytes = 0.0;   // both ends of every edge read once and written once
-            for (int l = l0; l < n_layers; ++l) {
-                const LayerGeom& g = lay.layers[l];
-                int nv = 0, slice = 0;
-                if (!g.pair_mode || done[l] || g.pair_mode != lay.layers[l0].pair_mode) continue;
-                group_of(g, &nv, &slice);
-                if (nv != nv0 || slice != slice0) continue;
-                done[l] = 1;
-                for (int e = 0; e < lay.max_edges; ++e)
-                    for (int rt = 0; rt < g.p_rtiles; ++rt) pairs.push_back(Tile{e, l, rt, 0});
-                bytes += 8.0 * 2.0 * lay.max_edges * static_cast<double>(g.n) * g.m;
-            }
-            const int count = static_cast<int>(pairs.size()) - first;
-            c->pair_groups.push_back(pg_ctx::PairGroup{lay.layers[l0].pair_mode, nv0, slice0, first, count, bytes});
-        }
-        // serpentine: the transposed sweep walks the stack in the opposite direction to the row
-        // sweeps that run before and after it, so each sweep starts on what is still in L2
-        if (!std::getenv("PG_NO_SERPENTINE")) std::reverse(cols.begin(), cols.end());
-        auto put = [](Tile* dst, const std::vector<Tile>& v) {
-            return v.empty() || cudaMemcpy(dst, v.data(), sizeof(Tile) * v.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-        };
-        ok = put(c->d_row_tiles, rows) && put(c->d_col_tiles, cols) && put(c->d_pair_tiles, pairs) &&
-             put(c->d_flush_tiles, flush);
-    }
+    ok = ok && upload_tile_lists(c);
     // Algorithm 2, initialisation: one standard-normal vector per pair, layer, column
     if (ok) {
         std::vector<Edge> all_pairs;
@@ -853,16 +985,28 @@ int pg_round(pg_ctx* c, void* stream_v) {
             DevState st = c->st;
             st.Ph = ph_prev;
             st.PhNext = ph_cur;
+            // rows with two readers: read the current copy of X, write the corrected rows to the other
+            const long long copy_elems = static_cast<long long>(c->topo.n_workers) * c->lay.x_stride;
+            const bool flip = c->lay.two_copies && c->pending;
+            st.X = c->st.X + c->xbuf * copy_elems;
+            st.Xw = flip ? c->st.X + (c->xbuf ^ 1) * copy_elems : st.X;
             for (const auto& grp : c->pair_groups) {
-                Timed t(c, PG_KERNEL_PAIR_SWEEP, stream, grp.bytes);
+                // without a pending correction the sweep only reads
+                Timed t(c, PG_KERNEL_PAIR_SWEEP, stream, c->pending ? grp.bytes : 0.5 * grp.bytes);
                 if (grp.mode == 1)
                     ok = ok && pg::launch_pair_sweep(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
-                                                     grp.count, grp.nv, stream) == cudaSuccess;
+                                                     grp.count, grp.nv, c->lay.pend_slots, stream) == cudaSuccess;
+                else if (grp.mode == 3)
+                    ok = ok && pg::launch_pair_sweep_mid(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
+                                                         grp.count, grp.nv, static_cast<int>(round_up(grp.slice, 4)),
+                                                         c->lay.pend_slots, stream) == cudaSuccess;
                 else
                     ok = ok && pg::launch_pair_sweep_wide(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
-                                                          grp.count, grp.nv, grp.slice, stream) == cudaSuccess;
+                                                          grp.count, grp.nv, grp.slice, c->lay.pend_slots,
+                                                          stream) == cudaSuccess;
                 c->launches += 1;
             }
+            if (flip) c->xbuf ^= 1;
             {
                 Timed t(c, PG_KERNEL_PAIR_EDGE, stream, 0.0);
                 ok = ok && pg::launch_pair_edge(st, tab, c->lay.max_edges, stream) == cudaSuccess;
@@ -886,7 +1030,9 @@ int pg_round(pg_ctx* c, void* stream_v) {
 int pg_set_half_step(pg_ctx* c, int32_t on) {
     if (!c) return PG_ERR_INVALID;
     if (c->round != 0 || c->pending || c->y_valid) return PG_ERR_STATE;
-    if (on && (c->rank != 1 || !c->static_graph || c->lay.n_pair_tiles > 0 || c->random_proj)) return PG_ERR_INVALID;
+    if (on && (c->rank != 1 || !c->static_graph || c->random_proj)) return PG_ERR_INVALID;
+    // the pair sweep has no half-step form: every layer goes to the three-sweep path
+    if (on && (!bind_device(c) || !leave_pair_mode(c))) return PG_ERR_CUDA;
     c->half_step = on != 0;
     c->iteration = 0;
     return PG_OK;
@@ -895,7 +1041,9 @@ int pg_set_half_step(pg_ctx* c, int32_t on) {
 int pg_set_random_projection(pg_ctx* c, int32_t mode) {
     if (!c || mode < 0 || mode > 2) return PG_ERR_INVALID;
     if (c->round != 0 || c->pending || c->y_valid || c->half_step) return PG_ERR_STATE;
-    if (mode != 0 && c->lay.n_pair_tiles > 0) return PG_ERR_INVALID;
+    // the pair sweep has no random-projection form: every layer goes to the three-sweep path
+    if (mode != 0 && !c->static_graph) return PG_ERR_INVALID;
+    if (mode != 0 && (!bind_device(c) || !leave_pair_mode(c))) return PG_ERR_CUDA;
     c->random_proj = mode;
     return PG_OK;
 }

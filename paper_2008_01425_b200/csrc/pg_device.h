@@ -20,6 +20,7 @@ constexpr int kColTileRowsMax = 256;   // rows of X per CTA in the transposed sw
 constexpr int kColTileCols = 256;      // columns per CTA in the transposed sweep (64 threads x float4)
 constexpr int kPairTileRows = 512;     // rows of both matrices per CTA in the pair sweep
 constexpr int kPairMaxLd = 1024;       // widest row a warp of the pair sweep keeps in registers
+constexpr int kPairMidMaxLd = 8192;    // widest row one CTA of the pair sweep keeps in registers (8 float4 per thread)
 constexpr int kPairCluster = 8;        // CTAs that share a row of a wider layer (thread-block cluster)
 constexpr int kPairWideRows = 32;      // rows per cluster tile of a wider layer when residency is unknown
 constexpr int kPairWideMaxTiles = 32;  // most row tiles per (edge, wide layer); sizes the partial-sum buffer
@@ -50,13 +51,14 @@ struct LayerGeom {
     long long y_off;   // forward partials inside a worker's block   (slots x f_csplit x npad)
     long long ph_off;  // P-hat inside an edge's block               (rank x npad)
     long long z_off;   // transposed partials inside a worker's block (slots x t_rtiles x ld)
-    // pair sweep (graphs of degree <= 1 at rank 1; rows of at most kPairMaxLd floats)
-    int pair_mode;     // 0: three sweeps; 1: pair sweep, row per warp; 2: pair sweep, row per cluster
+    // pair sweep (rank 1; a matching or a static graph of degree <= 2)
+    int pair_mode;     // 0: three sweeps; pair sweep with a row per 1: warp, 2: cluster, 3: CTA
     int p_rows;        // rows per tile of the pair sweep
     int p_rtiles;      // row tiles of the pair sweep
     int p_slice;       // mode 2: columns per CTA of the cluster (multiple of 4)
     long long up_off;  // partial sums of D^T p inside an edge's block (p_rtiles x ld)
     long long sp_off;  // partial sums of ||p||^2 inside an edge's block (p_rtiles doubles)
+    int e_chunks;      // CTAs that share the pair edge step of one edge on this layer (1..kEdgeChunks)
 };
 
 // One unit of work of a sweep: a tile of one worker's layer.
@@ -87,6 +89,8 @@ struct TabLayout {
 // Pointers into the workspace (device) plus sizes; passed to kernels by value.
 struct DevState {
     float* X;            // [worker][x_stride]
+    float* Xw;           // where corrected rows are written: X itself, or the second copy of the stack
+                         // when a row has two readers in one sweep (pair sweep on graphs of degree 2)
     float* Q;            // [pair][q_stride]     raw right factors
     float* Qinv;         // [pair][layer][rank]  1 / column norm (0 for a zero column)
     double* Qn2;         // [pair][layer][kEdgeChunks]  pair sweep layers: shares of ||Q||^2
@@ -103,6 +107,8 @@ struct DevState {
     int* live;           // [edge][layer][rank]  1 if the column took part in this step
     int* status;         // device status word (bit n set = error code n was raised)
     const LayerGeom* layers;
+    const int* edge_tab; // [e_total][2]  (layer, chunk) of every CTA of the pair edge step of one edge
+    int e_total;
     long long x_stride, q_stride, y_stride, ph_stride, z_stride, up_stride, sp_stride;
     int n_layers, rank, n_workers, max_degree;
     TabLayout tab;
@@ -130,12 +136,16 @@ cudaError_t launch_edge_raw(const DevState& st, const int* tab, int max_edges, c
 cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile* tiles, int n_tiles,
                           cudaStream_t stream);
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
-                              const Tile* tiles, int n_tiles, int nv, cudaStream_t stream);
+                              const Tile* tiles, int n_tiles, int nv, int pend_slots, cudaStream_t stream);
 cudaError_t launch_pair_sweep_wide(const DevState& st, const int* tab_prev, const int* tab_cur,
                                    bool apply_pending, const Tile* tiles, int n_tiles, int nv, int slice,
-                                   cudaStream_t stream);
+                                   int pend_slots, cudaStream_t stream);
+// `tiles`: tiles of layers whose rows one CTA holds (nv float4 per thread, rows of at most ld_pad floats)
+cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const int* tab_cur,
+                                  bool apply_pending, const Tile* tiles, int n_tiles, int nv, int ld_pad,
+                                  int pend_slots, cudaStream_t stream);
 // Clusters of the wide pair sweep that can be resident at once (0 if unknown).
-int pair_wide_resident_clusters(int nv, int slice);
+int pair_wide_resident_clusters(int nv, int slice, int pend_slots);
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 // One cooperative launch for `n_steps` power steps of a static graph (small stacks).
 cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* row_tiles, int n_rows,

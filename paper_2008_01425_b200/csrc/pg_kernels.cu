@@ -13,6 +13,8 @@
 // fixed order by the edge kernels, so results are bit-reproducible.
 #include <cooperative_groups.h>
 
+#include <algorithm>
+
 #include "pg_device.h"
 
 namespace pg {
@@ -125,6 +127,7 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
     const int w = tile.worker;
     const int rank = st.rank;
     float* __restrict__ X = st.X + (long long)w * st.x_stride + g.x_off;
+    float* Xw = st.Xw + (long long)w * st.x_stride + g.x_off;
 
     if (threadIdx.x < S) {
         const int v = threadIdx.x;
@@ -231,7 +234,11 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                 }
 #pragma unroll
                 for (int t = 0; t < RT; ++t)
-                    if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
+                    if (rb + t < r1) {
+                        // the update-only sweep may write to the other copy of the stack
+                        float* dst = FORWARD ? const_cast<float*>(xrow[t]) : Xw + (long long)(rb + t) * ld;
+                        st_stream(dst + c, x[t]);
+                    }
             }
             if (FORWARD && !(UPDATE && SAME)) {
 #pragma unroll
@@ -713,9 +720,37 @@ __device__ __forceinline__ float pair_qinv(const DevState& st, int pair, int lay
     return t > 0.0 ? (float)(1.0 / sqrt(t)) : 0.0f;
 }
 
+// Factors of the corrections that are still pending at one end of an edge: the
+// previous step left at most D of them at a worker (one per incident edge), each
+// coef * p-hat_r * q' with p-hat of that edge and the edge's new stored vector.
+template <int D>
+struct PendingEnd {
+    const float* vec[D];
+    const float* ph[D];
+    float coef[D];
+};
+template <int D>
+__device__ __forceinline__ void pending_of(const DevState& st, const int* __restrict__ tab_prev, int w,
+                                           const LayerGeom& g, const float* dflt, PendingEnd<D>& pe) {
+    const int deg = min(tab_prev[st.tab.off_degree + w], D);
+#pragma unroll
+    for (int s = 0; s < D; ++s) {
+        pe.vec[s] = dflt;
+        pe.ph[s] = nullptr;
+        pe.coef[s] = 0.0f;
+        if (s < deg) {
+            const int ep = tab_prev[st.tab.off_slot_edge + w * st.tab.max_degree + s];
+            pe.vec[s] = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            pe.ph[s] = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            pe.coef[s] = __int_as_float(tab_prev[st.tab.off_slot_coef + w * st.tab.max_degree + s]);
+        }
+    }
+}
+
 // --------------------------------------------------------------------------
-// Pair sweep (graphs of degree <= 1, rank 1).  One CTA owns a block of rows of
-// BOTH ends of an edge (i<j) and reads each row of X_i and X_j once:
+// Pair sweep (rank 1; a matching, or a static graph of degree <= 2, where the
+// TMA-fed variants below also take rows with two readers).  One CTA owns a block
+// of rows of BOTH ends of an edge (i<j) and reads each row of X_i and X_j once:
 //   - applies the correction that is still pending from the previous step to
 //     each row (each end has its own previous edge) and writes the rows back,
 //   - forms the row of D = X_i - X_j, its product with q-hat:  p_r = D_r . q-hat,
@@ -915,14 +950,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
     return false;
 }
 
-template <int NV, bool UPDATE>
+template <int NV, bool UPDATE, int D>
 __global__ void __launch_bounds__(256, PG_BULK_MIN_BLOCKS)
 pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles) {
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ __align__(16) float s_q[NV * 128];
-    __shared__ __align__(16) float s_ui[NV * 128];
-    __shared__ __align__(16) float s_uj[NV * 128];
+    __shared__ __align__(16) float s_ui[D][NV * 128];
+    __shared__ __align__(16) float s_uj[D][NV * 128];
     __shared__ __align__(8) unsigned long long s_full[kBulkStages];
     __shared__ double s_s[8];
     __shared__ int s_abort;
@@ -941,24 +976,17 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 
     const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
     const float qinv = pair_qinv(st, pair, tile.layer);
-    const float* ui = q;
-    const float* uj = q;
-    const float* phi = nullptr;
-    const float* phj = nullptr;
-    float coef_i = 0.0f, coef_j = 0.0f;
+    // only the edge in slot 0 of a worker writes that worker's rows back (to Xw, which
+    // is X itself unless rows have a second reader)
+    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
+    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
+    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    PendingEnd<D> pi, pj;
     if (UPDATE) {
-        if (tab_prev[st.tab.off_degree + wi] > 0) {
-            const int ep = tab_prev[st.tab.off_slot_edge + wi * st.tab.max_degree];
-            ui = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
-            phi = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
-            coef_i = __int_as_float(tab_prev[st.tab.off_slot_coef + wi * st.tab.max_degree]);
-        }
-        if (tab_prev[st.tab.off_degree + wj] > 0) {
-            const int ep = tab_prev[st.tab.off_slot_edge + wj * st.tab.max_degree];
-            uj = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
-            phj = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
-            coef_j = __int_as_float(tab_prev[st.tab.off_slot_coef + wj * st.tab.max_degree]);
-        }
+        pending_of<D>(st, tab_prev, wi, g, q, pi);
+        pending_of<D>(st, tab_prev, wj, g, q, pj);
     }
     const int r0 = tile.rtile * g.p_rows;
     const int r1 = min(g.n, r0 + g.p_rows);
@@ -973,8 +1001,11 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         const bool in = idx < ld;
         s_q[idx] = in ? q[idx] * qinv : 0.0f;
         if (UPDATE) {
-            s_ui[idx] = in ? ui[idx] : 0.0f;
-            s_uj[idx] = in ? uj[idx] : 0.0f;
+#pragma unroll
+            for (int s2 = 0; s2 < D; ++s2) {
+                s_ui[s2][idx] = in ? pi.vec[s2][idx] : 0.0f;
+                s_uj[s2][idx] = in ? pj.vec[s2][idx] : 0.0f;
+            }
         }
     }
     __syncthreads();
@@ -1027,22 +1058,29 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                 }
             }
             if (UPDATE) {
-                const float ai = phi ? coef_i * __ldg(phi + r) : 0.0f;
-                const float aj = phj ? coef_j * __ldg(phj + r) : 0.0f;
-                float* rowi = Xi + (long long)r * ld;
-                float* rowj = Xj + (long long)r * ld;
+                float ai[D], aj[D];
+#pragma unroll
+                for (int s2 = 0; s2 < D; ++s2) {
+                    ai[s2] = pi.ph[s2] ? pi.coef[s2] * __ldg(pi.ph[s2] + r) : 0.0f;
+                    aj[s2] = pj.ph[s2] ? pj.coef[s2] * __ldg(pj.ph[s2] + r) : 0.0f;
+                }
+                float* rowi = Xi_w + (long long)r * ld;
+                float* rowj = Xj_w + (long long)r * ld;
 #pragma unroll
                 for (int k = 0; k < NV; ++k) {
                     const int col = (k * 32 + lane) * 4;
-                    const float4 vi = *reinterpret_cast<const float4*>(&s_ui[col]);
-                    const float4 vj = *reinterpret_cast<const float4*>(&s_uj[col]);
-                    xi[k].x = fmaf(-ai, vi.x, xi[k].x); xi[k].y = fmaf(-ai, vi.y, xi[k].y);
-                    xi[k].z = fmaf(-ai, vi.z, xi[k].z); xi[k].w = fmaf(-ai, vi.w, xi[k].w);
-                    xj[k].x = fmaf(-aj, vj.x, xj[k].x); xj[k].y = fmaf(-aj, vj.y, xj[k].y);
-                    xj[k].z = fmaf(-aj, vj.z, xj[k].z); xj[k].w = fmaf(-aj, vj.w, xj[k].w);
+#pragma unroll
+                    for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
+                        const float4 vi = *reinterpret_cast<const float4*>(&s_ui[s2][col]);
+                        const float4 vj = *reinterpret_cast<const float4*>(&s_uj[s2][col]);
+                        xi[k].x = fmaf(-ai[s2], vi.x, xi[k].x); xi[k].y = fmaf(-ai[s2], vi.y, xi[k].y);
+                        xi[k].z = fmaf(-ai[s2], vi.z, xi[k].z); xi[k].w = fmaf(-ai[s2], vi.w, xi[k].w);
+                        xj[k].x = fmaf(-aj[s2], vj.x, xj[k].x); xj[k].y = fmaf(-aj[s2], vj.y, xj[k].y);
+                        xj[k].z = fmaf(-aj[s2], vj.z, xj[k].z); xj[k].w = fmaf(-aj[s2], vj.w, xj[k].w);
+                    }
                     if (col < ld) {
-                        st_stream(rowi + col, xi[k]);
-                        st_stream(rowj + col, xj[k]);
+                        if (own_i) st_stream(rowi + col, xi[k]);
+                        if (own_j) st_stream(rowj + col, xj[k]);
                     }
                 }
             }
@@ -1108,12 +1146,12 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 // owns: no reduction is needed for u.  The barrier is split (arrive ... wait)
 // and the loads of the next rows are issued in between.
 // --------------------------------------------------------------------------
-template <int NVW, bool UPDATE>
+template <int NVW, bool UPDATE, int D>
 __global__ void __cluster_dims__(kPairCluster, 1, 1) __launch_bounds__(256, PG_WIDE_MIN_BLOCKS)
 pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles, int slice_pad) {
     namespace cg = cooperative_groups;
-    extern __shared__ __align__(16) float s_vec[];               // q-hat, u_i, u_j slices
+    extern __shared__ __align__(16) float s_vec[];               // slices of q-hat, D x u_i, D x u_j
     __shared__ __align__(16) float s_share[2][kPairCluster][kPairWideStep];    // [parity][rank][row]
     __shared__ float s_warp[8][kPairWideStep];
     __shared__ __align__(8) unsigned long long s_arrived[2];     // one mbarrier per parity: counts the shares' bytes
@@ -1134,28 +1172,21 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     const int c_end = min(ld, c_begin + g.p_slice);
 
     float* s_q = s_vec;
-    float* s_ui = s_vec + slice_pad;
-    float* s_uj = s_vec + 2 * slice_pad;
+    float* s_ui = s_vec + slice_pad;                  // [D][slice_pad]
+    float* s_uj = s_vec + (1 + D) * slice_pad;        // [D][slice_pad]
     const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
     const float qinv = pair_qinv(st, pair, tile.layer);
-    const float* ui = q;
-    const float* uj = q;
-    const float* phi = nullptr;
-    const float* phj = nullptr;
-    float coef_i = 0.0f, coef_j = 0.0f;
+    // only the edge in slot 0 of a worker writes that worker's rows back (to Xw, which
+    // is X itself unless rows have a second reader)
+    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
+    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
+    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    PendingEnd<D> pi, pj;
     if (UPDATE) {
-        if (tab_prev[st.tab.off_degree + wi] > 0) {
-            const int ep = tab_prev[st.tab.off_slot_edge + wi * st.tab.max_degree];
-            ui = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
-            phi = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
-            coef_i = __int_as_float(tab_prev[st.tab.off_slot_coef + wi * st.tab.max_degree]);
-        }
-        if (tab_prev[st.tab.off_degree + wj] > 0) {
-            const int ep = tab_prev[st.tab.off_slot_edge + wj * st.tab.max_degree];
-            uj = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
-            phj = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
-            coef_j = __int_as_float(tab_prev[st.tab.off_slot_coef + wj * st.tab.max_degree]);
-        }
+        pending_of<D>(st, tab_prev, wi, g, q, pi);
+        pending_of<D>(st, tab_prev, wj, g, q, pj);
     }
     if (threadIdx.x == 0) {
         s_gave_up = 0;
@@ -1168,8 +1199,11 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         const bool in = col < c_end;
         s_q[idx] = in ? q[col] * qinv : 0.0f;
         if (UPDATE) {
-            s_ui[idx] = in ? ui[col] : 0.0f;
-            s_uj[idx] = in ? uj[col] : 0.0f;
+#pragma unroll
+            for (int s2 = 0; s2 < D; ++s2) {
+                s_ui[s2 * slice_pad + idx] = in ? pi.vec[s2][col] : 0.0f;
+                s_uj[s2 * slice_pad + idx] = in ? pj.vec[s2][col] : 0.0f;
+            }
         }
     }
     cluster.sync();      // every CTA's mbarriers exist before a peer signals them
@@ -1214,24 +1248,28 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
             dot[t] = 0.0f;
             const bool in_row = r + t < r1;
             const long long base = (long long)(in_row ? r + t : r1 - 1) * ld + c_begin;
-            float ai = 0.0f, aj = 0.0f;
-            if (UPDATE && in_row) {
-                ai = phi ? coef_i * __ldg(phi + r + t) : 0.0f;
-                aj = phj ? coef_j * __ldg(phj + r + t) : 0.0f;
+            float ai[D], aj[D];
+#pragma unroll
+            for (int s2 = 0; s2 < D; ++s2) {
+                ai[s2] = (UPDATE && in_row && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r + t) : 0.0f;
+                aj[s2] = (UPDATE && in_row && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r + t) : 0.0f;
             }
 #pragma unroll
             for (int k = 0; k < NVW; ++k) {
                 const int off = (k * 256 + threadIdx.x) * 4;
                 const bool in = in_row && c_begin + off < c_end;
                 if (UPDATE && in) {
-                    const float4 vi = *reinterpret_cast<const float4*>(&s_ui[off]);
-                    const float4 vj = *reinterpret_cast<const float4*>(&s_uj[off]);
-                    xi[t][k].x = fmaf(-ai, vi.x, xi[t][k].x); xi[t][k].y = fmaf(-ai, vi.y, xi[t][k].y);
-                    xi[t][k].z = fmaf(-ai, vi.z, xi[t][k].z); xi[t][k].w = fmaf(-ai, vi.w, xi[t][k].w);
-                    xj[t][k].x = fmaf(-aj, vj.x, xj[t][k].x); xj[t][k].y = fmaf(-aj, vj.y, xj[t][k].y);
-                    xj[t][k].z = fmaf(-aj, vj.z, xj[t][k].z); xj[t][k].w = fmaf(-aj, vj.w, xj[t][k].w);
-                    st_stream(Xi + base + off, xi[t][k]);
-                    st_stream(Xj + base + off, xj[t][k]);
+#pragma unroll
+                    for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
+                        const float4 vi = *reinterpret_cast<const float4*>(&s_ui[s2 * slice_pad + off]);
+                        const float4 vj = *reinterpret_cast<const float4*>(&s_uj[s2 * slice_pad + off]);
+                        xi[t][k].x = fmaf(-ai[s2], vi.x, xi[t][k].x); xi[t][k].y = fmaf(-ai[s2], vi.y, xi[t][k].y);
+                        xi[t][k].z = fmaf(-ai[s2], vi.z, xi[t][k].z); xi[t][k].w = fmaf(-ai[s2], vi.w, xi[t][k].w);
+                        xj[t][k].x = fmaf(-aj[s2], vj.x, xj[t][k].x); xj[t][k].y = fmaf(-aj[s2], vj.y, xj[t][k].y);
+                        xj[t][k].z = fmaf(-aj[s2], vj.z, xj[t][k].z); xj[t][k].w = fmaf(-aj[s2], vj.w, xj[t][k].w);
+                    }
+                    if (own_i) st_stream(Xi_w + base + off, xi[t][k]);
+                    if (own_j) st_stream(Xj_w + base + off, xj[t][k]);
                 }
                 d[t][k].x = xi[t][k].x - xj[t][k].x; d[t][k].y = xi[t][k].y - xj[t][k].y;
                 d[t][k].z = xi[t][k].z - xj[t][k].z; d[t][k].w = xi[t][k].w - xj[t][k].w;
@@ -1294,18 +1332,347 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     cluster.sync();              // nobody leaves while a peer could still address its shared memory
 }
 
+// --------------------------------------------------------------------------
+// Pair sweep for rows of up to kPairMidMaxLd floats: a CTA shares every row.
+// Thread t owns the columns 4*(k*256 + t) .. +3 for k < NVM of every row, keeps
+// them in registers and adds p_r D_r to its own columns of u, so u needs no
+// reduction.  The row product p_r is the sum of the eight warps' shares, added
+// in warp order by every thread; one barrier per row, with the next row's loads
+// issued before it.
+// --------------------------------------------------------------------------
+template <int NVM, bool UPDATE, int D>
+__global__ void __launch_bounds__(256, (NVM <= 2 ? 3 : (NVM <= 5 ? 2 : 1)))
+pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
+                      const Tile* __restrict__ tiles, int ld_pad) {
+    extern __shared__ __align__(16) float s_vec[];               // q-hat, D x u_i, D x u_j; ld_pad floats each
+    __shared__ float s_warp[2][8];
+
+    const Tile tile = tiles[blockIdx.x];
+    const int e = tile.worker;
+    if (e >= tab_cur[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[tile.layer];
+    const int wi = tab_cur[st.tab.off_edge_i + e], wj = tab_cur[st.tab.off_edge_j + e];
+    const int pair = tab_cur[st.tab.off_pair + e];
+    const float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
+    const float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
+    const int ld = g.ld;
+
+    float* s_q = s_vec;
+    float* s_ui = s_vec + ld_pad;                     // [D][ld_pad]
+    float* s_uj = s_vec + (1 + D) * ld_pad;           // [D][ld_pad]
+    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float qinv = pair_qinv(st, pair, tile.layer);
+    // only the edge in slot 0 of a worker writes that worker's rows back (to Xw, which
+    // is X itself unless rows have a second reader)
+    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
+    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
+    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    PendingEnd<D> pi, pj;
+    if (UPDATE) {
+        pending_of<D>(st, tab_prev, wi, g, q, pi);
+        pending_of<D>(st, tab_prev, wj, g, q, pj);
+    }
+    for (int idx = threadIdx.x; idx < ld_pad; idx += 256) {
+        const bool in = idx < ld;
+        s_q[idx] = in ? q[idx] * qinv : 0.0f;
+        if (UPDATE) {
+#pragma unroll
+            for (int s2 = 0; s2 < D; ++s2) {
+                s_ui[s2 * ld_pad + idx] = in ? pi.vec[s2][idx] : 0.0f;
+                s_uj[s2 * ld_pad + idx] = in ? pj.vec[s2][idx] : 0.0f;
+            }
+        }
+    }
+    __syncthreads();
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r0 = tile.rtile * g.p_rows;
+    const int r1 = min(g.n, r0 + g.p_rows);
+    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    float4 u[NVM];
+#pragma unroll
+    for (int k = 0; k < NVM; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float ssum = 0.0f;
+
+    float4 xi[NVM], xj[NVM];
+    auto load_row = [&](int r) {
+        const long long base = (long long)r * ld;
+#pragma unroll
+        for (int k = 0; k < NVM; ++k) {
+            const int off = (k * 256 + threadIdx.x) * 4;
+            if (off < ld) {
+                xi[k] = ld_stream(Xi + base + off);
+                xj[k] = ld_stream(Xj + base + off);
+            } else {
+                xi[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                xj[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+    };
+    load_row(r0);
+    int it = 0;
+    for (int r = r0; r < r1; ++r, ++it) {
+        float4 d[NVM];            // this thread's columns of row r of D
+        float dot = 0.0f;
+        const long long base = (long long)r * ld;
+        float ai[D], aj[D];
+#pragma unroll
+        for (int s2 = 0; s2 < D; ++s2) {
+            ai[s2] = (UPDATE && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r) : 0.0f;
+            aj[s2] = (UPDATE && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r) : 0.0f;
+        }
+#pragma unroll
+        for (int k = 0; k < NVM; ++k) {
+            const int off = (k * 256 + threadIdx.x) * 4;
+            const bool in = off < ld;
+            if (UPDATE && in) {
+#pragma unroll
+                for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
+                    const float4 vi = *reinterpret_cast<const float4*>(&s_ui[s2 * ld_pad + off]);
+                    const float4 vj = *reinterpret_cast<const float4*>(&s_uj[s2 * ld_pad + off]);
+                    xi[k].x = fmaf(-ai[s2], vi.x, xi[k].x); xi[k].y = fmaf(-ai[s2], vi.y, xi[k].y);
+                    xi[k].z = fmaf(-ai[s2], vi.z, xi[k].z); xi[k].w = fmaf(-ai[s2], vi.w, xi[k].w);
+                    xj[k].x = fmaf(-aj[s2], vj.x, xj[k].x); xj[k].y = fmaf(-aj[s2], vj.y, xj[k].y);
+                    xj[k].z = fmaf(-aj[s2], vj.z, xj[k].z); xj[k].w = fmaf(-aj[s2], vj.w, xj[k].w);
+                }
+                if (own_i) st_stream(Xi_w + base + off, xi[k]);
+                if (own_j) st_stream(Xj_w + base + off, xj[k]);
+            }
+            d[k].x = xi[k].x - xj[k].x; d[k].y = xi[k].y - xj[k].y;
+            d[k].z = xi[k].z - xj[k].z; d[k].w = xi[k].w - xj[k].w;
+            if (in) {
+                const float4 vq = *reinterpret_cast<const float4*>(&s_q[off]);
+                dot = fmaf(d[k].x, vq.x, dot); dot = fmaf(d[k].y, vq.y, dot);
+                dot = fmaf(d[k].z, vq.z, dot); dot = fmaf(d[k].w, vq.w, dot);
+            }
+        }
+        dot = warp_sum(dot);
+        if (lane == 0) s_warp[it & 1][warp] = dot;
+        if (r + 1 < r1) load_row(r + 1);          // in flight across the barrier
+        __syncthreads();
+        // the buffer of this parity is written again two rows on, after the next barrier
+        float p = 0.0f;
+#pragma unroll
+        for (int w8 = 0; w8 < 8; ++w8) p += s_warp[it & 1][w8];
+#pragma unroll
+        for (int k = 0; k < NVM; ++k) {
+            u[k].x = fmaf(p, d[k].x, u[k].x); u[k].y = fmaf(p, d[k].y, u[k].y);
+            u[k].z = fmaf(p, d[k].z, u[k].z); u[k].w = fmaf(p, d[k].w, u[k].w);
+        }
+        ssum = fmaf(p, p, ssum);
+        if (threadIdx.x == 0) Pw[r] = p;
+    }
+    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld;
+#pragma unroll
+    for (int k = 0; k < NVM; ++k) {
+        const int off = (k * 256 + threadIdx.x) * 4;
+        if (off < ld) *reinterpret_cast<float4*>(Up + off) = u[k];
+    }
+    if (threadIdx.x == 0) st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = (double)ssum;
+}
+
+// --------------------------------------------------------------------------
+// The same CTA-per-row sweep fed by bulk asynchronous copies (TMA), for rows of
+// up to kMidBulkNv * 1024 floats.  One thread moves kMidRows consecutive rows of
+// X_i and of X_j (contiguous in memory) into a shared-memory stage with two
+// cp.async.bulk copies, n_stage stages ahead of the arithmetic; an mbarrier per
+// stage counts the bytes.  A thread always works on the same columns, so it keeps
+// its part of q-hat and of the pending corrections' vectors in registers and
+// shared memory holds nothing but rows in flight.  The barrier that publishes
+// the warps' shares of the row products also tells that every thread has taken
+// its columns out of the stage, so the stage is refilled right after it.  Waits
+// are bounded as in the row-per-warp variant; a wait that runs out ends the CTA
+// at the next barrier.
+// --------------------------------------------------------------------------
+constexpr int kMidStagesMax = 4;
+constexpr int kMidRows = 2;       // rows per stage and per barrier
+constexpr int kMidBulkNv = 5;     // most float4 per thread and row (registers)
+
+template <int NVM, bool UPDATE, int D>
+__global__ void __launch_bounds__(256, 1)
+pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
+                           const Tile* __restrict__ tiles, int ld_pad, int n_stage) {
+    extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][kMidRows * ld_pad]
+    __shared__ __align__(8) unsigned long long s_full[kMidStagesMax];
+    __shared__ float s_warp[2][kMidRows][8];
+    __shared__ int s_abort;
+    constexpr int RS = kMidRows;
+
+    const Tile tile = tiles[blockIdx.x];
+    const int e = tile.worker;
+    if (e >= tab_cur[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[tile.layer];
+    const int wi = tab_cur[st.tab.off_edge_i + e], wj = tab_cur[st.tab.off_edge_j + e];
+    const int pair = tab_cur[st.tab.off_pair + e];
+    const float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
+    const float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
+    const int ld = g.ld;
+    const unsigned row_bytes = (unsigned)ld * 4u;     // multiple of 16: ld is a multiple of 4
+
+    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float qinv = pair_qinv(st, pair, tile.layer);
+    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
+    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
+    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    PendingEnd<D> pi, pj;
+    if (UPDATE) {
+        pending_of<D>(st, tab_prev, wi, g, q, pi);
+        pending_of<D>(st, tab_prev, wj, g, q, pj);
+    }
+    const int r0 = tile.rtile * g.p_rows;
+    const int r1 = min(g.n, r0 + g.p_rows);
+    const int n_iter = (r1 - r0 + RS - 1) / RS;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s2 = 0; s2 < n_stage; ++s2) mbar_init(&s_full[s2], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    auto issue = [&](int idx) {       // rows r0 + idx*RS ... into slot idx % n_stage
+        const int slot = idx % n_stage;
+        const int row = r0 + idx * RS;
+        const unsigned bytes = (unsigned)min(RS, r1 - row) * row_bytes;
+        float* dst = s_stage + (size_t)slot * 2 * RS * ld_pad;
+        mbar_expect_tx(&s_full[slot], 2 * bytes);
+        bulk_load(dst, Xi + (long long)row * ld, bytes, &s_full[slot]);
+        bulk_load(dst + (size_t)RS * ld_pad, Xj + (long long)row * ld, bytes, &s_full[slot]);
+    };
+    int issued = 0;
+    if (threadIdx.x == 0)
+        for (; issued < n_stage && issued < n_iter; ++issued) issue(issued);
+
+    // this thread's columns of the vectors, for the whole tile
+    float4 vq[NVM], vi[D][NVM], vj[D][NVM];
+#pragma unroll
+    for (int k = 0; k < NVM; ++k) {
+        const int off = (k * 256 + threadIdx.x) * 4;
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+        vq[k] = zero;
+        if (off < ld) {
+            vq[k] = *reinterpret_cast<const float4*>(q + off);
+            vq[k].x *= qinv; vq[k].y *= qinv; vq[k].z *= qinv; vq[k].w *= qinv;
+        }
+#pragma unroll
+        for (int s2 = 0; s2 < D; ++s2) {
+            vi[s2][k] = (UPDATE && off < ld) ? *reinterpret_cast<const float4*>(pi.vec[s2] + off) : zero;
+            vj[s2][k] = (UPDATE && off < ld) ? *reinterpret_cast<const float4*>(pj.vec[s2] + off) : zero;
+        }
+    }
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    float4 u[NVM];
+#pragma unroll
+    for (int k = 0; k < NVM; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float ssum = 0.0f;
+    bool ok = true;
+
+    for (int it = 0; it < n_iter; ++it) {
+        const int r = r0 + it * RS;
+        const int slot = it % n_stage;
+        const bool mine = mbar_wait_bounded(&s_full[slot], (unsigned)((it / n_stage) & 1), &s_abort, st.status);
+        const float* si = s_stage + (size_t)slot * 2 * RS * ld_pad;      // rows follow each other ld floats apart
+        const float* sj = si + (size_t)RS * ld_pad;
+        float4 d[RS][NVM];
+        float dot[RS];
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            const bool in_row = mine && r + t < r1;
+            const long long base = (long long)(r + t) * ld;
+            dot[t] = 0.0f;
+            float ai[D], aj[D];
+#pragma unroll
+            for (int s2 = 0; s2 < D; ++s2) {
+                ai[s2] = (UPDATE && in_row && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r + t) : 0.0f;
+                aj[s2] = (UPDATE && in_row && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r + t) : 0.0f;
+            }
+#pragma unroll
+            for (int k = 0; k < NVM; ++k) {
+                const int off = (k * 256 + threadIdx.x) * 4;
+                const bool in = in_row && off < ld;
+                float4 xi = make_float4(0.f, 0.f, 0.f, 0.f), xj = xi;
+                if (in) {
+                    xi = *reinterpret_cast<const float4*>(si + (size_t)t * ld + off);
+                    xj = *reinterpret_cast<const float4*>(sj + (size_t)t * ld + off);
+                }
+                if (UPDATE && in) {
+#pragma unroll
+                    for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
+                        xi.x = fmaf(-ai[s2], vi[s2][k].x, xi.x); xi.y = fmaf(-ai[s2], vi[s2][k].y, xi.y);
+                        xi.z = fmaf(-ai[s2], vi[s2][k].z, xi.z); xi.w = fmaf(-ai[s2], vi[s2][k].w, xi.w);
+                        xj.x = fmaf(-aj[s2], vj[s2][k].x, xj.x); xj.y = fmaf(-aj[s2], vj[s2][k].y, xj.y);
+                        xj.z = fmaf(-aj[s2], vj[s2][k].z, xj.z); xj.w = fmaf(-aj[s2], vj[s2][k].w, xj.w);
+                    }
+                    if (own_i) st_stream(Xi_w + base + off, xi);
+                    if (own_j) st_stream(Xj_w + base + off, xj);
+                }
+                d[t][k].x = xi.x - xj.x; d[t][k].y = xi.y - xj.y; d[t][k].z = xi.z - xj.z; d[t][k].w = xi.w - xj.w;
+                dot[t] = fmaf(d[t][k].x, vq[k].x, dot[t]); dot[t] = fmaf(d[t][k].y, vq[k].y, dot[t]);
+                dot[t] = fmaf(d[t][k].z, vq[k].z, dot[t]); dot[t] = fmaf(d[t][k].w, vq[k].w, dot[t]);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            dot[t] = warp_sum(dot[t]);
+            if (lane == 0) s_warp[it & 1][t][warp] = dot[t];
+        }
+        ok = __syncthreads_and(mine) != 0;        // shares visible, stage drained; all go on or all leave
+        if (!ok) break;
+        if (threadIdx.x == 0 && it + n_stage < n_iter) {
+            issue(it + n_stage);
+            issued = it + n_stage + 1;
+        }
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            float p = 0.0f;
+#pragma unroll
+            for (int w8 = 0; w8 < 8; ++w8) p += s_warp[it & 1][t][w8];
+#pragma unroll
+            for (int k = 0; k < NVM; ++k) {
+                u[k].x = fmaf(p, d[t][k].x, u[k].x); u[k].y = fmaf(p, d[t][k].y, u[k].y);
+                u[k].z = fmaf(p, d[t][k].z, u[k].z); u[k].w = fmaf(p, d[t][k].w, u[k].w);
+            }
+            ssum = fmaf(p, p, ssum);
+            if (threadIdx.x == 0 && r + t < r1) Pw[r + t] = p;
+        }
+    }
+    if (!ok) {
+        // leave only after the copies still in flight have landed (bounded)
+        if (threadIdx.x == 0)
+            for (int idx = 0; idx < issued; ++idx) {
+                const int slot = idx % n_stage;
+                for (int spin = 0; spin < kBulkSpinLimit; ++spin)
+                    if (mbar_try_wait(&s_full[slot], (unsigned)((idx / n_stage) & 1))) break;
+            }
+        return;
+    }
+    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld;
+#pragma unroll
+    for (int k = 0; k < NVM; ++k) {
+        const int off = (k * 256 + threadIdx.x) * 4;
+        if (off < ld) *reinterpret_cast<float4*>(Up + off) = u[k];
+    }
+    if (threadIdx.x == 0) st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = (double)ssum;
+}
+
 // Pair edge step: ||p||^2 from the tiles' shares, p-hat = p / ||p|| in place,
 // Q' = (sum of the tiles' shares of D^T p) / ||p||, and the shares of ||Q'||^2
 // (the sweep that uses Q' next adds them up).  A zero or non-finite norm leaves
-// the stored vector alone and zeroes p-hat.  kEdgeChunks CTAs per (edge, layer),
-// each taking a slice of the rows and of the columns.
+// the stored vector alone and zeroes p-hat.  LayerGeom::e_chunks CTAs per (edge,
+// layer), each taking a slice of the rows and of the columns; st.edge_tab lists
+// the (layer, chunk) pairs of one edge.
 __global__ void __launch_bounds__(256)
 pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     __shared__ double scratch[33];
     const int L = st.n_layers;
-    const int chunk = blockIdx.x % kEdgeChunks;
-    const int el = blockIdx.x / kEdgeChunks;
-    const int e = el / L, l = el - e * L;
+    const int e = blockIdx.x / st.e_total;
+    const int slot = blockIdx.x - e * st.e_total;
+    const int l = st.edge_tab[2 * slot], chunk = st.edge_tab[2 * slot + 1];
     if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
     if (!g.pair_mode) return;
@@ -1318,7 +1685,8 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     const bool live = finite && nn > 0.0;
     const double inv = live ? 1.0 / sqrt(nn) : 0.0;
     float* P = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
-    const int rw = (g.npad + kEdgeChunks - 1) / kEdgeChunks;
+    const int nch = g.e_chunks;
+    const int rw = (g.npad + nch - 1) / nch;
     for (int r = chunk * rw + threadIdx.x; r < min(g.npad, (chunk + 1) * rw); r += blockDim.x)
         P[r] = (live && r < g.n) ? (float)((double)P[r] * inv) : 0.0f;
     if (chunk == 0 && threadIdx.x == 0) {
@@ -1328,7 +1696,7 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     if (!live) return;   // uniform over the block
     const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
     float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
-    const int cw = (g.m + kEdgeChunks - 1) / kEdgeChunks;
+    const int cw = (g.m + nch - 1) / nch;
     const int c_lo = chunk * cw, c_hi = min(g.m, (chunk + 1) * cw);
     part = 0.0;
     if (cw <= 32) {
@@ -1521,33 +1889,33 @@ cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile*
     return launch_row<true, false, false>(st, tab_update, tab_update, tiles, n_tiles, stream);
 }
 
-template <int NV, bool UPDATE>
+template <int NV, bool UPDATE, int D>
 static cudaError_t launch_pair_bulk_t(const DevState& st, const int* tab_prev, const int* tab_cur,
                                       const Tile* tiles, int n_tiles, int max_ld, cudaStream_t stream) {
     // stage buffers; they also hold the 8 x NV*128 floats of the final reduction
     size_t smem = sizeof(float) * (size_t)kBulkStages * 2 * kBulkRows * max_ld;
     const size_t red = sizeof(float) * 8 * NV * 128;
     if (smem < red) smem = red;
-    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE>,
+    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE, D>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (rc != cudaSuccess) return rc;
-    pair_sweep_bulk_kernel<NV, UPDATE><<<n_tiles, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles);
+    pair_sweep_bulk_kernel<NV, UPDATE, D><<<n_tiles, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles);
     return cudaGetLastError();
 }
 
-template <bool UPDATE>
+template <bool UPDATE, int D>
 static cudaError_t launch_pair_bulk(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
                                     int n_tiles, int nv, cudaStream_t stream) {
     const int max_ld = nv * 128;
     switch (nv) {
-        case 1: return launch_pair_bulk_t<1, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 2: return launch_pair_bulk_t<2, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 3: return launch_pair_bulk_t<3, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 4: return launch_pair_bulk_t<4, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 5: return launch_pair_bulk_t<5, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 6: return launch_pair_bulk_t<6, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 7: return launch_pair_bulk_t<7, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        default: return launch_pair_bulk_t<8, UPDATE>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 1: return launch_pair_bulk_t<1, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 2: return launch_pair_bulk_t<2, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 3: return launch_pair_bulk_t<3, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 4: return launch_pair_bulk_t<4, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 5: return launch_pair_bulk_t<5, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 6: return launch_pair_bulk_t<6, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 7: return launch_pair_bulk_t<7, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        default: return launch_pair_bulk_t<8, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
     }
 }
 
@@ -1569,62 +1937,67 @@ static cudaError_t launch_pair(const DevState& st, const int* tab_prev, const in
 
 // `tiles` must list tiles of layers with the same number of float4 per lane
 // (ceil(ld / 128)); the host launches one group per value.
+// pend_slots: how many corrections can be pending at a worker (its largest degree).
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
-                              const Tile* tiles, int n_tiles, int nv, cudaStream_t stream) {
+                              const Tile* tiles, int n_tiles, int nv, int pend_slots, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
-    if (st.pair_bulk)
-        return apply_pending ? launch_pair_bulk<true>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
-                             : launch_pair_bulk<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (st.pair_bulk) {
+        if (!apply_pending) return launch_pair_bulk<false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+        return pend_slots > 1 ? launch_pair_bulk<true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
+                              : launch_pair_bulk<true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    }
+    if (pend_slots > 1) return cudaErrorInvalidValue;     // the register-fed variant holds one correction per end
     return apply_pending ? launch_pair<true>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
                          : launch_pair<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
 }
 
-template <int NVW, bool UPDATE>
+template <int NVW, bool UPDATE, int D>
 static cudaError_t launch_wide_t(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
                                  int n_tiles, int slice_pad, cudaStream_t stream) {
     const dim3 grid(static_cast<unsigned>(n_tiles) * kPairCluster);
-    const size_t smem = sizeof(float) * 3 * static_cast<size_t>(slice_pad);
+    const size_t smem = sizeof(float) * (1 + 2 * D) * static_cast<size_t>(slice_pad);
     if (smem > 48 * 1024) {
-        cudaError_t rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, UPDATE>,
+        cudaError_t rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, UPDATE, D>,
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (rc != cudaSuccess) return rc;
     }
-    pair_sweep_wide_kernel<NVW, UPDATE><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
+    pair_sweep_wide_kernel<NVW, UPDATE, D><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
     return cudaGetLastError();
 }
 
 template <int NVW>
-static cudaError_t launch_wide(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd,
+static cudaError_t launch_wide(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd, int pend_slots,
                                const Tile* tiles, int n_tiles, int slice_pad, cudaStream_t stream) {
-    return upd ? launch_wide_t<NVW, true>(st, tab_prev, tab_cur, tiles, n_tiles, slice_pad, stream)
-               : launch_wide_t<NVW, false>(st, tab_prev, tab_cur, tiles, n_tiles, slice_pad, stream);
+    if (!upd) return launch_wide_t<NVW, false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, slice_pad, stream);
+    return pend_slots > 1 ? launch_wide_t<NVW, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, slice_pad, stream)
+                          : launch_wide_t<NVW, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, slice_pad, stream);
 }
 
 // `tiles`: cluster tiles of layers with the same float4 count per thread `nv` and
 // the same slice width `slice` (columns per CTA).
 cudaError_t launch_pair_sweep_wide(const DevState& st, const int* tab_prev, const int* tab_cur,
                                    bool apply_pending, const Tile* tiles, int n_tiles, int nv, int slice,
-                                   cudaStream_t stream) {
+                                   int pend_slots, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
     const int slice_pad = (slice + 3) / 4 * 4;
     switch (nv) {
-        case 1: return launch_wide<1>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
-        case 2: return launch_wide<2>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
-        case 3: return launch_wide<3>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
-        case 4: return launch_wide<4>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
-        case 5: return launch_wide<5>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
-        case 6: return launch_wide<6>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
-        case 7: return launch_wide<7>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
-        default: return launch_wide<8>(st, tab_prev, tab_cur, apply_pending, tiles, n_tiles, slice_pad, stream);
+        case 1: return launch_wide<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
+        case 2: return launch_wide<2>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
+        case 3: return launch_wide<3>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
+        case 4: return launch_wide<4>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
+        case 5: return launch_wide<5>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
+        case 6: return launch_wide<6>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
+        case 7: return launch_wide<7>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
+        default: return launch_wide<8>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, slice_pad, stream);
     }
 }
 
-template <int NVW>
+template <int NVW, int D>
 static int resident_clusters(int slice_pad) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kPairCluster * 1024);
     cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = sizeof(float) * 3 * static_cast<size_t>(slice_pad);
+    cfg.dynamicSmemBytes = sizeof(float) * (1 + 2 * D) * static_cast<size_t>(slice_pad);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = kPairCluster;
@@ -1635,9 +2008,9 @@ static int resident_clusters(int slice_pad) {
     int n = 0;
     cudaError_t rc = cudaSuccess;
     if (cfg.dynamicSmemBytes > 48 * 1024)
-        rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        rc = cudaFuncSetAttribute(pair_sweep_wide_kernel<NVW, true, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)cfg.dynamicSmemBytes);
-    if (rc == cudaSuccess) rc = cudaOccupancyMaxActiveClusters(&n, pair_sweep_wide_kernel<NVW, true>, &cfg);
+    if (rc == cudaSuccess) rc = cudaOccupancyMaxActiveClusters(&n, pair_sweep_wide_kernel<NVW, true, D>, &cfg);
     if (rc != cudaSuccess) {
         cudaGetLastError();
         return 0;
@@ -1645,23 +2018,88 @@ static int resident_clusters(int slice_pad) {
     return n;
 }
 
-int pair_wide_resident_clusters(int nv, int slice) {
+int pair_wide_resident_clusters(int nv, int slice, int pend_slots) {
     const int slice_pad = (slice + 3) / 4 * 4;
+    if (pend_slots > 1) switch (nv) {
+        case 1: return resident_clusters<1, 2>(slice_pad);
+        case 2: return resident_clusters<2, 2>(slice_pad);
+        case 3: return resident_clusters<3, 2>(slice_pad);
+        case 4: return resident_clusters<4, 2>(slice_pad);
+        case 5: return resident_clusters<5, 2>(slice_pad);
+        case 6: return resident_clusters<6, 2>(slice_pad);
+        case 7: return resident_clusters<7, 2>(slice_pad);
+        default: return resident_clusters<8, 2>(slice_pad);
+    }
     switch (nv) {
-        case 1: return resident_clusters<1>(slice_pad);
-        case 2: return resident_clusters<2>(slice_pad);
-        case 3: return resident_clusters<3>(slice_pad);
-        case 4: return resident_clusters<4>(slice_pad);
-        case 5: return resident_clusters<5>(slice_pad);
-        case 6: return resident_clusters<6>(slice_pad);
-        case 7: return resident_clusters<7>(slice_pad);
-        default: return resident_clusters<8>(slice_pad);
+        case 1: return resident_clusters<1, 1>(slice_pad);
+        case 2: return resident_clusters<2, 1>(slice_pad);
+        case 3: return resident_clusters<3, 1>(slice_pad);
+        case 4: return resident_clusters<4, 1>(slice_pad);
+        case 5: return resident_clusters<5, 1>(slice_pad);
+        case 6: return resident_clusters<6, 1>(slice_pad);
+        case 7: return resident_clusters<7, 1>(slice_pad);
+        default: return resident_clusters<8, 1>(slice_pad);
     }
 }
 
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
-    pair_edge_kernel<<<max_edges * st.n_layers * kEdgeChunks, 256, 0, stream>>>(st, tab);
+    if (st.e_total <= 0) return cudaSuccess;
+    pair_edge_kernel<<<max_edges * st.e_total, 256, 0, stream>>>(st, tab);
     return cudaGetLastError();
+}
+
+// Shared memory one CTA may ask for, less the kernels' static part.
+constexpr size_t kMidSmemBudget = 227 * 1024 - 512;
+
+template <int NVM, bool UPDATE, int D>
+static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
+                                int n_tiles, int ld_pad, cudaStream_t stream) {
+    const size_t smem = sizeof(float) * (1 + 2 * D) * static_cast<size_t>(ld_pad);
+    // TMA-fed variant when the row fits its registers and at least two stages fit in shared memory
+    if constexpr (NVM <= kMidBulkNv) {
+        const size_t stage = sizeof(float) * 2 * kMidRows * static_cast<size_t>(ld_pad);
+        const int n_stage = (int)std::min<size_t>(kMidSmemBudget / stage, kMidStagesMax);
+        if (st.pair_bulk && n_stage >= 2) {
+            const size_t total = n_stage * stage;
+            cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_bulk_kernel<NVM, UPDATE, D>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
+            if (rc != cudaSuccess) return rc;
+            pair_sweep_mid_bulk_kernel<NVM, UPDATE, D><<<n_tiles, 256, total, stream>>>(st, tab_prev, tab_cur, tiles,
+                                                                                       ld_pad, n_stage);
+            return cudaGetLastError();
+        }
+    }
+    if (smem > 48 * 1024) {
+        cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_kernel<NVM, UPDATE, D>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (rc != cudaSuccess) return rc;
+    }
+    pair_sweep_mid_kernel<NVM, UPDATE, D><<<n_tiles, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, ld_pad);
+    return cudaGetLastError();
+}
+
+template <int NVM>
+static cudaError_t launch_mid(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd, int pend_slots,
+                              const Tile* tiles, int n_tiles, int ld_pad, cudaStream_t stream) {
+    if (!upd) return launch_mid_t<NVM, false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    return pend_slots > 1 ? launch_mid_t<NVM, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream)
+                          : launch_mid_t<NVM, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+}
+
+cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const int* tab_cur,
+                                  bool apply_pending, const Tile* tiles, int n_tiles, int nv, int ld_pad,
+                                  int pend_slots, cudaStream_t stream) {
+    if (n_tiles <= 0) return cudaSuccess;
+    switch (nv) {
+        case 1: return launch_mid<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        case 2: return launch_mid<2>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        case 3: return launch_mid<3>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        case 4: return launch_mid<4>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        case 5: return launch_mid<5>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        case 6: return launch_mid<6>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        case 7: return launch_mid<7>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        default: return launch_mid<8>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+    }
 }
 
 template <bool UPDATE>

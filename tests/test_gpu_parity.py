@@ -283,8 +283,11 @@ PERSISTENT_CASES = [
 
 
 @pytest.mark.parametrize("w", PERSISTENT_CASES, ids=lambda w: w.name)
-def test_pg_rounds_equals_repeated_pg_round_bit_for_bit(w):
-    """pg_rounds(n) runs the same arithmetic in the same order as n calls of pg_round."""
+def test_pg_rounds_equals_repeated_pg_round_bit_for_bit(w, monkeypatch):
+    """pg_rounds(n) runs the same arithmetic in the same order as n calls of pg_round.
+    (Rank-1 rings would take the pair sweep, which pg_rounds enqueues round by round; switched
+    off here so that the cooperative kernel is the one compared.)"""
+    monkeypatch.setenv("PG_DISABLE_PAIR_SWEEP", "1")
     a, b = common.network_for(w), common.network_for(w)
     common.load_both(w, None, a)
     common.load_both(w, None, b)
@@ -303,7 +306,10 @@ def test_pg_rounds_equals_repeated_pg_round_bit_for_bit(w):
     b.close()
 
 
-def test_pg_rounds_against_the_checker():
+@pytest.mark.parametrize("three_sweeps", [True, False], ids=["cooperative_kernel", "pair_sweep"])
+def test_pg_rounds_against_the_checker(three_sweeps, monkeypatch):
+    if three_sweeps:
+        monkeypatch.setenv("PG_DISABLE_PAIR_SWEEP", "1")
     w = wl.tiny_ring()
     oracle, net = common.oracle_for(w), common.network_for(w)
     common.load_both(w, oracle, net)
@@ -328,6 +334,77 @@ def test_grid_barrier_gives_up_instead_of_hanging():
     other.pg_rounds(2)
     assert other.pg_device_status() == pg.PG_OK
     other.close()
+
+
+# ---- pair sweep on graphs of degree 2 (a row has two readers) ------------------
+# thin rows (a warp per row), rows a CTA shares (TMA-fed up to 5120 floats, register-fed beyond),
+# rows a cluster shares; few rows each, so the stack is small and every layer takes the pair sweep
+DEGREE2_SHAPES = ((33, 130), (20, 1500), (40, 4612), (12, 6000), (9, 9000), (5, 3))
+DEGREE2_GRAPHS = {
+    "ring3": dict(n_workers=3, kind=wl.RING, custom_edges=()),
+    "ring7": dict(n_workers=7, kind=wl.RING, custom_edges=()),
+    "path5": dict(n_workers=5, kind=wl.CUSTOM, custom_edges=((0, 1), (1, 2), (2, 3), (3, 4))),
+    "pair_and_path": dict(n_workers=5, kind=wl.CUSTOM, custom_edges=((0, 1), (2, 3), (3, 4))),
+}
+
+
+@pytest.mark.parametrize("graph", sorted(DEGREE2_GRAPHS))
+def test_pair_sweep_on_graphs_of_degree_two(graph):
+    # uniform weights 1/3: with Metropolis weights the isolated pair would get 1/2, which deflates its
+    # difference exactly, and on these flat-spectrum matrices that makes the iteration follow rounding noise
+    # (the checker alone, with X rounded to fp32 once per round, is then 3e-1 away after four rounds)
+    w = wl.Workload("deg2_" + graph, 9, 4, wl.RING, 0, 0, wl.W_UNIFORM, None, DEGREE2_SHAPES, 1, 2, 6, 31,
+                    "normal1").replace(**DEGREE2_GRAPHS[graph])
+    _run(w, rebased=True)
+    _run(w, rounds=3, check_every=1)
+
+
+def test_three_sweeps_on_a_rank_one_ring(monkeypatch):
+    """The general path on a graph where the pair sweep is the default."""
+    monkeypatch.setenv("PG_DISABLE_PAIR_SWEEP", "1")
+    w = wl.Workload("ring_three_sweeps", 9, 6, wl.RING, 0, 0, wl.W_METROPOLIS, None, DEGREE2_SHAPES, 1, 2, 6, 31,
+                    "normal1")
+    _run(w, rebased=True)
+    _run(wl.resnet20_ring8(), rounds=20, check_every=10)
+
+
+def test_reads_between_steps_do_not_change_a_ring_run():
+    """On a ring the corrected rows alternate between two copies of the stack and a read folds
+    the pending correction into the first one: a run that is read (and check-pointed) after every
+    round ends on the same bits as one that is never touched."""
+    w = wl.Workload("ring_reads", 9, 5, wl.RING, 0, 0, wl.W_UNIFORM, None, ((70, 130), (24, 1500)), 1, 1, 7, 3,
+                    "normal1")
+    a, b = common.network_for(w), common.network_for(w)
+    common.load_both(w, None, a)
+    common.load_both(w, None, b)
+    for t in range(w.rounds):
+        a.pg_round()
+        b.pg_round()
+        b.read_all()
+    xa, xb = a.read_all(), b.read_all()
+    # resume from a snapshot taken after an odd number of steps
+    c = common.network_for(w)
+    common.load_both(w, None, c)
+    for t in range(3):
+        c.pg_round()
+    snap_x = c.read_all()
+    edges = [(int(i), int(j)) for i, j in c.pg_get_schedule(0)[0]]
+    snap_q = {(i, j): [c.pg_read_q(i, j, l) for l in range(2)] for i, j in edges}
+    d = common.network_for(w)
+    d.write_all(snap_x)
+    for (i, j), qs in snap_q.items():
+        for l, q in enumerate(qs):
+            d.pg_write_q(i, j, l, q)
+    d.pg_set_round(3)
+    for t in range(3, w.rounds):
+        d.pg_round()
+    xd = d.read_all()
+    for i in range(w.n_workers):
+        for l in range(2):
+            assert np.array_equal(xa[i][l], xb[i][l])
+            assert np.array_equal(xa[i][l], xd[i][l])
+    for n in (a, b, c, d):
+        n.close()
 
 
 # ---- Algorithm 2 read literally (half-step mode) ------------------------------
