@@ -187,6 +187,36 @@ PG_API int pg_params_device(pg_ctx *ctx, int32_t worker, int32_t layer, void *st
 PG_API int pg_round(pg_ctx *ctx, void *stream);
 
 /*
+ * One round of Algorithm 1 with the local term: pg_round, and with the round's
+ * last update every worker's matrices also lose eta * G (line 6 of Algorithm 1:
+ * X_i <- X_i + sum_j W_ij C(X_j - X_i) - eta G_i, the gossip term computed from
+ * the parameters the gradient was taken at).  The gradient is read in the sweep
+ * that applies the update, so it costs one extra read of G (4 B per parameter)
+ * and no pass of its own; on return (of the enqueued work) X in memory is
+ * fully updated, ready for the next gradient evaluation.
+ *   G_dev   device, caller-owned, pg_stack_elems floats, 16-byte aligned, laid out
+ *           like the parameter stack: the rows x cols matrix of (worker, layer)
+ *           starts at pg_stack_offset's offset, row-major with its leading
+ *           dimension ld >= cols.  Only the rows x cols entries are read for
+ *           their values; the padding may hold anything finite or not.  Must
+ *           stay unchanged until the enqueued work has run.
+ *   eta     finite step size.
+ * In half-step and random-projection modes the gradient step is a pass of its
+ * own after the round (12 B per parameter).  PG_ERR_INVALID for a null,
+ * misaligned, host or other-device G or a non-finite eta; otherwise as pg_round.
+ */
+PG_API int pg_round_sgd(pg_ctx *ctx, const float *G_dev, float eta, void *stream);
+
+/*
+ * Shape of one copy of the parameter stack, for caller-owned buffers that
+ * mirror it (gradients): total floats, and where (worker, layer) starts (in
+ * floats from the start of the buffer) with its leading dimension.  Offsets are
+ * multiples of 64 floats.  Host out-params, written only on PG_OK.
+ */
+PG_API int pg_stack_elems(pg_ctx *ctx, int64_t *elems_out);
+PG_API int pg_stack_offset(pg_ctx *ctx, int32_t worker, int32_t layer, int64_t *offset_out, int64_t *ld_out);
+
+/*
  * Algorithm 2 read literally ("half-step mode"): every iteration is ONE
  * mat-vec and one gossip update with that iteration's approximation, and the
  * stored vector alternates between R^cols and R^rows:

@@ -28,6 +28,7 @@ EXPORTS = (
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
     "pg_transposed_product_noalloc", "pg_rounds", "pg_selftest_barrier_timeout",
     "pg_set_half_step", "pg_params_device", "pg_set_random_projection",
+    "pg_round_sgd", "pg_stack_elems", "pg_stack_offset",
 )
 PG_POWER_ITERATION, PG_RANDOM_RIGHT, PG_RANDOM_LEFT = 0, 1, 2
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
@@ -73,6 +74,9 @@ def load_library() -> ctypes.CDLL:
     L.pg_write_params.argtypes = [vp, i32, i32, vp, vp]
     L.pg_read_params.argtypes = [vp, i32, i32, vp, vp]
     L.pg_round.argtypes = [vp, vp]
+    L.pg_round_sgd.argtypes = [vp, vp, ctypes.c_float, vp]
+    L.pg_stack_elems.argtypes = [vp, ctypes.POINTER(i64)]
+    L.pg_stack_offset.argtypes = [vp, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     L.pg_params_device.argtypes = [vp, i32, i32, vp, ctypes.POINTER(vp), ctypes.POINTER(i64)]
     L.pg_device_status.argtypes = [vp, vp]
     L.pg_rounds.argtypes = [vp, i32, vp]
@@ -282,6 +286,42 @@ class PowerGossip:
     # -- rounds -----------------------------------------------------------
     def pg_round(self, stream=None) -> None:
         _check(self._lib.pg_round(self._h, _stream_handle(stream)), "pg_round")
+
+    def pg_stack_elems(self) -> int:
+        n = ctypes.c_int64(0)
+        _check(self._lib.pg_stack_elems(self._h, ctypes.byref(n)), "pg_stack_elems")
+        return int(n.value)
+
+    def pg_stack_offset(self, worker: int, layer: int):
+        """(offset in floats, leading dimension) of a worker's matrix in a buffer shaped like the stack."""
+        off, ld = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(self._lib.pg_stack_offset(self._h, worker, layer, ctypes.byref(off), ctypes.byref(ld)),
+               "pg_stack_offset")
+        return int(off.value), int(ld.value)
+
+    def gradient_buffer(self):
+        """A zeroed fp32 CUDA tensor of pg_stack_elems floats on the workspace's device."""
+        import torch
+
+        return torch.zeros(self.pg_stack_elems(), dtype=torch.float32, device=self._workspace.device)
+
+    def gradient_view(self, grads, worker: int, layer: int):
+        """(rows x cols) view of a worker's matrix inside a buffer made by gradient_buffer()."""
+        import torch
+
+        off, ld = self.pg_stack_offset(worker, layer)
+        n, m = self.layer_shapes[layer]
+        return torch.as_strided(grads, (n, m), (ld, 1), storage_offset=off)
+
+    def pg_round_sgd(self, grads, eta: float, stream=None) -> None:
+        """grads: fp32 CUDA tensor of pg_stack_elems floats laid out like the parameter stack."""
+        import torch
+
+        if not (isinstance(grads, torch.Tensor) and grads.is_cuda and grads.dtype == torch.float32
+                and grads.is_contiguous() and grads.numel() >= self.pg_stack_elems()):
+            raise ValueError("grads must be a contiguous fp32 CUDA tensor of at least pg_stack_elems floats")
+        _check(self._lib.pg_round_sgd(self._h, ctypes.c_void_p(grads.data_ptr()), ctypes.c_float(eta),
+                                      _stream_handle(stream)), "pg_round_sgd")
 
     def pg_set_half_step(self, on: bool = True) -> None:
         _check(self._lib.pg_set_half_step(self._h, 1 if on else 0), "pg_set_half_step")

@@ -289,7 +289,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_status = take(sizeof(int) * 64);   // [0] status word, [16..17] grid barrier of the persistent kernel
     lay.off_layers = take(sizeof(LayerGeom) * static_cast<size_t>(n_layers));
     lay.off_edge_tab = take(sizeof(int) * 2 * static_cast<size_t>(n_layers) * pg::kEdgeChunks);
-    lay.off_tabs = take(sizeof(int) * static_cast<size_t>(kTabRing) * t.total_ints);
+    lay.off_tabs = take(sizeof(int) * static_cast<size_t>(kTabRing + 1) * t.total_ints);   // + one table of an empty graph
     lay.off_row_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.row_tile_cap));
     lay.off_col_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.col_tile_cap));
     lay.off_pair_tiles = take(sizeof(Tile) * static_cast<size_t>(lay.n_pair_tiles_cap));
@@ -433,7 +433,8 @@ bool bind_device(const pg_ctx* c) {
 
 // Apply the correction the pair sweep left pending, so that X in memory is the
 // live model (needed before X, Q or the round counter are read or overwritten).
-int flush_pending(pg_ctx* c, cudaStream_t stream) {
+// G, eta: the caller's gradient step, taken in the same pass (pair-sweep layers only).
+int flush_pending(pg_ctx* c, cudaStream_t stream, const float* G = nullptr, float eta = 0.0f) {
     if (c->half_pending) {
         // the odd iteration's update p q-hat^T, with the scaled coefficients
         const int* tab = nullptr;
@@ -461,8 +462,10 @@ int flush_pending(pg_ctx* c, cudaStream_t stream) {
     // the corrected stack always lands in the first copy of X, the one the caller sees
     st.X = c->st.X + c->xbuf * static_cast<long long>(c->topo.n_workers) * c->lay.x_stride;
     st.Xw = c->st.X;
+    st.G = G;
+    st.eta = eta;
     {
-        Timed t(c, PG_KERNEL_UPDATE_ONLY, stream, 2.0 * c->pair_param_bytes);
+        Timed t(c, PG_KERNEL_UPDATE_ONLY, stream, (G ? 3.0 : 2.0) * c->pair_param_bytes);
         if (pg::launch_update(st, tab_prev, c->d_flush_tiles, static_cast<int>(c->lay.n_flush_tiles), stream) !=
             cudaSuccess) {
             cudaGetLastError();
@@ -472,6 +475,24 @@ int flush_pending(pg_ctx* c, cudaStream_t stream) {
     c->launches += 1;
     c->pending = false;
     c->xbuf = 0;
+    return PG_OK;
+}
+
+// X <- X - eta * G on the layers of `tiles` with no correction pending: the update sweep
+// run against the table of an empty graph.
+int gradient_only_pass(pg_ctx* c, cudaStream_t stream, const Tile* tiles, long long n_tiles, double param_bytes,
+                       const float* G, float eta) {
+    if (n_tiles <= 0) return PG_OK;
+    DevState st = c->st;
+    st.G = G;
+    st.eta = eta;
+    const int* empty = c->d_tabs + static_cast<size_t>(kTabRing) * c->lay.tab.total_ints;
+    Timed t(c, PG_KERNEL_UPDATE_ONLY, stream, 3.0 * param_bytes);
+    if (pg::launch_update(st, empty, tiles, static_cast<int>(n_tiles), stream) != cudaSuccess) {
+        cudaGetLastError();
+        return PG_ERR_CUDA;
+    }
+    c->launches += 1;
     return PG_OK;
 }
 
@@ -842,7 +863,9 @@ int pg_device_status(pg_ctx* c, void* stream) {
     return device_status(c, static_cast<cudaStream_t>(stream));
 }
 
-int pg_round(pg_ctx* c, void* stream_v) {
+// One round; with G, X also loses eta * G with the round's last update (Algorithm 1, line 6)
+// and is left fully updated in memory.
+static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
     if (!c) return PG_ERR_INVALID;
     if (!bind_device(c)) return PG_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -893,6 +916,10 @@ int pg_round(pg_ctx* c, void* stream_v) {
         if (!ok) {
             cudaGetLastError();
             return PG_ERR_CUDA;
+        }
+        if (G) {
+            rc = gradient_only_pass(c, stream, c->d_row_tiles, n_rows, c->normal_param_bytes, G, eta);
+            if (rc != PG_OK) return rc;
         }
         c->round += 1;
         return PG_OK;
@@ -945,6 +972,14 @@ int pg_round(pg_ctx* c, void* stream_v) {
             return PG_ERR_CUDA;
         }
         c->round += 1;
+        if (G) {
+            // apply what is pending, then the gradient step in a pass of its own
+            rc = flush_pending(c, stream);
+            if (rc == PG_OK)
+                rc = gradient_only_pass(c, stream, c->d_row_tiles, n_rows, c->normal_param_bytes, G, eta);
+            c->y_valid = false;
+            if (rc != PG_OK) return rc;
+        }
         return PG_OK;
     }
     if (n_rows > 0 && !c->y_valid) {
@@ -972,7 +1007,12 @@ int pg_round(pg_ctx* c, void* stream_v) {
                 ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
             }
             {
-                Timed t(c, PG_KERNEL_UPDATE_FORWARD, stream, 2.0 * c->normal_param_bytes);
+                // the round's last update also takes the gradient step; the product for the
+                // next round is formed from the rows it has just written
+                const bool with_g = G && p + 1 == c->power_steps;
+                st.G = with_g ? G : nullptr;
+                st.eta = eta;
+                Timed t(c, PG_KERNEL_UPDATE_FORWARD, stream, (with_g ? 3.0 : 2.0) * c->normal_param_bytes);
                 ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, stream) == cudaSuccess;
             }
             c->launches += 4;
@@ -1024,6 +1064,36 @@ int pg_round(pg_ctx* c, void* stream_v) {
     }
     c->y_valid = true;
     c->round += 1;
+    // pair-sweep layers: the pending correction and the gradient step in one pass
+    if (G && has_pair) return flush_pending(c, stream, G, eta);
+    return PG_OK;
+}
+
+int pg_round(pg_ctx* c, void* stream) { return round_impl(c, stream, nullptr, 0.0f); }
+
+int pg_round_sgd(pg_ctx* c, const float* G_dev, float eta, void* stream) {
+    if (!c || !G_dev || !std::isfinite(eta)) return PG_ERR_INVALID;
+    if (reinterpret_cast<uintptr_t>(G_dev) % 16 != 0) return PG_ERR_INVALID;
+    cudaPointerAttributes attr{};
+    if (cudaPointerGetAttributes(&attr, G_dev) != cudaSuccess || attr.type != cudaMemoryTypeDevice ||
+        attr.device != c->device) {
+        cudaGetLastError();
+        return PG_ERR_INVALID;
+    }
+    return round_impl(c, stream, G_dev, eta);
+}
+
+int pg_stack_elems(pg_ctx* c, int64_t* elems_out) {
+    if (!c || !elems_out) return PG_ERR_INVALID;
+    *elems_out = static_cast<int64_t>(c->topo.n_workers) * c->lay.x_stride;
+    return PG_OK;
+}
+
+int pg_stack_offset(pg_ctx* c, int32_t worker, int32_t layer, int64_t* offset_out, int64_t* ld_out) {
+    const int rc = check_worker_layer(c, worker, layer);
+    if (rc != PG_OK || !offset_out || !ld_out) return PG_ERR_INVALID;
+    *offset_out = static_cast<int64_t>(worker) * c->lay.x_stride + c->lay.layers[layer].x_off;
+    *ld_out = c->lay.layers[layer].ld;
     return PG_OK;
 }
 

@@ -91,6 +91,8 @@ struct DevState {
     float* X;            // [worker][x_stride]
     float* Xw;           // where corrected rows are written: X itself, or the second copy of the stack
                          // when a row has two readers in one sweep (pair sweep on graphs of degree 2)
+    const float* G;      // null, or the caller's gradients laid out like X: updates also subtract eta * G
+    float eta;
     float* Q;            // [pair][q_stride]     raw right factors
     float* Qinv;         // [pair][layer][rank]  1 / column norm (0 for a zero column)
     double* Qn2;         // [pair][layer][kEdgeChunks]  pair sweep layers: shares of ||Q||^2

@@ -119,7 +119,8 @@ struct RowShared {
     int nu, nf;
 };
 
-template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH>
+// GRAD: the update also subtracts eta * G (Algorithm 1, line 6), G laid out like X.
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD = false>
 __device__ __forceinline__ void row_tile(const DevState& st, const int* __restrict__ tab_u,
                                          const int* __restrict__ tab_f, const Tile tile,
                                          RowShared<S>& sh) {
@@ -128,6 +129,8 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
     const int rank = st.rank;
     float* __restrict__ X = st.X + (long long)w * st.x_stride + g.x_off;
     float* Xw = st.Xw + (long long)w * st.x_stride + g.x_off;
+    const float* __restrict__ Gw = GRAD ? st.G + (long long)w * st.x_stride + g.x_off : nullptr;
+    const float eta = GRAD ? st.eta : 0.0f;
 
     if (threadIdx.x < S) {
         const int v = threadIdx.x;
@@ -203,6 +206,18 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                         }
                     }
                 }
+                if (GRAD) {
+#pragma unroll
+                    for (int t = 0; t < RT; ++t) {
+                        float4 gv = ld_stream(Gw + (xrow[t] - X) + c);
+                        // columns past the matrix are padding: X keeps zeros there whatever G holds
+                        if (c + 1 >= g.m) gv.y = 0.0f;
+                        if (c + 2 >= g.m) gv.z = 0.0f;
+                        if (c + 3 >= g.m) gv.w = 0.0f;
+                        x[t].x = fmaf(-eta, gv.x, x[t].x); x[t].y = fmaf(-eta, gv.y, x[t].y);
+                        x[t].z = fmaf(-eta, gv.z, x[t].z); x[t].w = fmaf(-eta, gv.w, x[t].w);
+                    }
+                }
 #pragma unroll
                 for (int t = 0; t < RT; ++t)
                     if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
@@ -230,6 +245,18 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                             x[t].z = fmaf(-a[t][v], q.z, x[t].z);
                             x[t].w = fmaf(-a[t][v], q.w, x[t].w);
                         }
+                    }
+                }
+                if (GRAD) {
+#pragma unroll
+                    for (int t = 0; t < RT; ++t) {
+                        float4 gv = ld_stream(Gw + (xrow[t] - X) + c);
+                        // columns past the matrix are padding: X keeps zeros there whatever G holds
+                        if (c + 1 >= g.m) gv.y = 0.0f;
+                        if (c + 2 >= g.m) gv.z = 0.0f;
+                        if (c + 3 >= g.m) gv.w = 0.0f;
+                        x[t].x = fmaf(-eta, gv.x, x[t].x); x[t].y = fmaf(-eta, gv.y, x[t].y);
+                        x[t].z = fmaf(-eta, gv.z, x[t].z); x[t].w = fmaf(-eta, gv.w, x[t].w);
                     }
                 }
 #pragma unroll
@@ -273,12 +300,12 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
     }
 }
 
-template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT>
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool GRAD = false>
 __global__ void __launch_bounds__(256, PG_ROW_MIN_BLOCKS)
 row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
                  const Tile* __restrict__ tiles) {
     __shared__ RowShared<S> sh;
-    row_tile<S, UPDATE, FORWARD, SAME, RT, false>(st, tab_u, tab_f, tiles[blockIdx.x], sh);
+    row_tile<S, UPDATE, FORWARD, SAME, RT, false, GRAD>(st, tab_u, tab_f, tiles[blockIdx.x], sh);
 }
 
 // --------------------------------------------------------------------------
@@ -1858,6 +1885,17 @@ cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, c
                        int n_tiles, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
     const int slots = st.max_degree * st.rank;
+    if (UPDATE && st.G) {     // the update also takes the caller's gradient step
+        if (slots <= 1)
+            row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        else if (slots <= 2)
+            row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        else if (slots <= 4)
+            row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        else
+            row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        return cudaGetLastError();
+    }
     if (slots <= 1)
         row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
     else if (slots <= 2)

@@ -504,6 +504,81 @@ def test_local_gradient_steps_between_rounds(w):
     oracle.close()
 
 
+SGD_CASES = {
+    "ring_pair_sweep": (wl.tiny_ring().replace(layer_shapes=((64, 32), (9, 1500), (5, 3))), None),
+    "ring_pair_sweep_two_steps": (wl.tiny_ring().replace(layer_shapes=((33, 130), (7, 9000)), power_steps=2), None),
+    "matching_pair_sweep": (wl.shrink(wl.lstm_matching32(), [(130, 70), (70, 1300)], 6).replace(n_workers=8), None),
+    "torus_rank2_two_steps": (wl.shrink(wl.torus8x8(2), [(200, 136), (5, 3)], 6).replace(rank=2), None),
+    "ring_three_sweeps": (wl.tiny_ring().replace(layer_shapes=((64, 32), (67, 131))), "three"),
+    "ring_half_step": (wl.tiny_ring().replace(power_steps=3), "half"),
+    "ring_random_projection": (wl.tiny_ring().replace(rank=2), "random"),
+}
+
+
+@pytest.mark.parametrize("case", sorted(SGD_CASES))
+def test_round_with_fused_gradient_step(case, monkeypatch):
+    """pg_round_sgd: X <- X + gossip - eta G with G read by the sweep that applies the update
+    (Algorithm 1, line 6).  The checker does the round, then add_params(-eta G) in fp64.  The
+    padding columns of the gradient buffer are filled with NaN: they must not be read into X."""
+    import torch
+
+    w, mode = SGD_CASES[case]
+    if mode == "three":
+        monkeypatch.setenv("PG_DISABLE_PAIR_SWEEP", "1")
+    oracle, net = common.oracle_for(w), common.network_for(w)
+    if mode == "half":
+        oracle.set_half_step()
+    if mode == "random":
+        oracle.set_random_projection(1)
+    common.load_both(w, oracle, net)
+    if mode == "half":
+        net.pg_set_half_step()
+    if mode == "random":
+        net.pg_set_random_projection(1)
+    grads = net.gradient_buffer()
+    grads.fill_(float("nan"))
+    eta = 0.05
+    for t in range(5):
+        for i in range(w.n_workers):
+            for l, (n, m) in enumerate(w.layer_shapes):
+                g = np.random.default_rng([t, i, l]).standard_normal((n, m)).astype(np.float32)
+                net.gradient_view(grads, i, l).copy_(torch.from_numpy(g))
+        net.pg_round_sgd(grads, eta)
+        oracle.round()
+        for i in range(w.n_workers):
+            for l, (n, m) in enumerate(w.layer_shapes):
+                g = np.random.default_rng([t, i, l]).standard_normal((n, m)).astype(np.float32)
+                oracle.add_params(i, l, -(np.float64(np.float32(eta)) * g.astype(np.float64)))
+        torch.cuda.synchronize()
+        if t % 2 == 1 or t == 4:        # some rounds follow each other without a read in between
+            err, where = common.max_relative_error(w, oracle, net)
+            assert err <= REL_TOL, (t, err, where)
+    assert net.pg_device_status() == 0
+    assert net.pg_get_round() == 5
+    net.close()
+    oracle.close()
+
+
+def test_round_with_gradient_rejects_bad_buffers():
+    import torch
+    from paper_2008_01425_b200 import binding as pg
+
+    w = wl.tiny_ring()
+    net = common.network_for(w)
+    common.load_both(w, None, net)
+    grads = net.gradient_buffer()
+    assert grads.numel() == net.pg_stack_elems() and net.pg_stack_offset(1, 0)[0] % 64 == 0
+    with pytest.raises(pg.PowerGossipError) as e:
+        net.pg_round_sgd(grads, float("inf"))
+    assert e.value.status == pg.PG_ERR_INVALID
+    bigger = torch.zeros(grads.numel() + 8, dtype=torch.float32, device=grads.device)
+    with pytest.raises(pg.PowerGossipError) as e:
+        net.pg_round_sgd(bigger[1:], 0.1)          # 4-byte aligned only
+    assert e.value.status == pg.PG_ERR_INVALID
+    assert net.pg_get_round() == 0
+    net.close()
+
+
 # ---- random-projection compressors (Section 5.1) ------------------------------
 RANDOM_CASES = [
     wl.tiny_ring().replace(rounds=30),
