@@ -179,7 +179,9 @@ PG_API int pg_params_device(pg_ctx *ctx, int32_t worker, int32_t layer, void *st
  * rows to a second copy of the stack and the copies swap roles every step; the
  * calls above always leave the result in the copy pg_params_device points to.
  * There, all layers take the pair sweep when the stack is at most 48 MiB, else
- * only layers of at least 256 rows and 2^20 elements.  PG_DISABLE_PAIR_SWEEP=1
+ * only layers of at least 256 rows and 2^20 elements, and the kernels of the
+ * other layers run on a stream of the library's own that is forked from and
+ * joined to `stream` with events inside the call.  PG_DISABLE_PAIR_SWEEP=1
  * in the environment at creation selects the general three-sweep path.
  * Host-side errors are returned at once; device-side ones show up in
  * pg_read_params / pg_device_status.

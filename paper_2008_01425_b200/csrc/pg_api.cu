@@ -313,6 +313,10 @@ struct pg_ctx {
     bool pending = false;
     int64_t pending_key = 0;    // round whose table describes the pending correction
     int xbuf = 0;               // which copy of X is current (always 0 unless a correction is pending)
+    // layers on the three sweeps and layers on the pair sweep are independent within a round: when a
+    // stack has both, the former are enqueued on a side stream forked from and joined to the caller's
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     int64_t step = 0;           // power steps enqueued so far (selects the P-hat buffer)
     float* ph_buf[2] = {nullptr, nullptr};
     Tile* d_pair_tiles = nullptr;
@@ -788,6 +792,9 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     ok = ok && cudaMallocHost(&c->h_tabs, sizeof(int) * static_cast<size_t>(kTabRing) * lay.tab.total_ints) == cudaSuccess;
     for (int s = 0; s < kTabRing && ok; ++s)
         ok = cudaEventCreateWithFlags(&c->tab_event[s], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
     if (ok) {
         ok = pg::launch_column_norms(st, lay.n_pairs, nullptr) == cudaSuccess;
         c->launches += 1;
@@ -810,6 +817,9 @@ void pg_destroy(pg_ctx* c) {
     }
     for (int s = 0; s < kTabRing; ++s)
         if (c->tab_event[s]) cudaEventDestroy(c->tab_event[s]);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side) cudaStreamDestroy(c->side);
     if (c->h_tabs) cudaFreeHost(c->h_tabs);
     delete c;
 }
@@ -982,9 +992,17 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
         }
         return PG_OK;
     }
+    // a stack with layers on both paths: the three sweeps of this round go to the side stream
+    const bool forked = n_rows > 0 && has_pair && !std::getenv("PG_NO_SIDE_STREAM");
+    cudaStream_t s3 = stream;
+    if (forked) {
+        ok = cudaEventRecord(c->ev_fork, stream) == cudaSuccess &&
+             cudaStreamWaitEvent(c->side, c->ev_fork, 0) == cudaSuccess;
+        s3 = c->side;
+    }
     if (n_rows > 0 && !c->y_valid) {
-        Timed t(c, PG_KERNEL_FORWARD, stream, c->normal_param_bytes);
-        ok = ok && pg::launch_forward(c->st, tab, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+        Timed t(c, PG_KERNEL_FORWARD, s3, c->normal_param_bytes);
+        ok = ok && pg::launch_forward(c->st, tab, c->d_row_tiles, n_rows, s3) == cudaSuccess;
         c->launches += 1;
     }
     for (int p = 0; p < c->power_steps && ok; ++p) {
@@ -995,16 +1013,16 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
             DevState st = c->st;
             st.Ph = ph_cur;
             {
-                Timed t(c, PG_KERNEL_EDGE_LEFT, stream, 0.0);
-                ok = ok && pg::launch_edge_left(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+                Timed t(c, PG_KERNEL_EDGE_LEFT, s3, 0.0);
+                ok = ok && pg::launch_edge_left(st, tab, c->lay.max_edges, s3) == cudaSuccess;
             }
             {
-                Timed t(c, PG_KERNEL_TRANSPOSED, stream, c->normal_param_bytes);
-                ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, stream) == cudaSuccess;
+                Timed t(c, PG_KERNEL_TRANSPOSED, s3, c->normal_param_bytes);
+                ok = ok && pg::launch_transposed(st, tab, c->d_col_tiles, n_cols, s3) == cudaSuccess;
             }
             {
-                Timed t(c, PG_KERNEL_EDGE_RIGHT, stream, 0.0);
-                ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, stream) == cudaSuccess;
+                Timed t(c, PG_KERNEL_EDGE_RIGHT, s3, 0.0);
+                ok = ok && pg::launch_edge_right(st, tab, c->lay.max_edges, s3) == cudaSuccess;
             }
             {
                 // the round's last update also takes the gradient step; the product for the
@@ -1012,8 +1030,8 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
                 const bool with_g = G && p + 1 == c->power_steps;
                 st.G = with_g ? G : nullptr;
                 st.eta = eta;
-                Timed t(c, PG_KERNEL_UPDATE_FORWARD, stream, (with_g ? 3.0 : 2.0) * c->normal_param_bytes);
-                ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, stream) == cudaSuccess;
+                Timed t(c, PG_KERNEL_UPDATE_FORWARD, s3, (with_g ? 3.0 : 2.0) * c->normal_param_bytes);
+                ok = ok && pg::launch_update_forward(st, tab, tab_fwd, c->d_row_tiles, n_rows, s3) == cudaSuccess;
             }
             c->launches += 4;
         }
@@ -1057,6 +1075,9 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
         }
         c->step += 1;
     }
+    if (forked)   // join even after a failed launch, so the caller's stream stays ordered after the side stream
+        ok = (cudaEventRecord(c->ev_join, c->side) == cudaSuccess &&
+              cudaStreamWaitEvent(stream, c->ev_join, 0) == cudaSuccess) && ok;
     if (!ok) {
         cudaGetLastError();
         c->y_valid = false;
