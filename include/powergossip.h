@@ -259,8 +259,14 @@ PG_API int pg_set_random_projection(pg_ctx *ctx, int32_t mode);
  * (at most 64 MiB of parameters, no layer on the pair sweep), all rounds run in ONE
  * cooperative kernel launch whose phases are separated by a grid barrier; the
  * barrier waits are bounded, and a wait that runs out ends the launch and sets
- * PG_ERR_TIMEOUT in the device status word.  Otherwise the rounds are enqueued
- * one by one.  Per-kernel timing (pg_timing_enable) forces the latter.
+ * PG_ERR_TIMEOUT in the device status word.  Otherwise, on a static graph and
+ * for four rounds or more, the first rounds are enqueued one by one until the
+ * launches repeat, then two rounds are captured once as a CUDA graph (on a
+ * stream of the library's own; nothing of the caller's is captured) and the graph
+ * is launched into `stream` as often as needed; a remainder, and every round of
+ * a time-varying graph, is enqueued one by one.  The same kernels run either way.
+ * While `stream` itself is being captured by the caller, and with per-kernel
+ * timing on (pg_timing_enable), only plain launches are used.
  */
 PG_API int pg_rounds(pg_ctx *ctx, int32_t n_rounds, void *stream);
 

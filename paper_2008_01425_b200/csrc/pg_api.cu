@@ -317,6 +317,12 @@ struct pg_ctx {
     // stack has both, the former are enqueued on a side stream forked from and joined to the caller's
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // pg_rounds on a static graph: two steady-state rounds captured once as a CUDA graph and replayed
+    cudaStream_t cap = nullptr;          // origin stream of the capture
+    cudaGraphExec_t loop_exec = nullptr;
+    int loop_key = -1;                   // buffer parities the captured rounds start from
+    int64_t loop_launches = 0;           // kernels in the captured pair of rounds
+    bool loop_failed = false;
     int64_t step = 0;           // power steps enqueued so far (selects the P-hat buffer)
     float* ph_buf[2] = {nullptr, nullptr};
     Tile* d_pair_tiles = nullptr;
@@ -631,6 +637,10 @@ bool upload_tile_lists(pg_ctx* c) {
 bool leave_pair_mode(pg_ctx* c) {
     if (c->lay.n_pair_tiles == 0) return true;
     for (LayerGeom& g : c->lay.layers) g.pair_mode = 0;
+    if (c->loop_exec) {
+        cudaGraphExecDestroy(c->loop_exec);
+        c->loop_exec = nullptr;
+    }
     return upload_tile_lists(c);
 }
 
@@ -792,6 +802,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     ok = ok && cudaMallocHost(&c->h_tabs, sizeof(int) * static_cast<size_t>(kTabRing) * lay.tab.total_ints) == cudaSuccess;
     for (int s = 0; s < kTabRing && ok; ++s)
         ok = cudaEventCreateWithFlags(&c->tab_event[s], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->cap, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess &&
          cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
@@ -820,6 +831,8 @@ void pg_destroy(pg_ctx* c) {
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
+    if (c->loop_exec) cudaGraphExecDestroy(c->loop_exec);
+    if (c->cap) cudaStreamDestroy(c->cap);
     if (c->h_tabs) cudaFreeHost(c->h_tabs);
     delete c;
 }
@@ -1139,6 +1152,46 @@ int pg_set_random_projection(pg_ctx* c, int32_t mode) {
     return PG_OK;
 }
 
+// Steady state of a static graph: the table is on the device, the pair sweep has a correction
+// pending and the three sweeps have their forward product cached, so every round enqueues the
+// same kernels with the same arguments up to the parity of the double buffers.
+static bool rounds_are_periodic(const pg_ctx* c) {
+    return c->static_graph && c->tab_used[0] && c->tab_round[0] == 0 &&
+           (c->lay.n_pair_tiles == 0 || c->pending) && (c->lay.n_row_tiles == 0 || c->y_valid);
+}
+
+// Capture two rounds (an even number of power steps: the buffer parities return) on the
+// library's own stream and instantiate them.  Nothing runs; the host state is put back.
+static void capture_two_rounds(pg_ctx* c, int key) {
+    const int64_t round = c->round, step = c->step, launches = c->launches, pending_key = c->pending_key;
+    const int xbuf = c->xbuf;
+    const bool pending = c->pending, y_valid = c->y_valid;
+    if (cudaStreamBeginCapture(c->cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        c->loop_failed = true;
+        return;
+    }
+    int rc = round_impl(c, c->cap, nullptr, 0.0f);
+    if (rc == PG_OK) rc = round_impl(c, c->cap, nullptr, 0.0f);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t end = cudaStreamEndCapture(c->cap, &graph);
+    c->loop_launches = c->launches - launches;
+    c->round = round; c->step = step; c->launches = launches; c->pending_key = pending_key;
+    c->xbuf = xbuf; c->pending = pending; c->y_valid = y_valid;
+    if (c->loop_exec) {
+        cudaGraphExecDestroy(c->loop_exec);
+        c->loop_exec = nullptr;
+    }
+    if (rc != PG_OK || end != cudaSuccess || !graph ||
+        cudaGraphInstantiate(&c->loop_exec, graph, 0) != cudaSuccess) {
+        cudaGetLastError();
+        c->loop_exec = nullptr;
+        c->loop_failed = true;
+    }
+    if (graph) cudaGraphDestroy(graph);
+    c->loop_key = key;
+}
+
 int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
     if (!c || n_rounds < 0) return PG_ERR_INVALID;
     if (n_rounds == 0) return PG_OK;
@@ -1150,7 +1203,41 @@ int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
     const bool persistent = c->static_graph && !c->half_step && !c->random_proj && c->lay.n_pair_tiles == 0 && c->coop_ok &&
                             x_bytes <= 64.0 * 1024 * 1024 && !c->timing;
     if (!persistent) {
-        for (int r = 0; r < n_rounds; ++r) {
+        int done = 0;
+        // launch-bound loops on a static graph: replay a captured pair of rounds
+        bool replay = c->static_graph && !c->half_step && !c->random_proj && !c->timing && !c->loop_failed &&
+                      n_rounds >= 4 && !std::getenv("PG_NO_GRAPH");
+        if (replay) {
+            cudaStreamCaptureStatus busy = cudaStreamCaptureStatusNone;
+            if (cudaStreamIsCapturing(stream, &busy) != cudaSuccess || busy != cudaStreamCaptureStatusNone) {
+                cudaGetLastError();
+                replay = false;      // the caller is capturing: enqueue plain launches into their graph
+            }
+        }
+        if (replay) {
+            while (done < n_rounds && !rounds_are_periodic(c)) {
+                const int rc = pg_round(c, stream_v);
+                if (rc != PG_OK) return rc;
+                ++done;
+            }
+            const int pairs_left = (n_rounds - done) / 2;
+            if (pairs_left > 0) {
+                const int key = static_cast<int>(c->step & 1) | (c->xbuf << 1);
+                if (!c->loop_exec || c->loop_key != key) capture_two_rounds(c, key);
+                if (c->loop_exec) {
+                    for (int r = 0; r < pairs_left; ++r)
+                        if (cudaGraphLaunch(c->loop_exec, stream) != cudaSuccess) {
+                            cudaGetLastError();
+                            return PG_ERR_CUDA;
+                        }
+                    c->round += 2LL * pairs_left;
+                    c->step += 2LL * pairs_left * c->power_steps;
+                    c->launches += c->loop_launches * pairs_left;
+                    done += 2 * pairs_left;
+                }
+            }
+        }
+        for (; done < n_rounds; ++done) {
             const int rc = pg_round(c, stream_v);
             if (rc != PG_OK) return rc;
         }

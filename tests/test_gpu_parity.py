@@ -306,6 +306,38 @@ def test_pg_rounds_equals_repeated_pg_round_bit_for_bit(w, monkeypatch):
     b.close()
 
 
+REPLAY_CASES = [
+    wl.tiny_ring(),                                   # pair sweep on a ring (two copies of X swap every step)
+    wl.resnet20_ring8().replace(rounds=13),
+    wl.vgg16_ring16(1).replace(rounds=7),             # layers on both paths: the side stream is part of the capture
+    wl.vgg16_ring16(2).replace(rounds=6),             # three sweeps, too large for the cooperative kernel
+]
+
+
+@pytest.mark.parametrize("w", REPLAY_CASES, ids=lambda w: w.name)
+def test_pg_rounds_graph_replay_equals_repeated_pg_round_bit_for_bit(w):
+    """Where pg_rounds replays a captured pair of rounds (static graph, steady state), the result
+    is that of the same number of pg_round calls, whatever the split and the parity it starts from."""
+    a, b = common.network_for(w), common.network_for(w)
+    common.load_both(w, None, a)
+    common.load_both(w, None, b)
+    for _ in range(2 * w.rounds):
+        a.pg_round()
+    b.pg_rounds(w.rounds - 1)      # warm-up rounds one by one, then replays, then a remainder
+    b.pg_round()                   # changes the parity the next replay starts from
+    b.pg_rounds(w.rounds)
+    assert a.pg_get_round() == b.pg_get_round() == 2 * w.rounds
+    assert a.pg_kernel_launches() == b.pg_kernel_launches()
+    assert a.pg_device_status() == 0 and b.pg_device_status() == 0
+    for i in range(w.n_workers):
+        for l in range(len(w.layer_shapes)):
+            assert np.array_equal(a.pg_read_params(i, l), b.pg_read_params(i, l))
+    e = a.pg_get_schedule(0)[0][0]
+    assert np.array_equal(a.pg_read_q(int(e[0]), int(e[1]), 0), b.pg_read_q(int(e[0]), int(e[1]), 0))
+    a.close()
+    b.close()
+
+
 @pytest.mark.parametrize("three_sweeps", [True, False], ids=["cooperative_kernel", "pair_sweep"])
 def test_pg_rounds_against_the_checker(three_sweeps, monkeypatch):
     if three_sweeps:
