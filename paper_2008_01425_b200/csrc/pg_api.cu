@@ -43,7 +43,8 @@ struct Layout {
     int max_edges = 0, max_degree = 0;
     TabLayout tab{};
     long long n_row_tiles = 0, n_col_tiles = 0;
-    size_t off_Qn2 = 0, off_Pn = 0, off_edge_tab = 0;
+    size_t off_Qn2 = 0, off_Pn = 0, off_edge_tab = 0, off_stage = 0;
+    long long stage_elems = 0;     // largest dense matrix whose rows need padding on upload
     size_t off_X = 0, off_Q = 0, off_Qinv = 0, off_Y = 0, off_Ph = 0, off_Z = 0, off_live = 0,
            off_Up = 0, off_Sp = 0, off_pair_tiles = 0, off_flush_tiles = 0, off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
     size_t total = 0;
@@ -287,6 +288,10 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_Z = take(sizeof(float) * static_cast<size_t>(N) * lay.z_stride);
     lay.off_live = take(sizeof(int) * static_cast<size_t>(lay.max_edges) * n_layers * rank);
     lay.off_status = take(sizeof(int) * 64);   // [0] status word, [16..17] grid barrier of the persistent kernel
+    lay.stage_elems = 0;
+    for (const LayerGeom& g : lay.layers)
+        if (g.ld != g.m) lay.stage_elems = std::max(lay.stage_elems, static_cast<long long>(g.n) * g.m);
+    lay.off_stage = take(sizeof(float) * static_cast<size_t>(lay.stage_elems));
     lay.off_layers = take(sizeof(LayerGeom) * static_cast<size_t>(n_layers));
     lay.off_edge_tab = take(sizeof(int) * 2 * static_cast<size_t>(n_layers) * pg::kEdgeChunks);
     lay.off_tabs = take(sizeof(int) * static_cast<size_t>(kTabRing + 1) * t.total_ints);   // + one table of an empty graph
@@ -846,9 +851,21 @@ int pg_write_params(pg_ctx* c, int32_t worker, int32_t layer, const float* host_
     const LayerGeom& g = c->lay.layers[layer];
     float* dst = c->st.X + static_cast<long long>(worker) * c->st.x_stride + g.x_off;
     c->y_valid = false;
-    if (cudaMemcpy2DAsync(dst, sizeof(float) * g.ld, host_src, sizeof(float) * g.m, sizeof(float) * g.m,
-                          g.n, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t dense = sizeof(float) * static_cast<size_t>(g.n) * g.m;
+    if (g.ld == g.m) {
+        if (cudaMemcpyAsync(dst, host_src, dense, cudaMemcpyHostToDevice, s) != cudaSuccess) return PG_ERR_CUDA;
+        return PG_OK;
+    }
+    // Rows that need padding: one contiguous copy into a staging area, then a kernel spreads the
+    // rows (a strided host-to-device copy of narrow rows runs at half the link rate).  The staging
+    // area is reused in stream order, like everything else in a context.
+    float* stage = reinterpret_cast<float*>(c->ws + c->lay.off_stage);
+    if (cudaMemcpyAsync(stage, host_src, dense, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        pg::launch_unpack_rows(dst, g.ld, stage, g.n, g.m, s) != cudaSuccess) {
+        cudaGetLastError();
         return PG_ERR_CUDA;
+    }
     return PG_OK;
 }
 

@@ -149,6 +149,8 @@ cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const
 // Clusters of the wide pair sweep that can be resident at once (0 if unknown).
 int pair_wide_resident_clusters(int nv, int slice, int pend_slots);
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
+// dense rows x cols at `src` (device) -> rows of leading dimension ld at `dst`
+cudaError_t launch_unpack_rows(float* dst, long long ld, const float* src, int rows, int cols, cudaStream_t stream);
 // One cooperative launch for `n_steps` power steps of a static graph (small stacks).
 cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* row_tiles, int n_rows,
                               const Tile* col_tiles, int n_cols, int n_steps, bool forward_first, int* bar,

@@ -2080,6 +2080,24 @@ int pair_wide_resident_clusters(int nv, int slice, int pend_slots) {
     }
 }
 
+// dst[r][c] = src[r * cols + c]: a dense matrix into its padded place in the stack.
+__global__ void __launch_bounds__(256)
+unpack_rows_kernel(float* __restrict__ dst, long long ld, const float* __restrict__ src, int rows, int cols) {
+    const long long total = (long long)rows * cols;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const long long r = idx / cols;
+        dst[r * ld + (idx - r * cols)] = src[idx];
+    }
+}
+
+cudaError_t launch_unpack_rows(float* dst, long long ld, const float* src, int rows, int cols, cudaStream_t stream) {
+    const long long total = (long long)rows * cols;
+    const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 16);
+    unpack_rows_kernel<<<blocks, 256, 0, stream>>>(dst, ld, src, rows, cols);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
     if (st.e_total <= 0) return cudaSuccess;
     pair_edge_kernel<<<max_edges * st.e_total, 256, 0, stream>>>(st, tab);
