@@ -129,7 +129,8 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     // row has one reader, so it is corrected in place.  On a static graph of degree 2
     // with no isolated worker (a ring, a path) a row has up to two readers: the edge in
     // the worker's slot 0 writes the corrected row to a second copy of X, which becomes
-    // the current one after the sweep.
+    // the current one after the sweep.  (Degree 4 was tried and is slower than the three
+    // sweeps: every row pair then needs eight corrections, applied by four CTAs each.)
     lay.pair_mode = false;
     lay.pend_slots = 1;
     lay.two_copies = false;
@@ -200,8 +201,8 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         // With two readers per row the pair sweep pays off in two regimes: a stack small
         // enough to live in L2, where it halves the launches of a step, and layers large
         // enough to keep every SM busy for many rows.  Other layers take the three sweeps.
-        if (lay.two_copies && !small_stack && !(g.n >= 256 && static_cast<long long>(g.n) * g.ld >= (1LL << 20)))
-            g.pair_mode = 0;
+        const bool large_layer = g.n >= 256 && static_cast<long long>(g.n) * g.ld >= (1LL << 20);
+        if (lay.two_copies && !small_stack && !large_layer) g.pair_mode = 0;
         g.p_slice = static_cast<int>(round_up((g.ld + pg::kPairCluster - 1) / pg::kPairCluster, 4));
         {   // equal tiles of at most kPairTileRows rows (a multiple of 8: one row per warp and stage);
             // on graphs of degree 2 short matrices are cut finer, down to 16 rows, so that a layer gives

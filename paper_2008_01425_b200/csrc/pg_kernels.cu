@@ -981,11 +981,12 @@ template <int NV, bool UPDATE, int D>
 __global__ void __launch_bounds__(256, PG_BULK_MIN_BLOCKS)
 pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles) {
+    constexpr int STAGES = kBulkStages;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ __align__(16) float s_q[NV * 128];
     __shared__ __align__(16) float s_ui[D][NV * 128];
     __shared__ __align__(16) float s_uj[D][NV * 128];
-    __shared__ __align__(8) unsigned long long s_full[kBulkStages];
+    __shared__ __align__(8) unsigned long long s_full[STAGES];
     __shared__ double s_s[8];
     __shared__ int s_abort;
 
@@ -1021,7 +1022,7 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 
     if (threadIdx.x == 0) {
         s_abort = 0;
-        for (int s2 = 0; s2 < kBulkStages; ++s2) mbar_init(&s_full[s2], 1);
+        for (int s2 = 0; s2 < STAGES; ++s2) mbar_init(&s_full[s2], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int idx = threadIdx.x; idx < NV * 128; idx += 256) {
@@ -1039,7 +1040,7 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 
     // stage `sidx` covers rows r0 + sidx*kBulkRows ...; both slabs are contiguous in global memory
     auto issue = [&](int sidx) {
-        const int slot = sidx % kBulkStages;
+        const int slot = sidx % STAGES;
         const int row = r0 + sidx * kBulkRows;
         const unsigned bytes = (unsigned)min(kBulkRows, r1 - row) * row_bytes;
         float* dst = s_stage + (size_t)slot * 2 * kBulkRows * ld;
@@ -1049,7 +1050,7 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     };
     int issued = 0;
     if (threadIdx.x == 0)
-        for (; issued < kBulkStages - 1 && issued < n_stages; ++issued) issue(issued);
+        for (; issued < STAGES - 1 && issued < n_stages; ++issued) issue(issued);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
@@ -1060,12 +1061,12 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     bool ok = true;
 
     for (int it = 0; it < n_stages; ++it) {
-        const int slot = it % kBulkStages;
-        if (threadIdx.x == 0 && it + kBulkStages - 1 < n_stages) {
-            issue(it + kBulkStages - 1);      // its slot was read for the last time before the barrier below
-            issued = it + kBulkStages;
+        const int slot = it % STAGES;
+        if (threadIdx.x == 0 && it + STAGES - 1 < n_stages) {
+            issue(it + STAGES - 1);      // its slot was read for the last time before the barrier below
+            issued = it + STAGES;
         }
-        const bool mine = mbar_wait_bounded(&s_full[slot], (unsigned)((it / kBulkStages) & 1), &s_abort, st.status);
+        const bool mine = mbar_wait_bounded(&s_full[slot], (unsigned)((it / STAGES) & 1), &s_abort, st.status);
         ok = __syncthreads_and(mine) != 0;        // either every thread goes on or all leave together
         if (!ok) break;
         const int r = r0 + it * kBulkRows + warp;
@@ -1135,9 +1136,9 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         // leave only after the copies still in flight have landed (bounded)
         if (threadIdx.x == 0)
             for (int sidx = 0; sidx < issued; ++sidx) {
-                const int slot = sidx % kBulkStages;
+                const int slot = sidx % STAGES;
                 for (int spin = 0; spin < kBulkSpinLimit; ++spin)
-                    if (mbar_try_wait(&s_full[slot], (unsigned)((sidx / kBulkStages) & 1))) break;
+                    if (mbar_try_wait(&s_full[slot], (unsigned)((sidx / STAGES) & 1))) break;
             }
         return;
     }
@@ -1514,18 +1515,27 @@ pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* 
 // at the next barrier.
 // --------------------------------------------------------------------------
 constexpr int kMidStagesMax = 4;
-constexpr int kMidRows = 2;       // rows per stage and per barrier
 constexpr int kMidBulkNv = 5;     // most float4 per thread and row (registers)
+#ifndef PG_MID_ROWS1
+#define PG_MID_ROWS1 4
+#endif
+#ifndef PG_MID_ROWS2
+#define PG_MID_ROWS2 4
+#endif
+// rows per stage and per barrier: more of them where a row is short
+__host__ __device__ constexpr int mid_rows(int nvm) { return nvm == 1 ? PG_MID_ROWS1 : (nvm == 2 ? PG_MID_ROWS2 : 2); }
+// two CTAs per SM where the registers allow it, so one CTA's prologue hides behind the other's rows
+__host__ __device__ constexpr int mid_min_blocks(int nvm, int d) { return (1 + 2 * d) * nvm <= 10 ? 2 : 1; }
 
 template <int NVM, bool UPDATE, int D>
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(256, mid_min_blocks(NVM, D))
 pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                            const Tile* __restrict__ tiles, int ld_pad, int n_stage) {
-    extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][kMidRows * ld_pad]
+    extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][RS * ld_pad]
     __shared__ __align__(8) unsigned long long s_full[kMidStagesMax];
-    __shared__ float s_warp[2][kMidRows][8];
+    constexpr int RS = mid_rows(NVM);
+    __shared__ float s_warp[2][RS][8];
     __shared__ int s_abort;
-    constexpr int RS = kMidRows;
 
     const Tile tile = tiles[blockIdx.x];
     const int e = tile.worker;
@@ -1981,6 +1991,7 @@ cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int
     if (n_tiles <= 0) return cudaSuccess;
     if (st.pair_bulk) {
         if (!apply_pending) return launch_pair_bulk<false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+        if (pend_slots > 2) return cudaErrorInvalidValue;
         return pend_slots > 1 ? launch_pair_bulk<true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
                               : launch_pair_bulk<true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
     }
@@ -2113,8 +2124,10 @@ static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const i
     const size_t smem = sizeof(float) * (1 + 2 * D) * static_cast<size_t>(ld_pad);
     // TMA-fed variant when the row fits its registers and at least two stages fit in shared memory
     if constexpr (NVM <= kMidBulkNv) {
-        const size_t stage = sizeof(float) * 2 * kMidRows * static_cast<size_t>(ld_pad);
-        const int n_stage = (int)std::min<size_t>(kMidSmemBudget / stage, kMidStagesMax);
+        const size_t stage = sizeof(float) * 2 * mid_rows(NVM) * static_cast<size_t>(ld_pad);
+        // leave room for the second CTA where the kernel is built for two per SM
+        const size_t budget = kMidSmemBudget / mid_min_blocks(NVM, D);
+        const int n_stage = (int)std::min<size_t>(budget / stage, kMidStagesMax);
         if (st.pair_bulk && n_stage >= 2) {
             const size_t total = n_stage * stage;
             cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_bulk_kernel<NVM, UPDATE, D>,
@@ -2138,6 +2151,7 @@ template <int NVM>
 static cudaError_t launch_mid(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd, int pend_slots,
                               const Tile* tiles, int n_tiles, int ld_pad, cudaStream_t stream) {
     if (!upd) return launch_mid_t<NVM, false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    if (pend_slots > 2) return cudaErrorInvalidValue;
     return pend_slots > 1 ? launch_mid_t<NVM, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream)
                           : launch_mid_t<NVM, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
 }
