@@ -225,7 +225,9 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         {   // pair edge step: about 2048 partial sums or rows per CTA
             const int max_tiles = g.pair_mode == 2 ? pg::kPairWideMaxTiles : g.p_rtiles;
             const long long work = static_cast<long long>(max_tiles) * g.ld + g.npad;
-            g.e_chunks = static_cast<int>(std::min<long long>(std::max<long long>((work + 2047) / 2048, 1), pg::kEdgeChunks));
+            long long per_cta = 2048;
+            if (const char* v = std::getenv("PG_EDGE_WORK")) per_cta = std::max(256LL, std::atoll(v));   // tuning aid
+            g.e_chunks = static_cast<int>(std::min<long long>(std::max<long long>((work + per_cta - 1) / per_cta, 1), pg::kEdgeChunks));
         }
         g.up_off = up;
         g.sp_off = sp;
