@@ -151,13 +151,15 @@ def whole_job_rate(world: int, steps: int, ms_total: float) -> float:
 # ----------------------------------------------------------------------------
 # the CPU checker as a timed baseline (bounded sample)
 # ----------------------------------------------------------------------------
-def time_oracle_sample(w, sample_workers: int, rounds: int, warmup: int = 1):
+def time_oracle_sample(w, sample_workers: int, rounds: int, warmup: int = 1, target_seconds: float = 0.0):
     """Times the fp64 CPU checker on `sample_workers` workers of the workload.
 
     The cost of a round is proportional to the number of workers (every worker
     takes part in `degree` edges whatever N is), so rounds/s of the full
     workload = rounds/s of the sample x sample_workers / n_workers.
-    Returns (scaled rounds/s, seconds timed, workers in the sample, threads).
+    With `target_seconds`, the number of timed rounds is chosen from the warm-up
+    rounds' pace so that about that much CPU time is measured (at least `rounds`).
+    Returns (scaled rounds/s, seconds timed, workers in the sample, threads, rounds timed).
     """
     from oracle import pg_oracle as po
     from paper_2008_01425_b200 import workloads as wl
@@ -174,13 +176,17 @@ def time_oracle_sample(w, sample_workers: int, rounds: int, warmup: int = 1):
     for i in range(sample.n_workers):
         for l in range(len(sample.layer_shapes)):
             o.set_params(i, l, wl.initial_params(sample, i, l))
+    t0 = time.perf_counter()
     o.round(max(warmup, 1))         # includes the first touch of every per-pair vector
+    if target_seconds > 0.0:
+        pace = (time.perf_counter() - t0) / max(warmup, 1)
+        rounds = int(min(max(rounds, target_seconds / max(pace, 1e-6)), 1000))
     t0 = time.perf_counter()
     o.round(rounds)
     dt = time.perf_counter() - t0
     o.close()
     scaled = (rounds / dt) * (sample.n_workers / w.n_workers)
-    return scaled, dt, sample.n_workers, po.num_threads()
+    return scaled, dt, sample.n_workers, po.num_threads(), rounds
 
 
 # ----------------------------------------------------------------------------
@@ -190,7 +196,7 @@ def run_reference(args, w):
     to the full worker count."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    value, dt, n_sample, cores = time_oracle_sample(w, 4, args.steps, args.warmup)
+    value, dt, n_sample, cores, _ = time_oracle_sample(w, 4, args.steps, args.warmup)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 / value,
@@ -377,10 +383,10 @@ def main():
     cpu = None
     if not args.no_cpu_baseline:
         try:
-            v, dt, n_sample, cores = time_oracle_sample(w, args.cpu_sample_workers, 2, 1)
+            v, dt, n_sample, cores, n_timed = time_oracle_sample(w, args.cpu_sample_workers, 2, 2, target_seconds=12.0)
             cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                   "sample": "%d of %d workers of %s, 2 timed rounds in %.1f s, scaled by workers"
-                             % (n_sample, w.n_workers, w.name, dt)}
+                   "sample": "%d of %d workers of %s, %d timed rounds in %.1f s, scaled by workers"
+                             % (n_sample, w.n_workers, w.name, n_timed, dt)}
         except Exception as exc:  # the baseline never decides the run
             cpu = {"value": None, "unit": UNIT, "cores": None, "kind": "oracle", "sample": "failed: %r" % (exc,)}
 
