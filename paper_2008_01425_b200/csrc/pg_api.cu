@@ -37,6 +37,7 @@ struct Layout {
     bool pair_mode = false;        // rank 1 and degree <= 2: layers run through the pair sweep
     int pend_slots = 1;            // corrections that can be pending at a worker in pair mode (its degree)
     bool two_copies = false;       // pair mode on a graph of degree 2: the sweep writes to a second copy of X
+    bool small_stack = false;      // at most 48 MiB of parameters: the latency regime
     long long n_pair_tiles = 0, n_flush_tiles = 0;
     long long row_tile_cap = 0, col_tile_cap = 0;   // room for the lists with every layer on the three-sweep path
     long long n_pair_tiles_cap = 0, n_flush_tiles_cap = 0;
@@ -109,6 +110,20 @@ int wide_tile_rows(int n, int max_edges, int resident) {
 // fit at once and shape its tiles accordingly.  Section sizes do not depend on
 // the answer, so a sizing pass without a device gives the same total.
 // PG_PAIR_BULK=0 in the environment selects the register-fed pair sweeps.
+// Which kernel families are launched with programmatic stream serialisation (the next
+// kernel is scheduled during the tail of the previous one and waits for it on the device).
+// Measured on B200: the sweeps gain (tiny ring 12.7 -> 9.2 us per round, torus 166 -> 159 us);
+// the cluster pair sweep loses badly as a dependent (1.98 -> 2.31 ms on the LSTM-shaped
+// stack), so it never is one; the pair edge step gains on small stacks and loses next to
+// a side stream, so it is one only on small stacks; a stack with layers on both paths,
+// whose round runs on two streams, launches plainly (0.85 vs 0.87 ms on the VGG-shaped ring).
+// PG_DEPENDENT_LAUNCH=<mask> overrides (0 = plain launches everywhere).
+int dependent_launch_mask(bool small_stack, bool two_streams) {
+    if (const char* v = std::getenv("PG_DEPENDENT_LAUNCH")) return std::atoi(v) & 31;
+    if (two_streams) return 0;
+    return pg::kDepSweep | pg::kDepPairRow | pg::kDepPairMid | (small_stack ? pg::kDepPairEdge : 0);
+}
+
 bool pair_bulk_wanted() {
     const char* v = std::getenv("PG_PAIR_BULK");
     return !(v && v[0] == '0');
@@ -161,6 +176,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     long long tile_elems = std::min<long long>(std::max<long long>(total_elems / 4096, 32 * 1024), 128 * 1024);
     if (const char* v = std::getenv("PG_TILE_ELEMS")) tile_elems = std::max(4096LL, std::atoll(v));   // tuning aid
     const bool small_stack = total_elems * 4 <= 48LL * 1024 * 1024;
+    lay.small_stack = small_stack;
     long long x = 0, q = 0, y = 0, ph = 0, z = 0, up = 0, sp = 0;
     lay.n_row_tiles = lay.n_col_tiles = lay.n_pair_tiles = lay.n_flush_tiles = 0;
     lay.row_tile_cap = lay.col_tile_cap = 0;
@@ -755,6 +771,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.Pn = reinterpret_cast<float*>(c->ws + lay.off_Pn);
     st.half_odd = 0;
     st.pair_bulk = pair_bulk_wanted() ? 1 : 0;
+    st.dep_launch = dependent_launch_mask(lay.small_stack, lay.n_row_tiles > 0 && lay.n_pair_tiles > 0);
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
     st.PhNext = st.Ph + static_cast<long long>(lay.max_edges) * lay.ph_stride;
@@ -1191,8 +1208,13 @@ static void capture_two_rounds(pg_ctx* c, int key) {
         c->loop_failed = true;
         return;
     }
+    // plain launches inside the graph: replay has no launch gaps to hide, and dependent
+    // launches measured equal or slower there
+    const int dep_launch = c->st.dep_launch;
+    c->st.dep_launch = 0;
     int rc = round_impl(c, c->cap, nullptr, 0.0f);
     if (rc == PG_OK) rc = round_impl(c, c->cap, nullptr, 0.0f);
+    c->st.dep_launch = dep_launch;
     cudaGraph_t graph = nullptr;
     const cudaError_t end = cudaStreamEndCapture(c->cap, &graph);
     c->loop_launches = c->launches - launches;

@@ -87,6 +87,9 @@ struct TabLayout {
 };
 
 // Pointers into the workspace (device) plus sizes; passed to kernels by value.
+// Kernel families for DevState::dep_launch.
+enum : int { kDepSweep = 1, kDepPairRow = 2, kDepPairMid = 4, kDepPairWide = 8, kDepPairEdge = 16 };
+
 struct DevState {
     float* X;            // [worker][x_stride]
     float* Xw;           // where corrected rows are written: X itself, or the second copy of the stack
@@ -104,6 +107,7 @@ struct DevState {
     double* Sp;          // [edge][sp_stride]    pair sweep: partial sums of ||p||^2
     float* Pn;           // [edge][layer]  half-step mode: ||p|| of the last odd iteration
     int pair_bulk;       // row-per-warp pair sweep fed by bulk asynchronous copies (TMA)
+    int dep_launch;      // host only: kernel families (kDep*) launched with programmatic stream serialisation
     int half_odd;        // half-step mode: the update being applied is an odd iteration's,
                          // p q-hat^T = (||p|| / ||q||) p-hat q^T: scale the coefficients accordingly
     int* live;           // [edge][layer][rank]  1 if the column took part in this step

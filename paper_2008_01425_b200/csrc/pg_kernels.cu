@@ -14,6 +14,7 @@
 #include <cooperative_groups.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "pg_device.h"
 
@@ -54,6 +55,17 @@ __device__ __forceinline__ void st_stream(float* p, const float4& v) {
     asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y),
                  "f"(v.z), "f"(v.w)
                  : "memory");
+}
+
+// Programmatic dependent launch.  Every kernel of a round starts with this pair:
+// the trigger lets the next kernel of the stream be scheduled while this one is
+// still running (its CTAs take the slots this kernel's tail leaves free), and the
+// wait returns once the previous kernel of the stream has completed and its
+// writes are visible.  Nothing before the wait touches global memory.  Without
+// the launch attribute both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_sync() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // Vector / scalar loads of data that other CTAs produce.  In the multi-launch
@@ -304,6 +316,7 @@ template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool GRAD = false
 __global__ void __launch_bounds__(256, PG_ROW_MIN_BLOCKS)
 row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
                  const Tile* __restrict__ tiles) {
+    grid_dependency_sync();
     __shared__ RowShared<S> sh;
     row_tile<S, UPDATE, FORWARD, SAME, RT, false, GRAD>(st, tab_u, tab_f, tiles[blockIdx.x], sh);
 }
@@ -440,6 +453,7 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
 template <int S, bool UPDATE>
 __global__ void __launch_bounds__(256)
 col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles) {
+    grid_dependency_sync();
     __shared__ ColShared<S> sh;
     col_tile<S, false, UPDATE>(st, tab, tiles[blockIdx.x], sh);
 }
@@ -450,6 +464,7 @@ col_sweep_kernel(DevState st, const int* __restrict__ tab, const Tile* __restric
 // non-finite p gives P-hat = 0 (the edge falls silent).  One CTA per (edge, layer).
 __global__ void __launch_bounds__(512)
 edge_odd_kernel(DevState st, const int* __restrict__ tab) {
+    grid_dependency_sync();
     __shared__ double scratch[33];
     const int L = st.n_layers;
     const int e = blockIdx.x / L, l = blockIdx.x - e * L;
@@ -568,6 +583,7 @@ __device__ __forceinline__ void edge_left_step(const DevState& st, const int* __
 
 __global__ void __launch_bounds__(512)
 edge_left_kernel(DevState st, const int* __restrict__ tab) {
+    grid_dependency_sync();
     __shared__ double scratch[33];
     const int e = blockIdx.x / st.n_layers, l = blockIdx.x - e * st.n_layers;
     if (e >= tab[st.tab.off_n_edges]) return;
@@ -618,6 +634,7 @@ __device__ __forceinline__ void edge_right_step(const DevState& st, const int* _
 
 __global__ void __launch_bounds__(512)
 edge_right_kernel(DevState st, const int* __restrict__ tab) {
+    grid_dependency_sync();
     __shared__ double scratch[33];
     const int e = blockIdx.x / st.n_layers, l = blockIdx.x - e * st.n_layers;
     if (e >= tab[st.tab.off_n_edges]) return;
@@ -651,6 +668,7 @@ __device__ __forceinline__ void philox4x32_10(unsigned c0, unsigned c1, unsigned
 
 __global__ void __launch_bounds__(256)
 random_directions_kernel(DevState st, const int* __restrict__ tab, unsigned key_lo, unsigned key_hi, int side) {
+    grid_dependency_sync();
     __shared__ double scratch[33];
     const int L = st.n_layers, rank = st.rank;
     const int e = blockIdx.x / L, l = blockIdx.x - e * L;
@@ -714,6 +732,7 @@ random_directions_kernel(DevState st, const int* __restrict__ tab, unsigned key_
 // left factor of the random right projection's update (X_i U - X_j U) U^T.
 __global__ void __launch_bounds__(256)
 edge_raw_kernel(DevState st, const int* __restrict__ tab) {
+    grid_dependency_sync();
     const int L = st.n_layers, rank = st.rank;
     const int e = blockIdx.x / L, l = blockIdx.x - e * L;
     if (e >= tab[st.tab.off_n_edges]) return;
@@ -791,6 +810,7 @@ template <int NV, bool UPDATE>
 __global__ void __launch_bounds__(256, 2)
 pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                   const Tile* __restrict__ tiles) {
+    grid_dependency_sync();
     __shared__ __align__(16) float s_q[NV * 128];
     __shared__ __align__(16) float s_ui[NV * 128];
     __shared__ __align__(16) float s_uj[NV * 128];
@@ -981,6 +1001,7 @@ template <int NV, bool UPDATE, int D>
 __global__ void __launch_bounds__(256, PG_BULK_MIN_BLOCKS)
 pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles) {
+    grid_dependency_sync();
     constexpr int STAGES = kBulkStages;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ __align__(16) float s_q[NV * 128];
@@ -1178,6 +1199,7 @@ template <int NVW, bool UPDATE, int D>
 __global__ void __cluster_dims__(kPairCluster, 1, 1) __launch_bounds__(256, PG_WIDE_MIN_BLOCKS)
 pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles, int slice_pad) {
+    grid_dependency_sync();
     namespace cg = cooperative_groups;
     extern __shared__ __align__(16) float s_vec[];               // slices of q-hat, D x u_i, D x u_j
     __shared__ __align__(16) float s_share[2][kPairCluster][kPairWideStep];    // [parity][rank][row]
@@ -1372,6 +1394,7 @@ template <int NVM, bool UPDATE, int D>
 __global__ void __launch_bounds__(256, (NVM <= 2 ? 3 : (NVM <= 5 ? 2 : 1)))
 pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                       const Tile* __restrict__ tiles, int ld_pad) {
+    grid_dependency_sync();
     extern __shared__ __align__(16) float s_vec[];               // q-hat, D x u_i, D x u_j; ld_pad floats each
     __shared__ float s_warp[2][8];
 
@@ -1531,6 +1554,7 @@ template <int NVM, bool UPDATE, int D>
 __global__ void __launch_bounds__(256, mid_min_blocks(NVM, D))
 pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                            const Tile* __restrict__ tiles, int ld_pad, int n_stage) {
+    grid_dependency_sync();
     extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][RS * ld_pad]
     __shared__ __align__(8) unsigned long long s_full[kMidStagesMax];
     constexpr int RS = mid_rows(NVM);
@@ -1705,6 +1729,7 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
 // the (layer, chunk) pairs of one edge.
 __global__ void __launch_bounds__(256)
 pair_edge_kernel(DevState st, const int* __restrict__ tab) {
+    grid_dependency_sync();
     __shared__ double scratch[33];
     const int L = st.n_layers;
     const int e = blockIdx.x / st.e_total;
@@ -1890,6 +1915,25 @@ barrier_timeout_probe_kernel(int* bar, int* status, long long spin_limit) {
     grid_barrier(bar, (int)gridDim.x + 1, status, spin_limit, &s_ok);
 }
 
+// Launch, with programmatic stream serialisation if `allowed`: the kernel may then be
+// scheduled before the previous kernel of the stream has finished, and waits for it on
+// the device (grid_dependency_sync).
+template <typename... Params, typename... Args>
+cudaError_t launch_dep(int allowed, void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = allowed ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 template <bool UPDATE, bool FORWARD, bool SAME>
 cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, const Tile* tiles,
                        int n_tiles, cudaStream_t stream) {
@@ -1897,23 +1941,23 @@ cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, c
     const int slots = st.max_degree * st.rank;
     if (UPDATE && st.G) {     // the update also takes the caller's gradient step
         if (slots <= 1)
-            row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         else if (slots <= 2)
-            row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         else if (slots <= 4)
-            row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         else
-            row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         return cudaGetLastError();
     }
     if (slots <= 1)
-        row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     else if (slots <= 2)
-        row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     else if (slots <= 4)
-        row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     else
-        row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8><<<n_tiles, 256, 0, stream>>>(st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     return cudaGetLastError();
 }
 
@@ -1947,7 +1991,7 @@ static cudaError_t launch_pair_bulk_t(const DevState& st, const int* tab_prev, c
     cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE, D>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (rc != cudaSuccess) return rc;
-    pair_sweep_bulk_kernel<NV, UPDATE, D><<<n_tiles, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles);
+    launch_dep(st.dep_launch & kDepPairRow, pair_sweep_bulk_kernel<NV, UPDATE, D>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles);
     return cudaGetLastError();
 }
 
@@ -1971,14 +2015,14 @@ template <bool UPDATE>
 static cudaError_t launch_pair(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
                                int n_tiles, int nv, cudaStream_t stream) {
     switch (nv) {
-        case 1: pair_sweep_kernel<1, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
-        case 2: pair_sweep_kernel<2, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
-        case 3: pair_sweep_kernel<3, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
-        case 4: pair_sweep_kernel<4, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
-        case 5: pair_sweep_kernel<5, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
-        case 6: pair_sweep_kernel<6, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
-        case 7: pair_sweep_kernel<7, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
-        default: pair_sweep_kernel<8, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab_prev, tab_cur, tiles); break;
+        case 1: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<1, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
+        case 2: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<2, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
+        case 3: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<3, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
+        case 4: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<4, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
+        case 5: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<5, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
+        case 6: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<6, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
+        case 7: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<7, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
+        default: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<8, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
     }
     return cudaGetLastError();
 }
@@ -2010,7 +2054,7 @@ static cudaError_t launch_wide_t(const DevState& st, const int* tab_prev, const 
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (rc != cudaSuccess) return rc;
     }
-    pair_sweep_wide_kernel<NVW, UPDATE, D><<<grid, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, slice_pad);
+    launch_dep(st.dep_launch & kDepPairWide, pair_sweep_wide_kernel<NVW, UPDATE, D>, dim3(grid), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles, slice_pad);
     return cudaGetLastError();
 }
 
@@ -2111,7 +2155,7 @@ cudaError_t launch_unpack_rows(float* dst, long long ld, const float* src, int r
 
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
     if (st.e_total <= 0) return cudaSuccess;
-    pair_edge_kernel<<<max_edges * st.e_total, 256, 0, stream>>>(st, tab);
+    launch_dep(st.dep_launch & kDepPairEdge, pair_edge_kernel, dim3(max_edges * st.e_total), dim3(256), 0, stream, st, tab);
     return cudaGetLastError();
 }
 
@@ -2133,8 +2177,7 @@ static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const i
             cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_bulk_kernel<NVM, UPDATE, D>,
                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
             if (rc != cudaSuccess) return rc;
-            pair_sweep_mid_bulk_kernel<NVM, UPDATE, D><<<n_tiles, 256, total, stream>>>(st, tab_prev, tab_cur, tiles,
-                                                                                       ld_pad, n_stage);
+            launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_bulk_kernel<NVM, UPDATE, D>, dim3(n_tiles), dim3(256), total, stream, st, tab_prev, tab_cur, tiles, ld_pad, n_stage);
             return cudaGetLastError();
         }
     }
@@ -2143,7 +2186,7 @@ static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const i
                                               cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (rc != cudaSuccess) return rc;
     }
-    pair_sweep_mid_kernel<NVM, UPDATE, D><<<n_tiles, 256, smem, stream>>>(st, tab_prev, tab_cur, tiles, ld_pad);
+    launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_kernel<NVM, UPDATE, D>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles, ld_pad);
     return cudaGetLastError();
 }
 
@@ -2178,13 +2221,13 @@ static cudaError_t launch_col(const DevState& st, const int* tab, const Tile* ti
     if (n_tiles <= 0) return cudaSuccess;
     const int slots = st.max_degree * st.rank;
     if (slots <= 1)
-        col_sweep_kernel<1, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        launch_dep(st.dep_launch & kDepSweep, col_sweep_kernel<1, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab, tiles);
     else if (slots <= 2)
-        col_sweep_kernel<2, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        launch_dep(st.dep_launch & kDepSweep, col_sweep_kernel<2, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab, tiles);
     else if (slots <= 4)
-        col_sweep_kernel<4, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        launch_dep(st.dep_launch & kDepSweep, col_sweep_kernel<4, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab, tiles);
     else
-        col_sweep_kernel<8, UPDATE><<<n_tiles, 256, 0, stream>>>(st, tab, tiles);
+        launch_dep(st.dep_launch & kDepSweep, col_sweep_kernel<8, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab, tiles);
     return cudaGetLastError();
 }
 
@@ -2200,27 +2243,27 @@ cudaError_t launch_transposed_update(const DevState& st, const int* tab, const T
 
 cudaError_t launch_random_directions(const DevState& st, const int* tab, int max_edges, unsigned key_lo,
                                      unsigned key_hi, int side, cudaStream_t stream) {
-    random_directions_kernel<<<max_edges * st.n_layers, 256, 0, stream>>>(st, tab, key_lo, key_hi, side);
+    launch_dep(st.dep_launch & kDepSweep, random_directions_kernel, dim3(max_edges * st.n_layers), dim3(256), 0, stream, st, tab, key_lo, key_hi, side);
     return cudaGetLastError();
 }
 
 cudaError_t launch_edge_raw(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
-    edge_raw_kernel<<<max_edges * st.n_layers, 256, 0, stream>>>(st, tab);
+    launch_dep(st.dep_launch & kDepSweep, edge_raw_kernel, dim3(max_edges * st.n_layers), dim3(256), 0, stream, st, tab);
     return cudaGetLastError();
 }
 
 cudaError_t launch_edge_odd(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
-    edge_odd_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    launch_dep(st.dep_launch & kDepSweep, edge_odd_kernel, dim3(max_edges * st.n_layers), dim3(512), 0, stream, st, tab);
     return cudaGetLastError();
 }
 
 cudaError_t launch_edge_left(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
-    edge_left_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    launch_dep(st.dep_launch & kDepSweep, edge_left_kernel, dim3(max_edges * st.n_layers), dim3(512), 0, stream, st, tab);
     return cudaGetLastError();
 }
 
 cudaError_t launch_edge_right(const DevState& st, const int* tab, int max_edges, cudaStream_t stream) {
-    edge_right_kernel<<<max_edges * st.n_layers, 512, 0, stream>>>(st, tab);
+    launch_dep(st.dep_launch & kDepSweep, edge_right_kernel, dim3(max_edges * st.n_layers), dim3(512), 0, stream, st, tab);
     return cudaGetLastError();
 }
 
