@@ -52,7 +52,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="lstm_matching32")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--cpu-sample-workers", type=int, default=8)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workers", type=int, default=0,
@@ -320,18 +320,36 @@ def main():
     value = whole_job_rate(world, args.steps, ms_total)
 
     # ---- end to end through the C ABI with host buffers -------------------------
+    # Every step uploads the whole stack from pinned memory, runs one round and reads the
+    # whole result back.  The read-back of step s runs on one stream beside the upload of
+    # step s + 1 on another (both directions of the link at once); a matrix is overwritten
+    # only after its own read-back has finished, and a round starts after all uploads.
     e2e_steps = max(1, args.e2e_steps)
     upload()
     net.pg_round(stream)
     download()
+    up_stream, down_stream = torch.cuda.Stream(), torch.cuda.Stream()
+    read_done = [[torch.cuda.Event() for _ in range(L)] for _ in range(w.n_workers)]
     barrier()
     e0.record(stream)
-    for _ in range(e2e_steps):
-        upload()
+    up_stream.wait_stream(stream)
+    for step in range(e2e_steps):
+        for i in range(w.n_workers):
+            for l in range(L):
+                if step > 0:
+                    up_stream.wait_event(read_done[i][l])
+                net.pg_write_params(i, l, views[i][l], up_stream)
+        stream.wait_stream(up_stream)
         net.pg_round(stream)
-        download()
+        down_stream.wait_stream(stream)
+        for i in range(w.n_workers):
+            for l in range(L):
+                net.pg_read_params_async(i, l, back_views[i][l], down_stream)
+                read_done[i][l].record(down_stream)
+    stream.wait_stream(down_stream)
     e1.record(stream)
     barrier()
+    status = status or net.pg_device_status(stream)
     ms_e2e = e0.elapsed_time(e1)
     ms_e2e = max_over_ranks(ms_e2e, dist, device)
     e2e_value = whole_job_rate(world, e2e_steps, ms_e2e)

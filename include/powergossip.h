@@ -147,6 +147,18 @@ PG_API int pg_write_params(pg_ctx *ctx, int32_t worker, int32_t layer, const flo
 PG_API int pg_read_params(pg_ctx *ctx, int32_t worker, int32_t layer, float *host_dst, void *stream);
 
 /*
+ * pg_read_params without the wait: the copy to host_dst (pinned memory, valid
+ * until the stream reaches the copy) is only enqueued on `stream`, and the device
+ * status word is not looked at - call pg_device_status when the results matter.
+ * A correction still pending from the last round (see pg_round) is first applied
+ * on `stream`, as in pg_read_params.  With it a caller can run the read-back of one
+ * round's result (Algorithm 1's output X_i) on one stream beside the upload of the
+ * next input on another, one matrix gated on the other by events of its own; the
+ * context does not order streams against each other.
+ */
+PG_API int pg_read_params_async(pg_ctx *ctx, int32_t worker, int32_t layer, float *host_dst, void *stream);
+
+/*
  * Device view of worker `worker`'s layer `layer` for local updates between
  * rounds - Algorithm 1's  - eta G  term: the caller subtracts its scaled
  * gradient in place with its own kernels.  *dev_ptr_out points at rows x cols

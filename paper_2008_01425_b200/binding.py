@@ -22,7 +22,7 @@ PG_RING, PG_TORUS, PG_MATCHING, PG_CUSTOM = 0, 1, 2, 3
 PG_W_UNIFORM, PG_W_METROPOLIS, PG_W_EXPLICIT = 0, 1, 2
 
 EXPORTS = (
-    "pg_workspace_bytes", "pg_create", "pg_destroy", "pg_write_params", "pg_read_params",
+    "pg_workspace_bytes", "pg_create", "pg_destroy", "pg_write_params", "pg_read_params", "pg_read_params_async",
     "pg_round", "pg_device_status", "pg_get_schedule", "pg_max_edges", "pg_read_q", "pg_write_q",
     "pg_get_round", "pg_set_round", "pg_kernel_launches", "pg_status_string",
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
@@ -73,6 +73,7 @@ def load_library() -> ctypes.CDLL:
     L.pg_destroy.restype = None
     L.pg_write_params.argtypes = [vp, i32, i32, vp, vp]
     L.pg_read_params.argtypes = [vp, i32, i32, vp, vp]
+    L.pg_read_params_async.argtypes = [vp, i32, i32, vp, vp]
     L.pg_round.argtypes = [vp, vp]
     L.pg_round_sgd.argtypes = [vp, vp, ctypes.c_float, vp]
     L.pg_stack_elems.argtypes = [vp, ctypes.POINTER(i64)]
@@ -255,6 +256,13 @@ class PowerGossip:
         ptr, _keep = _host_ptr(out, self.layer_shapes[layer])
         _check(self._lib.pg_read_params(self._h, worker, layer, ptr, _stream_handle(stream)),
                "pg_read_params")
+        return out
+
+    def pg_read_params_async(self, worker: int, layer: int, out, stream=None):
+        """Enqueue the copy into `out` (pinned CPU tensor or array) and return at once."""
+        ptr, _keep = _host_ptr(out, self.layer_shapes[layer])
+        _check(self._lib.pg_read_params_async(self._h, worker, layer, ptr, _stream_handle(stream)),
+               "pg_read_params_async")
         return out
 
     def pg_params_device(self, worker: int, layer: int, stream=None):

@@ -889,7 +889,7 @@ int pg_write_params(pg_ctx* c, int32_t worker, int32_t layer, const float* host_
     return PG_OK;
 }
 
-int pg_read_params(pg_ctx* c, int32_t worker, int32_t layer, float* host_dst, void* stream) {
+int pg_read_params_async(pg_ctx* c, int32_t worker, int32_t layer, float* host_dst, void* stream) {
     int rc = check_worker_layer(c, worker, layer);
     if (rc != PG_OK || !host_dst) return PG_ERR_INVALID;
     if (!bind_device(c)) return PG_ERR_CUDA;
@@ -900,6 +900,12 @@ int pg_read_params(pg_ctx* c, int32_t worker, int32_t layer, float* host_dst, vo
     if (cudaMemcpy2DAsync(host_dst, sizeof(float) * g.m, src, sizeof(float) * g.ld, sizeof(float) * g.m,
                           g.n, cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return PG_ERR_CUDA;
+    return PG_OK;
+}
+
+int pg_read_params(pg_ctx* c, int32_t worker, int32_t layer, float* host_dst, void* stream) {
+    const int rc = pg_read_params_async(c, worker, layer, host_dst, stream);
+    if (rc != PG_OK) return rc;
     return device_status(c, static_cast<cudaStream_t>(stream));
 }
 

@@ -261,6 +261,58 @@ def test_runs_are_bit_reproducible_and_checkpoint_resumes():
         n.close()
 
 
+def test_async_read_back_beside_the_next_upload():
+    """Upload, round, read back, several times over: the read-back of one result on one
+    stream beside the upload of the next input on another (each matrix gated on its own
+    event) ends on the same bits as the blocking calls on one stream."""
+    import torch
+
+    w = wl.shrink(wl.lstm_matching32(), [(130, 70), (70, 1300), (300, 652)], 4).replace(n_workers=8)
+    L = len(w.layer_shapes)
+    steps = 3
+    rng = np.random.default_rng(77)
+    inputs = [[[torch.from_numpy(rng.standard_normal(shape).astype(np.float32)).pin_memory()
+                for shape in w.layer_shapes] for _ in range(w.n_workers)] for _ in range(steps)]
+
+    ref = common.network_for(w)
+    expected = []
+    for s in range(steps):
+        for i in range(w.n_workers):
+            for l in range(L):
+                ref.pg_write_params(i, l, inputs[s][i][l])
+        ref.pg_round()
+        expected.append([[ref.pg_read_params(i, l) for l in range(L)] for i in range(w.n_workers)])
+    ref.close()
+
+    net = common.network_for(w)
+    main = torch.cuda.current_stream()
+    up, down = torch.cuda.Stream(), torch.cuda.Stream()
+    out = [[[torch.empty(shape, dtype=torch.float32).pin_memory() for shape in w.layer_shapes]
+            for _ in range(w.n_workers)] for _ in range(steps)]
+    read_done = [[torch.cuda.Event() for _ in range(L)] for _ in range(w.n_workers)]
+    for s in range(steps):
+        for i in range(w.n_workers):
+            for l in range(L):
+                if s > 0:
+                    up.wait_event(read_done[i][l])
+                net.pg_write_params(i, l, inputs[s][i][l], up)
+        main.wait_stream(up)
+        net.pg_round(main)
+        down.wait_stream(main)
+        for i in range(w.n_workers):
+            for l in range(L):
+                net.pg_read_params_async(i, l, out[s][i][l], down)
+                read_done[i][l].record(down)
+    main.wait_stream(down)
+    torch.cuda.synchronize()
+    assert net.pg_device_status(main) == 0
+    for s in range(steps):
+        for i in range(w.n_workers):
+            for l in range(L):
+                assert np.array_equal(out[s][i][l].numpy(), expected[s][i][l]), (s, i, l)
+    net.close()
+
+
 def test_initial_vectors_on_device_are_the_seeded_ones():
     from oracle import pg_oracle as po
 
