@@ -521,6 +521,43 @@ __device__ __forceinline__ void edge_left_step(const DevState& st, const int* __
     float* Ph = st.Ph + (long long)e * st.ph_stride + g.ph_off;
     double coef[kMaxRank];
 
+    if (rank == 1 && g.npad <= 4 * (int)blockDim.x) {
+        // one column and at most four rows per thread: the differences stay in registers
+        // between the norm and the scaling (same sums in the same order as the general case)
+        const float* yi = Yi + (long long)si * g.f_csplit * g.npad;
+        const float* yj = Yj + (long long)sj * g.f_csplit * g.npad;
+        double v[4];
+        double part = 0.0;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int r = threadIdx.x + t * blockDim.x;
+            v[t] = 0.0;
+            if (r < g.n) {
+                double a = 0.0, b = 0.0;
+                for (int cs = 0; cs < g.f_csplit; ++cs) {
+                    a += (double)ld_f<COH>(yi + (long long)cs * g.npad + r);
+                    b += (double)ld_f<COH>(yj + (long long)cs * g.npad + r);
+                }
+                v[t] = a - b;
+                part += v[t] * v[t];
+            }
+        }
+        const double nn = block_sum(part, scratch);
+        const bool finite = isfinite(nn);
+        const bool live = finite && nn > 0.0;
+        const double inv = live ? 1.0 / sqrt(nn) : 0.0;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int r = threadIdx.x + t * blockDim.x;
+            if (r < g.npad) Ph[r] = live ? (float)(v[t] * inv) : 0.0f;
+        }
+        if (threadIdx.x == 0) {
+            live_out[(long long)e * L + l] = live ? 1 : 0;
+            if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
+        }
+        return;
+    }
+
     for (int k = 0; k < rank; ++k) {
         const float* yi = Yi + (long long)(si * rank + k) * g.f_csplit * g.npad;
         const float* yj = Yj + (long long)(sj * rank + k) * g.f_csplit * g.npad;
@@ -614,15 +651,37 @@ __device__ __forceinline__ void edge_right_step(const DevState& st, const int* _
         const float* zi = Zi + (long long)(si * rank + k) * g.t_rtiles * g.ld;
         const float* zj = Zj + (long long)(sj * rank + k) * g.t_rtiles * g.ld;
         double part = 0.0;
-        for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
-            double a = 0.0, b = 0.0;
-            for (int rt = 0; rt < g.t_rtiles; ++rt) {        // added in tile order
-                a += (double)ld_own<COH>(zi + (long long)rt * g.ld + c);
-                b += (double)ld_own<COH>(zj + (long long)rt * g.ld + c);
+        // two columns per thread and pass, four tiles of both ends at a time: sixteen
+        // independent loads in flight, added in tile order
+        for (int c0 = threadIdx.x; c0 < g.m; c0 += 2 * blockDim.x) {
+            const int c1 = c0 + blockDim.x;
+            const bool two = c1 < g.m;
+            double a0 = 0.0, b0 = 0.0, a1 = 0.0, b1 = 0.0;
+            for (int rt = 0; rt < g.t_rtiles; rt += 4) {
+                float vi0[4], vj0[4], vi1[4], vj1[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool in = rt + j < g.t_rtiles;
+                    const long long row = (long long)(rt + j) * g.ld;
+                    vi0[j] = in ? ld_own<COH>(zi + row + c0) : 0.0f;
+                    vj0[j] = in ? ld_own<COH>(zj + row + c0) : 0.0f;
+                    vi1[j] = in && two ? ld_own<COH>(zi + row + c1) : 0.0f;
+                    vj1[j] = in && two ? ld_own<COH>(zj + row + c1) : 0.0f;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    a0 += (double)vi0[j]; b0 += (double)vj0[j];
+                    a1 += (double)vi1[j]; b1 += (double)vj1[j];
+                }
             }
-            const float q = (float)(a - b);
-            Q[(long long)k * g.ld + c] = q;
-            part += (double)q * (double)q;
+            const float q0 = (float)(a0 - b0);
+            Q[(long long)k * g.ld + c0] = q0;
+            part += (double)q0 * (double)q0;
+            if (two) {
+                const float q1 = (float)(a1 - b1);
+                Q[(long long)k * g.ld + c1] = q1;
+                part += (double)q1 * (double)q1;
+            }
         }
         const double nn = block_sum(part, scratch);
         if (threadIdx.x == 0) {
