@@ -149,9 +149,9 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.pair_mode = false;
     lay.pend_slots = 1;
     lay.two_copies = false;
-    if (rank == 1 && pair_sweep_allowed()) {
+    if (rank <= 2 && pair_sweep_allowed()) {
         if (lay.max_degree == 1) {
-            lay.pair_mode = true;
+            lay.pair_mode = rank == 1;
         } else if (lay.max_degree == 2 && topo.kind != PG_MATCHING && pair_bulk_wanted()) {
             std::vector<Edge> edges;
             if (!pg::build_edges(topo, 0, 0, edges)) return PG_ERR_INVALID;
@@ -219,6 +219,9 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         // enough to keep every SM busy for many rows.  Other layers take the three sweeps.
         const bool large_layer = g.n >= 256 && static_cast<long long>(g.n) * g.ld >= (1LL << 20);
         if (lay.two_copies && !small_stack && !large_layer) g.pair_mode = 0;
+        // Rank 2 (rings and paths only): the CTA-per-row sweep has a two-column form for rows its
+        // registers hold; everything else takes the three sweeps.
+        if (rank == 2 && !(g.pair_mode == 3 && large_layer && g.ld <= pg::kPairMid2MaxLd)) g.pair_mode = 0;
         g.p_slice = static_cast<int>(round_up((g.ld + pg::kPairCluster - 1) / pg::kPairCluster, 4));
         {   // equal tiles of at most kPairTileRows rows (a multiple of 8: one row per warp and stage);
             // on graphs of degree 2 short matrices are cut finer, down to 16 rows, so that a layer gives
@@ -241,7 +244,9 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         {   // pair edge step: about 2048 partial sums or rows per CTA
             const int max_tiles = g.pair_mode == 2 ? pg::kPairWideMaxTiles : g.p_rtiles;
             const long long work = static_cast<long long>(max_tiles) * g.ld + g.npad;
-            long long per_cta = 2048;
+            // (on a large ring every (edge, layer) of a step is in one launch: larger shares keep it to one wave;
+            //  VGG-shaped ring 0.877 -> 0.858 ms per round at rank 1, 1.237 -> 1.195 ms at rank 2)
+            long long per_cta = (lay.two_copies && !small_stack) ? 8192 : 2048;
             if (const char* v = std::getenv("PG_EDGE_WORK")) per_cta = std::max(256LL, std::atoll(v));   // tuning aid
             g.e_chunks = static_cast<int>(std::min<long long>(std::max<long long>((work + per_cta - 1) / per_cta, 1), pg::kEdgeChunks));
         }
@@ -252,14 +257,20 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         if (g.pair_mode != 0) {
             // wide layers: room for any tile count the device query may choose
             const int max_tiles = g.pair_mode == 2 ? pg::kPairWideMaxTiles : g.p_rtiles;
-            up += round_up(static_cast<long long>(max_tiles) * g.ld, 64);
-            sp += round_up(max_tiles, 8);
+            // per tile: `rank` vectors of D^T P, and ||p||^2 (rank 1) or the Gram matrix P^T P (rank 2, 4 doubles)
+            up += round_up(static_cast<long long>(max_tiles) * rank * g.ld, 64);
+            sp += round_up(static_cast<long long>(max_tiles) * (rank == 1 ? 1 : 4), 8);
             lay.n_pair_tiles += static_cast<long long>(lay.max_edges) * max_tiles;
             lay.n_flush_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
         } else {
             lay.n_row_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
             lay.n_col_tiles += static_cast<long long>(N) * g.t_rtiles * g.t_ctiles;
         }
+    }
+    if (rank == 2 && lay.n_pair_tiles == 0) {   // no layer for the rank-2 sweep: plain three-sweep context
+        lay.pair_mode = false;
+        lay.pend_slots = 1;
+        lay.two_copies = false;
     }
     lay.up_stride = up;
     lay.sp_stride = sp;
@@ -298,7 +309,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.off_X = take(sizeof(float) * static_cast<size_t>(N) * lay.x_stride * (lay.two_copies ? 2 : 1));
     lay.off_Q = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride);
     lay.off_Qinv = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * n_layers * rank);
-    lay.off_Qn2 = take(sizeof(double) * static_cast<size_t>(lay.n_pairs) * n_layers * pg::kEdgeChunks);
+    lay.off_Qn2 = take(sizeof(double) * static_cast<size_t>(lay.n_pairs) * n_layers * rank * pg::kEdgeChunks);
     lay.off_Pn = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * n_layers);
     lay.off_Y = take(sizeof(float) * static_cast<size_t>(N) * lay.y_stride);
     lay.off_Ph = take(sizeof(float) * 2 * static_cast<size_t>(lay.max_edges) * lay.ph_stride);  // two buffers

@@ -21,6 +21,7 @@ constexpr int kColTileCols = 256;      // columns per CTA in the transposed swee
 constexpr int kPairTileRows = 512;     // rows of both matrices per CTA in the pair sweep
 constexpr int kPairMaxLd = 1024;       // widest row a warp of the pair sweep keeps in registers
 constexpr int kPairMidMaxLd = 8192;    // widest row one CTA of the pair sweep keeps in registers (8 float4 per thread)
+constexpr int kPairMid2MaxLd = 5120;   // widest row of the rank-2 form of that sweep (5 float4 per thread)
 constexpr int kPairCluster = 8;        // CTAs that share a row of a wider layer (thread-block cluster)
 constexpr int kPairWideRows = 32;      // rows per cluster tile of a wider layer when residency is unknown
 constexpr int kPairWideMaxTiles = 32;  // most row tiles per (edge, wide layer); sizes the partial-sum buffer
@@ -51,13 +52,13 @@ struct LayerGeom {
     long long y_off;   // forward partials inside a worker's block   (slots x f_csplit x npad)
     long long ph_off;  // P-hat inside an edge's block               (rank x npad)
     long long z_off;   // transposed partials inside a worker's block (slots x t_rtiles x ld)
-    // pair sweep (rank 1; a matching or a static graph of degree <= 2)
+    // pair sweep (rank 1: a matching or a static graph of degree <= 2; rank 2: mode 3 on such a static graph)
     int pair_mode;     // 0: three sweeps; pair sweep with a row per 1: warp, 2: cluster, 3: CTA
     int p_rows;        // rows per tile of the pair sweep
     int p_rtiles;      // row tiles of the pair sweep
     int p_slice;       // mode 2: columns per CTA of the cluster (multiple of 4)
-    long long up_off;  // partial sums of D^T p inside an edge's block (p_rtiles x ld)
-    long long sp_off;  // partial sums of ||p||^2 inside an edge's block (p_rtiles doubles)
+    long long up_off;  // partial sums of D^T p inside an edge's block (p_rtiles x rank x ld)
+    long long sp_off;  // partial sums of ||p||^2 (p_rtiles doubles), at rank 2 of P^T P (p_rtiles x 4 doubles)
     int e_chunks;      // CTAs that share the pair edge step of one edge on this layer (1..kEdgeChunks)
 };
 
@@ -98,7 +99,7 @@ struct DevState {
     float eta;
     float* Q;            // [pair][q_stride]     raw right factors
     float* Qinv;         // [pair][layer][rank]  1 / column norm (0 for a zero column)
-    double* Qn2;         // [pair][layer][kEdgeChunks]  pair sweep layers: shares of ||Q||^2
+    double* Qn2;         // [pair][layer][rank][kEdgeChunks]  pair sweep layers: shares of ||Q_k||^2
     float* Y;            // [worker][y_stride]   partial sums of X q
     float* Ph;           // [edge][ph_stride]    orthonormal left factors of this step
     float* Z;            // [worker][z_stride]   partial sums of X^T p

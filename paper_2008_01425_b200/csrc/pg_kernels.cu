@@ -816,9 +816,9 @@ edge_raw_kernel(DevState st, const int* __restrict__ tab) {
     }
 }
 
-// 1 / ||Q|| of a pair-sweep layer from the shares the pair edge step left.
-__device__ __forceinline__ float pair_qinv(const DevState& st, int pair, int layer) {
-    const double* n2 = st.Qn2 + ((long long)pair * st.n_layers + layer) * kEdgeChunks;
+// 1 / ||Q_k|| of a pair-sweep layer from the shares the pair edge step left.
+__device__ __forceinline__ float pair_qinv(const DevState& st, int pair, int layer, int k = 0) {
+    const double* n2 = st.Qn2 + (((long long)pair * st.n_layers + layer) * st.rank + k) * kEdgeChunks;
     double t = 0.0;
 #pragma unroll
     for (int k = 0; k < kEdgeChunks; ++k) t += n2[k];
@@ -1780,6 +1780,340 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     if (threadIdx.x == 0) st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = (double)ssum;
 }
 
+// --------------------------------------------------------------------------
+// Rank 2 on a static graph of degree <= 2 (a ring, a path): the CTA-per-row sweep
+// with two columns.  For an edge (i<j) one pass over the rows of X_i and X_j gives
+//   P = D [q-hat_0 q-hat_1]   (rows x 2)      and      U = D^T P   (cols x 2),
+// and the pair edge step orthonormalises afterwards:  P-hat = P T,  Q' = D^T P-hat
+// = U T  with the 2 x 2 triangular T of the Gram-Schmidt step, taken from P^T P.
+// The graph is static, so the corrections still pending at a worker belong to its
+// current edges, and the vector of a pending correction of this edge is the edge's
+// stored Q itself (what q-hat is scaled from): a thread keeps its columns (float4
+// number k * 384 + thread of a row) of three vector pairs in registers - this edge's
+// and the other edge's of either end.
+// Corrections are applied in slot order, columns within a slot in order, as the
+// row sweep applies them; the edge in a worker's slot 0 writes the corrected row to
+// the second copy of the stack.  Rows arrive as in the rank-1 kernel above.
+// --------------------------------------------------------------------------
+// 384 threads (12 warps) a CTA: with 256 the two-column arithmetic of a row is latency-bound
+// (VGG-shaped ring, rank 2: 1.24 -> 1.13 ms per round); rows of up to 4 x 384 float4.
+constexpr int kMid2Threads = 384;
+__host__ __device__ constexpr int mid2_rows(int nvm) { return nvm <= 3 ? 2 : 1; }
+
+__device__ __forceinline__ void fma4(float4& x, float a, const float4& v) {
+    x.x = fmaf(a, v.x, x.x); x.y = fmaf(a, v.y, x.y); x.z = fmaf(a, v.z, x.z); x.w = fmaf(a, v.w, x.w);
+}
+
+template <int NVM, bool UPDATE>
+__global__ void __launch_bounds__(kMid2Threads, 1)
+pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles, int ld_pad,
+                       int n_stage) {
+    grid_dependency_sync();
+    constexpr int R = 2;
+    constexpr int NT = kMid2Threads;
+    constexpr int RS = mid2_rows(NVM);
+    extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][RS * ld_pad]
+    __shared__ __align__(8) unsigned long long s_full[kMidStagesMax];
+    __shared__ float s_warp[2][RS][R][NT / 32];
+    __shared__ int s_abort;
+
+    const Tile tile = tiles[blockIdx.x];
+    const int e = tile.worker;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[tile.layer];
+    const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
+    const int pair = tab[st.tab.off_pair + e];
+    const float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
+    const float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
+    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
+    const int ld = g.ld;
+    const unsigned row_bytes = (unsigned)ld * 4u;     // multiple of 16: ld is a multiple of 4
+    const int md = st.tab.max_degree;
+
+    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float qinv0 = pair_qinv(st, pair, tile.layer, 0), qinv1 = pair_qinv(st, pair, tile.layer, 1);
+    // slot of this edge at either end, and the other edge there (if the worker has two)
+    const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
+    const bool two_i = tab[st.tab.off_degree + wi] > 1, two_j = tab[st.tab.off_degree + wj] > 1;
+    const bool own_i = si == 0, own_j = sj == 0;      // the edge in slot 0 writes the corrected row
+    const float* ph_e = st.Ph + (long long)e * st.ph_stride + g.ph_off;
+    const float* ph_oi = ph_e;
+    const float* ph_oj = ph_e;
+    const float* q_oi = q;
+    const float* q_oj = q;
+    float ce_i = 0.f, ce_j = 0.f, co_i = 0.f, co_j = 0.f;
+    if (UPDATE) {
+        ce_i = __int_as_float(tab[st.tab.off_slot_coef + wi * md + si]);
+        ce_j = __int_as_float(tab[st.tab.off_slot_coef + wj * md + sj]);
+        if (two_i) {
+            const int eo = tab[st.tab.off_slot_edge + wi * md + (1 - si)];
+            q_oi = st.Q + (long long)tab[st.tab.off_pair + eo] * st.q_stride + g.q_off;
+            ph_oi = st.Ph + (long long)eo * st.ph_stride + g.ph_off;
+            co_i = __int_as_float(tab[st.tab.off_slot_coef + wi * md + (1 - si)]);
+        }
+        if (two_j) {
+            const int eo = tab[st.tab.off_slot_edge + wj * md + (1 - sj)];
+            q_oj = st.Q + (long long)tab[st.tab.off_pair + eo] * st.q_stride + g.q_off;
+            ph_oj = st.Ph + (long long)eo * st.ph_stride + g.ph_off;
+            co_j = __int_as_float(tab[st.tab.off_slot_coef + wj * md + (1 - sj)]);
+        }
+    }
+    const int r0 = tile.rtile * g.p_rows;
+    const int r1 = min(g.n, r0 + g.p_rows);
+    const int n_iter = (r1 - r0 + RS - 1) / RS;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s2 = 0; s2 < n_stage; ++s2) mbar_init(&s_full[s2], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    auto issue = [&](int idx) {       // rows r0 + idx*RS ... into slot idx % n_stage
+        const int slot = idx % n_stage;
+        const int row = r0 + idx * RS;
+        const unsigned bytes = (unsigned)min(RS, r1 - row) * row_bytes;
+        float* dst = s_stage + (size_t)slot * 2 * RS * ld_pad;
+        mbar_expect_tx(&s_full[slot], 2 * bytes);
+        bulk_load(dst, Xi + (long long)row * ld, bytes, &s_full[slot]);
+        bulk_load(dst + (size_t)RS * ld_pad, Xj + (long long)row * ld, bytes, &s_full[slot]);
+    };
+    int issued = 0;
+    if (threadIdx.x == 0)
+        for (; issued < n_stage && issued < n_iter; ++issued) issue(issued);
+
+    // this thread's columns of the three vector pairs, for the whole tile
+    float4 vq[R][NVM], vi[R][NVM], vj[R][NVM];
+#pragma unroll
+    for (int k = 0; k < NVM; ++k) {
+        const int off = (k * NT + threadIdx.x) * 4;
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < R; ++c) {
+            vq[c][k] = off < ld ? *reinterpret_cast<const float4*>(q + (long long)c * ld + off) : zero;
+            vi[c][k] = (UPDATE && two_i && off < ld) ? *reinterpret_cast<const float4*>(q_oi + (long long)c * ld + off) : zero;
+            vj[c][k] = (UPDATE && two_j && off < ld) ? *reinterpret_cast<const float4*>(q_oj + (long long)c * ld + off) : zero;
+        }
+    }
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    float4 u[R][NVM];
+#pragma unroll
+    for (int c = 0; c < R; ++c)
+#pragma unroll
+        for (int k = 0; k < NVM; ++k) u[c][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    double g00 = 0.0, g01 = 0.0, g11 = 0.0;       // this tile's share of P^T P (thread 0)
+    bool ok = true;
+
+    for (int it = 0; it < n_iter; ++it) {
+        const int r = r0 + it * RS;
+        const int slot = it % n_stage;
+        const bool mine = mbar_wait_bounded(&s_full[slot], (unsigned)((it / n_stage) & 1), &s_abort, st.status);
+        const float* si_rows = s_stage + (size_t)slot * 2 * RS * ld_pad;      // rows follow each other ld floats apart
+        const float* sj_rows = si_rows + (size_t)RS * ld_pad;
+        float4 d[RS][NVM];
+        float dot[RS][R];
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            const bool in_row = mine && r + t < r1;
+            const long long base = (long long)(r + t) * ld;
+            dot[t][0] = dot[t][1] = 0.0f;
+            // coefficients of the pending corrections of this row: this edge's and the other edge's, per column
+            float ae_i[R], ae_j[R], ao_i[R], ao_j[R];
+#pragma unroll
+            for (int c = 0; c < R; ++c) {
+                const bool on = UPDATE && in_row;
+                ae_i[c] = on ? -ce_i * __ldg(ph_e + (long long)c * g.npad + r + t) : 0.0f;
+                ae_j[c] = on ? -ce_j * __ldg(ph_e + (long long)c * g.npad + r + t) : 0.0f;
+                ao_i[c] = (on && two_i) ? -co_i * __ldg(ph_oi + (long long)c * g.npad + r + t) : 0.0f;
+                ao_j[c] = (on && two_j) ? -co_j * __ldg(ph_oj + (long long)c * g.npad + r + t) : 0.0f;
+            }
+#pragma unroll
+            for (int k = 0; k < NVM; ++k) {
+                const int off = (k * NT + threadIdx.x) * 4;
+                const bool in = in_row && off < ld;
+                float4 xi = make_float4(0.f, 0.f, 0.f, 0.f), xj = xi;
+                if (in) {
+                    xi = *reinterpret_cast<const float4*>(si_rows + (size_t)t * ld + off);
+                    xj = *reinterpret_cast<const float4*>(sj_rows + (size_t)t * ld + off);
+                }
+                if (UPDATE && in) {
+                    if (own_i) {       // this edge is in slot 0 of worker i: its correction first
+                        fma4(xi, ae_i[0], vq[0][k]); fma4(xi, ae_i[1], vq[1][k]);
+                        fma4(xi, ao_i[0], vi[0][k]); fma4(xi, ao_i[1], vi[1][k]);
+                        st_stream(Xi_w + base + off, xi);
+                    } else {
+                        fma4(xi, ao_i[0], vi[0][k]); fma4(xi, ao_i[1], vi[1][k]);
+                        fma4(xi, ae_i[0], vq[0][k]); fma4(xi, ae_i[1], vq[1][k]);
+                    }
+                    if (own_j) {
+                        fma4(xj, ae_j[0], vq[0][k]); fma4(xj, ae_j[1], vq[1][k]);
+                        fma4(xj, ao_j[0], vj[0][k]); fma4(xj, ao_j[1], vj[1][k]);
+                        st_stream(Xj_w + base + off, xj);
+                    } else {
+                        fma4(xj, ao_j[0], vj[0][k]); fma4(xj, ao_j[1], vj[1][k]);
+                        fma4(xj, ae_j[0], vq[0][k]); fma4(xj, ae_j[1], vq[1][k]);
+                    }
+                }
+                d[t][k].x = xi.x - xj.x; d[t][k].y = xi.y - xj.y; d[t][k].z = xi.z - xj.z; d[t][k].w = xi.w - xj.w;
+#pragma unroll
+                for (int c = 0; c < R; ++c) {
+                    dot[t][c] = fmaf(d[t][k].x, vq[c][k].x, dot[t][c]); dot[t][c] = fmaf(d[t][k].y, vq[c][k].y, dot[t][c]);
+                    dot[t][c] = fmaf(d[t][k].z, vq[c][k].z, dot[t][c]); dot[t][c] = fmaf(d[t][k].w, vq[c][k].w, dot[t][c]);
+                }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < RS; ++t)
+#pragma unroll
+            for (int c = 0; c < R; ++c) {
+                const float sum = warp_sum(dot[t][c]);
+                if (lane == 0) s_warp[it & 1][t][c][warp] = sum;
+            }
+        ok = __syncthreads_and(mine) != 0;        // shares visible, stage drained; all go on or all leave
+        if (!ok) break;
+        if (threadIdx.x == 0 && it + n_stage < n_iter) {
+            issue(it + n_stage);
+            issued = it + n_stage + 1;
+        }
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            float p[R];
+#pragma unroll
+            for (int c = 0; c < R; ++c) {
+                p[c] = 0.0f;
+#pragma unroll
+                for (int w8 = 0; w8 < NT / 32; ++w8) p[c] += s_warp[it & 1][t][c][w8];
+            }
+            p[0] *= qinv0;        // the products with the unit columns
+            p[1] *= qinv1;
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+#pragma unroll
+                for (int k = 0; k < NVM; ++k) fma4(u[c][k], p[c], d[t][k]);
+            if (threadIdx.x == 0 && r + t < r1) {
+                g00 += (double)p[0] * (double)p[0];
+                g01 += (double)p[0] * (double)p[1];
+                g11 += (double)p[1] * (double)p[1];
+                Pw[r + t] = p[0];
+                Pw[g.npad + r + t] = p[1];
+            }
+        }
+    }
+    if (!ok) {
+        // leave only after the copies still in flight have landed (bounded)
+        if (threadIdx.x == 0)
+            for (int idx = 0; idx < issued; ++idx) {
+                const int slot = idx % n_stage;
+                for (int spin = 0; spin < kBulkSpinLimit; ++spin)
+                    if (mbar_try_wait(&s_full[slot], (unsigned)((idx / n_stage) & 1))) break;
+            }
+        return;
+    }
+    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * R * ld;
+#pragma unroll
+    for (int c = 0; c < R; ++c)
+#pragma unroll
+        for (int k = 0; k < NVM; ++k) {
+            const int off = (k * NT + threadIdx.x) * 4;
+            if (off < ld) *reinterpret_cast<float4*>(Up + (long long)c * ld + off) = u[c][k];
+        }
+    if (threadIdx.x == 0) {
+        double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * 4;
+        sp[0] = g00;
+        sp[1] = g01;
+        sp[2] = g11;
+    }
+}
+
+// Pair edge step at rank 2: the Gram matrix P^T P from the tiles' shares, then the
+// Gram-Schmidt step in column order as a 2 x 2 triangular map applied to P (in place,
+// giving P-hat) and to U = D^T P (giving Q').  Column 0 is dead iff its squared norm
+// is 0; column 1 iff its residual's squared norm is at most 1e-10 of its own before
+// the projection.  A dead column leaves a zero P-hat column and its stored vector as
+// it was.  Same CTA layout as the rank-1 step below.
+__device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab, int e, int l, int chunk,
+                                double* scratch) {
+    const int L = st.n_layers;
+    const LayerGeom g = st.layers[l];
+    const int pair = tab[st.tab.off_pair + e];
+    const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
+    double a00 = 0.0, a01 = 0.0, a11 = 0.0;
+    for (int t = threadIdx.x; t < g.p_rtiles; t += blockDim.x) {
+        a00 += sp[4 * t];
+        a01 += sp[4 * t + 1];
+        a11 += sp[4 * t + 2];
+    }
+    const double g00 = block_sum(a00, scratch);      // same order, hence same bits, in every chunk
+    const double g01 = block_sum(a01, scratch);
+    const double g11 = block_sum(a11, scratch);
+    const bool finite = isfinite(g00) && isfinite(g01) && isfinite(g11);
+    const bool live0 = finite && g00 > 0.0;
+    const double inv0 = live0 ? 1.0 / sqrt(g00) : 0.0;
+    const double proj = live0 ? g01 * inv0 : 0.0;     // p-hat_0 . p_1
+    const double res = g11 - proj * proj;
+    const bool live1 = finite && res > 0.0 && res > 1e-10 * g11;
+    const double inv1 = live1 ? 1.0 / sqrt(res) : 0.0;
+    float* P = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    const int nch = g.e_chunks;
+    const int rw = (g.npad + nch - 1) / nch;
+    for (int r = chunk * rw + threadIdx.x; r < min(g.npad, (chunk + 1) * rw); r += blockDim.x) {
+        const bool in = r < g.n;
+        const float h0 = (live0 && in) ? (float)((double)P[r] * inv0) : 0.0f;
+        const float h1 = (live1 && in) ? (float)(((double)P[g.npad + r] - proj * (double)h0) * inv1) : 0.0f;
+        P[r] = h0;
+        P[g.npad + r] = h1;
+    }
+    if (chunk == 0 && threadIdx.x == 0) {
+        st.live[((long long)e * L + l) * 2] = live0 ? 1 : 0;
+        st.live[((long long)e * L + l) * 2 + 1] = live1 ? 1 : 0;
+        if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
+    }
+    if (!live0 && !live1) return;   // uniform over the block
+    const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
+    float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const int cw = (g.m + nch - 1) / nch;
+    const int c_lo = chunk * cw, c_hi = min(g.m, (chunk + 1) * cw);
+    double part0 = 0.0, part1 = 0.0;
+    for (int c = c_lo + threadIdx.x; c < c_hi; c += blockDim.x) {
+        double u0 = 0.0, u1 = 0.0;
+        for (int t = 0; t < g.p_rtiles; t += 4) {        // eight independent loads, added in tile order
+            float v0[4], v1[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool in = t + j < g.p_rtiles;
+                v0[j] = in ? up[((long long)(t + j) * 2) * g.ld + c] : 0.0f;
+                v1[j] = in ? up[((long long)(t + j) * 2 + 1) * g.ld + c] : 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                u0 += (double)v0[j];
+                u1 += (double)v1[j];
+            }
+        }
+        const double q0 = u0 * inv0;
+        if (live0) {
+            const float q = (float)q0;
+            Q[c] = q;
+            part0 += (double)q * (double)q;
+        }
+        if (live1) {
+            const float q = (float)((u1 - proj * q0) * inv1);
+            Q[g.ld + c] = q;
+            part1 += (double)q * (double)q;
+        }
+    }
+    const double qq0 = block_sum(part0, scratch);
+    const double qq1 = block_sum(part1, scratch);
+    if (threadIdx.x == 0) {
+        double* n2 = st.Qn2 + (((long long)pair * L + l) * 2) * kEdgeChunks;
+        if (live0) n2[chunk] = qq0;
+        if (live1) n2[kEdgeChunks + chunk] = qq1;
+        if (!isfinite(qq0) || !isfinite(qq1)) atomicOr(st.status, 1 << kStatusNumeric);
+    }
+}
+
 // Pair edge step: ||p||^2 from the tiles' shares, p-hat = p / ||p|| in place,
 // Q' = (sum of the tiles' shares of D^T p) / ||p||, and the shares of ||Q'||^2
 // (the sweep that uses Q' next adds them up).  A zero or non-finite norm leaves
@@ -1797,6 +2131,10 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
     if (!g.pair_mode) return;
+    if (st.rank == 2) {
+        pair_edge_rank2(st, tab, e, l, chunk, scratch);
+        return;
+    }
     const int pair = tab[st.tab.off_pair + e];
     const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
     double part = 0.0;
@@ -1880,8 +2218,8 @@ column_norms_kernel(DevState st) {
         const double nn = block_sum(part, scratch);
         if (threadIdx.x == 0) {
             st.Qinv[(pair * L + l) * rank + k] = nn > 0.0 ? (float)(1.0 / sqrt(nn)) : 0.0f;
-            if (k == 0) {   // the pair sweep reads the squared norm as kEdgeChunks shares
-                double* n2 = st.Qn2 + (pair * L + l) * kEdgeChunks;
+            {   // the pair sweep reads the squared norm as kEdgeChunks shares
+                double* n2 = st.Qn2 + ((pair * L + l) * rank + k) * kEdgeChunks;
                 n2[0] = nn;
                 for (int t = 1; t < kEdgeChunks; ++t) n2[t] = 0.0;
             }
@@ -2258,10 +2596,45 @@ static cudaError_t launch_mid(const DevState& st, const int* tab_prev, const int
                           : launch_mid_t<NVM, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
 }
 
+template <int NVM, bool UPDATE>
+static cudaError_t launch_mid2_t(const DevState& st, const int* tab, const Tile* tiles, int n_tiles, int ld_pad,
+                                 cudaStream_t stream) {
+    const size_t stage = sizeof(float) * 2 * mid2_rows(NVM) * static_cast<size_t>(ld_pad);
+    const int n_stage = (int)std::min<size_t>(kMidSmemBudget / stage, kMidStagesMax);
+    if (n_stage < 2) return cudaErrorInvalidValue;
+    const size_t total = n_stage * stage;
+    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid2_kernel<NVM, UPDATE>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
+    if (rc != cudaSuccess) return rc;
+    launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid2_kernel<NVM, UPDATE>, dim3(n_tiles), dim3(kMid2Threads),
+               total, stream, st, tab, tiles, ld_pad, n_stage);
+    return cudaGetLastError();
+}
+
+// Rank 2: static graphs only, so one table serves the pending corrections and the step.
+static cudaError_t launch_mid2(const DevState& st, const int* tab, bool upd, const Tile* tiles, int n_tiles,
+                               int ld_pad, cudaStream_t stream) {
+    switch ((ld_pad / 4 + kMid2Threads - 1) / kMid2Threads) {     // float4 per thread and row
+        case 1: return upd ? launch_mid2_t<1, true>(st, tab, tiles, n_tiles, ld_pad, stream)
+                           : launch_mid2_t<1, false>(st, tab, tiles, n_tiles, ld_pad, stream);
+        case 2: return upd ? launch_mid2_t<2, true>(st, tab, tiles, n_tiles, ld_pad, stream)
+                           : launch_mid2_t<2, false>(st, tab, tiles, n_tiles, ld_pad, stream);
+        case 3: return upd ? launch_mid2_t<3, true>(st, tab, tiles, n_tiles, ld_pad, stream)
+                           : launch_mid2_t<3, false>(st, tab, tiles, n_tiles, ld_pad, stream);
+        case 4: return upd ? launch_mid2_t<4, true>(st, tab, tiles, n_tiles, ld_pad, stream)
+                           : launch_mid2_t<4, false>(st, tab, tiles, n_tiles, ld_pad, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const int* tab_cur,
                                   bool apply_pending, const Tile* tiles, int n_tiles, int nv, int ld_pad,
                                   int pend_slots, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
+    if (st.rank == 2) {
+        if (tab_prev != tab_cur || pend_slots != 2) return cudaErrorInvalidValue;
+        return launch_mid2(st, tab_cur, apply_pending, tiles, n_tiles, ld_pad, stream);
+    }
     switch (nv) {
         case 1: return launch_mid<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
         case 2: return launch_mid<2>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);

@@ -443,6 +443,40 @@ def test_pair_sweep_on_graphs_of_degree_two(graph):
     _run(w, rounds=3, check_every=1)
 
 
+# rank 2 on graphs of degree 2: layers of at least 256 rows and 2^20 elements with rows of 1025..5120
+# floats take the two-column CTA-per-row sweep (2, 3, 4 and 5 float4 per thread here), the rest the
+# three sweeps on the side stream
+RANK2_SHAPES = ((1024, 1100), (512, 2304), (300, 3600), (256, 4612), (40, 130))
+
+
+@pytest.mark.parametrize("graph", ["ring3", "ring7", "path5", "pair_and_path"])
+def test_rank_two_pair_sweep_on_graphs_of_degree_two(graph):
+    w = wl.Workload("deg2_rank2_" + graph, 9, 4, wl.RING, 0, 0, wl.W_UNIFORM, None, RANK2_SHAPES, 2, 2, 4, 37,
+                    "normal1").replace(**DEGREE2_GRAPHS[graph])
+    _run(w, rebased=True)
+    _run(w, rounds=3, check_every=1)
+
+
+def test_rank_two_reads_between_steps_do_not_change_a_ring_run():
+    """The flush applies the pending rank-2 corrections with the same operations in the same
+    order as the sweep: reading after every round does not change a bit."""
+    w = wl.Workload("ring_reads_rank2", 9, 4, wl.RING, 0, 0, wl.W_UNIFORM, None, ((512, 2304), (24, 150)), 2, 1,
+                    5, 3, "normal1")
+    a, b = common.network_for(w), common.network_for(w)
+    common.load_both(w, None, a)
+    common.load_both(w, None, b)
+    for t in range(w.rounds):
+        a.pg_round()
+        b.pg_round()
+        b.read_all()
+    xa, xb = a.read_all(), b.read_all()
+    for i in range(w.n_workers):
+        for l in range(2):
+            assert np.array_equal(xa[i][l], xb[i][l])
+    a.close()
+    b.close()
+
+
 def test_three_sweeps_on_a_rank_one_ring(monkeypatch):
     """The general path on a graph where the pair sweep is the default."""
     monkeypatch.setenv("PG_DISABLE_PAIR_SWEEP", "1")
