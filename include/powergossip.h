@@ -96,8 +96,8 @@ typedef struct pg_ctx pg_ctx;  /* opaque; host memory owned by the library */
 /*
  * Size in bytes of the device workspace a context with these parameters needs
  * (parameters of all workers, per-pair vectors, exchange buffers, tables; on a
- * static graph of degree 2 at rank 1 a second copy of the parameters, see
- * pg_round).  `shapes`: host, n_layers entries.  PG_ERR_INVALID for a bad topology, rank
+ * static graph of degree 2 at rank 1, and at rank 2 with layers the pair sweep
+ * takes, a second copy of the parameters, see pg_round).  `shapes`: host, n_layers entries.  PG_ERR_INVALID for a bad topology, rank
  * outside 1..PG_MAX_RANK or degree*rank > PG_MAX_SLOTS.
  */
 PG_API int pg_workspace_bytes(const pg_topology *topo, const pg_layer_shape *shapes, int32_t n_layers,
@@ -193,7 +193,11 @@ PG_API int pg_params_device(pg_ctx *ctx, int32_t worker, int32_t layer, void *st
  * There, all layers take the pair sweep when the stack is at most 48 MiB, else
  * only layers of at least 256 rows and 2^20 elements, and the kernels of the
  * other layers run on a stream of the library's own that is forked from and
- * joined to `stream` with events inside the call.  PG_DISABLE_PAIR_SWEEP=1
+ * joined to `stream` with events inside the call.  At rank 2 the pair sweep
+ * exists for those graphs of degree 2 and layers of that size with rows of
+ * 1025 to 5120 floats: one read gives P = D [q-hat_0 q-hat_1] and D^T P, and
+ * the Gram-Schmidt step is applied afterwards as a 2 x 2 triangular map taken
+ * from P^T P (same column order and same dependent-column rule).  PG_DISABLE_PAIR_SWEEP=1
  * in the environment at creation selects the general three-sweep path.
  * Host-side errors are returned at once; device-side ones show up in
  * pg_read_params / pg_device_status.
@@ -357,7 +361,7 @@ enum {
     PG_KERNEL_TRANSPOSED = 2,      /* X^T p-hat                                          */
     PG_KERNEL_EDGE_RIGHT = 3,      /* difference of the two ends, new stored vector      */
     PG_KERNEL_UPDATE_FORWARD = 4,  /* rank-r update of X fused with the next X q         */
-    PG_KERNEL_PAIR_SWEEP = 5,      /* rank 1, degree <= 2: pending update + X q + X^T p from one read */
+    PG_KERNEL_PAIR_SWEEP = 5,      /* degree <= 2: pending update + X q + X^T p from one read */
     PG_KERNEL_PAIR_EDGE = 6,       /* its scalar edge step                               */
     PG_KERNEL_UPDATE_ONLY = 7,     /* applies a pending update before X is read or written */
     PG_KERNEL_KINDS = 8

@@ -1800,8 +1800,42 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
 constexpr int kMid2Threads = 384;
 __host__ __device__ constexpr int mid2_rows(int nvm) { return nvm <= 3 ? 2 : 1; }
 
+// Packed fp32 arithmetic (fma.rn.f32x2: two IEEE fused multiply-adds per instruction, each
+// lane rounded exactly like fmaf).  The two-column sweep is bound by instruction issue, and
+// most of its instructions are these.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// x += a * v
 __device__ __forceinline__ void fma4(float4& x, float a, const float4& v) {
-    x.x = fmaf(a, v.x, x.x); x.y = fmaf(a, v.y, x.y); x.z = fmaf(a, v.z, x.z); x.w = fmaf(a, v.w, x.w);
+    const unsigned long long aa = pack2(a, a);
+    unpack2(fma2(aa, pack2(v.x, v.y), pack2(x.x, x.y)), x.x, x.y);
+    unpack2(fma2(aa, pack2(v.z, v.w), pack2(x.z, x.w)), x.z, x.w);
+}
+// a - b (as fma(b, -1, a): the same rounding as the subtraction)
+__device__ __forceinline__ float4 sub4(const float4& a, const float4& b) {
+    const unsigned long long m = pack2(-1.0f, -1.0f);
+    float4 d;
+    unpack2(fma2(pack2(b.x, b.y), m, pack2(a.x, a.y)), d.x, d.y);
+    unpack2(fma2(pack2(b.z, b.w), m, pack2(a.z, a.w)), d.z, d.w);
+    return d;
+}
+// acc (two partial sums) += d * v, lane by lane
+__device__ __forceinline__ void dot4(float2& acc, const float4& d, const float4& v) {
+    unsigned long long t = pack2(acc.x, acc.y);
+    t = fma2(pack2(d.x, d.y), pack2(v.x, v.y), t);
+    t = fma2(pack2(d.z, d.w), pack2(v.z, v.w), t);
+    unpack2(t, acc.x, acc.y);
 }
 
 template <int NVM, bool UPDATE>
@@ -1913,12 +1947,12 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
         const float* si_rows = s_stage + (size_t)slot * 2 * RS * ld_pad;      // rows follow each other ld floats apart
         const float* sj_rows = si_rows + (size_t)RS * ld_pad;
         float4 d[RS][NVM];
-        float dot[RS][R];
+        float2 dot[RS][R];      // even and odd columns apart until the warp's sum
 #pragma unroll
         for (int t = 0; t < RS; ++t) {
             const bool in_row = mine && r + t < r1;
             const long long base = (long long)(r + t) * ld;
-            dot[t][0] = dot[t][1] = 0.0f;
+            dot[t][0] = dot[t][1] = make_float2(0.f, 0.f);
             // coefficients of the pending corrections of this row: this edge's and the other edge's, per column
             float ae_i[R], ae_j[R], ao_i[R], ao_j[R];
 #pragma unroll
@@ -1956,19 +1990,16 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
                         fma4(xj, ae_j[0], vq[0][k]); fma4(xj, ae_j[1], vq[1][k]);
                     }
                 }
-                d[t][k].x = xi.x - xj.x; d[t][k].y = xi.y - xj.y; d[t][k].z = xi.z - xj.z; d[t][k].w = xi.w - xj.w;
+                d[t][k] = sub4(xi, xj);
 #pragma unroll
-                for (int c = 0; c < R; ++c) {
-                    dot[t][c] = fmaf(d[t][k].x, vq[c][k].x, dot[t][c]); dot[t][c] = fmaf(d[t][k].y, vq[c][k].y, dot[t][c]);
-                    dot[t][c] = fmaf(d[t][k].z, vq[c][k].z, dot[t][c]); dot[t][c] = fmaf(d[t][k].w, vq[c][k].w, dot[t][c]);
-                }
+                for (int c = 0; c < R; ++c) dot4(dot[t][c], d[t][k], vq[c][k]);
             }
         }
 #pragma unroll
         for (int t = 0; t < RS; ++t)
 #pragma unroll
             for (int c = 0; c < R; ++c) {
-                const float sum = warp_sum(dot[t][c]);
+                const float sum = warp_sum(dot[t][c].x + dot[t][c].y);
                 if (lane == 0) s_warp[it & 1][t][c][warp] = sum;
             }
         ok = __syncthreads_and(mine) != 0;        // shares visible, stage drained; all go on or all leave
