@@ -261,6 +261,29 @@ def test_runs_are_bit_reproducible_and_checkpoint_resumes():
         n.close()
 
 
+@pytest.mark.parametrize("w", [wl.tiny_ring(), wl.shrink(wl.torus8x8(2), [(200, 136)], 6),
+                               wl.shrink(wl.lstm_matching32(), [(130, 70), (70, 1300)], 6).replace(n_workers=8)],
+                         ids=lambda w: w.name)
+def test_dependent_launches_do_not_change_a_bit(w, monkeypatch):
+    """Kernels scheduled during the previous kernel's tail wait for it on the device before they
+    touch memory: the run ends on the bits of a run with plain launches."""
+    def run():
+        net = common.network_for(w)
+        common.load_both(w, None, net)
+        for _ in range(w.rounds):
+            net.pg_round()
+        x = net.read_all()
+        assert net.pg_device_status() == 0
+        net.close()
+        return x
+    xa = run()
+    monkeypatch.setenv("PG_DEPENDENT_LAUNCH", "0")
+    xb = run()
+    for i in range(w.n_workers):
+        for l in range(len(w.layer_shapes)):
+            assert np.array_equal(xa[i][l], xb[i][l])
+
+
 def test_async_read_back_beside_the_next_upload():
     """Upload, round, read back, several times over: the read-back of one result on one
     stream beside the upload of the next input on another (each matrix gated on its own
