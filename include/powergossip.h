@@ -199,6 +199,10 @@ PG_API int pg_params_device(pg_ctx *ctx, int32_t worker, int32_t layer, void *st
  * the Gram-Schmidt step is applied afterwards as a 2 x 2 triangular map taken
  * from P^T P (same column order and same dependent-column rule).  PG_DISABLE_PAIR_SWEEP=1
  * in the environment at creation selects the general three-sweep path.
+ * The kernels of a round are launched with programmatic stream serialisation
+ * where that was measured to pay (each waits on the device for the kernel
+ * before it, so results do not depend on it); PG_DEPENDENT_LAUNCH=0 in the
+ * environment at creation gives plain launches.
  * Host-side errors are returned at once; device-side ones show up in
  * pg_read_params / pg_device_status.
  */
