@@ -650,6 +650,7 @@ SGD_CASES = {
     "ring_pair_sweep_two_steps": (wl.tiny_ring().replace(layer_shapes=((33, 130), (7, 9000)), power_steps=2), None),
     "matching_pair_sweep": (wl.shrink(wl.lstm_matching32(), [(130, 70), (70, 1300)], 6).replace(n_workers=8), None),
     "torus_rank2_two_steps": (wl.shrink(wl.torus8x8(2), [(200, 136), (5, 3)], 6).replace(rank=2), None),
+    "ring_rank2_pair_sweep": (wl.tiny_ring().replace(layer_shapes=((512, 2306), (33, 130)), rank=2, power_steps=2), None),
     "ring_three_sweeps": (wl.tiny_ring().replace(layer_shapes=((64, 32), (67, 131))), "three"),
     "ring_half_step": (wl.tiny_ring().replace(power_steps=3), "half"),
     "ring_random_projection": (wl.tiny_ring().replace(rank=2), "random"),
