@@ -385,7 +385,7 @@ REPLAY_CASES = [
     wl.tiny_ring(),                                   # pair sweep on a ring (two copies of X swap every step)
     wl.resnet20_ring8().replace(rounds=13),
     wl.vgg16_ring16(1).replace(rounds=7),             # layers on both paths: the side stream is part of the capture
-    wl.vgg16_ring16(2).replace(rounds=6),             # three sweeps, too large for the cooperative kernel
+    wl.vgg16_ring16(2).replace(rounds=6),             # the same at rank 2: two-column pair sweep beside the three sweeps
 ]
 
 
