@@ -89,7 +89,7 @@ typedef struct pg_layer_shape {
 
 typedef struct pg_ctx pg_ctx;  /* opaque; host memory owned by the library */
 
-/* Limits of this build. */
+/* Limits of the library as compiled. */
 #define PG_MAX_RANK 4          /* columns per edge                                    */
 #define PG_MAX_SLOTS 8         /* (max degree) * rank vectors handled per worker      */
 
