@@ -177,6 +177,29 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     if (const char* v = std::getenv("PG_TILE_ELEMS")) tile_elems = std::max(4096LL, std::atoll(v));   // tuning aid
     const bool small_stack = total_elems * 4 <= 48LL * 1024 * 1024;
     lay.small_stack = small_stack;
+    // Which sweep a layer takes.  A row per warp up to kPairMaxLd floats, per CTA up to kPairMidMaxLd,
+    // per cluster beyond.  With two readers per row the pair sweep pays off in two regimes: a stack small
+    // enough to live in L2, where it halves the launches of a step, and layers large enough to keep every
+    // SM busy for many rows; other layers take the three sweeps.  Rank 2 (rings and paths only): the
+    // CTA-per-row sweep has a two-column form for rows its registers hold; everything else takes the
+    // three sweeps.
+    auto pair_mode_of = [&](int rows, int ld) {
+        int mode = !lay.pair_mode ? 0
+                   : ld <= pg::kPairMaxLd ? 1
+                   : ld <= pg::kPairMidMaxLd ? 3
+                   : ld <= pg::kPairWideMaxLd ? 2 : 0;
+        const bool large_layer = rows >= 256 && static_cast<long long>(rows) * ld >= (1LL << 20);
+        if (lay.two_copies && !small_stack && !large_layer) mode = 0;
+        if (rank == 2 && !(mode == 3 && large_layer && ld <= pg::kPairMid2MaxLd)) mode = 0;
+        return mode;
+    };
+    // rows the CTA-per-row sweep covers on a large stack with two readers per row (one launch a step)
+    long long shared_launch_rows = 0;
+    if (lay.two_copies && !small_stack)
+        for (int l = 0; l < n_layers; ++l)
+            if (shapes[l].rows > 0 && shapes[l].cols > 0 &&
+                pair_mode_of(shapes[l].rows, static_cast<int>(round_up(shapes[l].cols, 4))) == 3)
+                shared_launch_rows += shapes[l].rows;
     long long x = 0, q = 0, y = 0, ph = 0, z = 0, up = 0, sp = 0;
     lay.n_row_tiles = lay.n_col_tiles = lay.n_pair_tiles = lay.n_flush_tiles = 0;
     lay.row_tile_cap = lay.col_tile_cap = 0;
@@ -209,19 +232,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         y += round_up(static_cast<long long>(slots) * g.f_csplit * g.npad, 64);
         ph += round_up(static_cast<long long>(rank) * g.npad, 64);
         z += round_up(static_cast<long long>(slots) * g.t_rtiles * g.ld, 64);
-        // a row per warp up to kPairMaxLd floats, per CTA up to kPairMidMaxLd, per cluster beyond
-        g.pair_mode = !lay.pair_mode ? 0
-                      : g.ld <= pg::kPairMaxLd ? 1
-                      : g.ld <= pg::kPairMidMaxLd ? 3
-                      : g.ld <= pg::kPairWideMaxLd ? 2 : 0;
-        // With two readers per row the pair sweep pays off in two regimes: a stack small
-        // enough to live in L2, where it halves the launches of a step, and layers large
-        // enough to keep every SM busy for many rows.  Other layers take the three sweeps.
-        const bool large_layer = g.n >= 256 && static_cast<long long>(g.n) * g.ld >= (1LL << 20);
-        if (lay.two_copies && !small_stack && !large_layer) g.pair_mode = 0;
-        // Rank 2 (rings and paths only): the CTA-per-row sweep has a two-column form for rows its
-        // registers hold; everything else takes the three sweeps.
-        if (rank == 2 && !(g.pair_mode == 3 && large_layer && g.ld <= pg::kPairMid2MaxLd)) g.pair_mode = 0;
+        g.pair_mode = pair_mode_of(g.n, g.ld);
         g.p_slice = static_cast<int>(round_up((g.ld + pg::kPairCluster - 1) / pg::kPairCluster, 4));
         {   // equal tiles of at most kPairTileRows rows (a multiple of 8: one row per warp and stage);
             // on graphs of degree 2 short matrices are cut finer, down to 16 rows, so that a layer gives
@@ -229,7 +240,15 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
             const int by_height = (g.n + pg::kPairTileRows - 1) / pg::kPairTileRows;
             const int by_count = std::min((296 + lay.max_edges - 1) / lay.max_edges, std::max(g.n / 16, 1));
             // (on a matching every layer of the stack shares one launch, which has tiles enough)
-            const int parts = lay.two_copies ? std::max(by_height, by_count) : by_height;
+            int parts = lay.two_copies ? std::max(by_height, by_count) : by_height;
+            if (g.pair_mode == 3 && shared_launch_rows > 0) {
+                // The large layers of such a stack share one launch: tall tiles, about two per SM over the
+                // whole launch (a tile's prologue - 5 to 6 vectors per thread - is not hidden by anything
+                // with one CTA per SM; VGG-shaped ring, tiles of 32 -> 176 rows: 0.854 -> 0.798 ms per round
+                // at rank 1, 1.049 -> 0.955 ms at rank 2; 256 rows, 1.3 CTAs per SM: 0.92 / 1.12 ms).
+                const long long target = std::max<long long>(16, shared_launch_rows * lay.max_edges / 296);
+                parts = std::max<int>(by_height, static_cast<int>(std::max<long long>(1, (g.n + target / 2) / target)));
+            }
             g.p_rows = static_cast<int>(round_up((g.n + parts - 1) / parts, 8));
         }
         if (g.pair_mode == 2) {
