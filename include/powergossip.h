@@ -394,8 +394,9 @@ PG_API int pg_timing_read(pg_ctx *ctx, double *ms_out, int64_t *launches_out, do
  *   All three on the current device.  Asynchronous on `stream`.
  *
  * Limit: ceil(rows/256) * (cols rounded up to 4) <= PG_NOALLOC_MAX_PARTIALS,
- * e.g. 28000 x 650, 650 x 28000 or 8192 x 8192; beyond it the call does nothing
- * and returns PG_ERR_TOO_LARGE.
+ * e.g. 28000 x 650, 650 x 28000 or 8192 x 8192, and at most 65535 * 256 rows;
+ * beyond either the call launches nothing, leaves z_dev alone and returns
+ * PG_ERR_TOO_LARGE.
  * Set-up: the first call on each device looks up the device address of the
  * array (cudaGetSymbolAddress, once per device, with that device current); make
  * that first call outside any stream capture.

@@ -20,6 +20,7 @@ constexpr int kTileRows = 256;                 // rows summed by one CTA
 constexpr int kTileCols = 256;                 // columns per CTA: 64 threads x 4
 constexpr long long kScratchFloats = PG_NOALLOC_MAX_PARTIALS;
 constexpr int kMaxDevices = 64;
+constexpr long long kMaxGridY = 65535;         // CUDA's limit on gridDim.y
 
 // The scratch itself.  Every GPU that loads this library keeps its own copy
 // until the process exits.  In host code this name is only a handle for the
@@ -121,9 +122,13 @@ bool on_current_device(const void* ptr) {
 extern "C" int pg_transposed_product_noalloc(const float* X_dev, int32_t rows, int32_t cols, int64_t ld,
                                              const float* p_dev, float* z_dev, void* stream_v) {
     if (!X_dev || !p_dev || !z_dev || rows < 1 || cols < 1 || ld < cols) return PG_ERR_INVALID;
-    const int rtiles = (rows + kTileRows - 1) / kTileRows;
-    const int width = (cols + 3) / 4 * 4;                    // one row of partials
-    if (static_cast<long long>(rtiles) * width > kScratchFloats) return PG_ERR_TOO_LARGE;
+    // sizes in 64 bits: cols near INT_MAX must not wrap while being rounded up
+    const long long rtiles_ll = (static_cast<long long>(rows) + kTileRows - 1) / kTileRows;
+    const long long width_ll = (static_cast<long long>(cols) + 3) / 4 * 4;      // one row of partials
+    if (rtiles_ll * width_ll > kScratchFloats) return PG_ERR_TOO_LARGE;
+    if (rtiles_ll > kMaxGridY) return PG_ERR_TOO_LARGE;      // row tiles are the launch's second grid dimension
+    const int rtiles = static_cast<int>(rtiles_ll);
+    const int width = static_cast<int>(width_ll);
     if (!on_current_device(X_dev) || !on_current_device(p_dev) || !on_current_device(z_dev)) return PG_ERR_INVALID;
     float* partials = nullptr;
     const int rc = scratch_address(&partials);
@@ -138,6 +143,8 @@ extern "C" int pg_transposed_product_noalloc(const float* X_dev, int32_t rows, i
         xtp_partial_kernel<true><<<grid, 256, 0, stream>>>(X_dev, rows, cols, ld, p_dev, partials, width);
     else
         xtp_partial_kernel<false><<<grid, 256, 0, stream>>>(X_dev, rows, cols, ld, p_dev, partials, width);
+    // z is written only if the partial sums were really enqueued
+    if (cudaGetLastError() != cudaSuccess) return PG_ERR_CUDA;
     xtp_reduce_kernel<<<(cols + 255) / 256, 256, 0, stream>>>(partials, rtiles, cols, width, z_dev);
     if (cudaGetLastError() != cudaSuccess) return PG_ERR_CUDA;
     return PG_OK;

@@ -6,6 +6,8 @@ import numpy as np
 
 from paper_2008_01425_b200 import workloads as wl
 
+PARITY_LINES = []     # one line per parity run, printed by conftest.py after the test summary
+
 
 def oracle_for(w: wl.Workload):
     from oracle import pg_oracle as po
@@ -36,10 +38,35 @@ def load_both(w: wl.Workload, oracle, net) -> None:
                 net.pg_write_params(i, l, x)
 
 
+def relative_errors(w: wl.Workload, oracle, net, x0=None):
+    """Two figures per (worker, layer), each returned as (maximum, where):
+
+    on_x        ||X_gpu - X_oracle||_F / ||X_oracle||_F, the tolerance figure;
+    on_change   ||X_gpu - X_oracle||_F / ||X_oracle - X0||_F, the same error against
+                what the rounds have changed since X0 (the seeded initial matrices,
+                or the caller's `x0[worker][layer]`, e.g. the state of the last
+                re-basing).  On stacks whose workers share a large common part this
+                is the stricter figure, because one round moves only a small part of ||X||.
+    """
+    on_x, on_change = (0.0, None), (0.0, None)
+    for i in range(w.n_workers):
+        for l in range(len(w.layer_shapes)):
+            ref = oracle.get_params(i, l)
+            got = net.pg_read_params(i, l).astype(np.float64)
+            start = wl.initial_params(w, i, l) if x0 is None else x0[i][l]
+            diff = np.linalg.norm(got - ref)
+            a = diff / max(np.linalg.norm(ref), 1e-300)
+            moved = np.linalg.norm(ref - start)
+            b = diff / moved if moved > 0.0 else (0.0 if diff == 0.0 else np.inf)
+            if not np.isfinite(a) or a > on_x[0]:
+                on_x = (float(a), (i, l))
+            if not np.isfinite(b) or b > on_change[0]:
+                on_change = (float(b), (i, l))
+    return on_x, on_change
+
+
 def max_relative_error(w: wl.Workload, oracle, net):
-    """max over (worker, layer) of ||X_gpu - X_oracle||_F / ||X_oracle||_F, and the
-    relative drift of the worker average on the GPU side is returned separately
-    by average_drift()."""
+    """max over (worker, layer) of ||X_gpu - X_oracle||_F / ||X_oracle||_F, and where."""
     worst = 0.0
     where = None
     for i in range(w.n_workers):
@@ -71,18 +98,24 @@ def rebase(w: wl.Workload, oracle, net, pairs) -> None:
 
     Data only flows from the checker to the CUDA path.  After this call both
     hold identical fp32 parameters and per-pair vectors; `pairs` lists the
-    pairs whose vectors have been touched so far.
+    pairs whose vectors have been touched so far.  Returns the loaded matrices,
+    [worker][layer], the state the next segment starts from.
     """
+    loaded = []
     for i in range(w.n_workers):
+        row = []
         for l in range(len(w.layer_shapes)):
             x32 = oracle.get_params(i, l).astype(np.float32)
             oracle.set_params(i, l, x32)
             net.pg_write_params(i, l, x32)
+            row.append(x32)
+        loaded.append(row)
     for (i, j) in sorted(pairs):
         for l in range(len(w.layer_shapes)):
             q32 = oracle.get_q(i, j, l).astype(np.float32)
             oracle.set_q(i, j, l, q32.astype(np.float64))
             net.pg_write_q(i, j, l, q32)
+    return loaded
 
 
 def gpu_consensus_distance(w: wl.Workload, net) -> float:

@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """The parity figures the GPU tests collected, one line per run, at the end of the log."""
+    from tests import common
+
+    if common.PARITY_LINES:
+        terminalreporter.write_sep("-", "parity against the fp64 CPU checker")
+        for line in common.PARITY_LINES:
+            terminalreporter.write_line(line)

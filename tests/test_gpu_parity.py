@@ -20,8 +20,6 @@ horizon.  Hence two kinds of test:
                  whole stated number of rounds.  This checks every round of the
                  computation along the checker's trajectory.
 """
-import os
-
 import numpy as np
 import pytest
 
@@ -31,9 +29,9 @@ from tests import common
 pytestmark = pytest.mark.gpu
 
 REL_TOL = 1e-4
+CHANGE_TOL = 1e-3            # the same error against ||X_ref - X_start||_F, what the rounds changed
 AVG_TOL = 1e-5
 SEGMENT_POWER_STEPS = 8      # re-base at least this often (in power steps)
-FULL = os.environ.get("PG_FULL_PARITY", "0") == "1"
 
 
 def _check_schedules(oracle, net, rounds):
@@ -53,10 +51,12 @@ def _check_average(w, net, avg0):
 def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance_tol=0.05):
     """Run `rounds` rounds on both sides.
 
-    free-running (rebased=False): assert 1e-4 at every check up to round
-    `horizon` (default: all rounds); past the horizon only the invariants.
-    rebased=True: re-base every SEGMENT_POWER_STEPS power steps, assert 1e-4 at
-    the end of every segment.
+    free-running (rebased=False): assert 1e-4 (on ||X||) and 1e-3 (on what the rounds
+    changed since the seeded start) at every check up to round `horizon` (default: all
+    rounds); past the horizon only the invariants.
+    rebased=True: re-base every SEGMENT_POWER_STEPS power steps, assert both figures at
+    the end of every segment, the second one against the state the segment started from.
+    One line per run with the largest of either figure goes to the end of the pytest log.
     """
     from paper_2008_01425_b200 import binding as pg
 
@@ -71,6 +71,7 @@ def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance
         check_every = max(1, SEGMENT_POWER_STEPS // w.power_steps)
     pairs = set()
     done, err = 0, 0.0
+    worst_x, worst_change, start = 0.0, 0.0, None
     while done < rounds:
         step = rounds - done if not check_every else min(check_every, rounds - done)
         for t in range(done, done + step):
@@ -79,16 +80,23 @@ def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance
         oracle.round(step)
         done += step
         if rebased or done <= horizon:
-            err, where = common.max_relative_error(w, oracle, net)
+            (err, where), (err_c, where_c) = common.relative_errors(w, oracle, net, start)
+            worst_x, worst_change = max(worst_x, err), max(worst_change, err_c)
             assert err <= REL_TOL, "round %d: relative error %.3e at (worker, layer) %r" % (done, err, where)
+            assert err_c <= CHANGE_TOL, ("round %d: error %.3e of what the rounds changed at (worker, layer) %r"
+                                         % (done, err_c, where_c))
         if rebased and done < rounds:
-            common.rebase(w, oracle, net, pairs)
+            start = common.rebase(w, oracle, net, pairs)
     assert net.pg_device_status() == pg.PG_OK
     assert net.pg_get_round() == rounds
     if not rebased:
         _check_average(w, net, avg0)
         d_ref, d_gpu = oracle.consensus_distance(), common.gpu_consensus_distance(w, net)
         assert abs(d_gpu - d_ref) <= distance_tol * d_ref, (d_gpu, d_ref)
+    common.PARITY_LINES.append(
+        "%-34s rank %d %s %3d rounds: max error %.2e of ||X||, %.2e of the change%s"
+        % (w.name, w.rank, "re-based" if rebased else "free-run", rounds, worst_x, worst_change,
+           "" if rebased or horizon >= rounds else " (asserted to round %d, invariants after)" % horizon))
     net.close()
     oracle.close()
     return err
@@ -121,19 +129,19 @@ def test_config3_torus_small_free_running(power_steps):
 
 def test_config3_torus_full_size_free_running():
     w = wl.torus8x8(1)
-    _run(w, rounds=w.rounds if FULL else 40, check_every=20, horizon=20)
+    _run(w, check_every=20, horizon=20)
 
 
 @pytest.mark.parametrize("power_steps", [1, 2, 4])
 def test_config3_torus_full_size_rebased(power_steps):
     w = wl.torus8x8(power_steps)
-    _run(w, rounds=w.rounds if FULL else 16 // power_steps, rebased=True)
+    _run(w, rebased=True)
 
 
 @pytest.mark.parametrize("rank", [1, 2])
 def test_config4_vgg16_ring16_full_size(rank):
     w = wl.vgg16_ring16(rank)
-    _run(w, rounds=w.rounds if FULL else 4, rebased=True)
+    _run(w, rebased=True)
 
 
 @pytest.mark.parametrize("rank", [1, 2])
@@ -163,7 +171,7 @@ def test_config5_lstm_matching_small_rebased():
 def test_config5_lstm_matching_full_size():
     """Full 5.96 GB stack, free-running; the checker needs about 12 GB of host memory."""
     w = wl.lstm_matching32()
-    _run(w, rounds=w.rounds if FULL else 3)
+    _run(w, check_every=10)
 
 
 # ---- edge cases -------------------------------------------------------------

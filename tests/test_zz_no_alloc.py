@@ -69,6 +69,13 @@ def test_two_calls_in_a_row_match_the_regular_path(shape):
         got = z.cpu().numpy().astype(np.float64)
         err = np.linalg.norm(got - q_expected) / np.linalg.norm(q_expected)
         assert err <= REL_TOL, "attempt %d: relative error %.3e" % (attempt, err)
+        # and each of the two products against the same product formed in double precision
+        # from the very operands the call was given (numpy on the host)
+        p_ref = x0.astype(np.float64) @ q_hat.cpu().numpy().astype(np.float64)
+        z_ref = x0.astype(np.float64).T @ p_hat.cpu().numpy().astype(np.float64)
+        for name, mine, ref in (("X q", p.cpu().numpy(), p_ref), ("X^T p", got, z_ref)):
+            e64 = np.linalg.norm(mine.astype(np.float64) - ref) / np.linalg.norm(ref)
+            assert e64 <= 1e-6, "attempt %d, %s: relative error %.3e against fp64" % (attempt, name, e64)
 
 
 def test_strided_rows_and_rejection_of_oversized_problems():
@@ -94,3 +101,12 @@ def test_strided_rows_and_rejection_of_oversized_problems():
     with pytest.raises(pg.PowerGossipError) as e:
         pg.pg_transposed_product_noalloc(big, p, z, rows=0, cols=4, ld=4)
     assert e.value.status == pg.PG_ERR_INVALID
+    # more row tiles than one launch can hold, although their partial sums would fit the scratch;
+    # and a column count whose rounding up would overflow: both refused on the host, z untouched
+    z.fill_(7.0)
+    for rows, cols in ((256 * 65536, 8), (1, 2 ** 31 - 2)):
+        with pytest.raises(pg.PowerGossipError) as e:
+            pg.pg_transposed_product_noalloc(big, p, z, rows=rows, cols=cols, ld=cols)
+        assert e.value.status == pg.PG_ERR_TOO_LARGE, (rows, cols)
+    torch.cuda.synchronize()
+    assert bool((z == 7.0).all())
