@@ -255,6 +255,9 @@ typedef struct pgo_ctx {
     int random_proj;     /* 0: power iteration; 1: random right projections R_k; 2: random left projections */
     int64_t step;        /* random projections: steps taken so far (keys the directions) */
     int64_t iteration;   /* half-step mode: Algorithm 2's counter k (shared: all pairs move in lockstep) */
+    /* diagnostics and test aids; neither changes what a power step computes */
+    double min_resid_ratio;  /* smallest (residual norm / norm before projection)^2 met at a column k > 0 */
+    int fp32_storage;        /* 1: X and Q are rounded to fp32 after every power step (see pgo_set_fp32_storage) */
 } pgo_ctx;
 
 static size_t pair_index(int N, int i, int j)  /* i < j, over all N(N-1)/2 pairs */
@@ -273,6 +276,7 @@ pgo_ctx *pgo_create(int kind, int N, int trows, int tcols, const int *custom, in
     c->N = N; c->L = L; c->rank = rank; c->power_steps = power_steps;
     c->kind = kind; c->trows = trows; c->tcols = tcols; c->rule = rule;
     c->seed = seed; c->round = 0;
+    c->min_resid_ratio = INFINITY;
     c->n_custom = n_custom;
     if (n_custom > 0) {
         c->custom = (int *)malloc(sizeof(int) * 2 * (size_t)n_custom);
@@ -437,7 +441,7 @@ static double dot(const double *a, const double *b, int n)
 /* One power step of one edge on one layer: fills Ph (n x rank, column-major),
  * Qn (m x rank, column-major) and live[k] (0 when column k was degenerate). */
 static void edge_power_step(const double *Xi, const double *Xj, int n, int m, int rank,
-                            const double *Q, double *Ph, double *Qn, int *live)
+                            const double *Q, double *Ph, double *Qn, int *live, double *min_ratio)
 {
     double *qh = (double *)malloc(sizeof(double) * (size_t)m);
     double *pi = (double *)malloc(sizeof(double) * (size_t)n);
@@ -468,6 +472,7 @@ static void edge_power_step(const double *Xi, const double *Xj, int n, int m, in
          * a linear combination of the earlier columns: what is left has no
          * meaningful direction), contributes nothing and keeps its vector */
         int ok = (nn > 0.0) && isfinite(nn) && (k == 0 || nn > 1e-10 * pre);
+        if (k > 0 && pre > 0.0 && isfinite(nn) && nn / pre < *min_ratio) *min_ratio = nn / pre;   /* diagnostic only */
         live[k] = ok;
         double inv = ok ? 1.0 / sqrt(nn) : 0.0;
         for (int r = 0; r < n; ++r) p[r] = ok ? p[r] * inv : 0.0;
@@ -685,6 +690,42 @@ static int random_projection_round(pgo_ctx *c)
     return 0;
 }
 
+/* Diagnostic: the smallest squared ratio (Gram-Schmidt residual / column before
+ * projection) met so far at any column k > 0; +inf if none was met.  The
+ * dependent-column rule compares this ratio with 1e-10, so a run whose minimum
+ * stays far above that threshold would have taken the same decisions under any
+ * smaller threshold. */
+double pgo_min_residual_ratio(pgo_ctx *c) { return c ? c->min_resid_ratio : -1.0; }
+
+/* Test aid, NOT part of the method: with this on, every entry of X and of the
+ * vectors of this round's pairs is rounded to fp32 and widened again after every
+ * power step, while all arithmetic stays in fp64.  That is the least
+ * perturbation any implementation that stores its state in fp32 applies to the
+ * iteration; a test runs this beside the untouched fp64 run to see how far such
+ * an implementation can be expected to drift.  Power-iteration mode only. */
+int pgo_set_fp32_storage(pgo_ctx *c, int on)
+{
+    if (!c || c->half_step || c->random_proj) return -1;
+    c->fp32_storage = on ? 1 : 0;
+    return 0;
+}
+
+static void round_state_to_fp32(pgo_ctx *c, const int *edges, int E)
+{
+    for (int i = 0; i < c->N; ++i)
+        for (int l = 0; l < c->L; ++l) {
+            double *x = c->X[(size_t)i * c->L + l];
+            size_t cnt = (size_t)c->rows[l] * (size_t)c->cols[l];
+            for (size_t t = 0; t < cnt; ++t) x[t] = (double)(float)x[t];
+        }
+    for (int e = 0; e < E; ++e)
+        for (int l = 0; l < c->L; ++l) {
+            double *q = c->Q[pair_index(c->N, edges[2 * e], edges[2 * e + 1]) * (size_t)c->L + (size_t)l];
+            size_t cnt = (size_t)c->cols[l] * (size_t)c->rank;
+            for (size_t t = 0; t < cnt; ++t) q[t] = (double)(float)q[t];
+        }
+}
+
 /* One gossip round = power_steps power steps on every layer and every edge of
  * this round's graph.  Returns 0, or -1 on an invalid schedule. */
 int pgo_round(pgo_ctx *c)
@@ -715,8 +756,11 @@ int pgo_round(pgo_ctx *c)
                 size_t t = pair_index(c->N, i, j) * (size_t)c->L + (size_t)l;
                 size_t u = (size_t)e * (size_t)c->L + (size_t)l;
                 Qn[u] = (double *)malloc(sizeof(double) * (size_t)m * (size_t)rank);
+                double ratio = INFINITY;
                 edge_power_step(c->X[(size_t)i * c->L + l], c->X[(size_t)j * c->L + l], n, m, rank,
-                                c->Q[t], c->Ph[t], Qn[u], live + u * (size_t)rank);
+                                c->Q[t], c->Ph[t], Qn[u], live + u * (size_t)rank, &ratio);
+#pragma omp critical(pgo_min_ratio)
+                if (ratio < c->min_resid_ratio) c->min_resid_ratio = ratio;
             }
         /* phase 2: X_i <- X_i - W_ij Ph Q'^T and X_j <- X_j + W_ij Ph Q'^T (what
          * is added to one endpoint is subtracted from the other), Q <- Q' */
@@ -746,6 +790,7 @@ int pgo_round(pgo_ctx *c)
                 Qn[u] = NULL;
             }
         }
+        if (c->fp32_storage) round_state_to_fp32(c, edges, E);
     }
     free(Qn); free(live); free(edges); free(w);
     c->round += 1;

@@ -89,6 +89,10 @@ def lib() -> ctypes.CDLL:
         L.pgo_set_half_step.restype = c_int
         L.pgo_get_vector.argtypes = [vp, c_int, c_int, c_int, vp]
         L.pgo_get_vector.restype = c_int
+        L.pgo_min_residual_ratio.argtypes = [vp]
+        L.pgo_min_residual_ratio.restype = c_dbl
+        L.pgo_set_fp32_storage.argtypes = [vp, c_int]
+        L.pgo_set_fp32_storage.restype = c_int
         L.pgo_num_threads.argtypes = []
         L.pgo_num_threads.restype = c_int
         _lib = L
@@ -236,6 +240,17 @@ class Oracle:
         `power_steps` then counts iterations per round.  Rank 1, static graphs."""
         if lib().pgo_set_half_step(self._h, int(on)) != 0:
             raise ValueError("half-step mode needs rank 1, a static graph and round 0")
+
+    def min_residual_ratio(self) -> float:
+        """Smallest squared (Gram-Schmidt residual / column before projection) met so far at a
+        column k > 0 (inf if none): what the dependent-column rule compares with 1e-10."""
+        return float(lib().pgo_min_residual_ratio(self._h))
+
+    def set_fp32_storage(self, on: bool = True) -> None:
+        """Test aid, not the method: round X and the touched vectors to fp32 after every power
+        step (arithmetic stays fp64), the least perturbation an fp32-storage implementation applies."""
+        if lib().pgo_set_fp32_storage(self._h, int(on)) != 0:
+            raise ValueError("fp32 storage emulation is for power-iteration mode only")
 
     def get_vector(self, i: int, j: int, layer: int) -> np.ndarray:
         """The pair's current vector (rows entries after an odd iteration, else cols)."""

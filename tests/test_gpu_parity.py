@@ -93,10 +93,17 @@ def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance
         _check_average(w, net, avg0)
         d_ref, d_gpu = oracle.consensus_distance(), common.gpu_consensus_distance(w, net)
         assert abs(d_gpu - d_ref) <= distance_tol * d_ref, (d_gpu, d_ref)
+    note = ""
+    if w.rank > 1 and all(min(n, m) >= w.rank for n, m in w.layer_shapes):
+        # no Gram-Schmidt residual came near the dependent-column threshold (1e-10): both sides
+        # took the same decisions whatever the threshold's exact value
+        smallest = oracle.min_residual_ratio()
+        assert smallest > 1e-8, smallest
+        note = ", smallest residual ratio %.1e" % smallest
     common.PARITY_LINES.append(
         "%-34s rank %d %s %3d rounds: max error %.2e of ||X||, %.2e of the change%s"
         % (w.name, w.rank, "re-based" if rebased else "free-run", rounds, worst_x, worst_change,
-           "" if rebased or horizon >= rounds else " (asserted to round %d, invariants after)" % horizon))
+           "" if rebased or horizon >= rounds else " (asserted to round %d, invariants after)" % horizon) + note)
     net.close()
     oracle.close()
     return err

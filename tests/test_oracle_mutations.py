@@ -29,6 +29,16 @@ MUTATIONS = {
     "ring_skips_wraparound": ("edges_out[2 * n + 1] = (i + 1) % N; ++n; }",
                               "edges_out[2 * n + 1] = (i + 1) % N; if (i + 1 < N) ++n; }"),
     "philox_round_count": ("round < 10; ++round", "round < 9; ++round"),
+    # rank > 1: the dependent-column rule
+    "dependent_rule_comparison_flipped": ("(k == 0 || nn > 1e-10 * pre);\n        if (k > 0",
+                                          "(k == 0 || nn < 1e-10 * pre);\n        if (k > 0"),
+    "dependent_rule_threshold_far_lower": ("(k == 0 || nn > 1e-10 * pre);\n        if (k > 0",
+                                           "(k == 0 || nn > 1e-20 * pre);\n        if (k > 0"),
+    "dependent_rule_threshold_far_higher": ("(k == 0 || nn > 1e-10 * pre);\n        if (k > 0",
+                                            "(k == 0 || nn > 1e-5 * pre);\n        if (k > 0"),
+    "dependent_rule_not_relative": ("(k == 0 || nn > 1e-10 * pre);\n        if (k > 0",
+                                    "(k == 0 || nn > 1e-10);\n        if (k > 0"),
+    "dropped_column_loses_its_vector": ("if (!live[u * (size_t)rank + k]) continue;", ";"),
     # Algorithm 2 read literally (half-step mode)
     "half_step_parity_swapped": ("const int odd = (int)(c->iteration % 2);",
                                  "const int odd = (int)(c->iteration % 2 == 0);"),
