@@ -295,12 +295,22 @@ PG_API int pg_rounds(pg_ctx *ctx, int32_t n_rounds, void *stream);
  * a few CTAs on a barrier that expects one arrival more than will come.  Every
  * CTA must give up after about a millisecond; the call waits for `stream` and
  * returns PG_ERR_TIMEOUT when that happened (the expected outcome), PG_OK if the
- * wait was not reported.  The status word keeps the time-out bit afterwards:
- * use a context of its own.
+ * wait was not reported.  The status word keeps the time-out bit afterwards and
+ * the context refuses further rounds (PG_ERR_STATE), as after any time-out: use a
+ * context of its own.
  */
 PG_API int pg_selftest_barrier_timeout(pg_ctx *ctx, void *stream);
 
-/* Wait for `stream` and return the device status word (PG_OK or PG_ERR_NUMERIC). */
+/*
+ * Wait for `stream` and return the device status word: PG_OK; PG_ERR_NUMERIC (a norm
+ * was not finite); PG_ERR_TIMEOUT (a bounded device-side wait gave up: an mbarrier or
+ * the grid barrier of pg_rounds); PG_ERR_STATE (any other bit); PG_ERR_CUDA if the copy
+ * or the wait failed.  The bits are sticky.  After PG_ERR_TIMEOUT a kernel has left in
+ * the middle of a step, so X, Q and the cached products no longer belong together: the
+ * context is marked failed, and pg_round, pg_round_sgd, pg_rounds and pg_set_round
+ * return PG_ERR_STATE from then on (reading parameters still works; create a new
+ * context to go on).  pg_read_params reports the same way.
+ */
 PG_API int pg_device_status(pg_ctx *ctx, void *stream);
 
 /*
@@ -322,9 +332,12 @@ PG_API int pg_read_q(pg_ctx *ctx, int32_t i, int32_t j, int32_t layer, float *ho
 PG_API int pg_write_q(pg_ctx *ctx, int32_t i, int32_t j, int32_t layer, const float *host_src, void *stream);
 
 /* Round counter (the index of the next round): read it, or set it when
- * restoring a checkpoint {all X, all Q, round}. */
+ * restoring a checkpoint {all X, all Q, round}.  Setting it first applies a
+ * correction still pending from the last round (see pg_round), enqueued on
+ * `stream`: pass the stream the rounds ran on, so that the correction is ordered
+ * after them.  Does not wait. */
 PG_API int pg_get_round(pg_ctx *ctx, int64_t *round_out);
-PG_API int pg_set_round(pg_ctx *ctx, int64_t round);
+PG_API int pg_set_round(pg_ctx *ctx, int64_t round, void *stream);
 
 /*
  * Context-free, host-only view of the schedule builder: the edge list (i<j,
@@ -408,6 +421,36 @@ PG_API int pg_timing_read(pg_ctx *ctx, double *ms_out, int64_t *launches_out, do
 #define PG_NOALLOC_MAX_PARTIALS (1 << 20)
 PG_API int pg_transposed_product_noalloc(const float *X_dev, int32_t rows, int32_t cols, int64_t ld,
                                          const float *p_dev, float *z_dev, void *stream);
+
+/*
+ * Communication volume of Algorithm 2: what the two ends of an edge would send
+ * each other if they sat on different machines (here the exchange is a read of
+ * device buffers).  In iteration k (the algorithm's counter, from 1) each end
+ * sends its product with the shared unit vector to the other end: rank * rows
+ * floats of every tensor when k is odd (p = X v-hat), rank * cols when k is even
+ * (the transposed iteration).  This is the count behind the per-tensor
+ * "compression" column of the paper's parameter tables (Appendix "Network
+ * architectures": rows * cols over (rows + cols) / 2 per iteration, "115/r x" for
+ * 64 x 576) and behind the bytes-per-epoch columns of its result tables.
+ *   pg_comm_floats        host only, no context: floats ONE end of ONE edge sends
+ *                         over `iterations` iterations starting at counter
+ *                         `first_iteration` >= 1, summed over the layers, to
+ *                         *floats_out; *dense_out (may be NULL) gets rows * cols
+ *                         summed over the layers, what one uncompressed exchange
+ *                         (D-PSGD, Eq. 1) sends.
+ *   pg_comm_floats_round  floats ALL workers of the context send in round `round`
+ *                         (both ends of every edge of that round's graph).  A power
+ *                         step is an odd and an even iteration; in half-step mode
+ *                         the round's `power_steps` iterations continue the count
+ *                         of the rounds before it; the random projections send the
+ *                         product only (rank * rows for PG_RANDOM_RIGHT, rank * cols
+ *                         for PG_RANDOM_LEFT per step; the directions are drawn
+ *                         from the shared seed at both ends).
+ * PG_ERR_INVALID for bad arguments.  Touches no GPU.
+ */
+PG_API int pg_comm_floats(const pg_layer_shape *shapes, int32_t n_layers, int32_t rank, int64_t first_iteration,
+                          int64_t iterations, int64_t *floats_out, int64_t *dense_out);
+PG_API int pg_comm_floats_round(pg_ctx *ctx, int64_t round, int64_t *floats_out, int64_t *dense_out);
 
 /* Number of kernels this context has launched so far. */
 PG_API int pg_kernel_launches(pg_ctx *ctx, int64_t *count_out);

@@ -28,7 +28,7 @@ EXPORTS = (
     "pg_build_schedule", "pg_initial_vector", "pg_timing_enable", "pg_timing_read",
     "pg_transposed_product_noalloc", "pg_rounds", "pg_selftest_barrier_timeout",
     "pg_set_half_step", "pg_params_device", "pg_set_random_projection",
-    "pg_round_sgd", "pg_stack_elems", "pg_stack_offset",
+    "pg_round_sgd", "pg_stack_elems", "pg_stack_offset", "pg_comm_floats", "pg_comm_floats_round",
 )
 PG_POWER_ITERATION, PG_RANDOM_RIGHT, PG_RANDOM_LEFT = 0, 1, 2
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
@@ -89,13 +89,16 @@ def load_library() -> ctypes.CDLL:
     L.pg_read_q.argtypes = [vp, i32, i32, i32, vp, vp]
     L.pg_write_q.argtypes = [vp, i32, i32, i32, vp, vp]
     L.pg_get_round.argtypes = [vp, ctypes.POINTER(i64)]
-    L.pg_set_round.argtypes = [vp, i64]
+    L.pg_set_round.argtypes = [vp, i64, vp]
     L.pg_kernel_launches.argtypes = [vp, ctypes.POINTER(i64)]
     L.pg_build_schedule.argtypes = [ctypes.POINTER(pg_topology), vp, u64, i64, vp, vp, i32, ctypes.POINTER(i32)]
     L.pg_initial_vector.argtypes = [u64, i32, i32, i32, i32, i32, vp]
     L.pg_timing_enable.argtypes = [vp, i32]
     L.pg_timing_read.argtypes = [vp, vp, vp, vp]
     L.pg_transposed_product_noalloc.argtypes = [vp, i32, i32, i64, vp, vp, vp]
+    L.pg_comm_floats.argtypes = [ctypes.POINTER(pg_layer_shape), i32, i32, i64, i64, ctypes.POINTER(i64),
+                                 ctypes.POINTER(i64)]
+    L.pg_comm_floats_round.argtypes = [vp, i64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     L.pg_status_string.argtypes = [ctypes.c_int]
     L.pg_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -160,6 +163,16 @@ def pg_initial_vector(seed: int, i: int, j: int, layer: int, col: int, m: int) -
     out = np.zeros(m, dtype=np.float32)
     _check(load_library().pg_initial_vector(seed, i, j, layer, col, m, out.ctypes.data), "pg_initial_vector")
     return out
+
+
+def pg_comm_floats(layer_shapes: Sequence[Tuple[int, int]], rank: int = 1, first_iteration: int = 1,
+                   iterations: int = 1) -> Tuple[int, int]:
+    """(floats one end of one edge sends over these iterations of Algorithm 2, floats of one
+    uncompressed exchange), summed over the layers; host only."""
+    sent, dense = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(load_library().pg_comm_floats(_shapes(layer_shapes), len(layer_shapes), rank, first_iteration,
+                                         iterations, ctypes.byref(sent), ctypes.byref(dense)), "pg_comm_floats")
+    return int(sent.value), int(dense.value)
 
 
 def pg_transposed_product_noalloc(X, p, z, stream=None, rows: Optional[int] = None,
@@ -361,8 +374,15 @@ class PowerGossip:
         _check(self._lib.pg_get_round(self._h, ctypes.byref(r)), "pg_get_round")
         return int(r.value)
 
-    def pg_set_round(self, r: int) -> None:
-        _check(self._lib.pg_set_round(self._h, int(r)), "pg_set_round")
+    def pg_set_round(self, r: int, stream=None) -> None:
+        _check(self._lib.pg_set_round(self._h, int(r), _stream_handle(stream)), "pg_set_round")
+
+    def pg_comm_floats_round(self, round_index: int) -> Tuple[int, int]:
+        """(floats all workers send in that round, floats uncompressed gossip would send)."""
+        sent, dense = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(self._lib.pg_comm_floats_round(self._h, int(round_index), ctypes.byref(sent), ctypes.byref(dense)),
+               "pg_comm_floats_round")
+        return int(sent.value), int(dense.value)
 
     def pg_kernel_launches(self) -> int:
         r = ctypes.c_int64(0)

@@ -35,12 +35,13 @@ def powergossip_curve(steps: int, every: int, device: str = "cuda:0"):
         net.pg_write_params(i, 0, x)
     net.pg_set_half_step()
     mean0 = sum(x.astype(np.float64) for x in x0) / w.n_workers
-    n, m = w.layer_shapes[0]
     curve = [(0.0, consensus_error(x0, mean0))]
     sent = 0.0
+    ends = 2 * len(net.pg_get_schedule(0)[0])       # every edge has two ends
     for t in range(1, steps + 1):
+        # what one worker sends one neighbour in this round: the library's count for all ends, per end
+        sent += net.pg_comm_floats_round(t - 1)[0] / ends
         net.pg_round()
-        sent += n if t % 2 == 1 else m          # an odd iteration sends p (rows), an even one q (cols)
         if t % every == 0 or t == steps:
             xs = [net.pg_read_params(i, 0) for i in range(w.n_workers)]
             curve.append((sent, consensus_error(xs, mean0)))

@@ -109,7 +109,6 @@ int wide_tile_rows(int n, int max_edges, int resident) {
 // query_device: ask the current device how many clusters of the wide pair sweep
 // fit at once and shape its tiles accordingly.  Section sizes do not depend on
 // the answer, so a sizing pass without a device gives the same total.
-// PG_PAIR_BULK=0 in the environment selects the register-fed pair sweeps.
 // Which kernel families are launched with programmatic stream serialisation (the next
 // kernel is scheduled during the tail of the previous one and waits for it on the device).
 // Measured on B200: the sweeps gain (tiny ring 12.7 -> 9.2 us per round, torus 166 -> 159 us);
@@ -122,11 +121,6 @@ int dependent_launch_mask(bool small_stack, bool two_streams) {
     if (const char* v = std::getenv("PG_DEPENDENT_LAUNCH")) return std::atoi(v) & 31;
     if (two_streams) return 0;
     return pg::kDepSweep | pg::kDepPairRow | pg::kDepPairMid | (small_stack ? pg::kDepPairEdge : 0);
-}
-
-bool pair_bulk_wanted() {
-    const char* v = std::getenv("PG_PAIR_BULK");
-    return !(v && v[0] == '0');
 }
 
 int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_layers, int rank,
@@ -152,7 +146,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     if (rank <= 2 && pair_sweep_allowed()) {
         if (lay.max_degree == 1) {
             lay.pair_mode = rank == 1;
-        } else if (lay.max_degree == 2 && topo.kind != PG_MATCHING && pair_bulk_wanted()) {
+        } else if (lay.max_degree == 2 && topo.kind != PG_MATCHING) {
             std::vector<Edge> edges;
             if (!pg::build_edges(topo, 0, 0, edges)) return PG_ERR_INVALID;
             std::vector<int> degree(N, 0);
@@ -174,7 +168,6 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         if (shapes[l].rows > 0 && shapes[l].cols > 0)
             total_elems += static_cast<long long>(N) * shapes[l].rows * round_up(shapes[l].cols, 4);
     long long tile_elems = std::min<long long>(std::max<long long>(total_elems / 4096, 32 * 1024), 128 * 1024);
-    if (const char* v = std::getenv("PG_TILE_ELEMS")) tile_elems = std::max(4096LL, std::atoll(v));   // tuning aid
     const bool small_stack = total_elems * 4 <= 48LL * 1024 * 1024;
     lay.small_stack = small_stack;
     // Which sweep a layer takes.  A row per warp up to kPairMaxLd floats, per CTA up to kPairMidMaxLd,
@@ -265,8 +258,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
             const long long work = static_cast<long long>(max_tiles) * g.ld + g.npad;
             // (on a large ring every (edge, layer) of a step is in one launch: larger shares keep it to one wave;
             //  VGG-shaped ring 0.877 -> 0.858 ms per round at rank 1, 1.237 -> 1.195 ms at rank 2)
-            long long per_cta = (lay.two_copies && !small_stack) ? 8192 : 2048;
-            if (const char* v = std::getenv("PG_EDGE_WORK")) per_cta = std::max(256LL, std::atoll(v));   // tuning aid
+            const long long per_cta = (lay.two_copies && !small_stack) ? 8192 : 2048;
             g.e_chunks = static_cast<int>(std::min<long long>(std::max<long long>((work + per_cta - 1) / per_cta, 1), pg::kEdgeChunks));
         }
         g.up_off = up;
@@ -399,6 +391,7 @@ struct pg_ctx {
     bool half_pending = false;  // an odd iteration's update has not been applied to X yet
     int random_proj = 0;        // 0 power iteration, 1 random right projections, 2 random left projections
     bool static_graph = true;
+    bool failed = false;        // a bounded device-side wait gave up: the state on the device is not trustworthy
     bool coop_ok = false;       // the device supports cooperative launches
     int device = 0;
     // optional per-kernel timing: one event pair per launch while enabled
@@ -657,7 +650,7 @@ bool upload_tile_lists(pg_ctx* c) {
     }
     // serpentine: the transposed sweep walks the stack in the opposite direction to the row
     // sweeps that run before and after it, so each sweep starts on what is still in L2
-    if (!std::getenv("PG_NO_SERPENTINE")) std::reverse(cols.begin(), cols.end());
+    std::reverse(cols.begin(), cols.end());
     if (static_cast<long long>(rows.size()) > lay.row_tile_cap || static_cast<long long>(cols.size()) > lay.col_tile_cap ||
         static_cast<long long>(pairs.size()) > lay.n_pair_tiles_cap || static_cast<long long>(flush.size()) > lay.n_flush_tiles_cap)
         return false;
@@ -709,7 +702,17 @@ int device_status(pg_ctx* c, cudaStream_t stream) {
     if (cudaMemcpyAsync(&word, c->st.status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return PG_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return PG_ERR_CUDA;
-    if (word & (1 << PG_ERR_TIMEOUT)) return PG_ERR_TIMEOUT;
+    if (word & (1 << PG_ERR_TIMEOUT)) {
+        // a kernel left in the middle of a step: X, Q and the cached products no longer belong
+        // together.  No further round runs on this context.
+        c->failed = true;
+        c->y_valid = false;
+        if (c->loop_exec) {
+            cudaGraphExecDestroy(c->loop_exec);
+            c->loop_exec = nullptr;
+        }
+        return PG_ERR_TIMEOUT;
+    }
     if (word & (1 << PG_ERR_NUMERIC)) return PG_ERR_NUMERIC;
     return word == 0 ? PG_OK : PG_ERR_STATE;
 }
@@ -800,7 +803,6 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
     st.Pn = reinterpret_cast<float*>(c->ws + lay.off_Pn);
     st.half_odd = 0;
-    st.pair_bulk = pair_bulk_wanted() ? 1 : 0;
     st.dep_launch = dependent_launch_mask(lay.small_stack, lay.n_row_tiles > 0 && lay.n_pair_tiles > 0);
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
@@ -963,6 +965,7 @@ int pg_device_status(pg_ctx* c, void* stream) {
 // and is left fully updated in memory.
 static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
     if (!c) return PG_ERR_INVALID;
+    if (c->failed) return PG_ERR_STATE;
     if (!bind_device(c)) return PG_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const int* tab = nullptr;
@@ -1079,7 +1082,7 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
         return PG_OK;
     }
     // a stack with layers on both paths: the three sweeps of this round go to the side stream
-    const bool forked = n_rows > 0 && has_pair && !std::getenv("PG_NO_SIDE_STREAM");
+    const bool forked = n_rows > 0 && has_pair;
     cudaStream_t s3 = stream;
     if (forked) {
         ok = cudaEventRecord(c->ev_fork, stream) == cudaSuccess &&
@@ -1272,6 +1275,7 @@ static void capture_two_rounds(pg_ctx* c, int key) {
 
 int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
     if (!c || n_rounds < 0) return PG_ERR_INVALID;
+    if (c->failed) return PG_ERR_STATE;
     if (n_rounds == 0) return PG_OK;
     if (!bind_device(c)) return PG_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -1284,7 +1288,7 @@ int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
         int done = 0;
         // launch-bound loops on a static graph: replay a captured pair of rounds
         bool replay = c->static_graph && !c->half_step && !c->random_proj && !c->timing && !c->loop_failed &&
-                      n_rounds >= 4 && !std::getenv("PG_NO_GRAPH");
+                      n_rounds >= 4;
         if (replay) {
             cudaStreamCaptureStatus busy = cudaStreamCaptureStatusNone;
             if (cudaStreamIsCapturing(stream, &busy) != cudaSuccess || busy != cudaStreamCaptureStatusNone) {
@@ -1436,19 +1440,66 @@ int pg_initial_vector(uint64_t seed, int32_t i, int32_t j, int32_t layer, int32_
     return PG_OK;
 }
 
+int pg_comm_floats(const pg_layer_shape* shapes, int32_t n_layers, int32_t rank, int64_t first_iteration,
+                   int64_t iterations, int64_t* floats_out, int64_t* dense_out) {
+    if (!shapes || n_layers < 1 || rank < 1 || first_iteration < 1 || iterations < 0 || !floats_out)
+        return PG_ERR_INVALID;
+    int64_t rows = 0, cols = 0, dense = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        if (shapes[l].rows < 1 || shapes[l].cols < 1) return PG_ERR_INVALID;
+        rows += shapes[l].rows;
+        cols += shapes[l].cols;
+        dense += static_cast<int64_t>(shapes[l].rows) * shapes[l].cols;
+    }
+    // odd counters among first_iteration .. first_iteration + iterations - 1
+    const int64_t last = first_iteration + iterations - 1;
+    const int64_t n_odd = (last + 1) / 2 - first_iteration / 2;
+    const int64_t n_even = iterations - n_odd;
+    *floats_out = rank * (n_odd * rows + n_even * cols);
+    if (dense_out) *dense_out = dense;
+    return PG_OK;
+}
+
+int pg_comm_floats_round(pg_ctx* c, int64_t round, int64_t* floats_out, int64_t* dense_out) {
+    if (!c || round < 0 || !floats_out) return PG_ERR_INVALID;
+    std::vector<Edge> edges;
+    if (!pg::build_edges(c->topo, c->seed, round, edges)) return PG_ERR_INVALID;
+    std::vector<pg_layer_shape> shapes(c->n_layers);
+    for (int l = 0; l < c->n_layers; ++l) shapes[l] = pg_layer_shape{c->lay.layers[l].n, c->lay.layers[l].m};
+    int64_t per_end = 0, dense = 0;
+    int rc;
+    if (c->random_proj) {
+        // one product per step: an "odd" iteration for right projections, an "even" one for left
+        rc = pg_comm_floats(shapes.data(), c->n_layers, c->rank, c->random_proj == 1 ? 1 : 2, 1, &per_end, &dense);
+        per_end *= c->power_steps;
+    } else if (c->half_step) {
+        rc = pg_comm_floats(shapes.data(), c->n_layers, c->rank, round * c->power_steps + 1, c->power_steps,
+                            &per_end, &dense);
+    } else {
+        rc = pg_comm_floats(shapes.data(), c->n_layers, c->rank, 1, 2LL * c->power_steps, &per_end, &dense);
+    }
+    if (rc != PG_OK) return rc;
+    const int64_t ends = 2 * static_cast<int64_t>(edges.size());
+    *floats_out = ends * per_end;
+    if (dense_out) *dense_out = ends * dense;
+    return PG_OK;
+}
+
 int pg_get_round(pg_ctx* c, int64_t* round_out) {
     if (!c || !round_out) return PG_ERR_INVALID;
     *round_out = c->round;
     return PG_OK;
 }
 
-int pg_set_round(pg_ctx* c, int64_t round) {
+int pg_set_round(pg_ctx* c, int64_t round, void* stream_v) {
     if (!c || round < 0) return PG_ERR_INVALID;
-    if (c->pending) {
+    if (c->failed) return PG_ERR_STATE;
+    if (c->pending || c->half_pending) {
+        // the pending correction belongs to the old round's graph: apply it first, on the
+        // stream the rounds were enqueued on
         if (!bind_device(c)) return PG_ERR_CUDA;
-        const int rc = flush_pending(c, nullptr);
+        const int rc = flush_pending(c, static_cast<cudaStream_t>(stream_v));
         if (rc != PG_OK) return rc;
-        if (cudaStreamSynchronize(nullptr) != cudaSuccess) return PG_ERR_CUDA;
     }
     c->round = round;
     c->y_valid = false;

@@ -25,13 +25,8 @@ constexpr int kPairMid2MaxLd = 5120;   // widest row of the rank-2 form of that 
 constexpr int kPairCluster = 8;        // CTAs that share a row of a wider layer (thread-block cluster)
 constexpr int kPairWideRows = 32;      // rows per cluster tile of a wider layer when residency is unknown
 constexpr int kPairWideMaxTiles = 32;  // most row tiles per (edge, wide layer); sizes the partial-sum buffer
-#ifndef PG_WIDE_STEP
-#define PG_WIDE_STEP 1
-#endif
-#ifndef PG_WIDE_MIN_BLOCKS
-#define PG_WIDE_MIN_BLOCKS 3
-#endif
-constexpr int kPairWideStep = PG_WIDE_STEP;  // rows a cluster handles between two barriers
+constexpr int kPairWideStep = 1;       // rows a cluster handles between two exchanges
+constexpr int kPairWideMinBlocks = 3;  // resident CTAs per SM the cluster sweep is compiled for
 constexpr int kPairWideMaxLd = 8 * 256 * 4 * kPairCluster;  // widest row the cluster variant covers
 constexpr int kEdgeChunks = 32;        // CTAs that share the pair edge step of one (edge, layer)
 
@@ -107,7 +102,6 @@ struct DevState {
     float* Up;           // [edge][up_stride]    pair sweep: partial sums of D^T p
     double* Sp;          // [edge][sp_stride]    pair sweep: partial sums of ||p||^2
     float* Pn;           // [edge][layer]  half-step mode: ||p|| of the last odd iteration
-    int pair_bulk;       // row-per-warp pair sweep fed by bulk asynchronous copies (TMA)
     int dep_launch;      // host only: kernel families (kDep*) launched with programmatic stream serialisation
     int half_odd;        // half-step mode: the update being applied is an odd iteration's,
                          // p q-hat^T = (||p|| / ||q||) p-hat q^T: scale the coefficients accordingly

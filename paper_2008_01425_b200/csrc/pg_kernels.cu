@@ -26,22 +26,9 @@ constexpr int kStatusTimeout = 5;  // PG_ERR_TIMEOUT
 constexpr long long kBarrierSpinLimit = 1LL << 23;   // polls before a grid barrier gives up (a few seconds)
 
 // Rows a warp of the row sweep works on at once, per number of vectors S.
-#ifndef PG_RT1
-#define PG_RT1 4
-#endif
-#ifndef PG_RT2
-#define PG_RT2 4
-#endif
-#ifndef PG_RT4
-#define PG_RT4 2
-#endif
-#ifndef PG_RT8
-#define PG_RT8 2
-#endif
+constexpr int kRowsPerWarp1 = 4, kRowsPerWarp2 = 4, kRowsPerWarp4 = 2, kRowsPerWarp8 = 2;
 // Resident CTAs per SM the row sweep is compiled for (caps its registers).
-#ifndef PG_ROW_MIN_BLOCKS
-#define PG_ROW_MIN_BLOCKS 4
-#endif
+constexpr int kRowMinBlocks = 4;
 
 __device__ __forceinline__ float4 ld_stream(const float* p) {
     float4 v;
@@ -313,7 +300,7 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
 }
 
 template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool GRAD = false>
-__global__ void __launch_bounds__(256, PG_ROW_MIN_BLOCKS)
+__global__ void __launch_bounds__(256, kRowMinBlocks)
 row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
                  const Tile* __restrict__ tiles) {
     grid_dependency_sync();
@@ -853,171 +840,34 @@ __device__ __forceinline__ void pending_of(const DevState& st, const int* __rest
 }
 
 // --------------------------------------------------------------------------
-// Pair sweep (rank 1; a matching, or a static graph of degree <= 2, where the
-// TMA-fed variants below also take rows with two readers).  One CTA owns a block
-// of rows of BOTH ends of an edge (i<j) and reads each row of X_i and X_j once:
+// Pair sweep (rank 1; a matching, or a static graph of degree <= 2, where a row
+// can have two readers).  One CTA owns a block of rows of BOTH ends of an edge
+// (i<j) and reads each row of X_i and X_j once:
 //   - applies the correction that is still pending from the previous step to
-//     each row (each end has its own previous edge) and writes the rows back,
+//     each row (each end has its own previous edges) and writes the rows back,
 //   - forms the row of D = X_i - X_j, its product with q-hat:  p_r = D_r . q-hat,
 //   - accumulates u += p_r D_r, i.e. its share of D^T p, and of ||p||^2.
 // The normalisation is a scalar, so it is applied afterwards by the pair edge
 // step:  p-hat = p / ||p||,  Q' = D^T p-hat = u / ||p||.  This is the same power
 // step as the three-sweep path with X read once instead of twice.
-// A warp keeps a whole row (up to 8 float4 per lane) in registers.
+// Four kernels by row length: a warp per row, a CTA per row (fed by bulk copies
+// where its registers hold the row, by plain loads beyond), a cluster per row.
 // --------------------------------------------------------------------------
-template <int NV, bool UPDATE>
-__global__ void __launch_bounds__(256, 2)
-pair_sweep_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
-                  const Tile* __restrict__ tiles) {
-    grid_dependency_sync();
-    __shared__ __align__(16) float s_q[NV * 128];
-    __shared__ __align__(16) float s_ui[NV * 128];
-    __shared__ __align__(16) float s_uj[NV * 128];
-    __shared__ __align__(16) float s_red[8][NV * 128];
-    __shared__ double s_s[8];
-
-    const Tile tile = tiles[blockIdx.x];
-    const int e = tile.worker;                       // edge index within the current round
-    if (e >= tab_cur[st.tab.off_n_edges]) return;
-    const LayerGeom g = st.layers[tile.layer];
-    const int wi = tab_cur[st.tab.off_edge_i + e], wj = tab_cur[st.tab.off_edge_j + e];
-    const int pair = tab_cur[st.tab.off_pair + e];
-    float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
-    float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
-    const int ld = g.ld;
-
-    // this edge's stored vector (unit length after scaling) and, per end, the
-    // factors of the pending correction
-    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
-    const float qinv = pair_qinv(st, pair, tile.layer);
-    const float* ui = q;
-    const float* uj = q;
-    const float* phi = nullptr;
-    const float* phj = nullptr;
-    float coef_i = 0.0f, coef_j = 0.0f;
-    if (UPDATE) {
-        if (tab_prev[st.tab.off_degree + wi] > 0) {
-            const int ep = tab_prev[st.tab.off_slot_edge + wi * st.tab.max_degree];
-            ui = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
-            phi = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
-            coef_i = __int_as_float(tab_prev[st.tab.off_slot_coef + wi * st.tab.max_degree]);
-        }
-        if (tab_prev[st.tab.off_degree + wj] > 0) {
-            const int ep = tab_prev[st.tab.off_slot_edge + wj * st.tab.max_degree];
-            uj = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
-            phj = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
-            coef_j = __int_as_float(tab_prev[st.tab.off_slot_coef + wj * st.tab.max_degree]);
-        }
-    }
-    for (int idx = threadIdx.x; idx < NV * 128; idx += 256) {
-        const bool in = idx < ld;
-        s_q[idx] = in ? q[idx] * qinv : 0.0f;
-        if (UPDATE) {
-            s_ui[idx] = in ? ui[idx] : 0.0f;
-            s_uj[idx] = in ? uj[idx] : 0.0f;
-        }
-    }
-    __syncthreads();
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int r0 = tile.rtile * g.p_rows;
-    const int r1 = min(g.n, r0 + g.p_rows);
-    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
-    float4 u[NV];
-#pragma unroll
-    for (int k = 0; k < NV; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    float ssum = 0.0f;
-
-    for (int r = r0 + warp; r < r1; r += 8) {
-        float4 xi[NV], xj[NV];
-        float* rowi = Xi + (long long)r * ld;
-        float* rowj = Xj + (long long)r * ld;
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int col = (k * 32 + lane) * 4;
-            if (col < ld) {
-                xi[k] = ld_stream(rowi + col);
-                xj[k] = ld_stream(rowj + col);
-            } else {
-                xi[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-                xj[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        }
-        if (UPDATE) {
-            const float ai = phi ? coef_i * __ldg(phi + r) : 0.0f;
-            const float aj = phj ? coef_j * __ldg(phj + r) : 0.0f;
-#pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const int col = (k * 32 + lane) * 4;
-                const float4 vi = *reinterpret_cast<const float4*>(&s_ui[col]);
-                const float4 vj = *reinterpret_cast<const float4*>(&s_uj[col]);
-                xi[k].x = fmaf(-ai, vi.x, xi[k].x); xi[k].y = fmaf(-ai, vi.y, xi[k].y);
-                xi[k].z = fmaf(-ai, vi.z, xi[k].z); xi[k].w = fmaf(-ai, vi.w, xi[k].w);
-                xj[k].x = fmaf(-aj, vj.x, xj[k].x); xj[k].y = fmaf(-aj, vj.y, xj[k].y);
-                xj[k].z = fmaf(-aj, vj.z, xj[k].z); xj[k].w = fmaf(-aj, vj.w, xj[k].w);
-                if (col < ld) {
-                    st_stream(rowi + col, xi[k]);
-                    st_stream(rowj + col, xj[k]);
-                }
-            }
-        }
-        float dot = 0.0f;
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            const int col = (k * 32 + lane) * 4;
-            const float4 vq = *reinterpret_cast<const float4*>(&s_q[col]);
-            xi[k].x -= xj[k].x; xi[k].y -= xj[k].y; xi[k].z -= xj[k].z; xi[k].w -= xj[k].w;   // row of D
-            dot = fmaf(xi[k].x, vq.x, dot); dot = fmaf(xi[k].y, vq.y, dot);
-            dot = fmaf(xi[k].z, vq.z, dot); dot = fmaf(xi[k].w, vq.w, dot);
-        }
-        const float p = warp_sum(dot);
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            u[k].x = fmaf(p, xi[k].x, u[k].x); u[k].y = fmaf(p, xi[k].y, u[k].y);
-            u[k].z = fmaf(p, xi[k].z, u[k].z); u[k].w = fmaf(p, xi[k].w, u[k].w);
-        }
-        ssum = fmaf(p, p, ssum);
-        if (lane == 0) Pw[r] = p;
-    }
-#pragma unroll
-    for (int k = 0; k < NV; ++k) *reinterpret_cast<float4*>(&s_red[warp][(k * 32 + lane) * 4]) = u[k];
-    if (lane == 0) s_s[warp] = (double)ssum;
-    __syncthreads();
-    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld;
-    for (int idx = threadIdx.x; idx < ld; idx += 256) {
-        float t = s_red[0][idx];
-#pragma unroll
-        for (int w8 = 1; w8 < 8; ++w8) t += s_red[w8][idx];
-        Up[idx] = t;
-    }
-    if (threadIdx.x == 0) {
-        double t = 0.0;
-        for (int w8 = 0; w8 < 8; ++w8) t += s_s[w8];
-        st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = t;
-    }
-}
 
 // --------------------------------------------------------------------------
-// Pair sweep, row-per-warp variant fed by bulk asynchronous copies (TMA).
-// The rows of a tile are contiguous in memory (full rows, padded leading
+// Pair sweep, a warp per row (rows of up to kPairMaxLd floats), fed by bulk
+// asynchronous copies (TMA).  The rows of a tile are contiguous in memory (full rows, padded leading
 // dimension), so one thread moves kBulkRows rows of X_i and of X_j into shared
 // memory with two cp.async.bulk copies per stage; an mbarrier per stage counts
 // the bytes.  kBulkStages stages are in flight, so the loads of the next stages
 // never wait for registers or for the arithmetic of the current one.  Every
-// warp then works on one row of the stage out of shared memory exactly as the
-// register variant does, and writes the corrected rows straight to global
-// memory.  All mbarrier waits are bounded: a wait that runs out raises the
+// warp then takes one row of the stage out of shared memory into registers (up
+// to 8 float4 per lane) and writes the corrected rows straight to global memory.  All mbarrier waits are bounded: a wait that runs out raises the
 // time-out bit of the status word and the CTA leaves after waiting (bounded
 // again) for the copies it still has in flight.
 // --------------------------------------------------------------------------
 constexpr int kBulkRows = 8;      // rows per stage = warps per CTA
-#ifndef PG_BULK_STAGES
-#define PG_BULK_STAGES 3
-#endif
-#ifndef PG_BULK_MIN_BLOCKS
-#define PG_BULK_MIN_BLOCKS 1
-#endif
-constexpr int kBulkStages = PG_BULK_STAGES;
+constexpr int kBulkStages = 3;
 constexpr int kBulkSpinLimit = 1 << 24;
 
 __device__ __forceinline__ unsigned smem_addr(const void* p) {
@@ -1057,7 +907,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
 }
 
 template <int NV, bool UPDATE, int D>
-__global__ void __launch_bounds__(256, PG_BULK_MIN_BLOCKS)
+__global__ void __launch_bounds__(256, 1)
 pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles) {
     grid_dependency_sync();
@@ -1255,7 +1105,7 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 // and the loads of the next rows are issued in between.
 // --------------------------------------------------------------------------
 template <int NVW, bool UPDATE, int D>
-__global__ void __cluster_dims__(kPairCluster, 1, 1) __launch_bounds__(256, PG_WIDE_MIN_BLOCKS)
+__global__ void __cluster_dims__(kPairCluster, 1, 1) __launch_bounds__(256, kPairWideMinBlocks)
 pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles, int slice_pad) {
     grid_dependency_sync();
@@ -1598,14 +1448,8 @@ pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* 
 // --------------------------------------------------------------------------
 constexpr int kMidStagesMax = 4;
 constexpr int kMidBulkNv = 5;     // most float4 per thread and row (registers)
-#ifndef PG_MID_ROWS1
-#define PG_MID_ROWS1 4
-#endif
-#ifndef PG_MID_ROWS2
-#define PG_MID_ROWS2 4
-#endif
 // rows per stage and per barrier: more of them where a row is short
-__host__ __device__ constexpr int mid_rows(int nvm) { return nvm == 1 ? PG_MID_ROWS1 : (nvm == 2 ? PG_MID_ROWS2 : 2); }
+__host__ __device__ constexpr int mid_rows(int nvm) { return nvm <= 2 ? 4 : 2; }
 // two CTAs per SM where the registers allow it, so one CTA's prologue hides behind the other's rows
 __host__ __device__ constexpr int mid_min_blocks(int nvm, int d) { return (1 + 2 * d) * nvm <= 10 ? 2 : 1; }
 
@@ -2369,23 +2213,23 @@ cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, c
     const int slots = st.max_degree * st.rank;
     if (UPDATE && st.G) {     // the update also takes the caller's gradient step
         if (slots <= 1)
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, kRowsPerWarp1, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         else if (slots <= 2)
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, kRowsPerWarp2, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         else if (slots <= 4)
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, kRowsPerWarp4, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         else
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, kRowsPerWarp8, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
         return cudaGetLastError();
     }
     if (slots <= 1)
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, PG_RT1>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, kRowsPerWarp1>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     else if (slots <= 2)
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, PG_RT2>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, kRowsPerWarp2>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     else if (slots <= 4)
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, PG_RT4>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, kRowsPerWarp4>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     else
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, PG_RT8>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
+        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, kRowsPerWarp8>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
     return cudaGetLastError();
 }
 
@@ -2439,37 +2283,16 @@ static cudaError_t launch_pair_bulk(const DevState& st, const int* tab_prev, con
     }
 }
 
-template <bool UPDATE>
-static cudaError_t launch_pair(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
-                               int n_tiles, int nv, cudaStream_t stream) {
-    switch (nv) {
-        case 1: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<1, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-        case 2: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<2, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-        case 3: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<3, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-        case 4: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<4, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-        case 5: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<5, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-        case 6: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<6, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-        case 7: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<7, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-        default: launch_dep(st.dep_launch & kDepPairRow, pair_sweep_kernel<8, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_prev, tab_cur, tiles); break;
-    }
-    return cudaGetLastError();
-}
-
 // `tiles` must list tiles of layers with the same number of float4 per lane
 // (ceil(ld / 128)); the host launches one group per value.
 // pend_slots: how many corrections can be pending at a worker (its largest degree).
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
                               const Tile* tiles, int n_tiles, int nv, int pend_slots, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
-    if (st.pair_bulk) {
-        if (!apply_pending) return launch_pair_bulk<false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
-        if (pend_slots > 2) return cudaErrorInvalidValue;
-        return pend_slots > 1 ? launch_pair_bulk<true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
-                              : launch_pair_bulk<true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
-    }
-    if (pend_slots > 1) return cudaErrorInvalidValue;     // the register-fed variant holds one correction per end
-    return apply_pending ? launch_pair<true>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
-                         : launch_pair<false>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (!apply_pending) return launch_pair_bulk<false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (pend_slots > 2) return cudaErrorInvalidValue;
+    return pend_slots > 1 ? launch_pair_bulk<true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
+                          : launch_pair_bulk<true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
 }
 
 template <int NVW, bool UPDATE, int D>
@@ -2600,7 +2423,7 @@ static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const i
         // leave room for the second CTA where the kernel is built for two per SM
         const size_t budget = kMidSmemBudget / mid_min_blocks(NVM, D);
         const int n_stage = (int)std::min<size_t>(budget / stage, kMidStagesMax);
-        if (st.pair_bulk && n_stage >= 2) {
+        if (n_stage >= 2) {
             const size_t total = n_stage * stage;
             cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_bulk_kernel<NVM, UPDATE, D>,
                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
@@ -2758,12 +2581,12 @@ cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* ro
     const int slots = st.max_degree * st.rank;
     const int max_blocks = n_rows > n_cols ? n_rows : n_cols;
     if (slots <= 1)
-        return launch_persistent_t<1, PG_RT1>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+        return launch_persistent_t<1, kRowsPerWarp1>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
     if (slots <= 2)
-        return launch_persistent_t<2, PG_RT2>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+        return launch_persistent_t<2, kRowsPerWarp2>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
     if (slots <= 4)
-        return launch_persistent_t<4, PG_RT4>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
-    return launch_persistent_t<8, PG_RT8>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+        return launch_persistent_t<4, kRowsPerWarp4>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+    return launch_persistent_t<8, kRowsPerWarp8>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
 }
 
 cudaError_t launch_barrier_timeout_probe(int* bar, int* status, cudaStream_t stream) {

@@ -38,6 +38,9 @@ def load_both(w: wl.Workload, oracle, net) -> None:
                 net.pg_write_params(i, l, x)
 
 
+FP32_FLOOR = 5e-7     # an error of this part of ||X|| is a few units in the last place of the fp32 values X is stored in
+
+
 def relative_errors(w: wl.Workload, oracle, net, x0=None):
     """Two figures per (worker, layer), each returned as (maximum, where):
 
@@ -47,6 +50,9 @@ def relative_errors(w: wl.Workload, oracle, net, x0=None):
                 or the caller's `x0[worker][layer]`, e.g. the state of the last
                 re-basing).  On stacks whose workers share a large common part this
                 is the stricter figure, because one round moves only a small part of ||X||.
+                Matrices whose on_x is below FP32_FLOOR are left out of this maximum:
+                their error is already at the resolution X is stored with, and once
+                the workers nearly agree a few rounds change less than that.
     """
     on_x, on_change = (0.0, None), (0.0, None)
     for i in range(w.n_workers):
@@ -60,7 +66,7 @@ def relative_errors(w: wl.Workload, oracle, net, x0=None):
             b = diff / moved if moved > 0.0 else (0.0 if diff == 0.0 else np.inf)
             if not np.isfinite(a) or a > on_x[0]:
                 on_x = (float(a), (i, l))
-            if not np.isfinite(b) or b > on_change[0]:
+            if a > FP32_FLOOR and (not np.isfinite(b) or b > on_change[0]):
                 on_change = (float(b), (i, l))
     return on_x, on_change
 

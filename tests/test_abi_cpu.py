@@ -129,3 +129,49 @@ def test_initial_vectors_match_the_checker_bit_for_bit():
     for (seed, i, j, layer, col, m) in [(0, 0, 1, 0, 0, 1), (1005, 3, 17, 7, 0, 28000), (1004, 0, 15, 12, 1, 4608),
                                          (2 ** 63 + 11, 30, 31, 2, 3, 651), (1, 0, 1, 0, 0, 27)]:
         assert np.array_equal(pg.pg_initial_vector(seed, i, j, layer, col, m), po.init_q(seed, i, j, layer, col, m))
+
+
+# --------------------------------------------------------------------------
+# communication volume (host-only call)
+# --------------------------------------------------------------------------
+def _golden(name):
+    rows = []
+    with open(os.path.join(ROOT, "tests", "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line.split())
+    return rows
+
+
+def test_comm_floats_reproduce_the_printed_per_tensor_ratios():
+    """Appendix, parameter tables: rank-1 PowerGossip with r iterations compresses an
+    n x m tensor n*m / ((n+m)/2) / r times; the tables print that ratio rounded ("115/r x")."""
+    for n, m, printed in _golden("compression_ratios.txt"):
+        n, m, printed = int(n), int(m), int(printed)
+        two, dense = pg.pg_comm_floats([(n, m)], 1, 1, 2)           # an odd and an even iteration
+        assert dense == n * m and two == n + m
+        assert round(dense / (two / 2)) == printed
+        odd, _ = pg.pg_comm_floats([(n, m)], 1, 1, 1)
+        even, _ = pg.pg_comm_floats([(n, m)], 1, 2, 1)
+        assert (odd, even) == (n, m)                                 # p has `rows` entries, the transposed step `cols`
+        assert pg.pg_comm_floats([(n, m)], 3, 4, 5)[0] == 3 * (2 * n + 3 * m)   # k = 4..8: three even, two odd
+    with pytest.raises(pg.PowerGossipError):
+        pg.pg_comm_floats([(4, 4)], 1, 0, 1)
+
+
+def test_comm_floats_reproduce_the_printed_whole_model_ratios():
+    """Result tables: bytes sent per epoch of PowerGossip against D-PSGD.  Every message carries
+    the matrices' vectors plus the 1-D tensors uncompressed, so the ratio is
+    (dense + bias) / (iterations x mean floats per iteration + bias)."""
+    lstm_paper = ((28869, 650),) + ((2600, 650),) * 6      # the paper's own LSTM table (tied decoder)
+    for model, iterations, printed, bias_bytes in _golden("comm_volume.txt"):
+        shapes = wl.RESNET20_SHAPES if model == "resnet20" else lstm_paper
+        iterations, printed, bias_bytes = int(iterations), int(printed), int(bias_bytes)
+        two, dense = pg.pg_comm_floats(shapes, 1, 1, 2)
+        sent_bytes = 4.0 * iterations * two / 2 + bias_bytes
+        ratio = (4.0 * dense + bias_bytes) / sent_bytes
+        if model == "resnet20":
+            assert round(ratio) == printed, (model, iterations, ratio)
+        else:
+            assert abs(ratio / printed - 1.0) < 0.025, (model, iterations, ratio)

@@ -30,6 +30,7 @@ pytestmark = pytest.mark.gpu
 
 REL_TOL = 1e-4
 CHANGE_TOL = 1e-3            # the same error against ||X_ref - X_start||_F, what the rounds changed
+                             # (matrices whose error is below common.FP32_FLOOR of ||X|| are exempt)
 AVG_TOL = 1e-5
 SEGMENT_POWER_STEPS = 8      # re-base at least this often (in power steps)
 
@@ -48,7 +49,20 @@ def _check_average(w, net, avg0):
         assert drift <= AVG_TOL, "layer %d: average drift %.3e" % (l, drift)
 
 
-def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance_tol=0.05):
+ENVELOPE = 8.0               # the GPU may drift this many times further than fp32 storage alone
+
+
+def _gap(w, a, b):
+    """max over (worker, layer) of ||X_a - X_b||_F / ||X_b||_F between two CPU checkers."""
+    worst = 0.0
+    for i in range(w.n_workers):
+        for l in range(len(w.layer_shapes)):
+            ref = b.get_params(i, l)
+            worst = max(worst, float(np.linalg.norm(a.get_params(i, l) - ref) / max(np.linalg.norm(ref), 1e-300)))
+    return worst
+
+
+def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance_tol=0.05, envelope=False):
     """Run `rounds` rounds on both sides.
 
     free-running (rebased=False): assert 1e-4 (on ||X||) and 1e-3 (on what the rounds
@@ -56,6 +70,10 @@ def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance
     rounds); past the horizon only the invariants.
     rebased=True: re-base every SEGMENT_POWER_STEPS power steps, assert both figures at
     the end of every segment, the second one against the state the segment started from.
+    envelope=True (free-running): a second fp64 checker runs beside the first with its state
+    rounded to fp32 after every power step, the least any fp32-storage implementation of
+    Algorithm 2 perturbs the iteration.  At the full round count the GPU's distance from the
+    untouched fp64 run must be within 1e-4, or within ENVELOPE times that checker's distance.
     One line per run with the largest of either figure goes to the end of the pytest log.
     """
     from paper_2008_01425_b200 import binding as pg
@@ -65,6 +83,11 @@ def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance
     oracle = common.oracle_for(w)
     net = common.network_for(w)
     common.load_both(w, oracle, net)
+    shadow = None
+    if envelope:
+        shadow = common.oracle_for(w)
+        shadow.set_fp32_storage()
+        common.load_both(w, shadow, None)
     _check_schedules(oracle, net, rounds)
     avg0 = [common.initial_average(w, l) for l in range(len(w.layer_shapes))]
     if rebased:
@@ -78,6 +101,8 @@ def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance
             pairs.update((int(a), int(b)) for a, b in oracle.round_schedule(t)[0])
             net.pg_round()
         oracle.round(step)
+        if shadow is not None:
+            shadow.round(step)
         done += step
         if rebased or done <= horizon:
             (err, where), (err_c, where_c) = common.relative_errors(w, oracle, net, start)
@@ -94,12 +119,19 @@ def _run(w, rounds=None, check_every=None, horizon=None, rebased=False, distance
         d_ref, d_gpu = oracle.consensus_distance(), common.gpu_consensus_distance(w, net)
         assert abs(d_gpu - d_ref) <= distance_tol * d_ref, (d_gpu, d_ref)
     note = ""
+    if shadow is not None:
+        gap_gpu, where = common.max_relative_error(w, oracle, net)
+        gap_shadow = _gap(w, shadow, oracle)
+        assert gap_gpu <= max(REL_TOL, ENVELOPE * gap_shadow), (gap_gpu, gap_shadow, where)
+        note += "; at round %d: GPU %.2e from the fp64 run, fp64 arithmetic with fp32 storage %.2e" % (
+            rounds, gap_gpu, gap_shadow)
+        shadow.close()
     if w.rank > 1 and all(min(n, m) >= w.rank for n, m in w.layer_shapes):
         # no Gram-Schmidt residual came near the dependent-column threshold (1e-10): both sides
         # took the same decisions whatever the threshold's exact value
         smallest = oracle.min_residual_ratio()
         assert smallest > 1e-8, smallest
-        note = ", smallest residual ratio %.1e" % smallest
+        note += ", smallest residual ratio %.1e" % smallest
     common.PARITY_LINES.append(
         "%-34s rank %d %s %3d rounds: max error %.2e of ||X||, %.2e of the change%s"
         % (w.name, w.rank, "re-based" if rebased else "free-run", rounds, worst_x, worst_change,
@@ -115,7 +147,7 @@ def test_config1_tiny_ring():
 
 def test_config2_resnet20_ring8_free_running():
     """All 100 rounds; the fp64 trajectory can be followed to 1e-4 for 20 rounds."""
-    _run(wl.resnet20_ring8(), check_every=10, horizon=20)
+    _run(wl.resnet20_ring8(), check_every=10, horizon=20, envelope=True)
 
 
 def test_config2_resnet20_ring8_rebased():
@@ -131,12 +163,12 @@ def test_config3_torus_small_rebased(power_steps):
 @pytest.mark.parametrize("power_steps", [1, 2, 4])
 def test_config3_torus_small_free_running(power_steps):
     w = wl.shrink(wl.torus8x8(power_steps), [(200, 136)], 200)
-    _run(w, check_every=max(1, 20 // power_steps), horizon=20 // power_steps)
+    _run(w, check_every=max(1, 20 // power_steps), horizon=20 // power_steps, envelope=True)
 
 
 def test_config3_torus_full_size_free_running():
     w = wl.torus8x8(1)
-    _run(w, check_every=20, horizon=20)
+    _run(w, check_every=20, horizon=20, envelope=True)
 
 
 @pytest.mark.parametrize("power_steps", [1, 2, 4])
@@ -152,6 +184,13 @@ def test_config4_vgg16_ring16_full_size(rank):
 
 
 @pytest.mark.parametrize("rank", [1, 2])
+def test_config4_vgg16_ring16_full_size_free_running(rank):
+    """All 50 rounds without contact: 1e-4 asserted over the first rounds, then the invariants
+    and the fp32-storage envelope."""
+    _run(wl.vgg16_ring16(rank), check_every=5, horizon=5, envelope=True)
+
+
+@pytest.mark.parametrize("rank", [1, 2])
 def test_config4_vgg16_small_rebased(rank):
     """VGG-shaped stack with every layer shrunk 8x per side: all 50 rounds."""
     shapes = [(max(n // 8, 3), max(m // 8, 5)) for n, m in wl.VGG16_SHAPES]
@@ -161,7 +200,7 @@ def test_config4_vgg16_small_rebased(rank):
 @pytest.mark.parametrize("rank", [1, 2])
 def test_config4_vgg16_small_free_running(rank):
     shapes = [(max(n // 8, 3), max(m // 8, 5)) for n, m in wl.VGG16_SHAPES]
-    _run(wl.shrink(wl.vgg16_ring16(rank), shapes, 50), check_every=5, horizon=5)
+    _run(wl.shrink(wl.vgg16_ring16(rank), shapes, 50), check_every=5, horizon=5, envelope=True)
 
 
 def test_config5_lstm_matching_small():
@@ -363,6 +402,57 @@ def test_initial_vectors_on_device_are_the_seeded_ones():
     net.close()
 
 
+def test_communication_volume_of_a_round():
+    """pg_comm_floats_round: both ends of every edge of the round send rank * rows floats per odd
+    iteration of Algorithm 2 and rank * cols per even one, summed over the layers."""
+    shapes = ((64, 32), (9, 5))
+    rows, cols, dense = 64 + 9, 32 + 5, 64 * 32 + 9 * 5
+    ring = wl.tiny_ring().replace(layer_shapes=shapes, rank=2, power_steps=3)
+    net = common.network_for(ring)
+    ends = 2 * 4                                            # ring of 4: four edges
+    assert net.pg_comm_floats_round(0) == (ends * 2 * 3 * (rows + cols), ends * dense)
+    assert net.pg_comm_floats_round(7) == net.pg_comm_floats_round(0)
+    net.close()
+    half = common.network_for(ring.replace(rank=1))
+    half.pg_set_half_step()                                  # three iterations a round: k = 1, 2, 3, then 4, 5, 6
+    assert half.pg_comm_floats_round(0)[0] == ends * (2 * rows + cols)
+    assert half.pg_comm_floats_round(1)[0] == ends * (rows + 2 * cols)
+    half.close()
+    for mode, per_step in ((1, rows), (2, cols)):
+        rp = common.network_for(ring)
+        rp.pg_set_random_projection(mode)
+        assert rp.pg_comm_floats_round(0)[0] == ends * 2 * 3 * per_step
+        rp.close()
+    match = common.network_for(wl.shrink(wl.lstm_matching32(), shapes, 1).replace(n_workers=6))
+    assert match.pg_comm_floats_round(3) == (6 * (rows + cols), 6 * dense)       # three pairs, six ends
+    match.close()
+
+
+def test_set_round_on_the_stream_of_the_rounds():
+    """A correction still pending when the round counter is set is applied on the stream the
+    caller names; with the rounds on a non-blocking stream the result is that of the default one."""
+    import torch
+
+    w = wl.Workload("ring_set_round", 9, 5, wl.RING, 0, 0, wl.W_UNIFORM, None, ((70, 130), (24, 1500)), 1, 1, 4, 3,
+                    "normal1")
+    results = []
+    for stream in (None, torch.cuda.Stream()):
+        net = common.network_for(w)
+        common.load_both(w, None, net)
+        if stream is not None:
+            stream.wait_stream(torch.cuda.current_stream())
+        for _ in range(3):
+            net.pg_round(stream)
+        net.pg_set_round(1, stream)            # flushes the pending correction, then replays round 1's counter
+        net.pg_round(stream)
+        assert net.pg_get_round() == 2
+        results.append(net.read_all(stream))
+        net.close()
+    for i in range(w.n_workers):
+        for l in range(2):
+            assert np.array_equal(results[0][i][l], results[1][i][l])
+
+
 # ---- one cooperative launch for many rounds (small stacks) --------------------
 PERSISTENT_CASES = [
     wl.tiny_ring(),
@@ -450,6 +540,12 @@ def test_grid_barrier_gives_up_instead_of_hanging():
     w = wl.tiny_ring()
     net = common.network_for(w)
     assert net.pg_selftest_barrier_timeout() == pg.PG_ERR_TIMEOUT
+    # a context that saw a time-out runs no further round: its state may be mid-step
+    for call in (net.pg_round, lambda: net.pg_rounds(3), lambda: net.pg_set_round(0)):
+        with pytest.raises(pg.PowerGossipError) as e:
+            call()
+        assert e.value.status == pg.PG_ERR_STATE
+    assert net.pg_device_status() == pg.PG_ERR_TIMEOUT          # sticky
     net.close()
     other = common.network_for(w)          # the device still works
     common.load_both(w, None, other)
