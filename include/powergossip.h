@@ -384,6 +384,16 @@ enum {
     PG_KERNEL_KINDS = 8
 };
 PG_API int pg_timing_enable(pg_ctx *ctx, int32_t on);
+/*
+ * Algorithmic bytes of X that one steady-state round of this context moves (measurement
+ * aid): per power step and parameter 8 B on layers the pair sweep takes (read once, written
+ * once), 12 B on the three sweeps (read for the transposed product, read and written by the
+ * update whose read doubles as the next forward product); 8 B per iteration in half-step
+ * mode, 12 B per step with random projections.  *pair_fraction_out (may be NULL): share of
+ * the parameters on the pair sweep.  Vectors and partial sums (under 1 %) are not counted.
+ */
+PG_API int pg_round_bytes(pg_ctx *ctx, double *bytes_out, double *pair_fraction_out);
+
 PG_API int pg_timing_read(pg_ctx *ctx, double *ms_out, int64_t *launches_out, double *bytes_out);
 
 /*

@@ -840,6 +840,16 @@ double pgo_compression_ratio(int n, int m, int rank, int iterations)
     return (double)n * (double)m / sent;
 }
 
+/* Threads the parallel loops use from now on (timing aid; results do not depend on it). */
+void pgo_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 int pgo_num_threads(void)
 {
 #ifdef _OPENMP

@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.pgo_min_residual_ratio.restype = c_dbl
         L.pgo_set_fp32_storage.argtypes = [vp, c_int]
         L.pgo_set_fp32_storage.restype = c_int
+        L.pgo_set_num_threads.argtypes = [c_int]
+        L.pgo_set_num_threads.restype = None
         L.pgo_num_threads.argtypes = []
         L.pgo_num_threads.restype = c_int
         _lib = L
@@ -150,6 +152,11 @@ def compression_ratio(n: int, m: int, rank: int = 1, iterations: int = 1) -> flo
 
 def num_threads() -> int:
     return int(lib().pgo_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    """Threads the checker's parallel loops use from now on (timing only)."""
+    lib().pgo_set_num_threads(int(n))
 
 
 RANDOM_RIGHT, RANDOM_LEFT = 1, 2

@@ -29,6 +29,7 @@ EXPORTS = (
     "pg_transposed_product_noalloc", "pg_rounds", "pg_selftest_barrier_timeout",
     "pg_set_half_step", "pg_params_device", "pg_set_random_projection",
     "pg_round_sgd", "pg_stack_elems", "pg_stack_offset", "pg_comm_floats", "pg_comm_floats_round",
+    "pg_round_bytes",
 )
 PG_POWER_ITERATION, PG_RANDOM_RIGHT, PG_RANDOM_LEFT = 0, 1, 2
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
@@ -99,6 +100,7 @@ def load_library() -> ctypes.CDLL:
     L.pg_comm_floats.argtypes = [ctypes.POINTER(pg_layer_shape), i32, i32, i64, i64, ctypes.POINTER(i64),
                                  ctypes.POINTER(i64)]
     L.pg_comm_floats_round.argtypes = [vp, i64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    L.pg_round_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]
     L.pg_status_string.argtypes = [ctypes.c_int]
     L.pg_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -388,6 +390,12 @@ class PowerGossip:
         r = ctypes.c_int64(0)
         _check(self._lib.pg_kernel_launches(self._h, ctypes.byref(r)), "pg_kernel_launches")
         return int(r.value)
+
+    def pg_round_bytes(self) -> Tuple[float, float]:
+        """(algorithmic bytes of X one steady-state round moves, share of the parameters on the pair sweep)."""
+        b, f = ctypes.c_double(0.0), ctypes.c_double(0.0)
+        _check(self._lib.pg_round_bytes(self._h, ctypes.byref(b), ctypes.byref(f)), "pg_round_bytes")
+        return float(b.value), float(f.value)
 
     def pg_timing_enable(self, on: bool) -> None:
         _check(self._lib.pg_timing_enable(self._h, 1 if on else 0), "pg_timing_enable")

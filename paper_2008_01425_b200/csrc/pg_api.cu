@@ -1506,6 +1506,17 @@ int pg_set_round(pg_ctx* c, int64_t round, void* stream_v) {
     return PG_OK;
 }
 
+int pg_round_bytes(pg_ctx* c, double* bytes_out, double* pair_fraction_out) {
+    if (!c || !bytes_out) return PG_ERR_INVALID;
+    // normal_param_bytes / pair_param_bytes: 4 B x the parameters on either path
+    const double per_step = c->half_step ? 2.0 * c->normal_param_bytes
+                                         : 3.0 * c->normal_param_bytes + 2.0 * c->pair_param_bytes;
+    *bytes_out = per_step * c->power_steps;
+    const double all = c->normal_param_bytes + c->pair_param_bytes;
+    if (pair_fraction_out) *pair_fraction_out = all > 0.0 ? c->pair_param_bytes / all : 0.0;
+    return PG_OK;
+}
+
 int pg_timing_enable(pg_ctx* c, int32_t on) {
     if (!c) return PG_ERR_INVALID;
     c->timing = on != 0;
