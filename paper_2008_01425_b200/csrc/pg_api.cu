@@ -36,7 +36,9 @@ struct Layout {
     long long n_pairs = 0;
     bool pair_mode = false;        // rank 1 and degree <= 2: layers run through the pair sweep
     int pend_slots = 1;            // corrections that can be pending at a worker in pair mode (its degree)
-    bool two_copies = false;       // pair mode on a graph of degree 2: the sweep writes to a second copy of X
+    bool two_copies = false;       // pair mode on a static graph where rows have several readers: the sweep writes
+                                   // to a second copy of X, and the pair vectors live in two copies as well
+    bool single_owner = false;     // there, no edge has to write the rows of both of its ends
     bool small_stack = false;      // at most 48 MiB of parameters: the latency regime
     long long n_pair_tiles = 0, n_flush_tiles = 0;
     long long row_tile_cap = 0, col_tile_cap = 0;   // room for the lists with every layer on the three-sweep path
@@ -44,7 +46,7 @@ struct Layout {
     int max_edges = 0, max_degree = 0;
     TabLayout tab{};
     long long n_row_tiles = 0, n_col_tiles = 0;
-    size_t off_Qn2 = 0, off_Pn = 0, off_edge_tab = 0, off_stage = 0;
+    size_t off_Qn2 = 0, off_Pn = 0, off_edge_tab = 0, off_stage = 0, off_Q2 = 0;
     long long stage_elems = 0;     // largest dense matrix whose rows need padding on upload
     size_t off_X = 0, off_Q = 0, off_Qinv = 0, off_Y = 0, off_Ph = 0, off_Z = 0, off_live = 0,
            off_Up = 0, off_Sp = 0, off_pair_tiles = 0, off_flush_tiles = 0, off_status = 0, off_layers = 0, off_tabs = 0, off_row_tiles = 0, off_col_tiles = 0;
@@ -123,6 +125,62 @@ int dependent_launch_mask(bool small_stack, bool two_streams) {
     return pg::kDepSweep | pg::kDepPairRow | pg::kDepPairMid | (small_stack ? pg::kDepPairEdge : 0);
 }
 
+// Which edge writes a worker's corrected rows in the pair sweep: every worker gets exactly one of
+// its edges.  Where possible no edge gets both of its ends (a bipartite matching of workers to
+// incident edges by augmenting paths; it exists unless a component of the graph is a tree), so that
+// the sweep's CTAs all do about the same work; the rest fall back to the worker's first edge.
+// own[e]: bit 0 = the smaller end, bit 1 = the larger end.  Returns true if no edge has both bits.
+bool assign_owners(int n_workers, const std::vector<Edge>& edges, std::vector<int>& own) {
+    const int E = static_cast<int>(edges.size());
+    std::vector<std::vector<int>> incident(n_workers);
+    for (int e = 0; e < E; ++e) {
+        incident[edges[e].i].push_back(e);
+        incident[edges[e].j].push_back(e);
+    }
+    std::vector<int> edge_owner(E, -1), worker_edge(n_workers, -1), seen(E, -1);
+    // iterative augmenting path search from worker `root`
+    auto augment = [&](int root) {
+        std::vector<int> stack_w{root}, stack_pos{0}, via;     // via[d]: edge taken at depth d
+        while (!stack_w.empty()) {
+            const int w = stack_w.back();
+            int& pos = stack_pos.back();
+            if (pos >= static_cast<int>(incident[w].size())) {
+                stack_w.pop_back();
+                stack_pos.pop_back();
+                if (!via.empty()) via.pop_back();
+                continue;
+            }
+            const int e = incident[w][pos++];
+            if (seen[e] == root) continue;
+            seen[e] = root;
+            if (edge_owner[e] < 0) {                           // free edge: flip the path
+                via.push_back(e);
+                for (size_t d = 0; d < via.size(); ++d) {
+                    edge_owner[via[d]] = stack_w[d];
+                    worker_edge[stack_w[d]] = via[d];
+                }
+                return true;
+            }
+            via.push_back(e);
+            stack_w.push_back(edge_owner[e]);
+            stack_pos.push_back(0);
+        }
+        return false;
+    };
+    bool single = true;
+    for (int w = 0; w < n_workers; ++w)
+        if (!incident[w].empty() && !augment(w)) single = false;
+    own.assign(E, 0);
+    for (int w = 0; w < n_workers; ++w) {
+        if (incident[w].empty()) continue;
+        const int e = worker_edge[w] >= 0 ? worker_edge[w] : incident[w][0];
+        own[e] |= edges[e].i == w ? 1 : 2;
+    }
+    for (int e = 0; e < E; ++e)
+        if (own[e] == 3) single = false;
+    return single;
+}
+
 int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_layers, int rank,
                 Layout& lay, bool query_device = false) {
     if (!shapes || n_layers < 1 || n_layers > 4096) return PG_ERR_INVALID;
@@ -143,21 +201,28 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     lay.pair_mode = false;
     lay.pend_slots = 1;
     lay.two_copies = false;
+    lay.single_owner = false;
     if (rank <= 2 && pair_sweep_allowed()) {
         if (lay.max_degree == 1) {
             lay.pair_mode = rank == 1;
-        } else if (lay.max_degree == 2 && topo.kind != PG_MATCHING) {
+        } else if (topo.kind != PG_MATCHING && (lay.max_degree == 2 || (rank == 1 && lay.max_degree <= 4))) {
+            // Rows with several readers: the sweep forms the difference from the rows as stored, only the
+            // edge that owns a worker corrects and writes its rows (to the second copy), and the pending
+            // terms enter as vector algebra.  Degree 3 and 4 (a torus) need an assignment in which no edge
+            // owns both of its ends.
             std::vector<Edge> edges;
             if (!pg::build_edges(topo, 0, 0, edges)) return PG_ERR_INVALID;
-            std::vector<int> degree(N, 0);
+            std::vector<int> degree(N, 0), own;
             for (const Edge& ed : edges) {
                 degree[ed.i] += 1;
                 degree[ed.j] += 1;
             }
-            if (*std::min_element(degree.begin(), degree.end()) >= 1) {
+            const bool single = assign_owners(N, edges, own);
+            if (*std::min_element(degree.begin(), degree.end()) >= 1 && (lay.max_degree == 2 || single)) {
                 lay.pair_mode = true;
-                lay.pend_slots = 2;
+                lay.pend_slots = lay.max_degree;
                 lay.two_copies = true;
+                lay.single_owner = single;
             }
         }
     }
@@ -184,7 +249,12 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         const bool large_layer = rows >= 256 && static_cast<long long>(rows) * ld >= (1LL << 20);
         if (lay.two_copies && !small_stack && !large_layer) mode = 0;
         if (rank == 2 && !(mode == 3 && large_layer && ld <= pg::kPairMid2MaxLd)) mode = 0;
+        if (lay.pend_slots > 2 && mode != 1) mode = 0;      // degree 3 and 4: the row-per-warp kernel only
         return mode;
+    };
+    // the raw form (see LayerGeom::raw) exists for a row per warp and for the TMA-fed CTA-per-row kernel at rank 1
+    auto raw_of = [&](int mode, int ld) {
+        return lay.two_copies && rank == 1 && (mode == 1 || (mode == 3 && ld <= 5 * 1024)) ? 1 : 0;
     };
     // rows the CTA-per-row sweep covers on a large stack with two readers per row (one launch a step)
     long long shared_launch_rows = 0;
@@ -226,6 +296,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         ph += round_up(static_cast<long long>(rank) * g.npad, 64);
         z += round_up(static_cast<long long>(slots) * g.t_rtiles * g.ld, 64);
         g.pair_mode = pair_mode_of(g.n, g.ld);
+        g.raw = raw_of(g.pair_mode, g.ld);
         g.p_slice = static_cast<int>(round_up((g.ld + pg::kPairCluster - 1) / pg::kPairCluster, 4));
         {   // equal tiles of at most kPairTileRows rows (a multiple of 8: one row per warp and stage);
             // on graphs of degree 2 short matrices are cut finer, down to 16 rows, so that a layer gives
@@ -268,9 +339,9 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         if (g.pair_mode != 0) {
             // wide layers: room for any tile count the device query may choose
             const int max_tiles = g.pair_mode == 2 ? pg::kPairWideMaxTiles : g.p_rtiles;
-            // per tile: `rank` vectors of D^T P, and ||p||^2 (rank 1) or the Gram matrix P^T P (rank 2, 4 doubles)
+            // per tile: `rank` vectors of D^T P, and kSpPerTile scalars (||p||^2 or P^T P, the pending terms' products)
             up += round_up(static_cast<long long>(max_tiles) * rank * g.ld, 64);
-            sp += round_up(static_cast<long long>(max_tiles) * (rank == 1 ? 1 : 4), 8);
+            sp += static_cast<long long>(max_tiles) * pg::kSpPerTile;
             lay.n_pair_tiles += static_cast<long long>(lay.max_edges) * max_tiles;
             lay.n_flush_tiles += static_cast<long long>(N) * g.f_rtiles * g.f_csplit;
         } else {
@@ -278,7 +349,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
             lay.n_col_tiles += static_cast<long long>(N) * g.t_rtiles * g.t_ctiles;
         }
     }
-    if (rank == 2 && lay.n_pair_tiles == 0) {   // no layer for the rank-2 sweep: plain three-sweep context
+    if (lay.two_copies && lay.n_pair_tiles == 0) {   // no layer for the pair sweep: plain three-sweep context
         lay.pair_mode = false;
         lay.pend_slots = 1;
         lay.two_copies = false;
@@ -309,6 +380,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     t.off_degree = o; o += N;
     t.off_slot_edge = o; o += N * lay.max_degree;
     t.off_slot_coef = o; o += N * lay.max_degree;
+    t.off_own = o; o += lay.max_edges;
     t.total_ints = static_cast<int>(round_up(o, 64));
 
     size_t off = 0;
@@ -319,6 +391,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     };
     lay.off_X = take(sizeof(float) * static_cast<size_t>(N) * lay.x_stride * (lay.two_copies ? 2 : 1));
     lay.off_Q = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride);
+    lay.off_Q2 = take(lay.two_copies ? sizeof(float) * static_cast<size_t>(lay.n_pairs) * lay.q_stride : 0);
     lay.off_Qinv = take(sizeof(float) * static_cast<size_t>(lay.n_pairs) * n_layers * rank);
     lay.off_Qn2 = take(sizeof(double) * static_cast<size_t>(lay.n_pairs) * n_layers * rank * pg::kEdgeChunks);
     lay.off_Pn = take(sizeof(float) * static_cast<size_t>(lay.max_edges) * n_layers);
@@ -371,10 +444,13 @@ struct pg_ctx {
     bool loop_failed = false;
     int64_t step = 0;           // power steps enqueued so far (selects the P-hat buffer)
     float* ph_buf[2] = {nullptr, nullptr};
+    // pair-sweep layers whose rows have several readers: step s reads the pair vectors in q_buf[s & 1]
+    // and writes the new ones to the other copy (both point at the one copy otherwise)
+    float* q_buf[2] = {nullptr, nullptr};
     Tile* d_pair_tiles = nullptr;
     Tile* d_flush_tiles = nullptr;
     // slice: widest per-CTA column slice (mode 2) or widest padded row (mode 3) in the group
-    struct PairGroup { int mode; int nv; int slice; int first; int count; double bytes; };
+    struct PairGroup { int mode; int nv; int slice; int first; int count; double bytes; bool raw; };
     std::vector<PairGroup> pair_groups;   // pair tiles grouped by float4 per lane
     int64_t launches = 0;
     char* ws = nullptr;
@@ -425,6 +501,13 @@ int fill_table(pg_ctx* c, int64_t round, int* tab) {
         std::memcpy(&tab[t.off_w + e], &w[e], sizeof(float));
         tab[t.off_slot_i + e] = slots.slot_at_i[e];
         tab[t.off_slot_j + e] = slots.slot_at_j[e];
+    }
+    {
+        // who writes a worker's corrected rows in the pair sweep: on a matching the one edge of either
+        // end; elsewhere an assignment of workers to incident edges, spread over the edges where possible
+        std::vector<int> own(edges.size(), 3);
+        if (c->lay.two_copies) assign_owners(c->topo.n_workers, edges, own);
+        for (size_t e = 0; e < edges.size(); ++e) tab[t.off_own + e] = own[e];
     }
     for (int v = 0; v < c->topo.n_workers; ++v) {
         if (slots.degree[v] > t.max_degree) return PG_ERR_INVALID;
@@ -516,6 +599,7 @@ int flush_pending(pg_ctx* c, cudaStream_t stream, const float* G = nullptr, floa
     if (rc != PG_OK) return rc;
     DevState st = c->st;
     st.Ph = c->ph_buf[(c->step + 1) & 1];
+    st.Q = c->q_buf[c->step & 1];     // the vectors the last step stored (the flush tiles are pair-sweep layers)
     // the corrected stack always lands in the first copy of X, the one the caller sees
     st.X = c->st.X + c->xbuf * static_cast<long long>(c->topo.n_workers) * c->lay.x_stride;
     st.Xw = c->st.X;
@@ -602,7 +686,7 @@ bool upload_tile_lists(pg_ctx* c) {
         for (int l = l0; l < n_layers; ++l) {
             const LayerGeom& g = lay.layers[l];
             int nv = 0, slice = 0;
-            if (!g.pair_mode || done[l] || g.pair_mode != lay.layers[l0].pair_mode) continue;
+            if (!g.pair_mode || done[l] || g.pair_mode != lay.layers[l0].pair_mode || g.raw != lay.layers[l0].raw) continue;
             group_of(g, &nv, &slice);
             if (nv != nv0) continue;
             slice0 = std::max(slice0, slice);     // sizes the shared-memory vectors of the launch
@@ -618,14 +702,15 @@ bool upload_tile_lists(pg_ctx* c) {
             bytes += 8.0 * N * static_cast<double>(g.n) * g.m;
         }
         const int count = static_cast<int>(pairs.size()) - first;
-        c->pair_groups.push_back(pg_ctx::PairGroup{lay.layers[l0].pair_mode, nv0, slice0, first, count, bytes});
+        c->pair_groups.push_back(pg_ctx::PairGroup{lay.layers[l0].pair_mode, nv0, slice0, first, count, bytes,
+                                                   lay.layers[l0].raw != 0});
     }
     // a group with fewer than two tiles per SM joins the next group of its kind with longer rows
     // (the kernels take any row up to their template's width): fewer, fuller launches
     {
         std::vector<pg_ctx::PairGroup>& gr = c->pair_groups;
         std::stable_sort(gr.begin(), gr.end(), [](const pg_ctx::PairGroup& a, const pg_ctx::PairGroup& b) {
-            return a.mode != b.mode ? a.mode < b.mode : a.nv < b.nv;
+            return a.mode != b.mode ? a.mode < b.mode : (a.raw != b.raw ? a.raw < b.raw : a.nv < b.nv);
         });
         std::vector<Tile> merged;
         std::vector<pg_ctx::PairGroup> out;
@@ -634,7 +719,8 @@ bool upload_tile_lists(pg_ctx* c) {
             pg_ctx::PairGroup cur = gr[i];
             const int first = static_cast<int>(merged.size());
             merged.insert(merged.end(), pairs.begin() + cur.first, pairs.begin() + cur.first + cur.count);
-            while (cur.mode != 2 && cur.count < 296 && i + 1 < gr.size() && gr[i + 1].mode == cur.mode) {
+            while (cur.mode != 2 && cur.count < 296 && i + 1 < gr.size() && gr[i + 1].mode == cur.mode &&
+                   gr[i + 1].raw == cur.raw) {
                 const pg_ctx::PairGroup& nx = gr[++i];
                 merged.insert(merged.end(), pairs.begin() + nx.first, pairs.begin() + nx.first + nx.count);
                 cur.nv = nx.nv;
@@ -683,7 +769,7 @@ bool upload_tile_lists(pg_ctx* c) {
 // need it).  Only before the first round, with nothing pending.
 bool leave_pair_mode(pg_ctx* c) {
     if (c->lay.n_pair_tiles == 0) return true;
-    for (LayerGeom& g : c->lay.layers) g.pair_mode = 0;
+    for (LayerGeom& g : c->lay.layers) g.pair_mode = g.raw = 0;
     if (c->loop_exec) {
         cudaGraphExecDestroy(c->loop_exec);
         c->loop_exec = nullptr;
@@ -799,6 +885,10 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.X = reinterpret_cast<float*>(c->ws + lay.off_X);
     st.Xw = st.X;
     st.Q = reinterpret_cast<float*>(c->ws + lay.off_Q);
+    st.Qr = st.Qw = st.Q;
+    st.raw_pending = 0;
+    c->q_buf[0] = st.Q;
+    c->q_buf[1] = lay.two_copies ? reinterpret_cast<float*>(c->ws + lay.off_Q2) : st.Q;
     st.Qinv = reinterpret_cast<float*>(c->ws + lay.off_Qinv);
     st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
     st.Pn = reinterpret_cast<float*>(c->ws + lay.off_Pn);
@@ -1132,7 +1222,10 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
             DevState st = c->st;
             st.Ph = ph_prev;
             st.PhNext = ph_cur;
-            // rows with two readers: read the current copy of X, write the corrected rows to the other
+            st.Qr = c->q_buf[c->step & 1];
+            st.Qw = c->q_buf[(c->step + 1) & 1];
+            st.raw_pending = c->pending ? 1 : 0;
+            // rows with several readers: read the current copy of X, write the corrected rows to the other
             const long long copy_elems = static_cast<long long>(c->topo.n_workers) * c->lay.x_stride;
             const bool flip = c->lay.two_copies && c->pending;
             st.X = c->st.X + c->xbuf * copy_elems;
@@ -1142,11 +1235,13 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
                 Timed t(c, PG_KERNEL_PAIR_SWEEP, stream, c->pending ? grp.bytes : 0.5 * grp.bytes);
                 if (grp.mode == 1)
                     ok = ok && pg::launch_pair_sweep(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
-                                                     grp.count, grp.nv, c->lay.pend_slots, stream) == cudaSuccess;
+                                                     grp.count, grp.nv, c->lay.pend_slots, grp.raw,
+                                                     c->lay.single_owner, stream) == cudaSuccess;
                 else if (grp.mode == 3)
                     ok = ok && pg::launch_pair_sweep_mid(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
                                                          grp.count, grp.nv, static_cast<int>(round_up(grp.slice, 4)),
-                                                         c->lay.pend_slots, stream) == cudaSuccess;
+                                                         c->lay.pend_slots, grp.raw, c->lay.single_owner,
+                                                         stream) == cudaSuccess;
                 else
                     ok = ok && pg::launch_pair_sweep_wide(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
                                                           grp.count, grp.nv, grp.slice, c->lay.pend_slots,
@@ -1387,7 +1482,7 @@ int pg_read_q(pg_ctx* c, int32_t i, int32_t j, int32_t layer, float* host_dst, v
     if (!bind_device(c)) return PG_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const LayerGeom& g = c->lay.layers[layer];
-    const float* src = c->st.Q + pair * c->st.q_stride + g.q_off;
+    const float* src = (g.pair_mode ? c->q_buf[c->step & 1] : c->st.Q) + pair * c->st.q_stride + g.q_off;
     if (cudaMemcpy2DAsync(host_dst, sizeof(float) * g.m, src, sizeof(float) * g.ld, sizeof(float) * g.m,
                           c->rank, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return PG_ERR_CUDA;
@@ -1401,14 +1496,18 @@ int pg_write_q(pg_ctx* c, int32_t i, int32_t j, int32_t layer, const float* host
     if (!bind_device(c)) return PG_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const LayerGeom& g = c->lay.layers[layer];
-    float* dst = c->st.Q + pair * c->st.q_stride + g.q_off;
+    float* dst = (g.pair_mode ? c->q_buf[c->step & 1] : c->st.Q) + pair * c->st.q_stride + g.q_off;
     const int frc = flush_pending(c, stream);     // the pending correction uses the stored vectors
     if (frc != PG_OK) return frc;
     c->y_valid = false;
     if (cudaMemcpy2DAsync(dst, sizeof(float) * g.ld, host_src, sizeof(float) * g.m, sizeof(float) * g.m,
                           c->rank, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return PG_ERR_CUDA;
-    if (pg::launch_column_norms(c->st, c->lay.n_pairs, stream) != cudaSuccess) return PG_ERR_CUDA;
+    {
+        DevState st = c->st;
+        st.Qr = c->q_buf[c->step & 1];
+        if (pg::launch_column_norms(st, c->lay.n_pairs, stream) != cudaSuccess) return PG_ERR_CUDA;
+    }
     c->launches += 1;
     return cudaStreamSynchronize(stream) == cudaSuccess ? PG_OK : PG_ERR_CUDA;
 }

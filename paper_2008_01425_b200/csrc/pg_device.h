@@ -29,6 +29,8 @@ constexpr int kPairWideStep = 1;       // rows a cluster handles between two exc
 constexpr int kPairWideMinBlocks = 3;  // resident CTAs per SM the cluster sweep is compiled for
 constexpr int kPairWideMaxLd = 8 * 256 * 4 * kPairCluster;  // widest row the cluster variant covers
 constexpr int kEdgeChunks = 32;        // CTAs that share the pair edge step of one (edge, layer)
+constexpr int kSpPerTile = 16;         // doubles a pair-sweep tile leaves for the pair edge step, see DevState::Sp
+constexpr int kMaxTerms = 7;           // rank-1 terms that can be pending on the difference of an edge (degree 4)
 
 // Geometry of one layer (same for every worker).
 struct LayerGeom {
@@ -53,8 +55,10 @@ struct LayerGeom {
     int p_rtiles;      // row tiles of the pair sweep
     int p_slice;       // mode 2: columns per CTA of the cluster (multiple of 4)
     long long up_off;  // partial sums of D^T p inside an edge's block (p_rtiles x rank x ld)
-    long long sp_off;  // partial sums of ||p||^2 (p_rtiles doubles), at rank 2 of P^T P (p_rtiles x 4 doubles)
+    long long sp_off;  // per-tile scalars for the pair edge step (p_rtiles x kSpPerTile doubles)
     int e_chunks;      // CTAs that share the pair edge step of one edge on this layer (1..kEdgeChunks)
+    int raw;           // pair sweep forms D from the rows as stored and leaves the pending terms to vector
+                       // algebra (graphs where a row has several readers), see pair_sweep_bulk_kernel
 };
 
 // One unit of work of a sweep: a tile of one worker's layer.
@@ -79,6 +83,8 @@ struct TabLayout {
     int off_degree;      // n_workers ints
     int off_slot_edge;   // n_workers * max_degree ints
     int off_slot_coef;   // n_workers * max_degree floats: sign * W
+    int off_own;         // max_edges ints: bit 0 / bit 1 set if the edge's CTAs write the corrected rows of
+                         // its smaller / larger end in the pair sweep (every worker has exactly one such edge)
     int total_ints;
 };
 
@@ -92,7 +98,12 @@ struct DevState {
                          // when a row has two readers in one sweep (pair sweep on graphs of degree 2)
     const float* G;      // null, or the caller's gradients laid out like X: updates also subtract eta * G
     float eta;
-    float* Q;            // [pair][q_stride]     raw right factors
+    float* Q;            // [pair][q_stride]     raw right factors (three-sweep layers; update sweeps)
+    float* Qr;           // pair-sweep layers: the stored vectors this step reads (q and the pending q') ...
+    float* Qw;           // ... and where the pair edge step writes the new ones.  Qr == Qw == Q unless rows
+                         // have several readers; there the two copies of Q swap roles every step, because an
+                         // edge's step still needs its neighbours' previous vectors while they write new ones
+    int raw_pending;     // pair edge step: the sweep ran on rows with corrections pending (their terms apply)
     float* Qinv;         // [pair][layer][rank]  1 / column norm (0 for a zero column)
     double* Qn2;         // [pair][layer][rank][kEdgeChunks]  pair sweep layers: shares of ||Q_k||^2
     float* Y;            // [worker][y_stride]   partial sums of X q
@@ -100,7 +111,8 @@ struct DevState {
     float* Z;            // [worker][z_stride]   partial sums of X^T p
     float* PhNext;       // same shape as Ph: where the pair sweep writes this step's p
     float* Up;           // [edge][up_stride]    pair sweep: partial sums of D^T p
-    double* Sp;          // [edge][sp_stride]    pair sweep: partial sums of ||p||^2
+    double* Sp;          // [edge][sp_stride]    pair sweep, per tile kSpPerTile doubles: [0] ||p||^2 (rank 2:
+                         // [0..2] P^T P), [4 + k] sum_r p_r p-hat_k[r] for pending term k (rank 2: [4 + 2k + c])
     float* Pn;           // [edge][layer]  half-step mode: ||p|| of the last odd iteration
     int dep_launch;      // host only: kernel families (kDep*) launched with programmatic stream serialisation
     int half_odd;        // half-step mode: the update being applied is an odd iteration's,
@@ -136,15 +148,18 @@ cudaError_t launch_random_directions(const DevState& st, const int* tab, int max
 cudaError_t launch_edge_raw(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile* tiles, int n_tiles,
                           cudaStream_t stream);
+// pend_slots: most corrections pending at a worker (its degree); raw / single_owner: see LayerGeom::raw and
+// TabLayout::off_own (single_owner: no edge writes both of its ends)
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
-                              const Tile* tiles, int n_tiles, int nv, int pend_slots, cudaStream_t stream);
+                              const Tile* tiles, int n_tiles, int nv, int pend_slots, bool raw, bool single_owner,
+                              cudaStream_t stream);
 cudaError_t launch_pair_sweep_wide(const DevState& st, const int* tab_prev, const int* tab_cur,
                                    bool apply_pending, const Tile* tiles, int n_tiles, int nv, int slice,
                                    int pend_slots, cudaStream_t stream);
 // `tiles`: tiles of layers whose rows one CTA holds (nv float4 per thread, rows of at most ld_pad floats)
 cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const int* tab_cur,
                                   bool apply_pending, const Tile* tiles, int n_tiles, int nv, int ld_pad,
-                                  int pend_slots, cudaStream_t stream);
+                                  int pend_slots, bool raw, bool single_owner, cudaStream_t stream);
 // Clusters of the wide pair sweep that can be resident at once (0 if unknown).
 int pair_wide_resident_clusters(int nv, int slice, int pend_slots);
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);

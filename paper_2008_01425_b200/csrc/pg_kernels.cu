@@ -832,11 +832,74 @@ __device__ __forceinline__ void pending_of(const DevState& st, const int* __rest
         pe.coef[s] = 0.0f;
         if (s < deg) {
             const int ep = tab_prev[st.tab.off_slot_edge + w * st.tab.max_degree + s];
-            pe.vec[s] = st.Q + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            pe.vec[s] = st.Qr + (long long)tab_prev[st.tab.off_pair + ep] * st.q_stride + g.q_off;
             pe.ph[s] = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
             pe.coef[s] = __int_as_float(tab_prev[st.tab.off_slot_coef + w * st.tab.max_degree + s]);
         }
     }
+}
+
+// The raw form of the pair sweep (graphs where a row has several readers).  With
+// the corrections of the previous step still pending, the difference of an edge
+// (i<j) is   D' = D - sum_k c_k p-hat_k q'_k^T   where D = X_i - X_j as stored and k
+// runs over the edges of the previous step at either end (c_k = coef at i, minus
+// coef at j; the edge itself, present at both ends, gets both).  Then
+//     p   = D' q-hat = D q-hat - sum_k c_k (q'_k . q-hat) p-hat_k
+//     D'^T p        = D^T p   - sum_k c_k (p-hat_k . p) q'_k
+// so the sweep needs the rows only as they are in memory: the pending terms enter p
+// as one scalar per row and D^T p as a few vectors, added by the pair edge step.
+// Only the one CTA that owns a worker's rows corrects and writes them.  Terms in the
+// order: the slots of worker i, then the slots of worker j without the edge itself.
+struct RawTerm {
+    int edge;
+    float coef;
+};
+__device__ __forceinline__ int raw_terms(const DevState& st, const int* __restrict__ tab, int e, int wi, int wj,
+                                         RawTerm* out) {
+    const int md = st.tab.max_degree;
+    const int di = min(tab[st.tab.off_degree + wi], md), dj = min(tab[st.tab.off_degree + wj], md);
+    int n = 0;
+    for (int s = 0; s < di && n < kMaxTerms; ++s) {
+        out[n].edge = tab[st.tab.off_slot_edge + wi * md + s];
+        out[n].coef = __int_as_float(tab[st.tab.off_slot_coef + wi * md + s]);
+        ++n;
+    }
+    for (int s = 0; s < dj; ++s) {
+        const int ep = tab[st.tab.off_slot_edge + wj * md + s];
+        const float c = __int_as_float(tab[st.tab.off_slot_coef + wj * md + s]);
+        if (ep == e) {
+            for (int k = 0; k < n; ++k)
+                if (out[k].edge == e) out[k].coef -= c;
+        } else if (n < kMaxTerms) {
+            out[n].edge = ep;
+            out[n].coef = -c;
+            ++n;
+        }
+    }
+    return n;
+}
+
+// Prologue of a raw sweep (whole CTA): the terms of edge e, each with its scalar
+// c_k (q'_k . q-hat) - the product in fp64 from the fp32 vectors, q_hat = `q` * qinv -
+// and the p-hat it multiplies.  s_ph / s_cb: kMaxTerms entries of shared memory.
+__device__ int raw_prologue(const DevState& st, const int* __restrict__ tab, int e, int wi, int wj,
+                            const LayerGeom& g, const float* __restrict__ q, float qinv, const float** s_ph,
+                            float* s_cb, double* scratch) {
+    RawTerm terms[kMaxTerms];
+    const int nt = raw_terms(st, tab, e, wi, wj, terms);
+    for (int k = 0; k < nt; ++k) {
+        const float* vk = st.Qr + (long long)tab[st.tab.off_pair + terms[k].edge] * st.q_stride + g.q_off;
+        double part = 0.0;
+        for (int idx = threadIdx.x; idx < g.m; idx += blockDim.x)
+            part += (double)vk[idx] * (double)(q[idx] * qinv);
+        const double beta = block_sum(part, scratch);
+        if (threadIdx.x == 0) {
+            s_ph[k] = st.Ph + (long long)terms[k].edge * st.ph_stride + g.ph_off;
+            s_cb[k] = (float)((double)terms[k].coef * beta);
+        }
+    }
+    __syncthreads();
+    return nt;
 }
 
 // --------------------------------------------------------------------------
@@ -906,7 +969,12 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
     return false;
 }
 
-template <int NV, bool UPDATE, int D>
+// RAW: the rows enter the products as stored, the pending terms as scalars (see
+// raw_terms); only the owning CTA corrects a worker's rows, and it keeps the pending
+// vectors of ENDS (1 or 2) ends of the edge in shared memory.  Otherwise (a matching:
+// each end has one previous edge and this edge is its only reader) both ends are
+// corrected before the difference is formed.
+template <int NV, bool UPDATE, int D, bool RAW, int ENDS>
 __global__ void __launch_bounds__(256, 1)
 pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles) {
@@ -914,10 +982,13 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     constexpr int STAGES = kBulkStages;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ __align__(16) float s_q[NV * 128];
-    __shared__ __align__(16) float s_ui[D][NV * 128];
-    __shared__ __align__(16) float s_uj[D][NV * 128];
+    __shared__ __align__(16) float s_u[ENDS][D][NV * 128];       // pending vectors of the ends this CTA corrects
     __shared__ __align__(8) unsigned long long s_full[STAGES];
     __shared__ double s_s[8];
+    __shared__ double s_g[8][kMaxTerms + 1];
+    __shared__ double s_scratch[33];
+    __shared__ const float* s_tph[kMaxTerms];
+    __shared__ float s_tcb[kMaxTerms];
     __shared__ int s_abort;
 
     const Tile tile = tiles[blockIdx.x];
@@ -932,15 +1003,16 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     const unsigned row_bytes = (unsigned)ld * 4u;                 // multiple of 16: ld is a multiple of 4
     float* s_stage = reinterpret_cast<float*>(s_dyn);             // [stage][matrix][row][ld]
 
-    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float* q = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const float qinv = pair_qinv(st, pair, tile.layer);
-    // only the edge in slot 0 of a worker writes that worker's rows back (to Xw, which
-    // is X itself unless rows have a second reader)
-    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
-    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
-    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
-    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // which ends' rows this CTA writes back (to Xw, which is X itself unless rows have several readers)
+    const int own = UPDATE ? tab_cur[st.tab.off_own + e] : 0;
+    const bool st_i = (own & 1) != 0, st_j = (own & 2) != 0;
+    // which ends' rows it corrects: all that it forms the difference from, or only its own
+    const bool act_i = UPDATE && (!RAW || st_i), act_j = UPDATE && (!RAW || st_j);
+    const int slot_i = 0, slot_j = ENDS == 2 ? 1 : 0;            // where s_u keeps either end's vectors
+    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
     PendingEnd<D> pi, pj;
     if (UPDATE) {
         pending_of<D>(st, tab_prev, wi, g, q, pi);
@@ -961,8 +1033,8 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         if (UPDATE) {
 #pragma unroll
             for (int s2 = 0; s2 < D; ++s2) {
-                s_ui[s2][idx] = in ? pi.vec[s2][idx] : 0.0f;
-                s_uj[s2][idx] = in ? pj.vec[s2][idx] : 0.0f;
+                if (act_i) s_u[slot_i][s2][idx] = in ? pi.vec[s2][idx] : 0.0f;
+                if (act_j) s_u[slot_j][s2][idx] = in ? pj.vec[s2][idx] : 0.0f;
             }
         }
     }
@@ -982,12 +1054,17 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     if (threadIdx.x == 0)
         for (; issued < STAGES - 1 && issued < n_stages; ++issued) issue(issued);
 
+    // the pending terms of this edge, while the first rows are on their way
+    int nt = 0;
+    if (RAW && UPDATE) nt = raw_prologue(st, tab_prev, e, wi, wj, g, q, qinv, s_tph, s_tcb, s_scratch);
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
     float4 u[NV];
 #pragma unroll
     for (int k = 0; k < NV; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     float ssum = 0.0f;
+    double gsum = 0.0;            // lane k: this warp's share of sum_r p_r p-hat_k[r]
     bool ok = true;
 
     for (int it = 0; it < n_stages; ++it) {
@@ -1015,30 +1092,45 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                     xj[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
+            float phv = 0.0f;                       // RAW, lane k: p-hat_k[r] of pending term k
+            if (RAW && UPDATE && lane < nt) phv = __ldg(s_tph[lane] + r);
             if (UPDATE) {
                 float ai[D], aj[D];
 #pragma unroll
                 for (int s2 = 0; s2 < D; ++s2) {
-                    ai[s2] = pi.ph[s2] ? pi.coef[s2] * __ldg(pi.ph[s2] + r) : 0.0f;
-                    aj[s2] = pj.ph[s2] ? pj.coef[s2] * __ldg(pj.ph[s2] + r) : 0.0f;
+                    ai[s2] = (act_i && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r) : 0.0f;
+                    aj[s2] = (act_j && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r) : 0.0f;
                 }
                 float* rowi = Xi_w + (long long)r * ld;
                 float* rowj = Xj_w + (long long)r * ld;
+                if (act_i) {
 #pragma unroll
-                for (int k = 0; k < NV; ++k) {
-                    const int col = (k * 32 + lane) * 4;
+                    for (int k = 0; k < NV; ++k) {
+                        const int col = (k * 32 + lane) * 4;
+                        float4 t = xi[k];
 #pragma unroll
-                    for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
-                        const float4 vi = *reinterpret_cast<const float4*>(&s_ui[s2][col]);
-                        const float4 vj = *reinterpret_cast<const float4*>(&s_uj[s2][col]);
-                        xi[k].x = fmaf(-ai[s2], vi.x, xi[k].x); xi[k].y = fmaf(-ai[s2], vi.y, xi[k].y);
-                        xi[k].z = fmaf(-ai[s2], vi.z, xi[k].z); xi[k].w = fmaf(-ai[s2], vi.w, xi[k].w);
-                        xj[k].x = fmaf(-aj[s2], vj.x, xj[k].x); xj[k].y = fmaf(-aj[s2], vj.y, xj[k].y);
-                        xj[k].z = fmaf(-aj[s2], vj.z, xj[k].z); xj[k].w = fmaf(-aj[s2], vj.w, xj[k].w);
+                        for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
+                            const float4 v = *reinterpret_cast<const float4*>(&s_u[slot_i][s2][col]);
+                            t.x = fmaf(-ai[s2], v.x, t.x); t.y = fmaf(-ai[s2], v.y, t.y);
+                            t.z = fmaf(-ai[s2], v.z, t.z); t.w = fmaf(-ai[s2], v.w, t.w);
+                        }
+                        if (st_i && col < ld) st_stream(rowi + col, t);
+                        if (!RAW) xi[k] = t;
                     }
-                    if (col < ld) {
-                        if (own_i) st_stream(rowi + col, xi[k]);
-                        if (own_j) st_stream(rowj + col, xj[k]);
+                }
+                if (act_j) {
+#pragma unroll
+                    for (int k = 0; k < NV; ++k) {
+                        const int col = (k * 32 + lane) * 4;
+                        float4 t = xj[k];
+#pragma unroll
+                        for (int s2 = 0; s2 < D; ++s2) {
+                            const float4 v = *reinterpret_cast<const float4*>(&s_u[slot_j][s2][col]);
+                            t.x = fmaf(-aj[s2], v.x, t.x); t.y = fmaf(-aj[s2], v.y, t.y);
+                            t.z = fmaf(-aj[s2], v.z, t.z); t.w = fmaf(-aj[s2], v.w, t.w);
+                        }
+                        if (st_j && col < ld) st_stream(rowj + col, t);
+                        if (!RAW) xj[k] = t;
                     }
                 }
             }
@@ -1051,6 +1143,7 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                 dot = fmaf(xi[k].x, vq.x, dot); dot = fmaf(xi[k].y, vq.y, dot);
                 dot = fmaf(xi[k].z, vq.z, dot); dot = fmaf(xi[k].w, vq.w, dot);
             }
+            if (RAW && UPDATE && lane < nt) dot = fmaf(-s_tcb[lane], phv, dot);   // the pending terms' part of p_r
             const float p = warp_sum(dot);
 #pragma unroll
             for (int k = 0; k < NV; ++k) {
@@ -1058,6 +1151,7 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                 u[k].z = fmaf(p, xi[k].z, u[k].z); u[k].w = fmaf(p, xi[k].w, u[k].w);
             }
             ssum = fmaf(p, p, ssum);
+            if (RAW && UPDATE) gsum += (double)p * (double)phv;
             if (lane == 0) Pw[r] = p;
         }
         __syncthreads();          // every warp is done with this slot before it is filled again
@@ -1077,6 +1171,7 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 #pragma unroll
     for (int k = 0; k < NV; ++k) *reinterpret_cast<float4*>(&s_red[warp * NV * 128 + (k * 32 + lane) * 4]) = u[k];
     if (lane == 0) s_s[warp] = (double)ssum;
+    if (lane <= kMaxTerms) s_g[warp][lane] = gsum;
     __syncthreads();
     float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld;
     for (int idx = threadIdx.x; idx < ld; idx += 256) {
@@ -1085,10 +1180,16 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         for (int w8 = 1; w8 < 8; ++w8) t += s_red[w8 * NV * 128 + idx];
         Up[idx] = t;
     }
+    double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile;
     if (threadIdx.x == 0) {
         double t = 0.0;
         for (int w8 = 0; w8 < 8; ++w8) t += s_s[w8];
-        st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = t;
+        sp[0] = t;
+    }
+    if (RAW && threadIdx.x < kMaxTerms) {
+        double t = 0.0;
+        for (int w8 = 0; w8 < 8; ++w8) t += s_g[w8][threadIdx.x];
+        sp[4 + threadIdx.x] = threadIdx.x < nt ? t : 0.0;
     }
 }
 
@@ -1133,15 +1234,14 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     float* s_q = s_vec;
     float* s_ui = s_vec + slice_pad;                  // [D][slice_pad]
     float* s_uj = s_vec + (1 + D) * slice_pad;        // [D][slice_pad]
-    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float* q = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const float qinv = pair_qinv(st, pair, tile.layer);
-    // only the edge in slot 0 of a worker writes that worker's rows back (to Xw, which
-    // is X itself unless rows have a second reader)
-    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
-    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
-    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
-    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // only the edge that owns a worker's rows writes them back (to Xw, which is X itself
+    // unless rows have a second reader; on a matching every edge owns both of its ends)
+    const int own = tab_cur[st.tab.off_own + e];
+    const bool own_i = (own & 1) != 0, own_j = (own & 2) != 0;
+    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
     PendingEnd<D> pi, pj;
     if (UPDATE) {
         pending_of<D>(st, tab_prev, wi, g, q, pi);
@@ -1287,7 +1387,7 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         if (c_begin + off < c_end) *reinterpret_cast<float4*>(Up + off) = u[k];
     }
     if (rank == 0 && threadIdx.x == 0)
-        st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = (double)ssum;
+        st.Sp[(long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile] = (double)ssum;
     cluster.sync();              // nobody leaves while a peer could still address its shared memory
 }
 
@@ -1320,15 +1420,14 @@ pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* 
     float* s_q = s_vec;
     float* s_ui = s_vec + ld_pad;                     // [D][ld_pad]
     float* s_uj = s_vec + (1 + D) * ld_pad;           // [D][ld_pad]
-    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float* q = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const float qinv = pair_qinv(st, pair, tile.layer);
-    // only the edge in slot 0 of a worker writes that worker's rows back (to Xw, which
-    // is X itself unless rows have a second reader)
-    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
-    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
-    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
-    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // only the edge that owns a worker's rows writes them back (to Xw, which is X itself
+    // unless rows have a second reader; on a matching every edge owns both of its ends)
+    const int own = tab_cur[st.tab.off_own + e];
+    const bool own_i = (own & 1) != 0, own_j = (own & 2) != 0;
+    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
     PendingEnd<D> pi, pj;
     if (UPDATE) {
         pending_of<D>(st, tab_prev, wi, g, q, pi);
@@ -1430,7 +1529,7 @@ pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* 
         const int off = (k * 256 + threadIdx.x) * 4;
         if (off < ld) *reinterpret_cast<float4*>(Up + off) = u[k];
     }
-    if (threadIdx.x == 0) st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = (double)ssum;
+    if (threadIdx.x == 0) st.Sp[(long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile] = (double)ssum;
 }
 
 // --------------------------------------------------------------------------
@@ -1453,8 +1552,11 @@ __host__ __device__ constexpr int mid_rows(int nvm) { return nvm <= 2 ? 4 : 2; }
 // two CTAs per SM where the registers allow it, so one CTA's prologue hides behind the other's rows
 __host__ __device__ constexpr int mid_min_blocks(int nvm, int d) { return (1 + 2 * d) * nvm <= 10 ? 2 : 1; }
 
-template <int NVM, bool UPDATE, int D>
-__global__ void __launch_bounds__(256, mid_min_blocks(NVM, D))
+// RAW / ENDS as in the row-per-warp kernel: the rows enter the products as stored, the
+// pending terms as one scalar per row, and the thread keeps in registers only the
+// pending vectors of the ENDS (1 or 2) ends whose rows this CTA may have to write.
+template <int NVM, bool UPDATE, int D, bool RAW, int ENDS>
+__global__ void __launch_bounds__(256, mid_min_blocks(NVM, RAW ? (ENDS * D + 1) / 2 : D))
 pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                            const Tile* __restrict__ tiles, int ld_pad, int n_stage) {
     grid_dependency_sync();
@@ -1462,6 +1564,9 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     __shared__ __align__(8) unsigned long long s_full[kMidStagesMax];
     constexpr int RS = mid_rows(NVM);
     __shared__ float s_warp[2][RS][8];
+    __shared__ double s_scratch[33];
+    __shared__ const float* s_tph[kMaxTerms];
+    __shared__ float s_tcb[kMaxTerms];
     __shared__ int s_abort;
 
     const Tile tile = tiles[blockIdx.x];
@@ -1475,18 +1580,23 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     const int ld = g.ld;
     const unsigned row_bytes = (unsigned)ld * 4u;     // multiple of 16: ld is a multiple of 4
 
-    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float* q = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const float qinv = pair_qinv(st, pair, tile.layer);
-    // (with one slot per worker every edge is in slot 0 and the rows are corrected in place)
-    const bool own_i = D == 1 || tab_cur[st.tab.off_slot_i + e] == 0;
-    const bool own_j = D == 1 || tab_cur[st.tab.off_slot_j + e] == 0;
-    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // which ends' rows this CTA writes back (to Xw, which is X itself unless rows have several readers),
+    // and which it corrects: all that it forms the difference from, or only the ones it writes
+    const int own = UPDATE ? tab_cur[st.tab.off_own + e] : 0;
+    const bool st_i = (own & 1) != 0, st_j = (own & 2) != 0;
+    const bool act_i = UPDATE && (!RAW || st_i), act_j = UPDATE && (!RAW || st_j);
+    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // ENDS == 1: the vectors of the one end this CTA corrects (worker j if `one_is_j`)
+    const bool one_is_j = ENDS == 1 && !act_i;
     PendingEnd<D> pi, pj;
     if (UPDATE) {
-        pending_of<D>(st, tab_prev, wi, g, q, pi);
-        pending_of<D>(st, tab_prev, wj, g, q, pj);
+        pending_of<D>(st, tab_prev, one_is_j ? wj : wi, g, q, pi);
+        if (ENDS == 2) pending_of<D>(st, tab_prev, wj, g, q, pj);
     }
+    const bool act_a = ENDS == 1 ? (act_i || act_j) : act_i;     // the end whose vectors are in va
     const int r0 = tile.rtile * g.p_rows;
     const int r1 = min(g.n, r0 + g.p_rows);
     const int n_iter = (r1 - r0 + RS - 1) / RS;
@@ -1510,8 +1620,12 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     if (threadIdx.x == 0)
         for (; issued < n_stage && issued < n_iter; ++issued) issue(issued);
 
+    // the pending terms of this edge, while the first rows are on their way
+    int nt = 0;
+    if (RAW && UPDATE) nt = raw_prologue(st, tab_prev, e, wi, wj, g, q, qinv, s_tph, s_tcb, s_scratch);
+
     // this thread's columns of the vectors, for the whole tile
-    float4 vq[NVM], vi[D][NVM], vj[D][NVM];
+    float4 vq[NVM], va[D][NVM], vb[ENDS == 2 ? D : 1][ENDS == 2 ? NVM : 1];
 #pragma unroll
     for (int k = 0; k < NVM; ++k) {
         const int off = (k * 256 + threadIdx.x) * 4;
@@ -1523,8 +1637,8 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
         }
 #pragma unroll
         for (int s2 = 0; s2 < D; ++s2) {
-            vi[s2][k] = (UPDATE && off < ld) ? *reinterpret_cast<const float4*>(pi.vec[s2] + off) : zero;
-            vj[s2][k] = (UPDATE && off < ld) ? *reinterpret_cast<const float4*>(pj.vec[s2] + off) : zero;
+            va[s2][k] = (act_a && off < ld) ? *reinterpret_cast<const float4*>(pi.vec[s2] + off) : zero;
+            if (ENDS == 2) vb[s2][k] = (act_j && off < ld) ? *reinterpret_cast<const float4*>(pj.vec[s2] + off) : zero;
         }
     }
 
@@ -1534,6 +1648,7 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
 #pragma unroll
     for (int k = 0; k < NVM; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     float ssum = 0.0f;
+    double gsum = 0.0;            // thread k < nt: this tile's sum_r p_r p-hat_k[r]
     bool ok = true;
 
     for (int it = 0; it < n_iter; ++it) {
@@ -1544,16 +1659,27 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
         const float* sj = si + (size_t)RS * ld_pad;
         float4 d[RS][NVM];
         float dot[RS];
+        float corr[RS];           // RAW: the pending terms' part of p_r
+        float mine_ph[RS];        // RAW, thread k < nt: p-hat_k[r]
 #pragma unroll
         for (int t = 0; t < RS; ++t) {
             const bool in_row = mine && r + t < r1;
             const long long base = (long long)(r + t) * ld;
             dot[t] = 0.0f;
-            float ai[D], aj[D];
+            corr[t] = 0.0f;
+            mine_ph[t] = 0.0f;
+            if (RAW && UPDATE && in_row) {
+                for (int k = 0; k < nt; ++k) {
+                    const float phv = __ldg(s_tph[k] + r + t);
+                    corr[t] = fmaf(s_tcb[k], phv, corr[t]);
+                    if (threadIdx.x == k) mine_ph[t] = phv;
+                }
+            }
+            float aa[D], ab[D];
 #pragma unroll
             for (int s2 = 0; s2 < D; ++s2) {
-                ai[s2] = (UPDATE && in_row && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r + t) : 0.0f;
-                aj[s2] = (UPDATE && in_row && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r + t) : 0.0f;
+                aa[s2] = (act_a && in_row && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r + t) : 0.0f;
+                ab[s2] = (ENDS == 2 && act_j && in_row && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r + t) : 0.0f;
             }
 #pragma unroll
             for (int k = 0; k < NVM; ++k) {
@@ -1564,18 +1690,42 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
                     xi = *reinterpret_cast<const float4*>(si + (size_t)t * ld + off);
                     xj = *reinterpret_cast<const float4*>(sj + (size_t)t * ld + off);
                 }
-                if (UPDATE && in) {
-#pragma unroll
-                    for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
-                        xi.x = fmaf(-ai[s2], vi[s2][k].x, xi.x); xi.y = fmaf(-ai[s2], vi[s2][k].y, xi.y);
-                        xi.z = fmaf(-ai[s2], vi[s2][k].z, xi.z); xi.w = fmaf(-ai[s2], vi[s2][k].w, xi.w);
-                        xj.x = fmaf(-aj[s2], vj[s2][k].x, xj.x); xj.y = fmaf(-aj[s2], vj[s2][k].y, xj.y);
-                        xj.z = fmaf(-aj[s2], vj[s2][k].z, xj.z); xj.w = fmaf(-aj[s2], vj[s2][k].w, xj.w);
-                    }
-                    if (own_i) st_stream(Xi_w + base + off, xi);
-                    if (own_j) st_stream(Xj_w + base + off, xj);
+                if (RAW) {   // the difference of the rows as stored; corrected rows only go back to memory
+                    d[t][k].x = xi.x - xj.x; d[t][k].y = xi.y - xj.y; d[t][k].z = xi.z - xj.z; d[t][k].w = xi.w - xj.w;
                 }
-                d[t][k].x = xi.x - xj.x; d[t][k].y = xi.y - xj.y; d[t][k].z = xi.z - xj.z; d[t][k].w = xi.w - xj.w;
+                if (UPDATE && in) {
+                    if (ENDS == 1) {
+                        if (act_a) {
+                            float4 x = one_is_j ? xj : xi;
+#pragma unroll
+                            for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
+                                x.x = fmaf(-aa[s2], va[s2][k].x, x.x); x.y = fmaf(-aa[s2], va[s2][k].y, x.y);
+                                x.z = fmaf(-aa[s2], va[s2][k].z, x.z); x.w = fmaf(-aa[s2], va[s2][k].w, x.w);
+                            }
+                            st_stream((one_is_j ? Xj_w : Xi_w) + base + off, x);
+                        }
+                    } else {
+                        if (act_i) {
+#pragma unroll
+                            for (int s2 = 0; s2 < D; ++s2) {
+                                xi.x = fmaf(-aa[s2], va[s2][k].x, xi.x); xi.y = fmaf(-aa[s2], va[s2][k].y, xi.y);
+                                xi.z = fmaf(-aa[s2], va[s2][k].z, xi.z); xi.w = fmaf(-aa[s2], va[s2][k].w, xi.w);
+                            }
+                            if (st_i) st_stream(Xi_w + base + off, xi);
+                        }
+                        if (act_j) {
+#pragma unroll
+                            for (int s2 = 0; s2 < D; ++s2) {
+                                xj.x = fmaf(-ab[s2], vb[s2][k].x, xj.x); xj.y = fmaf(-ab[s2], vb[s2][k].y, xj.y);
+                                xj.z = fmaf(-ab[s2], vb[s2][k].z, xj.z); xj.w = fmaf(-ab[s2], vb[s2][k].w, xj.w);
+                            }
+                            if (st_j) st_stream(Xj_w + base + off, xj);
+                        }
+                    }
+                }
+                if (!RAW) {
+                    d[t][k].x = xi.x - xj.x; d[t][k].y = xi.y - xj.y; d[t][k].z = xi.z - xj.z; d[t][k].w = xi.w - xj.w;
+                }
                 dot[t] = fmaf(d[t][k].x, vq[k].x, dot[t]); dot[t] = fmaf(d[t][k].y, vq[k].y, dot[t]);
                 dot[t] = fmaf(d[t][k].z, vq[k].z, dot[t]); dot[t] = fmaf(d[t][k].w, vq[k].w, dot[t]);
             }
@@ -1596,13 +1746,17 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
             float p = 0.0f;
 #pragma unroll
             for (int w8 = 0; w8 < 8; ++w8) p += s_warp[it & 1][t][w8];
+            if (RAW && UPDATE) p -= corr[t];
 #pragma unroll
             for (int k = 0; k < NVM; ++k) {
                 u[k].x = fmaf(p, d[t][k].x, u[k].x); u[k].y = fmaf(p, d[t][k].y, u[k].y);
                 u[k].z = fmaf(p, d[t][k].z, u[k].z); u[k].w = fmaf(p, d[t][k].w, u[k].w);
             }
-            ssum = fmaf(p, p, ssum);
-            if (threadIdx.x == 0 && r + t < r1) Pw[r + t] = p;
+            if (r + t < r1) {
+                ssum = fmaf(p, p, ssum);
+                if (RAW && UPDATE) gsum += (double)p * (double)mine_ph[t];
+                if (threadIdx.x == 0) Pw[r + t] = p;
+            }
         }
     }
     if (!ok) {
@@ -1621,7 +1775,9 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
         const int off = (k * 256 + threadIdx.x) * 4;
         if (off < ld) *reinterpret_cast<float4*>(Up + off) = u[k];
     }
-    if (threadIdx.x == 0) st.Sp[(long long)e * st.sp_stride + g.sp_off + tile.rtile] = (double)ssum;
+    double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile;
+    if (threadIdx.x == 0) sp[0] = (double)ssum;
+    if (RAW && threadIdx.x < kMaxTerms) sp[4 + threadIdx.x] = threadIdx.x < nt ? gsum : 0.0;
 }
 
 // --------------------------------------------------------------------------
@@ -1709,12 +1865,14 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
     const unsigned row_bytes = (unsigned)ld * 4u;     // multiple of 16: ld is a multiple of 4
     const int md = st.tab.max_degree;
 
-    const float* q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    const float* q = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const float qinv0 = pair_qinv(st, pair, tile.layer, 0), qinv1 = pair_qinv(st, pair, tile.layer, 1);
     // slot of this edge at either end, and the other edge there (if the worker has two)
     const int si = tab[st.tab.off_slot_i + e], sj = tab[st.tab.off_slot_j + e];
     const bool two_i = tab[st.tab.off_degree + wi] > 1, two_j = tab[st.tab.off_degree + wj] > 1;
-    const bool own_i = si == 0, own_j = sj == 0;      // the edge in slot 0 writes the corrected row
+    const bool first_i = si == 0, first_j = sj == 0;  // slot order: is this edge's correction the first at that end
+    const int own = tab[st.tab.off_own + e];          // the ends whose corrected rows this CTA writes
+    const bool own_i = (own & 1) != 0, own_j = (own & 2) != 0;
     const float* ph_e = st.Ph + (long long)e * st.ph_stride + g.ph_off;
     const float* ph_oi = ph_e;
     const float* ph_oj = ph_e;
@@ -1726,13 +1884,13 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
         ce_j = __int_as_float(tab[st.tab.off_slot_coef + wj * md + sj]);
         if (two_i) {
             const int eo = tab[st.tab.off_slot_edge + wi * md + (1 - si)];
-            q_oi = st.Q + (long long)tab[st.tab.off_pair + eo] * st.q_stride + g.q_off;
+            q_oi = st.Qr + (long long)tab[st.tab.off_pair + eo] * st.q_stride + g.q_off;
             ph_oi = st.Ph + (long long)eo * st.ph_stride + g.ph_off;
             co_i = __int_as_float(tab[st.tab.off_slot_coef + wi * md + (1 - si)]);
         }
         if (two_j) {
             const int eo = tab[st.tab.off_slot_edge + wj * md + (1 - sj)];
-            q_oj = st.Q + (long long)tab[st.tab.off_pair + eo] * st.q_stride + g.q_off;
+            q_oj = st.Qr + (long long)tab[st.tab.off_pair + eo] * st.q_stride + g.q_off;
             ph_oj = st.Ph + (long long)eo * st.ph_stride + g.ph_off;
             co_j = __int_as_float(tab[st.tab.off_slot_coef + wj * md + (1 - sj)]);
         }
@@ -1817,22 +1975,22 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
                     xj = *reinterpret_cast<const float4*>(sj_rows + (size_t)t * ld + off);
                 }
                 if (UPDATE && in) {
-                    if (own_i) {       // this edge is in slot 0 of worker i: its correction first
+                    if (first_i) {     // this edge is in slot 0 of worker i: its correction first
                         fma4(xi, ae_i[0], vq[0][k]); fma4(xi, ae_i[1], vq[1][k]);
                         fma4(xi, ao_i[0], vi[0][k]); fma4(xi, ao_i[1], vi[1][k]);
-                        st_stream(Xi_w + base + off, xi);
                     } else {
                         fma4(xi, ao_i[0], vi[0][k]); fma4(xi, ao_i[1], vi[1][k]);
                         fma4(xi, ae_i[0], vq[0][k]); fma4(xi, ae_i[1], vq[1][k]);
                     }
-                    if (own_j) {
+                    if (own_i) st_stream(Xi_w + base + off, xi);
+                    if (first_j) {
                         fma4(xj, ae_j[0], vq[0][k]); fma4(xj, ae_j[1], vq[1][k]);
                         fma4(xj, ao_j[0], vj[0][k]); fma4(xj, ao_j[1], vj[1][k]);
-                        st_stream(Xj_w + base + off, xj);
                     } else {
                         fma4(xj, ao_j[0], vj[0][k]); fma4(xj, ao_j[1], vj[1][k]);
                         fma4(xj, ae_j[0], vq[0][k]); fma4(xj, ae_j[1], vq[1][k]);
                     }
+                    if (own_j) st_stream(Xj_w + base + off, xj);
                 }
                 d[t][k] = sub4(xi, xj);
 #pragma unroll
@@ -1895,7 +2053,7 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
             if (off < ld) *reinterpret_cast<float4*>(Up + (long long)c * ld + off) = u[c][k];
         }
     if (threadIdx.x == 0) {
-        double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * 4;
+        double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile;
         sp[0] = g00;
         sp[1] = g01;
         sp[2] = g11;
@@ -1916,9 +2074,9 @@ __device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab,
     const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
     double a00 = 0.0, a01 = 0.0, a11 = 0.0;
     for (int t = threadIdx.x; t < g.p_rtiles; t += blockDim.x) {
-        a00 += sp[4 * t];
-        a01 += sp[4 * t + 1];
-        a11 += sp[4 * t + 2];
+        a00 += sp[kSpPerTile * t];
+        a01 += sp[kSpPerTile * t + 1];
+        a11 += sp[kSpPerTile * t + 2];
     }
     const double g00 = block_sum(a00, scratch);      // same order, hence same bits, in every chunk
     const double g01 = block_sum(a01, scratch);
@@ -1945,11 +2103,17 @@ __device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab,
         st.live[((long long)e * L + l) * 2 + 1] = live1 ? 1 : 0;
         if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
     }
-    if (!live0 && !live1) return;   // uniform over the block
     const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
-    float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    float* Q = st.Qw + (long long)pair * st.q_stride + g.q_off;
+    const float* Qold = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const int cw = (g.m + nch - 1) / nch;
     const int c_lo = chunk * cw, c_hi = min(g.m, (chunk + 1) * cw);
+    if (Q != Qold)   // the vectors live in two copies that swap roles: a dead column's vector moves over unchanged
+        for (int c = c_lo + threadIdx.x; c < c_hi; c += blockDim.x) {
+            if (!live0) Q[c] = Qold[c];
+            if (!live1) Q[g.ld + c] = Qold[g.ld + c];
+        }
+    if (!live0 && !live1) return;   // uniform over the block
     double part0 = 0.0, part1 = 0.0;
     for (int c = c_lo + threadIdx.x; c < c_hi; c += blockDim.x) {
         double u0 = 0.0, u1 = 0.0;
@@ -1999,6 +2163,7 @@ __global__ void __launch_bounds__(256)
 pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     grid_dependency_sync();
     __shared__ double scratch[33];
+    __shared__ double s_tot[kMaxTerms + 1];
     const int L = st.n_layers;
     const int e = blockIdx.x / st.e_total;
     const int slot = blockIdx.x - e * st.e_total;
@@ -2012,9 +2177,26 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     }
     const int pair = tab[st.tab.off_pair + e];
     const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
-    double part = 0.0;
-    for (int t = threadIdx.x; t < g.p_rtiles; t += blockDim.x) part += sp[t];
-    const double nn = block_sum(part, scratch);      // same order, hence same bits, in every chunk
+    // Raw sweep with corrections pending: the terms of this edge (same order as in the sweep).
+    // Warp w adds scalar w of every tile in tile order: ||p||^2 (w = 0) and sum_r p_r p-hat_k[r]
+    // (w = 1 + k); every chunk's CTA gets the same bits.
+    RawTerm terms[kMaxTerms];
+    int nt = 0;
+    if (g.raw && st.raw_pending)
+        nt = raw_terms(st, tab, e, tab[st.tab.off_edge_i + e], tab[st.tab.off_edge_j + e], terms);
+    {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        if (warp <= nt) {
+            const int which = warp == 0 ? 0 : 3 + warp;
+            double a = 0.0;
+            for (int t = lane; t < g.p_rtiles; t += 32) a += sp[(long long)t * kSpPerTile + which];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+            if (lane == 0) s_tot[warp] = a;
+        }
+        __syncthreads();
+    }
+    const double nn = s_tot[0];
     const bool finite = isfinite(nn);
     const bool live = finite && nn > 0.0;
     const double inv = live ? 1.0 / sqrt(nn) : 0.0;
@@ -2027,12 +2209,29 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
         st.live[(long long)e * L + l] = live ? 1 : 0;
         if (!finite) atomicOr(st.status, 1 << kStatusNumeric);
     }
-    if (!live) return;   // uniform over the block
-    const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
-    float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    float* Q = st.Qw + (long long)pair * st.q_stride + g.q_off;
+    const float* Qold = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const int cw = (g.m + nch - 1) / nch;
     const int c_lo = chunk * cw, c_hi = min(g.m, (chunk + 1) * cw);
-    part = 0.0;
+    if (!live) {   // uniform over the block; with two copies of the vectors the old one moves over unchanged
+        if (Q != Qold)
+            for (int c = c_lo + threadIdx.x; c < c_hi; c += blockDim.x) Q[c] = Qold[c];
+        return;
+    }
+    const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
+    // D'^T p = D^T p - sum_k c_k (p-hat_k . p) q'_k with the previous vectors of the pending edges
+    const float* tvec[kMaxTerms];
+    double tcoef[kMaxTerms];
+#pragma unroll
+    for (int k = 0; k < kMaxTerms; ++k) {
+        tvec[k] = Qold;
+        tcoef[k] = 0.0;
+        if (k < nt) {
+            tvec[k] = st.Qr + (long long)tab[st.tab.off_pair + terms[k].edge] * st.q_stride + g.q_off;
+            tcoef[k] = (double)terms[k].coef * s_tot[1 + k];
+        }
+    }
+    double part = 0.0;
     if (cw <= 32) {
         // few columns, many tiles: 8 thread groups each add every 8th tile's share, then the
         // groups are added in order (a fixed order, so the result is reproducible)
@@ -2048,6 +2247,9 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
             double tot = 0.0;
 #pragma unroll
             for (int k = 0; k < 8; ++k) tot += s_grp[k][col];
+#pragma unroll
+            for (int k = 0; k < kMaxTerms; ++k)
+                if (k < nt) tot -= tcoef[k] * (double)tvec[k][c];
             const float q = (float)(tot * inv);
             Q[c] = q;
             part = (double)q * (double)q;
@@ -2062,6 +2264,9 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) a += (double)v[j];
             }
+#pragma unroll
+            for (int k = 0; k < kMaxTerms; ++k)
+                if (k < nt) a -= tcoef[k] * (double)tvec[k][c];
             const float q = (float)(a * inv);
             Q[c] = q;
             part += (double)q * (double)q;
@@ -2083,7 +2288,7 @@ column_norms_kernel(DevState st) {
     const long long pair = blockIdx.x / L;
     const int l = blockIdx.x - (int)pair * L;
     const LayerGeom g = st.layers[l];
-    const float* Q = st.Q + pair * st.q_stride + g.q_off;
+    const float* Q = (g.pair_mode ? st.Qr : st.Q) + pair * st.q_stride + g.q_off;
     for (int k = 0; k < rank; ++k) {
         double part = 0.0;
         for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
@@ -2253,33 +2458,33 @@ cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile*
     return launch_row<true, false, false>(st, tab_update, tab_update, tiles, n_tiles, stream);
 }
 
-template <int NV, bool UPDATE, int D>
+template <int NV, bool UPDATE, int D, bool RAW, int ENDS>
 static cudaError_t launch_pair_bulk_t(const DevState& st, const int* tab_prev, const int* tab_cur,
                                       const Tile* tiles, int n_tiles, int max_ld, cudaStream_t stream) {
     // stage buffers; they also hold the 8 x NV*128 floats of the final reduction
     size_t smem = sizeof(float) * (size_t)kBulkStages * 2 * kBulkRows * max_ld;
     const size_t red = sizeof(float) * 8 * NV * 128;
     if (smem < red) smem = red;
-    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE, D>,
+    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE, D, RAW, ENDS>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (rc != cudaSuccess) return rc;
-    launch_dep(st.dep_launch & kDepPairRow, pair_sweep_bulk_kernel<NV, UPDATE, D>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles);
+    launch_dep(st.dep_launch & kDepPairRow, pair_sweep_bulk_kernel<NV, UPDATE, D, RAW, ENDS>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles);
     return cudaGetLastError();
 }
 
-template <bool UPDATE, int D>
+template <bool UPDATE, int D, bool RAW, int ENDS>
 static cudaError_t launch_pair_bulk(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
                                     int n_tiles, int nv, cudaStream_t stream) {
     const int max_ld = nv * 128;
     switch (nv) {
-        case 1: return launch_pair_bulk_t<1, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 2: return launch_pair_bulk_t<2, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 3: return launch_pair_bulk_t<3, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 4: return launch_pair_bulk_t<4, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 5: return launch_pair_bulk_t<5, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 6: return launch_pair_bulk_t<6, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 7: return launch_pair_bulk_t<7, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        default: return launch_pair_bulk_t<8, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 1: return launch_pair_bulk_t<1, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 2: return launch_pair_bulk_t<2, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 3: return launch_pair_bulk_t<3, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 4: return launch_pair_bulk_t<4, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 5: return launch_pair_bulk_t<5, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 6: return launch_pair_bulk_t<6, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 7: return launch_pair_bulk_t<7, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        default: return launch_pair_bulk_t<8, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
     }
 }
 
@@ -2287,12 +2492,17 @@ static cudaError_t launch_pair_bulk(const DevState& st, const int* tab_prev, con
 // (ceil(ld / 128)); the host launches one group per value.
 // pend_slots: how many corrections can be pending at a worker (its largest degree).
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
-                              const Tile* tiles, int n_tiles, int nv, int pend_slots, cudaStream_t stream) {
+                              const Tile* tiles, int n_tiles, int nv, int pend_slots, bool raw, bool single_owner,
+                              cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
-    if (!apply_pending) return launch_pair_bulk<false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
-    if (pend_slots > 2) return cudaErrorInvalidValue;
-    return pend_slots > 1 ? launch_pair_bulk<true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
-                          : launch_pair_bulk<true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (!apply_pending) return launch_pair_bulk<false, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (pend_slots <= 1) return launch_pair_bulk<true, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (!raw || pend_slots > 4) return cudaErrorInvalidValue;
+    if (pend_slots == 2)
+        return single_owner ? launch_pair_bulk<true, 2, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
+                            : launch_pair_bulk<true, 2, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (!single_owner) return cudaErrorInvalidValue;      // degree 3 and 4: one owned end per edge only
+    return launch_pair_bulk<true, 4, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
 }
 
 template <int NVW, bool UPDATE, int D>
@@ -2413,41 +2623,51 @@ cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, 
 // Shared memory one CTA may ask for, less the kernels' static part.
 constexpr size_t kMidSmemBudget = 227 * 1024 - 512;
 
-template <int NVM, bool UPDATE, int D>
+template <int NVM, bool UPDATE, int D, bool RAW, int ENDS>
 static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
                                 int n_tiles, int ld_pad, cudaStream_t stream) {
-    const size_t smem = sizeof(float) * (1 + 2 * D) * static_cast<size_t>(ld_pad);
     // TMA-fed variant when the row fits its registers and at least two stages fit in shared memory
     if constexpr (NVM <= kMidBulkNv) {
         const size_t stage = sizeof(float) * 2 * mid_rows(NVM) * static_cast<size_t>(ld_pad);
         // leave room for the second CTA where the kernel is built for two per SM
-        const size_t budget = kMidSmemBudget / mid_min_blocks(NVM, D);
+        const size_t budget = kMidSmemBudget / mid_min_blocks(NVM, RAW ? (ENDS * D + 1) / 2 : D);
         const int n_stage = (int)std::min<size_t>(budget / stage, kMidStagesMax);
         if (n_stage >= 2) {
             const size_t total = n_stage * stage;
-            cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_bulk_kernel<NVM, UPDATE, D>,
+            cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_bulk_kernel<NVM, UPDATE, D, RAW, ENDS>,
                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
             if (rc != cudaSuccess) return rc;
-            launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_bulk_kernel<NVM, UPDATE, D>, dim3(n_tiles), dim3(256), total, stream, st, tab_prev, tab_cur, tiles, ld_pad, n_stage);
+            launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_bulk_kernel<NVM, UPDATE, D, RAW, ENDS>, dim3(n_tiles), dim3(256), total, stream, st, tab_prev, tab_cur, tiles, ld_pad, n_stage);
             return cudaGetLastError();
         }
     }
-    if (smem > 48 * 1024) {
-        cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_kernel<NVM, UPDATE, D>,
-                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (rc != cudaSuccess) return rc;
+    if constexpr (RAW) {
+        return cudaErrorInvalidValue;      // the host gives the raw form only rows the TMA-fed kernel takes
+    } else {
+        const size_t smem = sizeof(float) * (1 + 2 * D) * static_cast<size_t>(ld_pad);
+        if (smem > 48 * 1024) {
+            cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_kernel<NVM, UPDATE, D>,
+                                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (rc != cudaSuccess) return rc;
+        }
+        launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_kernel<NVM, UPDATE, D>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles, ld_pad);
+        return cudaGetLastError();
     }
-    launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_kernel<NVM, UPDATE, D>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles, ld_pad);
-    return cudaGetLastError();
 }
 
 template <int NVM>
 static cudaError_t launch_mid(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd, int pend_slots,
-                              const Tile* tiles, int n_tiles, int ld_pad, cudaStream_t stream) {
-    if (!upd) return launch_mid_t<NVM, false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+                              bool raw, bool single_owner, const Tile* tiles, int n_tiles, int ld_pad,
+                              cudaStream_t stream) {
+    if (!upd) return launch_mid_t<NVM, false, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
     if (pend_slots > 2) return cudaErrorInvalidValue;
-    return pend_slots > 1 ? launch_mid_t<NVM, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream)
-                          : launch_mid_t<NVM, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    if (pend_slots <= 1) return launch_mid_t<NVM, true, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    if constexpr (NVM <= kMidBulkNv) {
+        if (raw)
+            return single_owner ? launch_mid_t<NVM, true, 2, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream)
+                                : launch_mid_t<NVM, true, 2, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    }
+    return launch_mid_t<NVM, true, 2, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
 }
 
 template <int NVM, bool UPDATE>
@@ -2483,21 +2703,21 @@ static cudaError_t launch_mid2(const DevState& st, const int* tab, bool upd, con
 
 cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const int* tab_cur,
                                   bool apply_pending, const Tile* tiles, int n_tiles, int nv, int ld_pad,
-                                  int pend_slots, cudaStream_t stream) {
+                                  int pend_slots, bool raw, bool single_owner, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
     if (st.rank == 2) {
         if (tab_prev != tab_cur || pend_slots != 2) return cudaErrorInvalidValue;
         return launch_mid2(st, tab_cur, apply_pending, tiles, n_tiles, ld_pad, stream);
     }
     switch (nv) {
-        case 1: return launch_mid<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
-        case 2: return launch_mid<2>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
-        case 3: return launch_mid<3>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
-        case 4: return launch_mid<4>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
-        case 5: return launch_mid<5>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
-        case 6: return launch_mid<6>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
-        case 7: return launch_mid<7>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
-        default: return launch_mid<8>(st, tab_prev, tab_cur, apply_pending, pend_slots, tiles, n_tiles, ld_pad, stream);
+        case 1: return launch_mid<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        case 2: return launch_mid<2>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        case 3: return launch_mid<3>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        case 4: return launch_mid<4>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        case 5: return launch_mid<5>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        case 6: return launch_mid<6>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        case 7: return launch_mid<7>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        default: return launch_mid<8>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
     }
 }
 
