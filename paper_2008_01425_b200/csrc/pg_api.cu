@@ -89,6 +89,8 @@ bool pair_sweep_allowed() {
     return !(v && v[0] == '1');
 }
 
+constexpr int kPairChains = 2;       // chains the pair-sweep layers of a large stack are spread over
+
 // Rows per cluster tile of a wide pair-sweep layer: with `resident` clusters
 // running at once, split every edge's rows into S equal parts so that the
 // max_edges * S tiles fill whole waves as nearly as possible.
@@ -181,6 +183,8 @@ bool assign_owners(int n_workers, const std::vector<Edge>& edges, std::vector<in
     return single;
 }
 
+constexpr int kSmCount = 148;        // SMs of the one GPU this library is built for
+
 int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_layers, int rank,
                 Layout& lay, bool query_device = false) {
     if (!shapes || n_layers < 1 || n_layers > 4096) return PG_ERR_INVALID;
@@ -205,11 +209,11 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
     if (rank <= 2 && pair_sweep_allowed()) {
         if (lay.max_degree == 1) {
             lay.pair_mode = rank == 1;
-        } else if (topo.kind != PG_MATCHING && (lay.max_degree == 2 || (rank == 1 && lay.max_degree <= 4))) {
-            // Rows with several readers: the sweep forms the difference from the rows as stored, only the
-            // edge that owns a worker corrects and writes its rows (to the second copy), and the pending
-            // terms enter as vector algebra.  Degree 3 and 4 (a torus) need an assignment in which no edge
-            // owns both of its ends.
+        } else if (topo.kind != PG_MATCHING && lay.max_degree == 2) {
+            // Rows with two readers (a ring, a path): the edge that owns a worker writes its corrected
+            // rows to the second copy of X.  (Degree 4 was tried twice - every reader applying all eight
+            // corrections of a row pair, and the raw form below with one owner per worker - and both are
+            // slower than the three sweeps: a row then passes through four CTAs.)
             std::vector<Edge> edges;
             if (!pg::build_edges(topo, 0, 0, edges)) return PG_ERR_INVALID;
             std::vector<int> degree(N, 0), own;
@@ -218,7 +222,7 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
                 degree[ed.j] += 1;
             }
             const bool single = assign_owners(N, edges, own);
-            if (*std::min_element(degree.begin(), degree.end()) >= 1 && (lay.max_degree == 2 || single)) {
+            if (*std::min_element(degree.begin(), degree.end()) >= 1) {
                 lay.pair_mode = true;
                 lay.pend_slots = lay.max_degree;
                 lay.two_copies = true;
@@ -249,14 +253,13 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         const bool large_layer = rows >= 256 && static_cast<long long>(rows) * ld >= (1LL << 20);
         if (lay.two_copies && !small_stack && !large_layer) mode = 0;
         if (rank == 2 && !(mode == 3 && large_layer && ld <= pg::kPairMid2MaxLd)) mode = 0;
-        if (lay.pend_slots > 2 && mode != 1) mode = 0;      // degree 3 and 4: the row-per-warp kernel only
         return mode;
     };
-    // the raw form (see LayerGeom::raw) exists for a row per warp and for the TMA-fed CTA-per-row kernel at rank 1
+    // the raw form (see LayerGeom::raw) exists for the TMA-fed CTA-per-row kernel at rank 1
     auto raw_of = [&](int mode, int ld) {
-        return lay.two_copies && rank == 1 && (mode == 1 || (mode == 3 && ld <= 5 * 1024)) ? 1 : 0;
+        return lay.two_copies && rank == 1 && mode == 3 && ld <= 5 * 1024 ? 1 : 0;
     };
-    // rows the CTA-per-row sweep covers on a large stack with two readers per row (one launch a step)
+    // rows the CTA-per-row sweep covers on a large stack with two readers per row (their tiles are sized together)
     long long shared_launch_rows = 0;
     if (lay.two_copies && !small_stack)
         for (int l = 0; l < n_layers; ++l)
@@ -306,11 +309,13 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
             // (on a matching every layer of the stack shares one launch, which has tiles enough)
             int parts = lay.two_copies ? std::max(by_height, by_count) : by_height;
             if (g.pair_mode == 3 && shared_launch_rows > 0) {
-                // The large layers of such a stack share one launch: tall tiles, about two per SM over the
-                // whole launch (a tile's prologue - 5 to 6 vectors per thread - is not hidden by anything
-                // with one CTA per SM; VGG-shaped ring, tiles of 32 -> 176 rows: 0.854 -> 0.798 ms per round
-                // at rank 1, 1.049 -> 0.955 ms at rank 2; 256 rows, 1.3 CTAs per SM: 0.92 / 1.12 ms).
-                const long long target = std::max<long long>(16, shared_launch_rows * lay.max_edges / 296);
+                // The large layers of such a stack run as two chains of launches side by side (see
+                // pg_ctx::chain): tall tiles, about four for every three SMs over both chains.  A tile's
+                // prologue (the pending terms' products, the vectors into registers) is hidden by nothing
+                // with one CTA per SM, and an SM left without a tile costs as much: measured on the VGG-shaped
+                // ring of 16 at rank 1 / rank 2, tiles of 256 rows (192 tiles) 0.732 / 0.904 ms per round,
+                // 176 rows (288 tiles) 0.760 / 0.933 ms; one chain with 176 rows 0.777 / 0.934 ms.
+                const long long target = std::max<long long>(16, shared_launch_rows * lay.max_edges * 3 / (4 * kSmCount));
                 parts = std::max<int>(by_height, static_cast<int>(std::max<long long>(1, (g.n + target / 2) / target)));
             }
             g.p_rows = static_cast<int>(round_up((g.n + parts - 1) / parts, 8));
@@ -432,10 +437,23 @@ struct pg_ctx {
     bool pending = false;
     int64_t pending_key = 0;    // round whose table describes the pending correction
     int xbuf = 0;               // which copy of X is current (always 0 unless a correction is pending)
-    // layers on the three sweeps and layers on the pair sweep are independent within a round: when a
-    // stack has both, the former are enqueued on a side stream forked from and joined to the caller's
-    cudaStream_t side = nullptr;
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // Layers are independent of each other, and a power step is a chain of kernels with a short
+    // vector-only step between two sweeps over X, during which memory idles.  On large stacks the
+    // layers are therefore spread over several chains, each on a stream of the library's own: while
+    // one chain is between sweeps another one streams.  chain[0] takes the layers on the three
+    // sweeps, chain[1..] the pair-sweep layers.  The chains are forked from the caller's stream
+    // (everything enqueued there so far is waited for) and the caller's stream is made to wait for
+    // all of them at the end of every call; consecutive rounds on the same stream, with no other call
+    // on this context in between, continue the chains without a new fork, so a chain never waits
+    // for another one.
+    static constexpr int kMaxChains = 4;
+    cudaStream_t chain[kMaxChains] = {};
+    cudaEvent_t ev_fork = nullptr, ev_join[kMaxChains] = {};
+    int n_pair_chains = 0;               // chains the pair-sweep layers are spread over (0: caller's stream)
+    bool use_chains = false;
+    bool chains_open = false;            // the chains are ordered after all earlier work on chain_origin
+    cudaStream_t chain_origin = nullptr;
+    int edge_first[kMaxChains] = {}, edge_count[kMaxChains] = {};   // CTAs per edge of a chain's pair edge step
     // pg_rounds on a static graph: two steady-state rounds captured once as a CUDA graph and replayed
     cudaStream_t cap = nullptr;          // origin stream of the capture
     cudaGraphExec_t loop_exec = nullptr;
@@ -450,7 +468,7 @@ struct pg_ctx {
     Tile* d_pair_tiles = nullptr;
     Tile* d_flush_tiles = nullptr;
     // slice: widest per-CTA column slice (mode 2) or widest padded row (mode 3) in the group
-    struct PairGroup { int mode; int nv; int slice; int first; int count; double bytes; bool raw; };
+    struct PairGroup { int mode; int nv; int slice; int first; int count; double bytes; bool raw; int max_rows; int chain; };
     std::vector<PairGroup> pair_groups;   // pair tiles grouped by float4 per lane
     int64_t launches = 0;
     char* ws = nullptr;
@@ -575,6 +593,7 @@ bool bind_device(const pg_ctx* c) {
 // live model (needed before X, Q or the round counter are read or overwritten).
 // G, eta: the caller's gradient step, taken in the same pass (pair-sweep layers only).
 int flush_pending(pg_ctx* c, cudaStream_t stream, const float* G = nullptr, float eta = 0.0f) {
+    c->chains_open = false;      // whatever follows on the caller's stream must be waited for by the next round
     if (c->half_pending) {
         // the odd iteration's update p q-hat^T, with the scaled coefficients
         const int* tab = nullptr;
@@ -663,7 +682,33 @@ bool upload_tile_lists(pg_ctx* c) {
             for (int rt = 0; rt < g.t_rtiles; ++rt)
                 for (int ct = 0; ct < g.t_ctiles; ++ct) cols.push_back(Tile{v, l, rt, ct});
         }
-    // one launch per group of layers that share the kernel instantiation
+    // Chains (see pg_ctx::chain): on a large stack the pair-sweep layers are spread over two chains of
+    // about equal size (largest layer first, each to the chain with the least so far; three chains
+    // measured 2 % slower than two on the VGG-shaped ring, one chain 6 % slower).
+    std::vector<int> chain_of(n_layers, 0);
+    c->n_pair_chains = 0;
+    c->use_chains = false;
+    if (!lay.small_stack) {
+        std::vector<int> order;
+        for (int l = 0; l < n_layers; ++l)
+            if (lay.layers[l].pair_mode) order.push_back(l);
+        const int want = std::min<int>({kPairChains, pg_ctx::kMaxChains - 1, static_cast<int>(order.size())});
+        if (want >= 2 || (want >= 1 && !rows.empty())) {
+            std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+                return static_cast<long long>(lay.layers[a].n) * lay.layers[a].ld >
+                       static_cast<long long>(lay.layers[b].n) * lay.layers[b].ld;
+            });
+            std::vector<double> load(want, 0.0);
+            for (int l : order) {
+                const int k = static_cast<int>(std::min_element(load.begin(), load.end()) - load.begin());
+                chain_of[l] = k;
+                load[k] += static_cast<double>(lay.layers[l].n) * lay.layers[l].ld;
+            }
+            c->n_pair_chains = want;
+            c->use_chains = true;
+        }
+    }
+    // one launch per group of layers that share the kernel instantiation (and the chain)
     auto group_of = [&](const LayerGeom& g, int* nv, int* slice) {
         if (g.pair_mode == 1) {
             *nv = (g.ld + 127) / 128;
@@ -683,13 +728,17 @@ bool upload_tile_lists(pg_ctx* c) {
         group_of(lay.layers[l0], &nv0, &slice0);
         const int first = static_cast<int>(pairs.size());
         double bytes = 0.0;   // every worker's rows read from memory once and written once
+        int max_rows = 0;     // tallest tile of the group
         for (int l = l0; l < n_layers; ++l) {
             const LayerGeom& g = lay.layers[l];
             int nv = 0, slice = 0;
-            if (!g.pair_mode || done[l] || g.pair_mode != lay.layers[l0].pair_mode || g.raw != lay.layers[l0].raw) continue;
+            if (!g.pair_mode || done[l] || g.pair_mode != lay.layers[l0].pair_mode || g.raw != lay.layers[l0].raw ||
+                chain_of[l] != chain_of[l0])
+                continue;
             group_of(g, &nv, &slice);
             if (nv != nv0) continue;
             slice0 = std::max(slice0, slice);     // sizes the shared-memory vectors of the launch
+            max_rows = std::max(max_rows, g.p_rows);
             done[l] = 1;
             if (lay.two_copies) {
                 // the readers of a row block run next to each other, so the second one finds it in L2
@@ -703,33 +752,35 @@ bool upload_tile_lists(pg_ctx* c) {
         }
         const int count = static_cast<int>(pairs.size()) - first;
         c->pair_groups.push_back(pg_ctx::PairGroup{lay.layers[l0].pair_mode, nv0, slice0, first, count, bytes,
-                                                   lay.layers[l0].raw != 0});
+                                                   lay.layers[l0].raw != 0, max_rows, chain_of[l0]});
     }
-    // a group with fewer than two tiles per SM joins the next group of its kind with longer rows
-    // (the kernels take any row up to their template's width): fewer, fuller launches
+    // Launch order: longest rows first (the costliest tiles start first, the cheaper ones fill the end of
+    // the launch).  A group with fewer than two tiles per SM joins the group before it, of its kind with
+    // longer rows (the kernels take any row up to their template's width): fewer, fuller launches.
     {
         std::vector<pg_ctx::PairGroup>& gr = c->pair_groups;
         std::stable_sort(gr.begin(), gr.end(), [](const pg_ctx::PairGroup& a, const pg_ctx::PairGroup& b) {
-            return a.mode != b.mode ? a.mode < b.mode : (a.raw != b.raw ? a.raw < b.raw : a.nv < b.nv);
+            if (a.chain != b.chain) return a.chain < b.chain;
+            return a.mode != b.mode ? a.mode < b.mode : (a.raw != b.raw ? a.raw < b.raw : a.nv > b.nv);
         });
         std::vector<Tile> merged;
         std::vector<pg_ctx::PairGroup> out;
         merged.reserve(pairs.size());
         for (size_t i = 0; i < gr.size(); ++i) {
-            pg_ctx::PairGroup cur = gr[i];
+            const pg_ctx::PairGroup& cur = gr[i];
             const int first = static_cast<int>(merged.size());
             merged.insert(merged.end(), pairs.begin() + cur.first, pairs.begin() + cur.first + cur.count);
-            while (cur.mode != 2 && cur.count < 296 && i + 1 < gr.size() && gr[i + 1].mode == cur.mode &&
-                   gr[i + 1].raw == cur.raw) {
-                const pg_ctx::PairGroup& nx = gr[++i];
-                merged.insert(merged.end(), pairs.begin() + nx.first, pairs.begin() + nx.first + nx.count);
-                cur.nv = nx.nv;
-                cur.slice = std::max(cur.slice, nx.slice);
-                cur.count += nx.count;
-                cur.bytes += nx.bytes;
+            if (!out.empty() && cur.mode != 2 && cur.count < 2 * kSmCount && out.back().mode == cur.mode &&
+                out.back().raw == cur.raw && out.back().chain == cur.chain) {
+                pg_ctx::PairGroup& prev = out.back();       // its tiles end where these begin
+                prev.slice = std::max(prev.slice, cur.slice);
+                prev.count += cur.count;
+                prev.bytes += cur.bytes;
+                prev.max_rows = std::max(prev.max_rows, cur.max_rows);
+            } else {
+                out.push_back(cur);
+                out.back().first = first;
             }
-            cur.first = first;
-            out.push_back(cur);
         }
         pairs.swap(merged);
         gr.swap(out);
@@ -747,18 +798,24 @@ bool upload_tile_lists(pg_ctx* c) {
     auto put = [](Tile* dst, const std::vector<Tile>& v) {
         return v.empty() || cudaMemcpy(dst, v.data(), sizeof(Tile) * v.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     };
-    // the CTAs of the pair edge step of one edge: (layer, chunk)
+    // the CTAs of the pair edge step of one edge, chain by chain: (layer, chunk)
     std::vector<int> edge_tab;
-    for (int l = 0; l < n_layers; ++l)
-        if (lay.layers[l].pair_mode)
-            for (int ch = 0; ch < lay.layers[l].e_chunks; ++ch) {
-                edge_tab.push_back(l);
-                edge_tab.push_back(ch);
-            }
+    for (int k = 0; k < std::max(c->n_pair_chains, 1); ++k) {
+        c->edge_first[k] = static_cast<int>(edge_tab.size() / 2);
+        for (int l = 0; l < n_layers; ++l)
+            if (lay.layers[l].pair_mode && chain_of[l] == k)
+                for (int ch = 0; ch < lay.layers[l].e_chunks; ++ch) {
+                    edge_tab.push_back(l);
+                    edge_tab.push_back(ch);
+                }
+        c->edge_count[k] = static_cast<int>(edge_tab.size() / 2) - c->edge_first[k];
+    }
     c->st.e_total = static_cast<int>(edge_tab.size() / 2);
     if (!edge_tab.empty() && cudaMemcpy(c->ws + lay.off_edge_tab, edge_tab.data(), sizeof(int) * edge_tab.size(),
                                         cudaMemcpyHostToDevice) != cudaSuccess)
         return false;
+    // kernels that share the GPU with another chain's are launched plainly
+    c->st.dep_launch = dependent_launch_mask(lay.small_stack, c->use_chains);
     return cudaMemcpy(c->ws + lay.off_layers, lay.layers.data(), sizeof(LayerGeom) * n_layers, cudaMemcpyHostToDevice) ==
                cudaSuccess &&
            put(c->d_row_tiles, rows) && put(c->d_col_tiles, cols) && put(c->d_pair_tiles, pairs) &&
@@ -893,7 +950,6 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.Qn2 = reinterpret_cast<double*>(c->ws + lay.off_Qn2);
     st.Pn = reinterpret_cast<float*>(c->ws + lay.off_Pn);
     st.half_odd = 0;
-    st.dep_launch = dependent_launch_mask(lay.small_stack, lay.n_row_tiles > 0 && lay.n_pair_tiles > 0);
     st.Y = reinterpret_cast<float*>(c->ws + lay.off_Y);
     st.Ph = reinterpret_cast<float*>(c->ws + lay.off_Ph);
     st.PhNext = st.Ph + static_cast<long long>(lay.max_edges) * lay.ph_stride;
@@ -950,9 +1006,10 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     for (int s = 0; s < kTabRing && ok; ++s)
         ok = cudaEventCreateWithFlags(&c->tab_event[s], cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->cap, cudaStreamNonBlocking) == cudaSuccess;
-    ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess &&
-         cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
-         cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int k = 0; k < pg_ctx::kMaxChains && ok; ++k)
+        ok = cudaStreamCreateWithFlags(&c->chain[k], cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->ev_join[k], cudaEventDisableTiming) == cudaSuccess;
     if (ok) {
         ok = pg::launch_column_norms(st, lay.n_pairs, nullptr) == cudaSuccess;
         c->launches += 1;
@@ -976,8 +1033,10 @@ void pg_destroy(pg_ctx* c) {
     for (int s = 0; s < kTabRing; ++s)
         if (c->tab_event[s]) cudaEventDestroy(c->tab_event[s]);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
-    if (c->ev_join) cudaEventDestroy(c->ev_join);
-    if (c->side) cudaStreamDestroy(c->side);
+    for (int k = 0; k < pg_ctx::kMaxChains; ++k) {
+        if (c->ev_join[k]) cudaEventDestroy(c->ev_join[k]);
+        if (c->chain[k]) cudaStreamDestroy(c->chain[k]);
+    }
     if (c->loop_exec) cudaGraphExecDestroy(c->loop_exec);
     if (c->cap) cudaStreamDestroy(c->cap);
     if (c->h_tabs) cudaFreeHost(c->h_tabs);
@@ -1171,14 +1230,21 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
         }
         return PG_OK;
     }
-    // a stack with layers on both paths: the three sweeps of this round go to the side stream
-    const bool forked = n_rows > 0 && has_pair;
-    cudaStream_t s3 = stream;
-    if (forked) {
-        ok = cudaEventRecord(c->ev_fork, stream) == cudaSuccess &&
-             cudaStreamWaitEvent(c->side, c->ev_fork, 0) == cudaSuccess;
-        s3 = c->side;
+    // Large stacks: the layers' chains of kernels go to the library's streams (see pg_ctx::chain)
+    const bool chained = c->use_chains;
+    cudaStream_t s3 = stream;                       // the three sweeps
+    if (chained) {
+        if (!c->chains_open || c->chain_origin != stream || !c->static_graph) {
+            // fork: every chain waits for what the caller's stream holds now (uploads, this round's table)
+            ok = cudaEventRecord(c->ev_fork, stream) == cudaSuccess;
+            for (int k = 0; k <= c->n_pair_chains && ok; ++k)
+                ok = cudaStreamWaitEvent(c->chain[k], c->ev_fork, 0) == cudaSuccess;
+            c->chains_open = true;
+            c->chain_origin = stream;
+        }
+        s3 = c->chain[0];
     }
+    auto pair_stream = [&](int chain) { return chained ? c->chain[1 + chain] : stream; };
     if (n_rows > 0 && !c->y_valid) {
         Timed t(c, PG_KERNEL_FORWARD, s3, c->normal_param_bytes);
         ok = ok && pg::launch_forward(c->st, tab, c->d_row_tiles, n_rows, s3) == cudaSuccess;
@@ -1230,41 +1296,51 @@ static int round_impl(pg_ctx* c, void* stream_v, const float* G, float eta) {
             const bool flip = c->lay.two_copies && c->pending;
             st.X = c->st.X + c->xbuf * copy_elems;
             st.Xw = flip ? c->st.X + (c->xbuf ^ 1) * copy_elems : st.X;
-            for (const auto& grp : c->pair_groups) {
-                // without a pending correction the sweep only reads
-                Timed t(c, PG_KERNEL_PAIR_SWEEP, stream, c->pending ? grp.bytes : 0.5 * grp.bytes);
-                if (grp.mode == 1)
-                    ok = ok && pg::launch_pair_sweep(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
-                                                     grp.count, grp.nv, c->lay.pend_slots, grp.raw,
-                                                     c->lay.single_owner, stream) == cudaSuccess;
-                else if (grp.mode == 3)
-                    ok = ok && pg::launch_pair_sweep_mid(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
-                                                         grp.count, grp.nv, static_cast<int>(round_up(grp.slice, 4)),
-                                                         c->lay.pend_slots, grp.raw, c->lay.single_owner,
-                                                         stream) == cudaSuccess;
-                else
-                    ok = ok && pg::launch_pair_sweep_wide(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
-                                                          grp.count, grp.nv, grp.slice, c->lay.pend_slots,
-                                                          stream) == cudaSuccess;
-                c->launches += 1;
+            const int n_chains = std::max(c->n_pair_chains, 1);
+            for (int k = 0; k < n_chains && ok; ++k) {
+                cudaStream_t sp = pair_stream(k);
+                for (const auto& grp : c->pair_groups) {
+                    if (grp.chain != k) continue;
+                    // without a pending correction the sweep only reads
+                    Timed t(c, PG_KERNEL_PAIR_SWEEP, sp, c->pending ? grp.bytes : 0.5 * grp.bytes);
+                    if (grp.mode == 1)
+                        ok = ok && pg::launch_pair_sweep(st, tab_prev, tab, c->pending, c->d_pair_tiles + grp.first,
+                                                         grp.count, grp.nv, c->lay.pend_slots, sp) == cudaSuccess;
+                    else if (grp.mode == 3)
+                        ok = ok && pg::launch_pair_sweep_mid(st, tab_prev, tab, c->pending,
+                                                             c->d_pair_tiles + grp.first, grp.count, grp.nv,
+                                                             static_cast<int>(round_up(grp.slice, 4)),
+                                                             c->lay.pend_slots, grp.raw, c->lay.single_owner,
+                                                             grp.max_rows, sp) == cudaSuccess;
+                    else
+                        ok = ok && pg::launch_pair_sweep_wide(st, tab_prev, tab, c->pending,
+                                                              c->d_pair_tiles + grp.first, grp.count, grp.nv, grp.slice,
+                                                              c->lay.pend_slots, sp) == cudaSuccess;
+                    c->launches += 1;
+                }
+                if (c->edge_count[k] > 0) {     // the pair edge step of this chain's layers
+                    DevState se = st;
+                    se.edge_tab = c->st.edge_tab + 2 * c->edge_first[k];
+                    se.e_total = c->edge_count[k];
+                    Timed t(c, PG_KERNEL_PAIR_EDGE, sp, 0.0);
+                    ok = ok && pg::launch_pair_edge(se, tab, c->lay.max_edges, sp) == cudaSuccess;
+                    c->launches += 1;
+                }
             }
             if (flip) c->xbuf ^= 1;
-            {
-                Timed t(c, PG_KERNEL_PAIR_EDGE, stream, 0.0);
-                ok = ok && pg::launch_pair_edge(st, tab, c->lay.max_edges, stream) == cudaSuccess;
-                c->launches += 1;
-            }
             c->pending = true;
             c->pending_key = c->static_graph ? 0 : c->round;
         }
         c->step += 1;
     }
-    if (forked)   // join even after a failed launch, so the caller's stream stays ordered after the side stream
-        ok = (cudaEventRecord(c->ev_join, c->side) == cudaSuccess &&
-              cudaStreamWaitEvent(stream, c->ev_join, 0) == cudaSuccess) && ok;
+    if (chained)   // join even after a failed launch, so the caller's stream stays ordered after the chains
+        for (int k = 0; k <= c->n_pair_chains; ++k)
+            ok = (cudaEventRecord(c->ev_join[k], c->chain[k]) == cudaSuccess &&
+                  cudaStreamWaitEvent(stream, c->ev_join[k], 0) == cudaSuccess) && ok;
     if (!ok) {
         cudaGetLastError();
         c->y_valid = false;
+        c->chains_open = false;
         return PG_ERR_CUDA;
     }
     c->y_valid = true;
@@ -1337,6 +1413,7 @@ static void capture_two_rounds(pg_ctx* c, int key) {
     const int64_t round = c->round, step = c->step, launches = c->launches, pending_key = c->pending_key;
     const int xbuf = c->xbuf;
     const bool pending = c->pending, y_valid = c->y_valid;
+    c->chains_open = false;              // the captured rounds fork the chains from the capturing stream
     if (cudaStreamBeginCapture(c->cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         cudaGetLastError();
         c->loop_failed = true;
@@ -1354,6 +1431,7 @@ static void capture_two_rounds(pg_ctx* c, int key) {
     c->loop_launches = c->launches - launches;
     c->round = round; c->step = step; c->launches = launches; c->pending_key = pending_key;
     c->xbuf = xbuf; c->pending = pending; c->y_valid = y_valid;
+    c->chains_open = false;
     if (c->loop_exec) {
         cudaGraphExecDestroy(c->loop_exec);
         c->loop_exec = nullptr;
@@ -1407,6 +1485,7 @@ int pg_rounds(pg_ctx* c, int32_t n_rounds, void* stream_v) {
                             cudaGetLastError();
                             return PG_ERR_CUDA;
                         }
+                    c->chains_open = false;
                     c->round += 2LL * pairs_left;
                     c->step += 2LL * pairs_left * c->power_steps;
                     c->launches += c->loop_launches * pairs_left;
@@ -1593,6 +1672,7 @@ int pg_get_round(pg_ctx* c, int64_t* round_out) {
 int pg_set_round(pg_ctx* c, int64_t round, void* stream_v) {
     if (!c || round < 0) return PG_ERR_INVALID;
     if (c->failed) return PG_ERR_STATE;
+    c->chains_open = false;
     if (c->pending || c->half_pending) {
         // the pending correction belongs to the old round's graph: apply it first, on the
         // stream the rounds were enqueued on

@@ -30,7 +30,7 @@ constexpr int kPairWideMinBlocks = 3;  // resident CTAs per SM the cluster sweep
 constexpr int kPairWideMaxLd = 8 * 256 * 4 * kPairCluster;  // widest row the cluster variant covers
 constexpr int kEdgeChunks = 32;        // CTAs that share the pair edge step of one (edge, layer)
 constexpr int kSpPerTile = 16;         // doubles a pair-sweep tile leaves for the pair edge step, see DevState::Sp
-constexpr int kMaxTerms = 7;           // rank-1 terms that can be pending on the difference of an edge (degree 4)
+constexpr int kMaxTerms = 3;           // edges whose corrections can be pending on the difference of an edge (degree 2)
 
 // Geometry of one layer (same for every worker).
 struct LayerGeom {
@@ -58,7 +58,7 @@ struct LayerGeom {
     long long sp_off;  // per-tile scalars for the pair edge step (p_rtiles x kSpPerTile doubles)
     int e_chunks;      // CTAs that share the pair edge step of one edge on this layer (1..kEdgeChunks)
     int raw;           // pair sweep forms D from the rows as stored and leaves the pending terms to vector
-                       // algebra (graphs where a row has several readers), see pair_sweep_bulk_kernel
+                       // algebra (graphs where a row has two readers), see raw_terms
 };
 
 // One unit of work of a sweep: a tile of one worker's layer.
@@ -148,18 +148,18 @@ cudaError_t launch_random_directions(const DevState& st, const int* tab, int max
 cudaError_t launch_edge_raw(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);
 cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile* tiles, int n_tiles,
                           cudaStream_t stream);
-// pend_slots: most corrections pending at a worker (its degree); raw / single_owner: see LayerGeom::raw and
-// TabLayout::off_own (single_owner: no edge writes both of its ends)
+// pend_slots: most corrections pending at a worker (its degree)
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
-                              const Tile* tiles, int n_tiles, int nv, int pend_slots, bool raw, bool single_owner,
-                              cudaStream_t stream);
+                              const Tile* tiles, int n_tiles, int nv, int pend_slots, cudaStream_t stream);
 cudaError_t launch_pair_sweep_wide(const DevState& st, const int* tab_prev, const int* tab_cur,
                                    bool apply_pending, const Tile* tiles, int n_tiles, int nv, int slice,
                                    int pend_slots, cudaStream_t stream);
 // `tiles`: tiles of layers whose rows one CTA holds (nv float4 per thread, rows of at most ld_pad floats)
+// raw / single_owner: see LayerGeom::raw and TabLayout::off_own (single_owner: no edge writes both of its
+// ends); max_rows: tallest tile in `tiles`
 cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const int* tab_cur,
                                   bool apply_pending, const Tile* tiles, int n_tiles, int nv, int ld_pad,
-                                  int pend_slots, bool raw, bool single_owner, cudaStream_t stream);
+                                  int pend_slots, bool raw, bool single_owner, int max_rows, cudaStream_t stream);
 // Clusters of the wide pair sweep that can be resident at once (0 if unknown).
 int pair_wide_resident_clusters(int nv, int slice, int pend_slots);
 cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, cudaStream_t stream);

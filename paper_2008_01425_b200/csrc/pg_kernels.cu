@@ -879,27 +879,54 @@ __device__ __forceinline__ int raw_terms(const DevState& st, const int* __restri
     return n;
 }
 
-// Prologue of a raw sweep (whole CTA): the terms of edge e, each with its scalar
-// c_k (q'_k . q-hat) - the product in fp64 from the fp32 vectors, q_hat = `q` * qinv -
-// and the p-hat it multiplies.  s_ph / s_cb: kMaxTerms entries of shared memory.
+// Prologue of a raw sweep (whole CTA of 256 threads): the terms of edge e and, for the
+// rows [r0, r1) of the tile, the scalar each row's product loses to them,
+//     corr[r] = sum_k c_k (q'_k . q-hat) p-hat_k[r],
+// the products q'_k . q-hat taken in fp64 from the fp32 vectors (q-hat = `q` * qinv).
+// Returns the number of terms; s_ph[k] points at p-hat_k.
 __device__ int raw_prologue(const DevState& st, const int* __restrict__ tab, int e, int wi, int wj,
-                            const LayerGeom& g, const float* __restrict__ q, float qinv, const float** s_ph,
-                            float* s_cb, double* scratch) {
+                            const LayerGeom& g, const float* __restrict__ q, float qinv, int r0, int r1,
+                            float* s_corr, const float** s_ph, double* s_red /* 8 x kMaxTerms + kMaxTerms */) {
     RawTerm terms[kMaxTerms];
     const int nt = raw_terms(st, tab, e, wi, wj, terms);
-    for (int k = 0; k < nt; ++k) {
-        const float* vk = st.Qr + (long long)tab[st.tab.off_pair + terms[k].edge] * st.q_stride + g.q_off;
-        double part = 0.0;
-        for (int idx = threadIdx.x; idx < g.m; idx += blockDim.x)
-            part += (double)vk[idx] * (double)(q[idx] * qinv);
-        const double beta = block_sum(part, scratch);
-        if (threadIdx.x == 0) {
-            s_ph[k] = st.Ph + (long long)terms[k].edge * st.ph_stride + g.ph_off;
-            s_cb[k] = (float)((double)terms[k].coef * beta);
-        }
+    const float* vec[kMaxTerms];
+    double part[kMaxTerms];
+#pragma unroll
+    for (int k = 0; k < kMaxTerms; ++k) {
+        part[k] = 0.0;
+        vec[k] = q;
+        if (k < nt) vec[k] = st.Qr + (long long)tab[st.tab.off_pair + terms[k].edge] * st.q_stride + g.q_off;
+    }
+    for (int idx = threadIdx.x; idx < g.m; idx += blockDim.x) {
+        const double qh = (double)(q[idx] * qinv);
+#pragma unroll
+        for (int k = 0; k < kMaxTerms; ++k)
+            if (k < nt) part[k] += (double)vec[k][idx] * qh;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int k = 0; k < kMaxTerms; ++k) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
+        if (lane == 0) s_red[warp * kMaxTerms + k] = part[k];
     }
     __syncthreads();
-    return nt;
+    if (threadIdx.x < kMaxTerms) {
+        double beta = 0.0;
+        for (int w8 = 0; w8 < 8; ++w8) beta += s_red[w8 * kMaxTerms + threadIdx.x];
+        const int k = threadIdx.x;
+        s_red[8 * kMaxTerms + k] = k < nt ? (double)terms[k].coef * beta : 0.0;
+        s_ph[k] = st.Ph + (long long)(k < nt ? terms[k].edge : e) * st.ph_stride + g.ph_off;
+    }
+    __syncthreads();
+    for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x) {
+        float c = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kMaxTerms; ++k)
+            if (k < nt) c = fmaf((float)s_red[8 * kMaxTerms + k], __ldg(s_ph[k] + r), c);
+        s_corr[r - r0] = c;
+    }
+    return nt;      // the caller's next barrier publishes s_corr
 }
 
 // --------------------------------------------------------------------------
@@ -969,12 +996,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
     return false;
 }
 
-// RAW: the rows enter the products as stored, the pending terms as scalars (see
-// raw_terms); only the owning CTA corrects a worker's rows, and it keeps the pending
-// vectors of ENDS (1 or 2) ends of the edge in shared memory.  Otherwise (a matching:
-// each end has one previous edge and this edge is its only reader) both ends are
-// corrected before the difference is formed.
-template <int NV, bool UPDATE, int D, bool RAW, int ENDS>
+template <int NV, bool UPDATE, int D>
 __global__ void __launch_bounds__(256, 1)
 pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
                        const Tile* __restrict__ tiles) {
@@ -982,13 +1004,10 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     constexpr int STAGES = kBulkStages;
     extern __shared__ __align__(128) unsigned char s_dyn[];
     __shared__ __align__(16) float s_q[NV * 128];
-    __shared__ __align__(16) float s_u[ENDS][D][NV * 128];       // pending vectors of the ends this CTA corrects
+    __shared__ __align__(16) float s_ui[D][NV * 128];
+    __shared__ __align__(16) float s_uj[D][NV * 128];
     __shared__ __align__(8) unsigned long long s_full[STAGES];
     __shared__ double s_s[8];
-    __shared__ double s_g[8][kMaxTerms + 1];
-    __shared__ double s_scratch[33];
-    __shared__ const float* s_tph[kMaxTerms];
-    __shared__ float s_tcb[kMaxTerms];
     __shared__ int s_abort;
 
     const Tile tile = tiles[blockIdx.x];
@@ -1005,12 +1024,10 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 
     const float* q = st.Qr + (long long)pair * st.q_stride + g.q_off;
     const float qinv = pair_qinv(st, pair, tile.layer);
-    // which ends' rows this CTA writes back (to Xw, which is X itself unless rows have several readers)
-    const int own = UPDATE ? tab_cur[st.tab.off_own + e] : 0;
-    const bool st_i = (own & 1) != 0, st_j = (own & 2) != 0;
-    // which ends' rows it corrects: all that it forms the difference from, or only its own
-    const bool act_i = UPDATE && (!RAW || st_i), act_j = UPDATE && (!RAW || st_j);
-    const int slot_i = 0, slot_j = ENDS == 2 ? 1 : 0;            // where s_u keeps either end's vectors
+    // only the edge that owns a worker's rows writes them back (to Xw, which is X itself
+    // unless rows have a second reader; on a matching every edge owns both of its ends)
+    const int own = tab_cur[st.tab.off_own + e];
+    const bool own_i = (own & 1) != 0, own_j = (own & 2) != 0;
     float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
     float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
     PendingEnd<D> pi, pj;
@@ -1033,8 +1050,8 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         if (UPDATE) {
 #pragma unroll
             for (int s2 = 0; s2 < D; ++s2) {
-                if (act_i) s_u[slot_i][s2][idx] = in ? pi.vec[s2][idx] : 0.0f;
-                if (act_j) s_u[slot_j][s2][idx] = in ? pj.vec[s2][idx] : 0.0f;
+                s_ui[s2][idx] = in ? pi.vec[s2][idx] : 0.0f;
+                s_uj[s2][idx] = in ? pj.vec[s2][idx] : 0.0f;
             }
         }
     }
@@ -1054,17 +1071,12 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     if (threadIdx.x == 0)
         for (; issued < STAGES - 1 && issued < n_stages; ++issued) issue(issued);
 
-    // the pending terms of this edge, while the first rows are on their way
-    int nt = 0;
-    if (RAW && UPDATE) nt = raw_prologue(st, tab_prev, e, wi, wj, g, q, qinv, s_tph, s_tcb, s_scratch);
-
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
     float4 u[NV];
 #pragma unroll
     for (int k = 0; k < NV; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     float ssum = 0.0f;
-    double gsum = 0.0;            // lane k: this warp's share of sum_r p_r p-hat_k[r]
     bool ok = true;
 
     for (int it = 0; it < n_stages; ++it) {
@@ -1092,45 +1104,30 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                     xj[k] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
-            float phv = 0.0f;                       // RAW, lane k: p-hat_k[r] of pending term k
-            if (RAW && UPDATE && lane < nt) phv = __ldg(s_tph[lane] + r);
             if (UPDATE) {
                 float ai[D], aj[D];
 #pragma unroll
                 for (int s2 = 0; s2 < D; ++s2) {
-                    ai[s2] = (act_i && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r) : 0.0f;
-                    aj[s2] = (act_j && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r) : 0.0f;
+                    ai[s2] = pi.ph[s2] ? pi.coef[s2] * __ldg(pi.ph[s2] + r) : 0.0f;
+                    aj[s2] = pj.ph[s2] ? pj.coef[s2] * __ldg(pj.ph[s2] + r) : 0.0f;
                 }
                 float* rowi = Xi_w + (long long)r * ld;
                 float* rowj = Xj_w + (long long)r * ld;
-                if (act_i) {
 #pragma unroll
-                    for (int k = 0; k < NV; ++k) {
-                        const int col = (k * 32 + lane) * 4;
-                        float4 t = xi[k];
+                for (int k = 0; k < NV; ++k) {
+                    const int col = (k * 32 + lane) * 4;
 #pragma unroll
-                        for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
-                            const float4 v = *reinterpret_cast<const float4*>(&s_u[slot_i][s2][col]);
-                            t.x = fmaf(-ai[s2], v.x, t.x); t.y = fmaf(-ai[s2], v.y, t.y);
-                            t.z = fmaf(-ai[s2], v.z, t.z); t.w = fmaf(-ai[s2], v.w, t.w);
-                        }
-                        if (st_i && col < ld) st_stream(rowi + col, t);
-                        if (!RAW) xi[k] = t;
+                    for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
+                        const float4 vi = *reinterpret_cast<const float4*>(&s_ui[s2][col]);
+                        const float4 vj = *reinterpret_cast<const float4*>(&s_uj[s2][col]);
+                        xi[k].x = fmaf(-ai[s2], vi.x, xi[k].x); xi[k].y = fmaf(-ai[s2], vi.y, xi[k].y);
+                        xi[k].z = fmaf(-ai[s2], vi.z, xi[k].z); xi[k].w = fmaf(-ai[s2], vi.w, xi[k].w);
+                        xj[k].x = fmaf(-aj[s2], vj.x, xj[k].x); xj[k].y = fmaf(-aj[s2], vj.y, xj[k].y);
+                        xj[k].z = fmaf(-aj[s2], vj.z, xj[k].z); xj[k].w = fmaf(-aj[s2], vj.w, xj[k].w);
                     }
-                }
-                if (act_j) {
-#pragma unroll
-                    for (int k = 0; k < NV; ++k) {
-                        const int col = (k * 32 + lane) * 4;
-                        float4 t = xj[k];
-#pragma unroll
-                        for (int s2 = 0; s2 < D; ++s2) {
-                            const float4 v = *reinterpret_cast<const float4*>(&s_u[slot_j][s2][col]);
-                            t.x = fmaf(-aj[s2], v.x, t.x); t.y = fmaf(-aj[s2], v.y, t.y);
-                            t.z = fmaf(-aj[s2], v.z, t.z); t.w = fmaf(-aj[s2], v.w, t.w);
-                        }
-                        if (st_j && col < ld) st_stream(rowj + col, t);
-                        if (!RAW) xj[k] = t;
+                    if (col < ld) {
+                        if (own_i) st_stream(rowi + col, xi[k]);
+                        if (own_j) st_stream(rowj + col, xj[k]);
                     }
                 }
             }
@@ -1143,7 +1140,6 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                 dot = fmaf(xi[k].x, vq.x, dot); dot = fmaf(xi[k].y, vq.y, dot);
                 dot = fmaf(xi[k].z, vq.z, dot); dot = fmaf(xi[k].w, vq.w, dot);
             }
-            if (RAW && UPDATE && lane < nt) dot = fmaf(-s_tcb[lane], phv, dot);   // the pending terms' part of p_r
             const float p = warp_sum(dot);
 #pragma unroll
             for (int k = 0; k < NV; ++k) {
@@ -1151,7 +1147,6 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
                 u[k].z = fmaf(p, xi[k].z, u[k].z); u[k].w = fmaf(p, xi[k].w, u[k].w);
             }
             ssum = fmaf(p, p, ssum);
-            if (RAW && UPDATE) gsum += (double)p * (double)phv;
             if (lane == 0) Pw[r] = p;
         }
         __syncthreads();          // every warp is done with this slot before it is filled again
@@ -1171,7 +1166,6 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
 #pragma unroll
     for (int k = 0; k < NV; ++k) *reinterpret_cast<float4*>(&s_red[warp * NV * 128 + (k * 32 + lane) * 4]) = u[k];
     if (lane == 0) s_s[warp] = (double)ssum;
-    if (lane <= kMaxTerms) s_g[warp][lane] = gsum;
     __syncthreads();
     float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld;
     for (int idx = threadIdx.x; idx < ld; idx += 256) {
@@ -1180,16 +1174,10 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
         for (int w8 = 1; w8 < 8; ++w8) t += s_red[w8 * NV * 128 + idx];
         Up[idx] = t;
     }
-    double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile;
     if (threadIdx.x == 0) {
         double t = 0.0;
         for (int w8 = 0; w8 < 8; ++w8) t += s_s[w8];
-        sp[0] = t;
-    }
-    if (RAW && threadIdx.x < kMaxTerms) {
-        double t = 0.0;
-        for (int w8 = 0; w8 < 8; ++w8) t += s_g[w8][threadIdx.x];
-        sp[4 + threadIdx.x] = threadIdx.x < nt ? t : 0.0;
+        st.Sp[(long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile] = t;
     }
 }
 
@@ -1552,21 +1540,23 @@ __host__ __device__ constexpr int mid_rows(int nvm) { return nvm <= 2 ? 4 : 2; }
 // two CTAs per SM where the registers allow it, so one CTA's prologue hides behind the other's rows
 __host__ __device__ constexpr int mid_min_blocks(int nvm, int d) { return (1 + 2 * d) * nvm <= 10 ? 2 : 1; }
 
-// RAW / ENDS as in the row-per-warp kernel: the rows enter the products as stored, the
-// pending terms as one scalar per row, and the thread keeps in registers only the
-// pending vectors of the ENDS (1 or 2) ends whose rows this CTA may have to write.
+// RAW (graphs where a row has two readers; see raw_terms): the rows enter the products
+// as stored and the pending terms as one scalar per row; only the CTA that owns a worker
+// corrects and writes its rows, and the thread keeps in registers the pending vectors of
+// just the ENDS (1 or 2) ends this CTA may own.  The per-row scalars (that correction of
+// p_r, the coefficients of the owned rows' corrections, and p_r itself for the terms'
+// products at the end) sit in shared memory behind the stages, `rows_pad` floats each.
 template <int NVM, bool UPDATE, int D, bool RAW, int ENDS>
 __global__ void __launch_bounds__(256, mid_min_blocks(NVM, RAW ? (ENDS * D + 1) / 2 : D))
 pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int* __restrict__ tab_cur,
-                           const Tile* __restrict__ tiles, int ld_pad, int n_stage) {
+                           const Tile* __restrict__ tiles, int ld_pad, int n_stage, int rows_pad) {
     grid_dependency_sync();
-    extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][RS * ld_pad]
+    extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][RS * ld_pad], then the scalars
     __shared__ __align__(8) unsigned long long s_full[kMidStagesMax];
     constexpr int RS = mid_rows(NVM);
     __shared__ float s_warp[2][RS][8];
-    __shared__ double s_scratch[33];
+    __shared__ double s_red[8 * kMaxTerms + kMaxTerms];
     __shared__ const float* s_tph[kMaxTerms];
-    __shared__ float s_tcb[kMaxTerms];
     __shared__ int s_abort;
 
     const Tile tile = tiles[blockIdx.x];
@@ -1591,15 +1581,20 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
     // ENDS == 1: the vectors of the one end this CTA corrects (worker j if `one_is_j`)
     const bool one_is_j = ENDS == 1 && !act_i;
-    PendingEnd<D> pi, pj;
-    if (UPDATE) {
-        pending_of<D>(st, tab_prev, one_is_j ? wj : wi, g, q, pi);
-        if (ENDS == 2) pending_of<D>(st, tab_prev, wj, g, q, pj);
-    }
     const bool act_a = ENDS == 1 ? (act_i || act_j) : act_i;     // the end whose vectors are in va
+    PendingEnd<D> pa, pb;
+    if (UPDATE) {
+        pending_of<D>(st, tab_prev, one_is_j ? wj : wi, g, q, pa);
+        if (ENDS == 2) pending_of<D>(st, tab_prev, wj, g, q, pb);
+    }
     const int r0 = tile.rtile * g.p_rows;
     const int r1 = min(g.n, r0 + g.p_rows);
     const int n_iter = (r1 - r0 + RS - 1) / RS;
+    // per-row scalars behind the stages (RAW only)
+    float* s_corr = s_stage + (size_t)n_stage * 2 * RS * ld_pad;
+    float* s_p = s_corr + rows_pad;
+    float* s_ca = s_p + rows_pad;                     // [D][rows_pad]: coefficients of end a's corrections
+    float* s_cb = s_ca + (size_t)D * rows_pad;        // [D][rows_pad]: end b's (ENDS == 2)
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -1620,9 +1615,19 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     if (threadIdx.x == 0)
         for (; issued < n_stage && issued < n_iter; ++issued) issue(issued);
 
-    // the pending terms of this edge, while the first rows are on their way
+    // while the first rows are on their way: the pending terms of this edge and the scalars of the tile's rows
     int nt = 0;
-    if (RAW && UPDATE) nt = raw_prologue(st, tab_prev, e, wi, wj, g, q, qinv, s_tph, s_tcb, s_scratch);
+    if (RAW && UPDATE) {
+        nt = raw_prologue(st, tab_prev, e, wi, wj, g, q, qinv, r0, r1, s_corr, s_tph, s_red);
+        for (int r = r0 + threadIdx.x; r < r1; r += 256) {
+#pragma unroll
+            for (int s2 = 0; s2 < D; ++s2) {
+                s_ca[s2 * rows_pad + r - r0] = (act_a && pa.ph[s2]) ? pa.coef[s2] * __ldg(pa.ph[s2] + r) : 0.0f;
+                if (ENDS == 2) s_cb[s2 * rows_pad + r - r0] = (act_j && pb.ph[s2]) ? pb.coef[s2] * __ldg(pb.ph[s2] + r) : 0.0f;
+            }
+        }
+        __syncthreads();
+    }
 
     // this thread's columns of the vectors, for the whole tile
     float4 vq[NVM], va[D][NVM], vb[ENDS == 2 ? D : 1][ENDS == 2 ? NVM : 1];
@@ -1637,8 +1642,8 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
         }
 #pragma unroll
         for (int s2 = 0; s2 < D; ++s2) {
-            va[s2][k] = (act_a && off < ld) ? *reinterpret_cast<const float4*>(pi.vec[s2] + off) : zero;
-            if (ENDS == 2) vb[s2][k] = (act_j && off < ld) ? *reinterpret_cast<const float4*>(pj.vec[s2] + off) : zero;
+            va[s2][k] = (act_a && off < ld) ? *reinterpret_cast<const float4*>(pa.vec[s2] + off) : zero;
+            if (ENDS == 2) vb[s2][k] = (act_j && off < ld) ? *reinterpret_cast<const float4*>(pb.vec[s2] + off) : zero;
         }
     }
 
@@ -1648,7 +1653,6 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
 #pragma unroll
     for (int k = 0; k < NVM; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     float ssum = 0.0f;
-    double gsum = 0.0;            // thread k < nt: this tile's sum_r p_r p-hat_k[r]
     bool ok = true;
 
     for (int it = 0; it < n_iter; ++it) {
@@ -1659,27 +1663,21 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
         const float* sj = si + (size_t)RS * ld_pad;
         float4 d[RS][NVM];
         float dot[RS];
-        float corr[RS];           // RAW: the pending terms' part of p_r
-        float mine_ph[RS];        // RAW, thread k < nt: p-hat_k[r]
 #pragma unroll
         for (int t = 0; t < RS; ++t) {
             const bool in_row = mine && r + t < r1;
             const long long base = (long long)(r + t) * ld;
             dot[t] = 0.0f;
-            corr[t] = 0.0f;
-            mine_ph[t] = 0.0f;
-            if (RAW && UPDATE && in_row) {
-                for (int k = 0; k < nt; ++k) {
-                    const float phv = __ldg(s_tph[k] + r + t);
-                    corr[t] = fmaf(s_tcb[k], phv, corr[t]);
-                    if (threadIdx.x == k) mine_ph[t] = phv;
-                }
-            }
             float aa[D], ab[D];
 #pragma unroll
             for (int s2 = 0; s2 < D; ++s2) {
-                aa[s2] = (act_a && in_row && pi.ph[s2]) ? pi.coef[s2] * __ldg(pi.ph[s2] + r + t) : 0.0f;
-                ab[s2] = (ENDS == 2 && act_j && in_row && pj.ph[s2]) ? pj.coef[s2] * __ldg(pj.ph[s2] + r + t) : 0.0f;
+                if (RAW) {
+                    aa[s2] = (UPDATE && in_row) ? s_ca[s2 * rows_pad + r + t - r0] : 0.0f;
+                    ab[s2] = (UPDATE && ENDS == 2 && in_row) ? s_cb[s2 * rows_pad + r + t - r0] : 0.0f;
+                } else {
+                    aa[s2] = (act_a && in_row && pa.ph[s2]) ? pa.coef[s2] * __ldg(pa.ph[s2] + r + t) : 0.0f;
+                    ab[s2] = (act_j && in_row && pb.ph[s2]) ? pb.coef[s2] * __ldg(pb.ph[s2] + r + t) : 0.0f;
+                }
             }
 #pragma unroll
             for (int k = 0; k < NVM; ++k) {
@@ -1699,8 +1697,9 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
                             float4 x = one_is_j ? xj : xi;
 #pragma unroll
                             for (int s2 = 0; s2 < D; ++s2) {      // slot order, as the row sweep applies them
-                                x.x = fmaf(-aa[s2], va[s2][k].x, x.x); x.y = fmaf(-aa[s2], va[s2][k].y, x.y);
-                                x.z = fmaf(-aa[s2], va[s2][k].z, x.z); x.w = fmaf(-aa[s2], va[s2][k].w, x.w);
+                                const float4 v = va[s2][k];
+                                x.x = fmaf(-aa[s2], v.x, x.x); x.y = fmaf(-aa[s2], v.y, x.y);
+                                x.z = fmaf(-aa[s2], v.z, x.z); x.w = fmaf(-aa[s2], v.w, x.w);
                             }
                             st_stream((one_is_j ? Xj_w : Xi_w) + base + off, x);
                         }
@@ -1708,8 +1707,9 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
                         if (act_i) {
 #pragma unroll
                             for (int s2 = 0; s2 < D; ++s2) {
-                                xi.x = fmaf(-aa[s2], va[s2][k].x, xi.x); xi.y = fmaf(-aa[s2], va[s2][k].y, xi.y);
-                                xi.z = fmaf(-aa[s2], va[s2][k].z, xi.z); xi.w = fmaf(-aa[s2], va[s2][k].w, xi.w);
+                                const float4 v = va[s2][k];
+                                xi.x = fmaf(-aa[s2], v.x, xi.x); xi.y = fmaf(-aa[s2], v.y, xi.y);
+                                xi.z = fmaf(-aa[s2], v.z, xi.z); xi.w = fmaf(-aa[s2], v.w, xi.w);
                             }
                             if (st_i) st_stream(Xi_w + base + off, xi);
                         }
@@ -1746,7 +1746,7 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
             float p = 0.0f;
 #pragma unroll
             for (int w8 = 0; w8 < 8; ++w8) p += s_warp[it & 1][t][w8];
-            if (RAW && UPDATE) p -= corr[t];
+            if (RAW && UPDATE && r + t < r1) p -= s_corr[r + t - r0];
 #pragma unroll
             for (int k = 0; k < NVM; ++k) {
                 u[k].x = fmaf(p, d[t][k].x, u[k].x); u[k].y = fmaf(p, d[t][k].y, u[k].y);
@@ -1754,8 +1754,10 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
             }
             if (r + t < r1) {
                 ssum = fmaf(p, p, ssum);
-                if (RAW && UPDATE) gsum += (double)p * (double)mine_ph[t];
-                if (threadIdx.x == 0) Pw[r + t] = p;
+                if (threadIdx.x == 0) {
+                    Pw[r + t] = p;
+                    if (RAW && UPDATE) s_p[r + t - r0] = p;
+                }
             }
         }
     }
@@ -1777,7 +1779,18 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     }
     double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile;
     if (threadIdx.x == 0) sp[0] = (double)ssum;
-    if (RAW && threadIdx.x < kMaxTerms) sp[4 + threadIdx.x] = threadIdx.x < nt ? gsum : 0.0;
+    if (RAW) {
+        // this tile's share of p-hat_k . p for every pending term: warp k adds it up in row order
+        __syncthreads();          // s_p complete
+        if (warp < kMaxTerms) {
+            double a = 0.0;
+            if (warp < nt)
+                for (int r = r0 + lane; r < r1; r += 32) a += (double)s_p[r - r0] * (double)__ldg(s_tph[warp] + r);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+            if (lane == 0) sp[4 + warp] = a;
+        }
+    }
 }
 
 // --------------------------------------------------------------------------
@@ -2159,22 +2172,14 @@ __device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab,
 // the stored vector alone and zeroes p-hat.  LayerGeom::e_chunks CTAs per (edge,
 // layer), each taking a slice of the rows and of the columns; st.edge_tab lists
 // the (layer, chunk) pairs of one edge.
-__global__ void __launch_bounds__(256)
-pair_edge_kernel(DevState st, const int* __restrict__ tab) {
-    grid_dependency_sync();
+// `pending`: the sweep ran on rows with corrections pending (the raw form's terms apply).
+__device__ void pair_edge_rank1(const DevState& st, const int* __restrict__ tab, int e, int l, int chunk, int nch,
+                                bool pending) {
     __shared__ double scratch[33];
     __shared__ double s_tot[kMaxTerms + 1];
+    __shared__ double s_grp[8][32];
     const int L = st.n_layers;
-    const int e = blockIdx.x / st.e_total;
-    const int slot = blockIdx.x - e * st.e_total;
-    const int l = st.edge_tab[2 * slot], chunk = st.edge_tab[2 * slot + 1];
-    if (e >= tab[st.tab.off_n_edges]) return;
     const LayerGeom g = st.layers[l];
-    if (!g.pair_mode) return;
-    if (st.rank == 2) {
-        pair_edge_rank2(st, tab, e, l, chunk, scratch);
-        return;
-    }
     const int pair = tab[st.tab.off_pair + e];
     const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
     // Raw sweep with corrections pending: the terms of this edge (same order as in the sweep).
@@ -2182,7 +2187,7 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     // (w = 1 + k); every chunk's CTA gets the same bits.
     RawTerm terms[kMaxTerms];
     int nt = 0;
-    if (g.raw && st.raw_pending)
+    if (g.raw && pending)
         nt = raw_terms(st, tab, e, tab[st.tab.off_edge_i + e], tab[st.tab.off_edge_j + e], terms);
     {
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -2201,7 +2206,6 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     const bool live = finite && nn > 0.0;
     const double inv = live ? 1.0 / sqrt(nn) : 0.0;
     float* P = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
-    const int nch = g.e_chunks;
     const int rw = (g.npad + nch - 1) / nch;
     for (int r = chunk * rw + threadIdx.x; r < min(g.npad, (chunk + 1) * rw); r += blockDim.x)
         P[r] = (live && r < g.n) ? (float)((double)P[r] * inv) : 0.0f;
@@ -2235,7 +2239,6 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
     if (cw <= 32) {
         // few columns, many tiles: 8 thread groups each add every 8th tile's share, then the
         // groups are added in order (a fixed order, so the result is reproducible)
-        __shared__ double s_grp[8][32];
         const int col = threadIdx.x & 31, grp = threadIdx.x >> 5;
         const int c = c_lo + col;
         double a = 0.0;
@@ -2277,6 +2280,23 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
         st.Qn2[((long long)pair * L + l) * kEdgeChunks + chunk] = qq;
         if (!isfinite(qq)) atomicOr(st.status, 1 << kStatusNumeric);
     }
+}
+
+__global__ void __launch_bounds__(256)
+pair_edge_kernel(DevState st, const int* __restrict__ tab) {
+    grid_dependency_sync();
+    __shared__ double scratch[33];
+    const int e = blockIdx.x / st.e_total;
+    const int slot = blockIdx.x - e * st.e_total;
+    const int l = st.edge_tab[2 * slot], chunk = st.edge_tab[2 * slot + 1];
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[l];
+    if (!g.pair_mode) return;
+    if (st.rank == 2) {
+        pair_edge_rank2(st, tab, e, l, chunk, scratch);
+        return;
+    }
+    pair_edge_rank1(st, tab, e, l, chunk, g.e_chunks, st.raw_pending != 0);
 }
 
 // 1 / ||column|| of every stored right factor (after initialisation or an
@@ -2458,33 +2478,33 @@ cudaError_t launch_update(const DevState& st, const int* tab_update, const Tile*
     return launch_row<true, false, false>(st, tab_update, tab_update, tiles, n_tiles, stream);
 }
 
-template <int NV, bool UPDATE, int D, bool RAW, int ENDS>
+template <int NV, bool UPDATE, int D>
 static cudaError_t launch_pair_bulk_t(const DevState& st, const int* tab_prev, const int* tab_cur,
                                       const Tile* tiles, int n_tiles, int max_ld, cudaStream_t stream) {
     // stage buffers; they also hold the 8 x NV*128 floats of the final reduction
     size_t smem = sizeof(float) * (size_t)kBulkStages * 2 * kBulkRows * max_ld;
     const size_t red = sizeof(float) * 8 * NV * 128;
     if (smem < red) smem = red;
-    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE, D, RAW, ENDS>,
+    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_bulk_kernel<NV, UPDATE, D>,
                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (rc != cudaSuccess) return rc;
-    launch_dep(st.dep_launch & kDepPairRow, pair_sweep_bulk_kernel<NV, UPDATE, D, RAW, ENDS>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles);
+    launch_dep(st.dep_launch & kDepPairRow, pair_sweep_bulk_kernel<NV, UPDATE, D>, dim3(n_tiles), dim3(256), smem, stream, st, tab_prev, tab_cur, tiles);
     return cudaGetLastError();
 }
 
-template <bool UPDATE, int D, bool RAW, int ENDS>
+template <bool UPDATE, int D>
 static cudaError_t launch_pair_bulk(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
                                     int n_tiles, int nv, cudaStream_t stream) {
     const int max_ld = nv * 128;
     switch (nv) {
-        case 1: return launch_pair_bulk_t<1, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 2: return launch_pair_bulk_t<2, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 3: return launch_pair_bulk_t<3, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 4: return launch_pair_bulk_t<4, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 5: return launch_pair_bulk_t<5, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 6: return launch_pair_bulk_t<6, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        case 7: return launch_pair_bulk_t<7, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
-        default: return launch_pair_bulk_t<8, UPDATE, D, RAW, ENDS>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 1: return launch_pair_bulk_t<1, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 2: return launch_pair_bulk_t<2, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 3: return launch_pair_bulk_t<3, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 4: return launch_pair_bulk_t<4, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 5: return launch_pair_bulk_t<5, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 6: return launch_pair_bulk_t<6, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        case 7: return launch_pair_bulk_t<7, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
+        default: return launch_pair_bulk_t<8, UPDATE, D>(st, tab_prev, tab_cur, tiles, n_tiles, max_ld, stream);
     }
 }
 
@@ -2492,17 +2512,12 @@ static cudaError_t launch_pair_bulk(const DevState& st, const int* tab_prev, con
 // (ceil(ld / 128)); the host launches one group per value.
 // pend_slots: how many corrections can be pending at a worker (its largest degree).
 cudaError_t launch_pair_sweep(const DevState& st, const int* tab_prev, const int* tab_cur, bool apply_pending,
-                              const Tile* tiles, int n_tiles, int nv, int pend_slots, bool raw, bool single_owner,
-                              cudaStream_t stream) {
+                              const Tile* tiles, int n_tiles, int nv, int pend_slots, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
-    if (!apply_pending) return launch_pair_bulk<false, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
-    if (pend_slots <= 1) return launch_pair_bulk<true, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
-    if (!raw || pend_slots > 4) return cudaErrorInvalidValue;
-    if (pend_slots == 2)
-        return single_owner ? launch_pair_bulk<true, 2, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
-                            : launch_pair_bulk<true, 2, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
-    if (!single_owner) return cudaErrorInvalidValue;      // degree 3 and 4: one owned end per edge only
-    return launch_pair_bulk<true, 4, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (!apply_pending) return launch_pair_bulk<false, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
+    if (pend_slots > 2) return cudaErrorInvalidValue;
+    return pend_slots > 1 ? launch_pair_bulk<true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream)
+                          : launch_pair_bulk<true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, nv, stream);
 }
 
 template <int NVW, bool UPDATE, int D>
@@ -2621,23 +2636,26 @@ cudaError_t launch_pair_edge(const DevState& st, const int* tab, int max_edges, 
 }
 
 // Shared memory one CTA may ask for, less the kernels' static part.
-constexpr size_t kMidSmemBudget = 227 * 1024 - 512;
+constexpr size_t kMidSmemBudget = 227 * 1024 - 1024;
 
 template <int NVM, bool UPDATE, int D, bool RAW, int ENDS>
 static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const int* tab_cur, const Tile* tiles,
-                                int n_tiles, int ld_pad, cudaStream_t stream) {
+                                int n_tiles, int ld_pad, int max_rows, cudaStream_t stream) {
     // TMA-fed variant when the row fits its registers and at least two stages fit in shared memory
     if constexpr (NVM <= kMidBulkNv) {
+        // the raw form keeps 2 + ENDS * D scalars per row of the tile behind the stages
+        const int rows_pad = (max_rows + 3) / 4 * 4;
+        const size_t scalars = RAW ? sizeof(float) * (2 + ENDS * D) * static_cast<size_t>(rows_pad) : 0;
         const size_t stage = sizeof(float) * 2 * mid_rows(NVM) * static_cast<size_t>(ld_pad);
         // leave room for the second CTA where the kernel is built for two per SM
         const size_t budget = kMidSmemBudget / mid_min_blocks(NVM, RAW ? (ENDS * D + 1) / 2 : D);
-        const int n_stage = (int)std::min<size_t>(budget / stage, kMidStagesMax);
+        const int n_stage = budget > scalars ? (int)std::min<size_t>((budget - scalars) / stage, kMidStagesMax) : 0;
         if (n_stage >= 2) {
-            const size_t total = n_stage * stage;
+            const size_t total = n_stage * stage + scalars;
             cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid_bulk_kernel<NVM, UPDATE, D, RAW, ENDS>,
                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
             if (rc != cudaSuccess) return rc;
-            launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_bulk_kernel<NVM, UPDATE, D, RAW, ENDS>, dim3(n_tiles), dim3(256), total, stream, st, tab_prev, tab_cur, tiles, ld_pad, n_stage);
+            launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid_bulk_kernel<NVM, UPDATE, D, RAW, ENDS>, dim3(n_tiles), dim3(256), total, stream, st, tab_prev, tab_cur, tiles, ld_pad, n_stage, rows_pad);
             return cudaGetLastError();
         }
     }
@@ -2657,17 +2675,17 @@ static cudaError_t launch_mid_t(const DevState& st, const int* tab_prev, const i
 
 template <int NVM>
 static cudaError_t launch_mid(const DevState& st, const int* tab_prev, const int* tab_cur, bool upd, int pend_slots,
-                              bool raw, bool single_owner, const Tile* tiles, int n_tiles, int ld_pad,
+                              bool raw, bool single_owner, const Tile* tiles, int n_tiles, int ld_pad, int max_rows,
                               cudaStream_t stream) {
-    if (!upd) return launch_mid_t<NVM, false, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    if (!upd) return launch_mid_t<NVM, false, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, max_rows, stream);
     if (pend_slots > 2) return cudaErrorInvalidValue;
-    if (pend_slots <= 1) return launch_mid_t<NVM, true, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    if (pend_slots <= 1) return launch_mid_t<NVM, true, 1, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, max_rows, stream);
     if constexpr (NVM <= kMidBulkNv) {
         if (raw)
-            return single_owner ? launch_mid_t<NVM, true, 2, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream)
-                                : launch_mid_t<NVM, true, 2, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+            return single_owner ? launch_mid_t<NVM, true, 2, true, 1>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, max_rows, stream)
+                                : launch_mid_t<NVM, true, 2, true, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, max_rows, stream);
     }
-    return launch_mid_t<NVM, true, 2, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, stream);
+    return launch_mid_t<NVM, true, 2, false, 2>(st, tab_prev, tab_cur, tiles, n_tiles, ld_pad, max_rows, stream);
 }
 
 template <int NVM, bool UPDATE>
@@ -2703,21 +2721,21 @@ static cudaError_t launch_mid2(const DevState& st, const int* tab, bool upd, con
 
 cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const int* tab_cur,
                                   bool apply_pending, const Tile* tiles, int n_tiles, int nv, int ld_pad,
-                                  int pend_slots, bool raw, bool single_owner, cudaStream_t stream) {
+                                  int pend_slots, bool raw, bool single_owner, int max_rows, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
     if (st.rank == 2) {
         if (tab_prev != tab_cur || pend_slots != 2) return cudaErrorInvalidValue;
         return launch_mid2(st, tab_cur, apply_pending, tiles, n_tiles, ld_pad, stream);
     }
     switch (nv) {
-        case 1: return launch_mid<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
-        case 2: return launch_mid<2>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
-        case 3: return launch_mid<3>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
-        case 4: return launch_mid<4>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
-        case 5: return launch_mid<5>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
-        case 6: return launch_mid<6>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
-        case 7: return launch_mid<7>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
-        default: return launch_mid<8>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, stream);
+        case 1: return launch_mid<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 2: return launch_mid<2>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 3: return launch_mid<3>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 4: return launch_mid<4>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 5: return launch_mid<5>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 6: return launch_mid<6>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 7: return launch_mid<7>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
+        default: return launch_mid<8>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
     }
 }
 
