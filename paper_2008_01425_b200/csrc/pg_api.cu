@@ -255,9 +255,10 @@ int make_layout(const pg::Topology& topo, const pg_layer_shape* shapes, int n_la
         if (rank == 2 && !(mode == 3 && large_layer && ld <= pg::kPairMid2MaxLd)) mode = 0;
         return mode;
     };
-    // the raw form (see LayerGeom::raw) exists for the TMA-fed CTA-per-row kernel at rank 1
+    // the raw form (see LayerGeom::raw) exists for the TMA-fed CTA-per-row kernels: at rank 1, and at rank 2
+    // where no edge owns both of its ends
     auto raw_of = [&](int mode, int ld) {
-        return lay.two_copies && rank == 1 && mode == 3 && ld <= 5 * 1024 ? 1 : 0;
+        return lay.two_copies && mode == 3 && ld <= 5 * 1024 && (rank == 1 || (rank == 2 && lay.single_owner)) ? 1 : 0;
     };
     // rows the CTA-per-row sweep covers on a large stack with two readers per row (their tiles are sized together)
     long long shared_launch_rows = 0;
@@ -688,7 +689,9 @@ bool upload_tile_lists(pg_ctx* c) {
     std::vector<int> chain_of(n_layers, 0);
     c->n_pair_chains = 0;
     c->use_chains = false;
-    if (!lay.small_stack) {
+    // (not on a time-varying graph: a round there is two long launches and a new table, and side by side
+    //  they ran 5 % slower on the LSTM-shaped stack: the cluster sweep wants the GPU to itself)
+    if (!lay.small_stack && c->static_graph) {
         std::vector<int> order;
         for (int l = 0; l < n_layers; ++l)
             if (lay.layers[l].pair_mode) order.push_back(l);

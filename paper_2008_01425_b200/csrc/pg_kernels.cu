@@ -2073,6 +2073,296 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
     }
 }
 
+// The raw form of the rank-2 sweep (see raw_terms), for graphs in which no edge owns both of
+// its ends, with corrections pending.  The rows enter P = D [q-hat_0 q-hat_1] and U = D^T P as
+// stored; with D' = D - sum_k c_k (p-hat_{k,0} q'_{k,0}^T + p-hat_{k,1} q'_{k,1}^T) over the pending
+// edges k,
+//     P[r][c]   -= sum_{k,c'} c_k (q'_{k,c'} . q-hat_c) p-hat_{k,c'}[r]        (one scalar per row and column)
+//     U[:, c]   -= sum_{k,c'} c_k (p-hat_{k,c'} . P[:, c]) q'_{k,c'}            (by the pair edge step)
+// and only the CTA that owns a worker's rows applies its four pending rank-1 terms (slot order,
+// columns in order) and writes the rows.  A thread keeps the columns of the edge's two vectors and
+// of the owned end's four in registers; the per-row scalars sit behind the stages.
+template <int NVM>
+__global__ void __launch_bounds__(kMid2Threads, 1)
+pair_sweep_mid2_raw_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles, int ld_pad,
+                           int n_stage, int rows_pad) {
+    grid_dependency_sync();
+    constexpr int R = 2;
+    constexpr int NT = kMid2Threads;
+    constexpr int RS = mid2_rows(NVM);
+    constexpr int NB = kMaxTerms * R * R;      // products q'_{k,c'} . q-hat_c
+    extern __shared__ __align__(128) float s_stage[];            // [slot][matrix][RS * ld_pad], then the scalars
+    __shared__ __align__(8) unsigned long long s_full[kMidStagesMax];
+    __shared__ float s_warp[2][RS][R][NT / 32];
+    __shared__ double s_red[NT / 32][NB];
+    __shared__ float s_beta[NB];                // c_k (q'_{k,c'} . q-hat_c), index (k * 2 + c') * 2 + c
+    __shared__ const float* s_tph[kMaxTerms];
+    __shared__ int s_abort;
+
+    const Tile tile = tiles[blockIdx.x];
+    const int e = tile.worker;
+    if (e >= tab[st.tab.off_n_edges]) return;
+    const LayerGeom g = st.layers[tile.layer];
+    const int wi = tab[st.tab.off_edge_i + e], wj = tab[st.tab.off_edge_j + e];
+    const int pair = tab[st.tab.off_pair + e];
+    const float* __restrict__ Xi = st.X + (long long)wi * st.x_stride + g.x_off;
+    const float* __restrict__ Xj = st.X + (long long)wj * st.x_stride + g.x_off;
+    const int ld = g.ld;
+    const unsigned row_bytes = (unsigned)ld * 4u;     // multiple of 16: ld is a multiple of 4
+    const int md = st.tab.max_degree;
+
+    const float* q = st.Qr + (long long)pair * st.q_stride + g.q_off;
+    const float qinv0 = pair_qinv(st, pair, tile.layer, 0), qinv1 = pair_qinv(st, pair, tile.layer, 1);
+    // the end whose rows this CTA corrects and writes (if any), and its pending edges in slot order
+    const int own = tab[st.tab.off_own + e];
+    const bool act = own != 0;
+    const bool own_j = (own & 1) == 0;
+    const int wo = own_j ? wj : wi;
+    float* Xo_w = st.Xw + (long long)wo * st.x_stride + g.x_off;
+    const float* o_vec[2] = {q, q};
+    const float* o_ph[2] = {nullptr, nullptr};
+    float o_coef[2] = {0.f, 0.f};
+    if (act) {
+        const int deg = min(tab[st.tab.off_degree + wo], 2);
+        for (int s2 = 0; s2 < deg; ++s2) {
+            const int ep = tab[st.tab.off_slot_edge + wo * md + s2];
+            o_vec[s2] = st.Qr + (long long)tab[st.tab.off_pair + ep] * st.q_stride + g.q_off;
+            o_ph[s2] = st.Ph + (long long)ep * st.ph_stride + g.ph_off;
+            o_coef[s2] = __int_as_float(tab[st.tab.off_slot_coef + wo * md + s2]);
+        }
+    }
+    const int r0 = tile.rtile * g.p_rows;
+    const int r1 = min(g.n, r0 + g.p_rows);
+    const int n_iter = (r1 - r0 + RS - 1) / RS;
+    // per-row scalars behind the stages
+    float* s_corr = s_stage + (size_t)n_stage * 2 * RS * ld_pad;     // [R][rows_pad]
+    float* s_p = s_corr + (size_t)R * rows_pad;                       // [R][rows_pad]
+    float* s_oa = s_p + (size_t)R * rows_pad;                         // [2 slots][R][rows_pad]
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s2 = 0; s2 < n_stage; ++s2) mbar_init(&s_full[s2], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    auto issue = [&](int idx) {       // rows r0 + idx*RS ... into slot idx % n_stage
+        const int slot = idx % n_stage;
+        const int row = r0 + idx * RS;
+        const unsigned bytes = (unsigned)min(RS, r1 - row) * row_bytes;
+        float* dst = s_stage + (size_t)slot * 2 * RS * ld_pad;
+        mbar_expect_tx(&s_full[slot], 2 * bytes);
+        bulk_load(dst, Xi + (long long)row * ld, bytes, &s_full[slot]);
+        bulk_load(dst + (size_t)RS * ld_pad, Xj + (long long)row * ld, bytes, &s_full[slot]);
+    };
+    int issued = 0;
+    if (threadIdx.x == 0)
+        for (; issued < n_stage && issued < n_iter; ++issued) issue(issued);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // while the first rows are on their way: the pending terms, their products with the unit columns ...
+    RawTerm terms[kMaxTerms];
+    const int nt = raw_terms(st, tab, e, wi, wj, terms);
+    {
+        double part[NB];
+        const float* tv[kMaxTerms];
+#pragma unroll
+        for (int k = 0; k < kMaxTerms; ++k)
+            tv[k] = k < nt ? st.Qr + (long long)tab[st.tab.off_pair + terms[k].edge] * st.q_stride + g.q_off : q;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) part[b] = 0.0;
+        for (int idx = threadIdx.x; idx < g.m; idx += NT) {
+            const double qh0 = (double)(q[idx] * qinv0), qh1 = (double)(q[(long long)ld + idx] * qinv1);
+#pragma unroll
+            for (int k = 0; k < kMaxTerms; ++k)
+                if (k < nt) {
+#pragma unroll
+                    for (int c2 = 0; c2 < R; ++c2) {
+                        const double v = (double)tv[k][(long long)c2 * ld + idx];
+                        part[(k * R + c2) * R + 0] += v * qh0;
+                        part[(k * R + c2) * R + 1] += v * qh1;
+                    }
+                }
+        }
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) part[b] += __shfl_xor_sync(0xffffffffu, part[b], o);
+            if (lane == 0) s_red[warp][b] = part[b];
+        }
+        __syncthreads();
+        if (threadIdx.x < NB) {
+            double t = 0.0;
+            for (int w8 = 0; w8 < NT / 32; ++w8) t += s_red[w8][threadIdx.x];
+            const int k = threadIdx.x / (R * R);
+            s_beta[threadIdx.x] = k < nt ? (float)((double)terms[k].coef * t) : 0.0f;
+        }
+        if (threadIdx.x < kMaxTerms)
+            s_tph[threadIdx.x] = st.Ph + (long long)(threadIdx.x < nt ? terms[threadIdx.x].edge : e) * st.ph_stride + g.ph_off;
+        __syncthreads();
+    }
+    // ... and the scalars of the tile's rows: what the pending terms take from P[r][c], and the
+    // coefficients of the owned rows' four corrections
+    for (int r = r0 + threadIdx.x; r < r1; r += NT) {
+        float c0 = 0.0f, c1 = 0.0f;
+        for (int k = 0; k < nt; ++k)
+#pragma unroll
+            for (int c2 = 0; c2 < R; ++c2) {
+                const float phv = __ldg(s_tph[k] + (long long)c2 * g.npad + r);
+                c0 = fmaf(s_beta[(k * R + c2) * R + 0], phv, c0);
+                c1 = fmaf(s_beta[(k * R + c2) * R + 1], phv, c1);
+            }
+        s_corr[r - r0] = c0;
+        s_corr[rows_pad + r - r0] = c1;
+#pragma unroll
+        for (int s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+            for (int c2 = 0; c2 < R; ++c2)
+                s_oa[(size_t)(s2 * R + c2) * rows_pad + r - r0] =
+                    o_ph[s2] ? -o_coef[s2] * __ldg(o_ph[s2] + (long long)c2 * g.npad + r) : 0.0f;
+    }
+    __syncthreads();
+
+    // this thread's columns of the edge's two vectors and of the owned end's four, for the whole tile
+    float4 vq[R][NVM], vo[2][R][NVM];
+#pragma unroll
+    for (int k = 0; k < NVM; ++k) {
+        const int off = (k * NT + threadIdx.x) * 4;
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < R; ++c) {
+            vq[c][k] = off < ld ? *reinterpret_cast<const float4*>(q + (long long)c * ld + off) : zero;
+#pragma unroll
+            for (int s2 = 0; s2 < 2; ++s2)
+                vo[s2][c][k] = (act && off < ld) ? *reinterpret_cast<const float4*>(o_vec[s2] + (long long)c * ld + off) : zero;
+        }
+    }
+
+    float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    float4 u[R][NVM];
+#pragma unroll
+    for (int c = 0; c < R; ++c)
+#pragma unroll
+        for (int k = 0; k < NVM; ++k) u[c][k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    double g00 = 0.0, g01 = 0.0, g11 = 0.0;       // this tile's share of P^T P (thread 0)
+    bool ok = true;
+
+    for (int it = 0; it < n_iter; ++it) {
+        const int r = r0 + it * RS;
+        const int slot = it % n_stage;
+        const bool mine = mbar_wait_bounded(&s_full[slot], (unsigned)((it / n_stage) & 1), &s_abort, st.status);
+        const float* si_rows = s_stage + (size_t)slot * 2 * RS * ld_pad;      // rows follow each other ld floats apart
+        const float* sj_rows = si_rows + (size_t)RS * ld_pad;
+        float4 d[RS][NVM];
+        float2 dot[RS][R];      // even and odd columns apart until the warp's sum
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            const bool in_row = mine && r + t < r1;
+            const long long base = (long long)(r + t) * ld;
+            dot[t][0] = dot[t][1] = make_float2(0.f, 0.f);
+            float oa[2][R];
+#pragma unroll
+            for (int s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+                for (int c = 0; c < R; ++c)
+                    oa[s2][c] = (act && in_row) ? s_oa[(size_t)(s2 * R + c) * rows_pad + r + t - r0] : 0.0f;
+#pragma unroll
+            for (int k = 0; k < NVM; ++k) {
+                const int off = (k * NT + threadIdx.x) * 4;
+                const bool in = in_row && off < ld;
+                float4 xi = make_float4(0.f, 0.f, 0.f, 0.f), xj = xi;
+                if (in) {
+                    xi = *reinterpret_cast<const float4*>(si_rows + (size_t)t * ld + off);
+                    xj = *reinterpret_cast<const float4*>(sj_rows + (size_t)t * ld + off);
+                }
+                d[t][k] = sub4(xi, xj);
+                if (act && in) {
+                    float4 x = own_j ? xj : xi;
+                    fma4(x, oa[0][0], vo[0][0][k]); fma4(x, oa[0][1], vo[0][1][k]);
+                    fma4(x, oa[1][0], vo[1][0][k]); fma4(x, oa[1][1], vo[1][1][k]);
+                    st_stream(Xo_w + base + off, x);
+                }
+#pragma unroll
+                for (int c = 0; c < R; ++c) dot4(dot[t][c], d[t][k], vq[c][k]);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < RS; ++t)
+#pragma unroll
+            for (int c = 0; c < R; ++c) {
+                const float sum = warp_sum(dot[t][c].x + dot[t][c].y);
+                if (lane == 0) s_warp[it & 1][t][c][warp] = sum;
+            }
+        ok = __syncthreads_and(mine) != 0;        // shares visible, stage drained; all go on or all leave
+        if (!ok) break;
+        if (threadIdx.x == 0 && it + n_stage < n_iter) {
+            issue(it + n_stage);
+            issued = it + n_stage + 1;
+        }
+#pragma unroll
+        for (int t = 0; t < RS; ++t) {
+            float p[R];
+#pragma unroll
+            for (int c = 0; c < R; ++c) {
+                p[c] = 0.0f;
+#pragma unroll
+                for (int w8 = 0; w8 < NT / 32; ++w8) p[c] += s_warp[it & 1][t][c][w8];
+            }
+            const int rr = min(r + t, r1 - 1) - r0;
+            p[0] = p[0] * qinv0 - s_corr[rr];        // the products with the unit columns, less the pending terms' part
+            p[1] = p[1] * qinv1 - s_corr[rows_pad + rr];
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+#pragma unroll
+                for (int k = 0; k < NVM; ++k) fma4(u[c][k], p[c], d[t][k]);
+            if (threadIdx.x == 0 && r + t < r1) {
+                g00 += (double)p[0] * (double)p[0];
+                g01 += (double)p[0] * (double)p[1];
+                g11 += (double)p[1] * (double)p[1];
+                Pw[r + t] = p[0];
+                Pw[g.npad + r + t] = p[1];
+                s_p[rr] = p[0];
+                s_p[rows_pad + rr] = p[1];
+            }
+        }
+    }
+    if (!ok) {
+        // leave only after the copies still in flight have landed (bounded)
+        if (threadIdx.x == 0)
+            for (int idx = 0; idx < issued; ++idx) {
+                const int slot = idx % n_stage;
+                for (int spin = 0; spin < kBulkSpinLimit; ++spin)
+                    if (mbar_try_wait(&s_full[slot], (unsigned)((idx / n_stage) & 1))) break;
+            }
+        return;
+    }
+    float* __restrict__ Up = st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * R * ld;
+#pragma unroll
+    for (int c = 0; c < R; ++c)
+#pragma unroll
+        for (int k = 0; k < NVM; ++k) {
+            const int off = (k * NT + threadIdx.x) * 4;
+            if (off < ld) *reinterpret_cast<float4*>(Up + (long long)c * ld + off) = u[c][k];
+        }
+    double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile;
+    if (threadIdx.x == 0) {
+        sp[0] = g00;
+        sp[1] = g01;
+        sp[2] = g11;
+    }
+    // this tile's share of p-hat_{k,c'} . P[:, c] for every pending term: warp (k, c', c) adds it up in row order
+    __syncthreads();          // s_p complete
+    if (warp < NB) {
+        const int k = warp / (R * R), c2 = (warp / R) % R, c = warp % R;
+        double a = 0.0;
+        if (k < nt)
+            for (int r = r0 + lane; r < r1; r += 32)
+                a += (double)s_p[(size_t)c * rows_pad + r - r0] * (double)__ldg(s_tph[k] + (long long)c2 * g.npad + r);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane == 0) sp[4 + warp] = a;
+    }
+}
+
 // Pair edge step at rank 2: the Gram matrix P^T P from the tiles' shares, then the
 // Gram-Schmidt step in column order as a 2 x 2 triangular map applied to P (in place,
 // giving P-hat) and to U = D^T P (giving Q').  Column 0 is dead iff its squared norm
@@ -2094,6 +2384,24 @@ __device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab,
     const double g00 = block_sum(a00, scratch);      // same order, hence same bits, in every chunk
     const double g01 = block_sum(a01, scratch);
     const double g11 = block_sum(a11, scratch);
+    // Raw sweep with corrections pending: U[:, c] -= sum_{k,c'} c_k (p-hat_{k,c'} . P[:, c]) q'_{k,c'}.
+    // Warp w < 12 adds product w = (k * 2 + c') * 2 + c of every tile in tile order.
+    __shared__ double s_gam[kMaxTerms * 4];
+    RawTerm terms[kMaxTerms];
+    int nt = 0;
+    if (g.raw && st.raw_pending)
+        nt = raw_terms(st, tab, e, tab[st.tab.off_edge_i + e], tab[st.tab.off_edge_j + e], terms);
+    {
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        for (int w = warp; w < nt * 4; w += (int)blockDim.x / 32) {
+            double a = 0.0;
+            for (int t = lane; t < g.p_rtiles; t += 32) a += sp[(long long)t * kSpPerTile + 4 + w];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+            if (lane == 0) s_gam[w] = a * (double)terms[w / 4].coef;
+        }
+        __syncthreads();
+    }
     const bool finite = isfinite(g00) && isfinite(g01) && isfinite(g11);
     const bool live0 = finite && g00 > 0.0;
     const double inv0 = live0 ? 1.0 / sqrt(g00) : 0.0;
@@ -2143,6 +2451,12 @@ __device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab,
                 u0 += (double)v0[j];
                 u1 += (double)v1[j];
             }
+        }
+        for (int k = 0; k < nt; ++k) {
+            const float* tv = st.Qr + (long long)tab[st.tab.off_pair + terms[k].edge] * st.q_stride + g.q_off;
+            const double t0 = (double)tv[c], t1 = (double)tv[g.ld + c];
+            u0 -= s_gam[(k * 2 + 0) * 2 + 0] * t0 + s_gam[(k * 2 + 1) * 2 + 0] * t1;
+            u1 -= s_gam[(k * 2 + 0) * 2 + 1] * t0 + s_gam[(k * 2 + 1) * 2 + 1] * t1;
         }
         const double q0 = u0 * inv0;
         if (live0) {
@@ -2703,10 +3017,36 @@ static cudaError_t launch_mid2_t(const DevState& st, const int* tab, const Tile*
     return cudaGetLastError();
 }
 
+template <int NVM>
+static cudaError_t launch_mid2_raw_t(const DevState& st, const int* tab, const Tile* tiles, int n_tiles, int ld_pad,
+                                     int max_rows, cudaStream_t stream) {
+    const size_t stage = sizeof(float) * 2 * mid2_rows(NVM) * static_cast<size_t>(ld_pad);
+    const int rows_pad = (max_rows + 3) / 4 * 4;
+    const size_t scalars = sizeof(float) * 8 * static_cast<size_t>(rows_pad);       // 2 + 2 + 4 per row
+    const size_t budget = kMidSmemBudget - 2048;                                    // the kernel's static part
+    const int n_stage = budget > scalars ? (int)std::min<size_t>((budget - scalars) / stage, kMidStagesMax) : 0;
+    if (n_stage < 2) return cudaErrorInvalidValue;
+    const size_t total = n_stage * stage + scalars;
+    cudaError_t rc = cudaFuncSetAttribute(pair_sweep_mid2_raw_kernel<NVM>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)total);
+    if (rc != cudaSuccess) return rc;
+    launch_dep(st.dep_launch & kDepPairMid, pair_sweep_mid2_raw_kernel<NVM>, dim3(n_tiles), dim3(kMid2Threads),
+               total, stream, st, tab, tiles, ld_pad, n_stage, rows_pad);
+    return cudaGetLastError();
+}
+
 // Rank 2: static graphs only, so one table serves the pending corrections and the step.
-static cudaError_t launch_mid2(const DevState& st, const int* tab, bool upd, const Tile* tiles, int n_tiles,
-                               int ld_pad, cudaStream_t stream) {
-    switch ((ld_pad / 4 + kMid2Threads - 1) / kMid2Threads) {     // float4 per thread and row
+static cudaError_t launch_mid2(const DevState& st, const int* tab, bool upd, bool raw, const Tile* tiles, int n_tiles,
+                               int ld_pad, int max_rows, cudaStream_t stream) {
+    const int nvm = (ld_pad / 4 + kMid2Threads - 1) / kMid2Threads;     // float4 per thread and row
+    if (upd && raw) switch (nvm) {
+        case 1: return launch_mid2_raw_t<1>(st, tab, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 2: return launch_mid2_raw_t<2>(st, tab, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 3: return launch_mid2_raw_t<3>(st, tab, tiles, n_tiles, ld_pad, max_rows, stream);
+        case 4: return launch_mid2_raw_t<4>(st, tab, tiles, n_tiles, ld_pad, max_rows, stream);
+        default: return cudaErrorInvalidValue;
+    }
+    switch (nvm) {
         case 1: return upd ? launch_mid2_t<1, true>(st, tab, tiles, n_tiles, ld_pad, stream)
                            : launch_mid2_t<1, false>(st, tab, tiles, n_tiles, ld_pad, stream);
         case 2: return upd ? launch_mid2_t<2, true>(st, tab, tiles, n_tiles, ld_pad, stream)
@@ -2725,7 +3065,7 @@ cudaError_t launch_pair_sweep_mid(const DevState& st, const int* tab_prev, const
     if (n_tiles <= 0) return cudaSuccess;
     if (st.rank == 2) {
         if (tab_prev != tab_cur || pend_slots != 2) return cudaErrorInvalidValue;
-        return launch_mid2(st, tab_cur, apply_pending, tiles, n_tiles, ld_pad, stream);
+        return launch_mid2(st, tab_cur, apply_pending, raw, tiles, n_tiles, ld_pad, max_rows, stream);
     }
     switch (nv) {
         case 1: return launch_mid<1>(st, tab_prev, tab_cur, apply_pending, pend_slots, raw, single_owner, tiles, n_tiles, ld_pad, max_rows, stream);
