@@ -51,7 +51,8 @@ typedef enum pg_status {
     PG_ERR_STATE = 4,      /* call not allowed in the context's current state      */
     PG_ERR_TIMEOUT = 5,    /* a bounded device-side wait gave up                   */
     PG_ERR_NUMERIC = 6,    /* a norm was not finite (NaN / Inf in the parameters)  */
-    PG_ERR_TOO_LARGE = 7   /* problem exceeds the fixed scratch of a no-allocation call */
+    PG_ERR_TOO_LARGE = 7,  /* problem exceeds the fixed scratch of a no-allocation call */
+    PG_ERR_BOUNDS = 8      /* bounds-checked build only: a kernel computed an address outside its section */
 } pg_status;
 
 /* Graph kinds.  The paper's experiments use rings; Assumption A4 (Section 5.1)
@@ -302,9 +303,19 @@ PG_API int pg_rounds(pg_ctx *ctx, int32_t n_rounds, void *stream);
 PG_API int pg_selftest_barrier_timeout(pg_ctx *ctx, void *stream);
 
 /*
+ * Self-test of the bounds-checked build (the paper has no counterpart): a kernel asks the
+ * check about a range that ends one float past the parameter section, without touching it.
+ * Waits for `stream` and returns PG_ERR_BOUNDS from a library built with -DPG_BOUNDS_CHECK
+ * (python -m paper_2008_01425_b200.build --checked), PG_OK from the regular one, where the
+ * checks are compiled out.  The status word keeps the bit: use a context of its own.
+ */
+PG_API int pg_selftest_bounds_check(pg_ctx *ctx, void *stream);
+
+/*
  * Wait for `stream` and return the device status word: PG_OK; PG_ERR_NUMERIC (a norm
  * was not finite); PG_ERR_TIMEOUT (a bounded device-side wait gave up: an mbarrier or
- * the grid barrier of pg_rounds); PG_ERR_STATE (any other bit); PG_ERR_CUDA if the copy
+ * the grid barrier of pg_rounds); PG_ERR_BOUNDS (bounds-checked build only: a kernel
+ * computed an address outside its section and skipped the access); PG_ERR_STATE (any other bit); PG_ERR_CUDA if the copy
  * or the wait failed.  The bits are sticky.  After PG_ERR_TIMEOUT a kernel has left in
  * the middle of a step, so X, Q and the cached products no longer belong together: the
  * context is marked failed, and pg_round, pg_round_sgd, pg_rounds and pg_set_round

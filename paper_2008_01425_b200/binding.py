@@ -14,9 +14,11 @@ from typing import List, Optional, Sequence, Tuple
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libpowergossip.so")
+# PG_LIBRARY selects another build of the same library (the bounds-checked one, see build.py)
+LIB_PATH = os.environ.get("PG_LIBRARY") or os.path.join(_HERE, "libpowergossip.so")
 
-PG_OK, PG_ERR_INVALID, PG_ERR_WORKSPACE, PG_ERR_CUDA, PG_ERR_STATE, PG_ERR_TIMEOUT, PG_ERR_NUMERIC, PG_ERR_TOO_LARGE = range(8)
+(PG_OK, PG_ERR_INVALID, PG_ERR_WORKSPACE, PG_ERR_CUDA, PG_ERR_STATE, PG_ERR_TIMEOUT, PG_ERR_NUMERIC, PG_ERR_TOO_LARGE,
+ PG_ERR_BOUNDS) = range(9)
 PG_NOALLOC_MAX_PARTIALS = 1 << 20
 PG_RING, PG_TORUS, PG_MATCHING, PG_CUSTOM = 0, 1, 2, 3
 PG_W_UNIFORM, PG_W_METROPOLIS, PG_W_EXPLICIT = 0, 1, 2
@@ -29,7 +31,7 @@ EXPORTS = (
     "pg_transposed_product_noalloc", "pg_rounds", "pg_selftest_barrier_timeout",
     "pg_set_half_step", "pg_params_device", "pg_set_random_projection",
     "pg_round_sgd", "pg_stack_elems", "pg_stack_offset", "pg_comm_floats", "pg_comm_floats_round",
-    "pg_round_bytes",
+    "pg_round_bytes", "pg_selftest_bounds_check",
 )
 PG_POWER_ITERATION, PG_RANDOM_RIGHT, PG_RANDOM_LEFT = 0, 1, 2
 KERNEL_KINDS = ("forward", "edge_left", "transposed", "edge_right", "update_forward",
@@ -85,6 +87,7 @@ def load_library() -> ctypes.CDLL:
     L.pg_set_half_step.argtypes = [vp, i32]
     L.pg_set_random_projection.argtypes = [vp, i32]
     L.pg_selftest_barrier_timeout.argtypes = [vp, vp]
+    L.pg_selftest_bounds_check.argtypes = [vp, vp]
     L.pg_get_schedule.argtypes = [vp, i64, vp, vp, ctypes.POINTER(i32)]
     L.pg_max_edges.argtypes = [vp, ctypes.POINTER(i32)]
     L.pg_read_q.argtypes = [vp, i32, i32, i32, vp, vp]
@@ -357,6 +360,9 @@ class PowerGossip:
 
     def pg_selftest_barrier_timeout(self, stream=None) -> int:
         return int(self._lib.pg_selftest_barrier_timeout(self._h, _stream_handle(stream)))
+
+    def pg_selftest_bounds_check(self, stream=None) -> int:
+        return int(self._lib.pg_selftest_bounds_check(self._h, _stream_handle(stream)))
 
     def pg_device_status(self, stream=None) -> int:
         return int(self._lib.pg_device_status(self._h, _stream_handle(stream)))

@@ -859,6 +859,7 @@ int device_status(pg_ctx* c, cudaStream_t stream) {
         }
         return PG_ERR_TIMEOUT;
     }
+    if (word & (1 << PG_ERR_BOUNDS)) return PG_ERR_BOUNDS;
     if (word & (1 << PG_ERR_NUMERIC)) return PG_ERR_NUMERIC;
     return word == 0 ? PG_OK : PG_ERR_STATE;
 }
@@ -980,6 +981,28 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.n_workers = c->topo.n_workers;
     st.max_degree = lay.max_degree;
     st.tab = lay.tab;
+    {   // section bounds for the bounds-checked build
+        auto sec = [&](int id, size_t lo, size_t bytes) {
+            st.sec_lo[id] = c->ws + lo;
+            st.sec_hi[id] = c->ws + lo + bytes;
+        };
+        const size_t N = static_cast<size_t>(c->topo.n_workers), E = static_cast<size_t>(lay.max_edges);
+        const size_t P = static_cast<size_t>(lay.n_pairs), L = static_cast<size_t>(n_layers);
+        sec(pg::kSecX, lay.off_X, sizeof(float) * N * lay.x_stride * (lay.two_copies ? 2 : 1));
+        sec(pg::kSecQ, lay.off_Q, (lay.two_copies ? lay.off_Q2 - lay.off_Q : 0) + sizeof(float) * P * lay.q_stride);
+        sec(pg::kSecQinv, lay.off_Qinv, sizeof(float) * P * L * rank);
+        sec(pg::kSecQn2, lay.off_Qn2, sizeof(double) * P * L * rank * pg::kEdgeChunks);
+        sec(pg::kSecPn, lay.off_Pn, sizeof(float) * E * L);
+        sec(pg::kSecY, lay.off_Y, sizeof(float) * N * lay.y_stride);
+        sec(pg::kSecPh, lay.off_Ph, sizeof(float) * 2 * E * lay.ph_stride);
+        sec(pg::kSecUp, lay.off_Up, sizeof(float) * E * lay.up_stride);
+        sec(pg::kSecSp, lay.off_Sp, sizeof(double) * E * lay.sp_stride);
+        sec(pg::kSecZ, lay.off_Z, sizeof(float) * N * lay.z_stride);
+        sec(pg::kSecLive, lay.off_live, sizeof(int) * E * L * rank);
+        sec(pg::kSecTabs, lay.off_tabs, sizeof(int) * static_cast<size_t>(kTabRing + 1) * lay.tab.total_ints);
+        sec(pg::kSecTiles, lay.off_row_tiles, lay.total - lay.off_row_tiles);
+        sec(pg::kSecLayers, lay.off_layers, sizeof(LayerGeom) * L);
+    }
     c->d_tabs = reinterpret_cast<int*>(c->ws + lay.off_tabs);
     c->d_row_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_row_tiles);
     c->d_col_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_col_tiles);
@@ -1536,6 +1559,18 @@ int pg_selftest_barrier_timeout(pg_ctx* c, void* stream_v) {
     return device_status(c, stream);
 }
 
+int pg_selftest_bounds_check(pg_ctx* c, void* stream_v) {
+    if (!c) return PG_ERR_INVALID;
+    if (!bind_device(c)) return PG_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    if (pg::launch_bounds_probe(c->st, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return PG_ERR_CUDA;
+    }
+    c->launches += 1;
+    return device_status(c, stream);
+}
+
 int pg_max_edges(pg_ctx* c, int32_t* max_edges_out) {
     if (!c || !max_edges_out) return PG_ERR_INVALID;
     *max_edges_out = c->lay.max_edges;
@@ -1746,6 +1781,7 @@ const char* pg_status_string(int status) {
         case PG_ERR_TIMEOUT: return "a bounded device-side wait gave up";
         case PG_ERR_NUMERIC: return "a norm was not finite";
         case PG_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
+        case PG_ERR_BOUNDS: return "a kernel of the bounds-checked build computed an address outside its section";
         default: return "unknown status";
     }
 }

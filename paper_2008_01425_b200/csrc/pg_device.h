@@ -88,6 +88,12 @@ struct TabLayout {
     int total_ints;
 };
 
+// Sections of the workspace, for the bounds-checked build (-DPG_BOUNDS_CHECK): every kernel checks the
+// address ranges it is about to touch against the section they belong to; a range outside raises
+// the bounds bit of the status word and the access is skipped (nothing traps).
+enum : int { kSecX, kSecQ, kSecQinv, kSecQn2, kSecPn, kSecY, kSecPh, kSecUp, kSecSp, kSecZ, kSecLive, kSecTabs,
+             kSecTiles, kSecLayers, kSecCount };
+
 // Pointers into the workspace (device) plus sizes; passed to kernels by value.
 // Kernel families for DevState::dep_launch.
 enum : int { kDepSweep = 1, kDepPairRow = 2, kDepPairMid = 4, kDepPairWide = 8, kDepPairEdge = 16 };
@@ -125,6 +131,8 @@ struct DevState {
     long long x_stride, q_stride, y_stride, ph_stride, z_stride, up_stride, sp_stride;
     int n_layers, rank, n_workers, max_degree;
     TabLayout tab;
+    const char* sec_lo[kSecCount];   // first byte and one past the last byte of every workspace section
+    const char* sec_hi[kSecCount];
 };
 
 // Launchers (all asynchronous on `stream`; return the cudaError of the launch).
@@ -170,6 +178,7 @@ cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* ro
                               const Tile* col_tiles, int n_cols, int n_steps, bool forward_first, int* bar,
                               cudaStream_t stream);
 cudaError_t launch_barrier_timeout_probe(int* bar, int* status, cudaStream_t stream);
+cudaError_t launch_bounds_probe(const DevState& st, cudaStream_t stream);
 cudaError_t launch_column_norms(const DevState& st, long long n_pairs, cudaStream_t stream);
 
 }  // namespace pg

@@ -23,6 +23,23 @@ namespace {
 
 constexpr int kStatusNumeric = 6;  // PG_ERR_NUMERIC
 constexpr int kStatusTimeout = 5;  // PG_ERR_TIMEOUT
+constexpr int kStatusBounds = 8;   // PG_ERR_BOUNDS
+
+// Bounds-checked build (-DPG_BOUNDS_CHECK; the stand-in for a memory checker): PG_OOB(st, section,
+// pointer, count) is true, and raises the bounds bit of the status word, if the `count` elements at
+// `pointer` do not lie inside that section of the workspace; the caller then skips the work that
+// would touch them.  In the normal build it is the constant false and costs nothing.
+#ifdef PG_BOUNDS_CHECK
+__device__ __noinline__ bool pg_out_of_bounds(const DevState& st, int sec, const void* p, long long bytes) {
+    const char* a = static_cast<const char*>(p);
+    if (bytes <= 0 || (a >= st.sec_lo[sec] && a + bytes <= st.sec_hi[sec])) return false;
+    atomicOr(st.status, 1 << kStatusBounds);
+    return true;
+}
+#define PG_OOB(st, sec, ptr, count) pg_out_of_bounds(st, sec, ptr, (long long)(count) * (long long)sizeof(*(ptr)))
+#else
+#define PG_OOB(st, sec, ptr, count) false
+#endif
 constexpr long long kBarrierSpinLimit = 1LL << 23;   // polls before a grid barrier gives up (a few seconds)
 
 // Rows a warp of the row sweep works on at once, per number of vectors S.
@@ -169,6 +186,18 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
     const int c1 = min(g.ld, c0 + g.f_chunk);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ld = g.ld;
+    if (r1 > r0 && c1 > c0) {      // (checked build) everything this tile touches; the same for every thread
+        const long long span = (long long)(r1 - 1 - r0) * ld + (c1 - c0);
+        bool bad = PG_OOB(st, kSecX, X + (long long)r0 * ld + c0, span);
+        if (UPDATE && !FORWARD) bad = PG_OOB(st, kSecX, Xw + (long long)r0 * ld + c0, span) || bad;
+        for (int v = 0; v < nu; ++v)
+            bad = PG_OOB(st, kSecQ, sh.uq[v] + c0, c1 - c0) || PG_OOB(st, kSecPh, sh.up[v] + r0, r1 - r0) || bad;
+        for (int v = 0; v < nf; ++v)
+            bad = PG_OOB(st, kSecQ, sh.fq[v] + c0, c1 - c0) ||
+                  PG_OOB(st, kSecY, st.Y + (long long)w * st.y_stride + g.y_off +
+                                        ((long long)v * g.f_csplit + tile.ctile) * g.npad + r0, r1 - r0) || bad;
+        if (bad) return;
+    }
 
     for (int rb = r0 + warp * RT; rb < r1; rb += 8 * RT) {
         float a[RT][S];
@@ -335,6 +364,21 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
     const int r1 = min(g.n, r0 + g.t_rows);
     const int deg = tab[st.tab.off_degree + w];
     const int nv = deg * rank;
+    if (r1 > r0) {      // (checked build) everything this tile touches; the same for every thread
+        const int cb = tile.ctile * kColTileCols, ce = min(g.ld, cb + kColTileCols);
+        bool bad = ce > cb && PG_OOB(st, kSecX, X + (long long)r0 * g.ld + cb, (long long)(r1 - 1 - r0) * g.ld + (ce - cb));
+        for (int v = 0; v < nv && ce > cb; ++v) {
+            const int slot = v / rank, k = v - slot * rank;
+            const int e = tab[st.tab.off_slot_edge + w * st.tab.max_degree + slot];
+            bad = PG_OOB(st, kSecPh, st.Ph + (long long)e * st.ph_stride + g.ph_off + (long long)k * g.npad + r0, r1 - r0) ||
+                  PG_OOB(st, kSecZ, st.Z + (long long)w * st.z_stride + g.z_off +
+                                        ((long long)v * g.t_rtiles + tile.rtile) * g.ld + cb, ce - cb) || bad;
+            if (UPDATE)
+                bad = PG_OOB(st, kSecQ, st.Q + (long long)tab[st.tab.off_pair + e] * st.q_stride + g.q_off +
+                                            (long long)k * g.ld + cb, ce - cb) || bad;
+        }
+        if (bad) return;
+    }
 
     for (int idx = threadIdx.x; idx < S * kColTileRowsMax; idx += 256) {
         const int v = idx / kColTileRowsMax, rr = idx - v * kColTileRowsMax;
@@ -462,6 +506,9 @@ edge_odd_kernel(DevState st, const int* __restrict__ tab) {
     const float* yi = st.Y + (long long)wi * st.y_stride + g.y_off + (long long)si * g.f_csplit * g.npad;
     const float* yj = st.Y + (long long)wj * st.y_stride + g.y_off + (long long)sj * g.f_csplit * g.npad;
     float* Ph = st.Ph + (long long)e * st.ph_stride + g.ph_off;
+    if (PG_OOB(st, kSecY, yi, (long long)g.f_csplit * g.npad) || PG_OOB(st, kSecY, yj, (long long)g.f_csplit * g.npad) ||
+        PG_OOB(st, kSecPh, Ph, g.npad) || PG_OOB(st, kSecPn, st.Pn + (long long)e * L + l, 1))
+        return;
     auto raw = [&](int r) {
         double a = 0.0, b = 0.0;
         for (int cs = 0; cs < g.f_csplit; ++cs) {
@@ -507,6 +554,13 @@ __device__ __forceinline__ void edge_left_step(const DevState& st, const int* __
     const float* Yj = st.Y + (long long)wj * st.y_stride + g.y_off;
     float* Ph = st.Ph + (long long)e * st.ph_stride + g.ph_off;
     double coef[kMaxRank];
+    {   // (checked build) the slices of both ends' partial sums, the factor and its flags
+        const long long slice = (long long)rank * g.f_csplit * g.npad;
+        if (PG_OOB(st, kSecY, Yi + (long long)si * slice, slice) || PG_OOB(st, kSecY, Yj + (long long)sj * slice, slice) ||
+            PG_OOB(st, kSecPh, Ph, (long long)rank * g.npad) ||
+            PG_OOB(st, kSecLive, live_out + ((long long)e * L + l) * rank, rank))
+            return;
+    }
 
     if (rank == 1 && g.npad <= 4 * (int)blockDim.x) {
         // one column and at most four rows per thread: the differences stay in registers
@@ -632,6 +686,14 @@ __device__ __forceinline__ void edge_right_step(const DevState& st, const int* _
     const float* Zi = st.Z + (long long)wi * st.z_stride + g.z_off;
     const float* Zj = st.Z + (long long)wj * st.z_stride + g.z_off;
     float* Q = st.Q + (long long)pair * st.q_stride + g.q_off;
+    {   // (checked build) the slices of both ends' partial sums and the stored vectors
+        const long long slice = (long long)rank * g.t_rtiles * g.ld;
+        if (PG_OOB(st, kSecZ, Zi + (long long)si * slice, slice) || PG_OOB(st, kSecZ, Zj + (long long)sj * slice, slice) ||
+            PG_OOB(st, kSecQ, Q, (long long)rank * g.ld) ||
+            PG_OOB(st, kSecQinv, st.Qinv + ((long long)pair * L + l) * rank, rank) ||
+            PG_OOB(st, kSecLive, live_in + ((long long)e * L + l) * rank, rank))
+            return;
+    }
 
     for (int k = 0; k < rank; ++k) {
         if (!ld_i<COH>(&live_in[((long long)e * L + l) * rank + k])) continue;  // uniform over the block
@@ -727,6 +789,7 @@ random_directions_kernel(DevState st, const int* __restrict__ tab, unsigned key_
     float* dst = side == 0 ? st.Q + (long long)pair * st.q_stride + g.q_off
                            : st.Ph + (long long)e * st.ph_stride + g.ph_off;
     double coef[kMaxRank];
+    if (PG_OOB(st, side == 0 ? kSecQ : kSecPh, dst, (long long)rank * stride)) return;
     for (int k = 0; k < rank; ++k) {
         float* col = dst + (long long)k * stride;
         for (int b = threadIdx.x; 4 * b < stride; b += blockDim.x) {
@@ -788,6 +851,12 @@ edge_raw_kernel(DevState st, const int* __restrict__ tab) {
     const float* Yi = st.Y + (long long)wi * st.y_stride + g.y_off;
     const float* Yj = st.Y + (long long)wj * st.y_stride + g.y_off;
     float* Ph = st.Ph + (long long)e * st.ph_stride + g.ph_off;
+    {
+        const long long slice = (long long)rank * g.f_csplit * g.npad;
+        if (PG_OOB(st, kSecY, Yi + (long long)si * slice, slice) || PG_OOB(st, kSecY, Yj + (long long)sj * slice, slice) ||
+            PG_OOB(st, kSecPh, Ph, (long long)rank * g.npad))
+            return;
+    }
     for (int k = 0; k < rank; ++k) {
         const float* yi = Yi + (long long)(si * rank + k) * g.f_csplit * g.npad;
         const float* yj = Yj + (long long)(sj * rank + k) * g.f_csplit * g.npad;
@@ -879,6 +948,33 @@ __device__ __forceinline__ int raw_terms(const DevState& st, const int* __restri
     return n;
 }
 
+// (checked build) what a pair-sweep tile touches: rows [r0, r1) of both ends where it reads and where it
+// writes, the edge's stored vectors (`rank` columns), the rows of its raw left factor, its shares of
+// D^T P and its scalars.  True if any of it lies outside its section; the same for every thread.
+__device__ __forceinline__ bool pair_tile_out_of_bounds(const DevState& st, const LayerGeom& g, const float* Xi,
+                                                        const float* Xj, const float* Xi_w, const float* Xj_w,
+                                                        int r0, int r1, const float* q, const float* Pw,
+                                                        const float* up, int up_count, const double* sp) {
+    if (r1 <= r0) return false;
+    const long long first = (long long)r0 * g.ld, span = (long long)(r1 - r0) * g.ld;
+    bool bad = PG_OOB(st, kSecX, Xi + first, span) || PG_OOB(st, kSecX, Xj + first, span);
+    bad = PG_OOB(st, kSecX, Xi_w + first, span) || PG_OOB(st, kSecX, Xj_w + first, span) || bad;
+    bad = PG_OOB(st, kSecQ, q, (long long)st.rank * g.ld) || bad;
+    for (int k = 0; k < st.rank; ++k) bad = PG_OOB(st, kSecPh, Pw + (long long)k * g.npad + r0, r1 - r0) || bad;
+    bad = PG_OOB(st, kSecUp, up, up_count) || PG_OOB(st, kSecSp, sp, kSpPerTile) || bad;
+    return bad;
+}
+// (checked build) the vectors and left factors of the corrections pending at one end
+template <int D>
+__device__ __forceinline__ bool pending_out_of_bounds(const DevState& st, const LayerGeom& g, const PendingEnd<D>& pe,
+                                                      int r0, int r1) {
+    bool bad = false;
+#pragma unroll
+    for (int s = 0; s < D; ++s)
+        if (pe.ph[s]) bad = PG_OOB(st, kSecQ, pe.vec[s], g.ld) || PG_OOB(st, kSecPh, pe.ph[s] + r0, r1 - r0) || bad;
+    return bad;
+}
+
 // Prologue of a raw sweep (whole CTA of 256 threads): the terms of edge e and, for the
 // rows [r0, r1) of the tile, the scalar each row's product loses to them,
 //     corr[r] = sum_k c_k (q'_k . q-hat) p-hat_k[r],
@@ -888,7 +984,7 @@ __device__ int raw_prologue(const DevState& st, const int* __restrict__ tab, int
                             const LayerGeom& g, const float* __restrict__ q, float qinv, int r0, int r1,
                             float* s_corr, const float** s_ph, double* s_red /* 8 x kMaxTerms + kMaxTerms */) {
     RawTerm terms[kMaxTerms];
-    const int nt = raw_terms(st, tab, e, wi, wj, terms);
+    int nt = raw_terms(st, tab, e, wi, wj, terms);
     const float* vec[kMaxTerms];
     double part[kMaxTerms];
 #pragma unroll
@@ -897,6 +993,10 @@ __device__ int raw_prologue(const DevState& st, const int* __restrict__ tab, int
         vec[k] = q;
         if (k < nt) vec[k] = st.Qr + (long long)tab[st.tab.off_pair + terms[k].edge] * st.q_stride + g.q_off;
     }
+    for (int k = 0; k < nt; ++k)      // (checked build) a term that points outside drops all of them
+        if (PG_OOB(st, kSecQ, vec[k], g.ld) ||
+            (r1 > r0 && PG_OOB(st, kSecPh, st.Ph + (long long)terms[k].edge * st.ph_stride + g.ph_off + r0, r1 - r0)))
+            nt = 0;
     for (int idx = threadIdx.x; idx < g.m; idx += blockDim.x) {
         const double qh = (double)(q[idx] * qinv);
 #pragma unroll
@@ -1038,6 +1138,11 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     const int r0 = tile.rtile * g.p_rows;
     const int r1 = min(g.n, r0 + g.p_rows);
     const int n_stages = (r1 - r0 + kBulkRows - 1) / kBulkRows;
+    if (pair_tile_out_of_bounds(st, g, Xi, Xj, Xi_w, Xj_w, r0, r1, q, st.PhNext + (long long)e * st.ph_stride + g.ph_off,
+                                st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld, ld,
+                                st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile) ||
+        (UPDATE && (pending_out_of_bounds<D>(st, g, pi, r0, r1) || pending_out_of_bounds<D>(st, g, pj, r0, r1))))
+        return;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -1259,6 +1364,13 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     const int r0 = tile.rtile * g.p_rows;
     const int r1 = min(g.n, r0 + g.p_rows);
     float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    // (checked build; after the cluster's barrier, so that a CTA that backs out leaves no peer waiting for
+    //  its mbarriers to exist - the whole cluster sees the same tile and backs out together)
+    if (pair_tile_out_of_bounds(st, g, Xi, Xj, Xi_w, Xj_w, r0, r1, q, Pw,
+                                st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld, ld,
+                                st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile) ||
+        (UPDATE && (pending_out_of_bounds<D>(st, g, pi, r0, r1) || pending_out_of_bounds<D>(st, g, pj, r0, r1))))
+        return;
     constexpr int RS = kPairWideStep;
     float4 u[NVW];
 #pragma unroll
@@ -1438,6 +1550,11 @@ pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* 
     const int r0 = tile.rtile * g.p_rows;
     const int r1 = min(g.n, r0 + g.p_rows);
     float* __restrict__ Pw = st.PhNext + (long long)e * st.ph_stride + g.ph_off;
+    if (pair_tile_out_of_bounds(st, g, Xi, Xj, Xi_w, Xj_w, r0, r1, q, Pw,
+                                st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld, ld,
+                                st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile) ||
+        (UPDATE && (pending_out_of_bounds<D>(st, g, pi, r0, r1) || pending_out_of_bounds<D>(st, g, pj, r0, r1))))
+        return;
     float4 u[NVM];
 #pragma unroll
     for (int k = 0; k < NVM; ++k) u[k] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1595,6 +1712,13 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     float* s_p = s_corr + rows_pad;
     float* s_ca = s_p + rows_pad;                     // [D][rows_pad]: coefficients of end a's corrections
     float* s_cb = s_ca + (size_t)D * rows_pad;        // [D][rows_pad]: end b's (ENDS == 2)
+    if (pair_tile_out_of_bounds(st, g, Xi, Xj, Xi_w, Xj_w, r0, r1, q, st.PhNext + (long long)e * st.ph_stride + g.ph_off,
+                                st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * ld, ld,
+                                st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile) ||
+        (UPDATE && (pending_out_of_bounds<D>(st, g, pa, r0, r1) ||
+                    (ENDS == 2 && pending_out_of_bounds<D>(st, g, pb, r0, r1)))) ||
+        (RAW && r1 - r0 > rows_pad))
+        return;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -1911,6 +2035,13 @@ pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __r
     const int r0 = tile.rtile * g.p_rows;
     const int r1 = min(g.n, r0 + g.p_rows);
     const int n_iter = (r1 - r0 + RS - 1) / RS;
+    if (pair_tile_out_of_bounds(st, g, Xi, Xj, Xi_w, Xj_w, r0, r1, q, st.PhNext + (long long)e * st.ph_stride + g.ph_off,
+                                st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * 2 * ld, 2 * ld,
+                                st.Sp + (long long)e * st.sp_stride + g.sp_off + (long long)tile.rtile * kSpPerTile) ||
+        (UPDATE && (PG_OOB(st, kSecQ, q_oi, 2LL * ld) || PG_OOB(st, kSecQ, q_oj, 2LL * ld))) ||
+        (UPDATE && r1 > r0 && (PG_OOB(st, kSecPh, ph_e + g.npad + r0, r1 - r0) || PG_OOB(st, kSecPh, ph_oi + g.npad + r0, r1 - r0) ||
+                               PG_OOB(st, kSecPh, ph_oj + g.npad + r0, r1 - r0) || PG_OOB(st, kSecPh, ph_e + r0, r1 - r0))))
+        return;
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -2138,6 +2269,19 @@ pair_sweep_mid2_raw_kernel(DevState st, const int* __restrict__ tab, const Tile*
     float* s_corr = s_stage + (size_t)n_stage * 2 * RS * ld_pad;     // [R][rows_pad]
     float* s_p = s_corr + (size_t)R * rows_pad;                       // [R][rows_pad]
     float* s_oa = s_p + (size_t)R * rows_pad;                         // [2 slots][R][rows_pad]
+    {
+        bool bad = pair_tile_out_of_bounds(st, g, Xi, Xj, Xo_w, Xo_w, r0, r1, q,
+                                           st.PhNext + (long long)e * st.ph_stride + g.ph_off,
+                                           st.Up + (long long)e * st.up_stride + g.up_off + (long long)tile.rtile * 2 * ld,
+                                           2 * ld, st.Sp + (long long)e * st.sp_stride + g.sp_off +
+                                                       (long long)tile.rtile * kSpPerTile) ||
+                   r1 - r0 > rows_pad;
+        for (int s2 = 0; s2 < 2; ++s2)
+            if (o_ph[s2] && r1 > r0)
+                bad = PG_OOB(st, kSecQ, o_vec[s2], 2LL * ld) || PG_OOB(st, kSecPh, o_ph[s2] + r0, r1 - r0) ||
+                      PG_OOB(st, kSecPh, o_ph[s2] + g.npad + r0, r1 - r0) || bad;
+        if (bad) return;
+    }
 
     if (threadIdx.x == 0) {
         s_abort = 0;
@@ -2375,6 +2519,13 @@ __device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab,
     const LayerGeom g = st.layers[l];
     const int pair = tab[st.tab.off_pair + e];
     const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
+    if (PG_OOB(st, kSecSp, sp, (long long)g.p_rtiles * kSpPerTile) ||
+        PG_OOB(st, kSecPh, st.PhNext + (long long)e * st.ph_stride + g.ph_off, 2LL * g.npad) ||
+        PG_OOB(st, kSecUp, st.Up + (long long)e * st.up_stride + g.up_off, (long long)g.p_rtiles * 2 * g.ld) ||
+        PG_OOB(st, kSecQ, st.Qw + (long long)pair * st.q_stride + g.q_off, 2LL * g.ld) ||
+        PG_OOB(st, kSecQ, st.Qr + (long long)pair * st.q_stride + g.q_off, 2LL * g.ld) ||
+        PG_OOB(st, kSecQn2, st.Qn2 + ((long long)pair * L + l) * 2 * kEdgeChunks, 2 * kEdgeChunks))
+        return;
     double a00 = 0.0, a01 = 0.0, a11 = 0.0;
     for (int t = threadIdx.x; t < g.p_rtiles; t += blockDim.x) {
         a00 += sp[kSpPerTile * t];
@@ -2496,6 +2647,13 @@ __device__ void pair_edge_rank1(const DevState& st, const int* __restrict__ tab,
     const LayerGeom g = st.layers[l];
     const int pair = tab[st.tab.off_pair + e];
     const double* sp = st.Sp + (long long)e * st.sp_stride + g.sp_off;
+    if (PG_OOB(st, kSecSp, sp, (long long)g.p_rtiles * kSpPerTile) ||
+        PG_OOB(st, kSecPh, st.PhNext + (long long)e * st.ph_stride + g.ph_off, g.npad) ||
+        PG_OOB(st, kSecUp, st.Up + (long long)e * st.up_stride + g.up_off, (long long)g.p_rtiles * g.ld) ||
+        PG_OOB(st, kSecQ, st.Qw + (long long)pair * st.q_stride + g.q_off, g.ld) ||
+        PG_OOB(st, kSecQ, st.Qr + (long long)pair * st.q_stride + g.q_off, g.ld) ||
+        PG_OOB(st, kSecQn2, st.Qn2 + ((long long)pair * L + l) * kEdgeChunks, kEdgeChunks))
+        return;
     // Raw sweep with corrections pending: the terms of this edge (same order as in the sweep).
     // Warp w adds scalar w of every tile in tile order: ||p||^2 (w = 0) and sum_r p_r p-hat_k[r]
     // (w = 1 + k); every chunk's CTA gets the same bits.
@@ -2623,6 +2781,9 @@ column_norms_kernel(DevState st) {
     const int l = blockIdx.x - (int)pair * L;
     const LayerGeom g = st.layers[l];
     const float* Q = (g.pair_mode ? st.Qr : st.Q) + pair * st.q_stride + g.q_off;
+    if (PG_OOB(st, kSecQ, Q, (long long)rank * g.ld) || PG_OOB(st, kSecQinv, st.Qinv + (pair * L + l) * rank, rank) ||
+        PG_OOB(st, kSecQn2, st.Qn2 + (pair * L + l) * rank * kEdgeChunks, rank * kEdgeChunks))
+        return;
     for (int k = 0; k < rank; ++k) {
         double part = 0.0;
         for (int c = threadIdx.x; c < g.m; c += blockDim.x) {
@@ -3165,6 +3326,19 @@ cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* ro
     if (slots <= 4)
         return launch_persistent_t<4, kRowsPerWarp4>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
     return launch_persistent_t<8, kRowsPerWarp8>(st, tab, row_tiles, n_rows, col_tiles, n_cols, n_steps, forward_first, bar, max_blocks, stream);
+}
+
+// Asks the bounds check about one range inside the parameter section and one that ends a float past
+// it; nothing is read or written.  The checked build raises the bounds bit for the second range.
+__global__ void bounds_probe_kernel(DevState st) {
+    const float* last = reinterpret_cast<const float*>(st.sec_hi[kSecX]) - 4;
+    if (PG_OOB(st, kSecX, last, 4)) atomicOr(st.status, 1 << kStatusTimeout);     // must not happen
+    (void)PG_OOB(st, kSecX, last, 5);
+}
+
+cudaError_t launch_bounds_probe(const DevState& st, cudaStream_t stream) {
+    bounds_probe_kernel<<<1, 32, 0, stream>>>(st);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_barrier_timeout_probe(int* bar, int* status, cudaStream_t stream) {
