@@ -981,6 +981,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.n_workers = c->topo.n_workers;
     st.max_degree = lay.max_degree;
     st.tab = lay.tab;
+#ifdef PG_BOUNDS_CHECK
     {   // section bounds for the bounds-checked build
         auto sec = [&](int id, size_t lo, size_t bytes) {
             st.sec_lo[id] = c->ws + lo;
@@ -1003,6 +1004,7 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
         sec(pg::kSecTiles, lay.off_row_tiles, lay.total - lay.off_row_tiles);
         sec(pg::kSecLayers, lay.off_layers, sizeof(LayerGeom) * L);
     }
+#endif
     c->d_tabs = reinterpret_cast<int*>(c->ws + lay.off_tabs);
     c->d_row_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_row_tiles);
     c->d_col_tiles = reinterpret_cast<Tile*>(c->ws + lay.off_col_tiles);

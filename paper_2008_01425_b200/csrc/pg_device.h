@@ -131,8 +131,10 @@ struct DevState {
     long long x_stride, q_stride, y_stride, ph_stride, z_stride, up_stride, sp_stride;
     int n_layers, rank, n_workers, max_degree;
     TabLayout tab;
+#ifdef PG_BOUNDS_CHECK
     const char* sec_lo[kSecCount];   // first byte and one past the last byte of every workspace section
-    const char* sec_hi[kSecCount];
+    const char* sec_hi[kSecCount];   // (kernel parameters: only the checked build carries them)
+#endif
 };
 
 // Launchers (all asynchronous on `stream`; return the cudaError of the launch).

@@ -1126,10 +1126,11 @@ pair_sweep_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     const float qinv = pair_qinv(st, pair, tile.layer);
     // only the edge that owns a worker's rows writes them back (to Xw, which is X itself
     // unless rows have a second reader; on a matching every edge owns both of its ends)
-    const int own = tab_cur[st.tab.off_own + e];
-    const bool own_i = (own & 1) != 0, own_j = (own & 2) != 0;
-    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // (with one slot per worker every edge owns both ends and the rows are corrected in place: known at compile time)
+    const int own = D == 1 ? 3 : tab_cur[st.tab.off_own + e];
+    const bool own_i = D == 1 || (own & 1) != 0, own_j = D == 1 || (own & 2) != 0;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
     PendingEnd<D> pi, pj;
     if (UPDATE) {
         pending_of<D>(st, tab_prev, wi, g, q, pi);
@@ -1331,10 +1332,11 @@ pair_sweep_wide_kernel(DevState st, const int* __restrict__ tab_prev, const int*
     const float qinv = pair_qinv(st, pair, tile.layer);
     // only the edge that owns a worker's rows writes them back (to Xw, which is X itself
     // unless rows have a second reader; on a matching every edge owns both of its ends)
-    const int own = tab_cur[st.tab.off_own + e];
-    const bool own_i = (own & 1) != 0, own_j = (own & 2) != 0;
-    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // (with one slot per worker every edge owns both ends and the rows are corrected in place: known at compile time)
+    const int own = D == 1 ? 3 : tab_cur[st.tab.off_own + e];
+    const bool own_i = D == 1 || (own & 1) != 0, own_j = D == 1 || (own & 2) != 0;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
     PendingEnd<D> pi, pj;
     if (UPDATE) {
         pending_of<D>(st, tab_prev, wi, g, q, pi);
@@ -1524,10 +1526,11 @@ pair_sweep_mid_kernel(DevState st, const int* __restrict__ tab_prev, const int* 
     const float qinv = pair_qinv(st, pair, tile.layer);
     // only the edge that owns a worker's rows writes them back (to Xw, which is X itself
     // unless rows have a second reader; on a matching every edge owns both of its ends)
-    const int own = tab_cur[st.tab.off_own + e];
-    const bool own_i = (own & 1) != 0, own_j = (own & 2) != 0;
-    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
+    // (with one slot per worker every edge owns both ends and the rows are corrected in place: known at compile time)
+    const int own = D == 1 ? 3 : tab_cur[st.tab.off_own + e];
+    const bool own_i = D == 1 || (own & 1) != 0, own_j = D == 1 || (own & 2) != 0;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
     PendingEnd<D> pi, pj;
     if (UPDATE) {
         pending_of<D>(st, tab_prev, wi, g, q, pi);
@@ -1691,11 +1694,12 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
     const float qinv = pair_qinv(st, pair, tile.layer);
     // which ends' rows this CTA writes back (to Xw, which is X itself unless rows have several readers),
     // and which it corrects: all that it forms the difference from, or only the ones it writes
-    const int own = UPDATE ? tab_cur[st.tab.off_own + e] : 0;
-    const bool st_i = (own & 1) != 0, st_j = (own & 2) != 0;
+    // (with one slot per worker every edge owns both ends and the rows are corrected in place: known at compile time)
+    const int own = !UPDATE ? 0 : (D == 1 ? 3 : tab_cur[st.tab.off_own + e]);
+    const bool st_i = UPDATE && (D == 1 || (own & 1) != 0), st_j = UPDATE && (D == 1 || (own & 2) != 0);
     const bool act_i = UPDATE && (!RAW || st_i), act_j = UPDATE && (!RAW || st_j);
-    float* Xi_w = st.Xw + (long long)wi * st.x_stride + g.x_off;
-    float* Xj_w = st.Xw + (long long)wj * st.x_stride + g.x_off;
+    float* Xi_w = D == 1 ? const_cast<float*>(Xi) : st.Xw + (long long)wi * st.x_stride + g.x_off;
+    float* Xj_w = D == 1 ? const_cast<float*>(Xj) : st.Xw + (long long)wj * st.x_stride + g.x_off;
     // ENDS == 1: the vectors of the one end this CTA corrects (worker j if `one_is_j`)
     const bool one_is_j = ENDS == 1 && !act_i;
     const bool act_a = ENDS == 1 ? (act_i || act_j) : act_i;     // the end whose vectors are in va
@@ -2637,7 +2641,9 @@ __device__ void pair_edge_rank2(const DevState& st, const int* __restrict__ tab,
 // the stored vector alone and zeroes p-hat.  LayerGeom::e_chunks CTAs per (edge,
 // layer), each taking a slice of the rows and of the columns; st.edge_tab lists
 // the (layer, chunk) pairs of one edge.
-// `pending`: the sweep ran on rows with corrections pending (the raw form's terms apply).
+// RAW: the layer's sweep takes the raw form; `pending`: it ran on rows with corrections pending, so
+// the pending terms apply.
+template <bool RAW>
 __device__ void pair_edge_rank1(const DevState& st, const int* __restrict__ tab, int e, int l, int chunk, int nch,
                                 bool pending) {
     __shared__ double scratch[33];
@@ -2657,9 +2663,9 @@ __device__ void pair_edge_rank1(const DevState& st, const int* __restrict__ tab,
     // Raw sweep with corrections pending: the terms of this edge (same order as in the sweep).
     // Warp w adds scalar w of every tile in tile order: ||p||^2 (w = 0) and sum_r p_r p-hat_k[r]
     // (w = 1 + k); every chunk's CTA gets the same bits.
-    RawTerm terms[kMaxTerms];
+    RawTerm terms[RAW ? kMaxTerms : 1];
     int nt = 0;
-    if (g.raw && pending)
+    if (RAW && pending)
         nt = raw_terms(st, tab, e, tab[st.tab.off_edge_i + e], tab[st.tab.off_edge_j + e], terms);
     {
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -2696,10 +2702,11 @@ __device__ void pair_edge_rank1(const DevState& st, const int* __restrict__ tab,
     }
     const float* up = st.Up + (long long)e * st.up_stride + g.up_off;
     // D'^T p = D^T p - sum_k c_k (p-hat_k . p) q'_k with the previous vectors of the pending edges
-    const float* tvec[kMaxTerms];
-    double tcoef[kMaxTerms];
+    constexpr int NTERM = RAW ? kMaxTerms : 0;
+    const float* tvec[RAW ? kMaxTerms : 1];
+    double tcoef[RAW ? kMaxTerms : 1];
 #pragma unroll
-    for (int k = 0; k < kMaxTerms; ++k) {
+    for (int k = 0; k < NTERM; ++k) {
         tvec[k] = Qold;
         tcoef[k] = 0.0;
         if (k < nt) {
@@ -2723,7 +2730,7 @@ __device__ void pair_edge_rank1(const DevState& st, const int* __restrict__ tab,
 #pragma unroll
             for (int k = 0; k < 8; ++k) tot += s_grp[k][col];
 #pragma unroll
-            for (int k = 0; k < kMaxTerms; ++k)
+            for (int k = 0; k < NTERM; ++k)
                 if (k < nt) tot -= tcoef[k] * (double)tvec[k][c];
             const float q = (float)(tot * inv);
             Q[c] = q;
@@ -2740,7 +2747,7 @@ __device__ void pair_edge_rank1(const DevState& st, const int* __restrict__ tab,
                 for (int j = 0; j < 8; ++j) a += (double)v[j];
             }
 #pragma unroll
-            for (int k = 0; k < kMaxTerms; ++k)
+            for (int k = 0; k < NTERM; ++k)
                 if (k < nt) a -= tcoef[k] * (double)tvec[k][c];
             const float q = (float)(a * inv);
             Q[c] = q;
@@ -2768,7 +2775,10 @@ pair_edge_kernel(DevState st, const int* __restrict__ tab) {
         pair_edge_rank2(st, tab, e, l, chunk, scratch);
         return;
     }
-    pair_edge_rank1(st, tab, e, l, chunk, g.e_chunks, st.raw_pending != 0);
+    if (g.raw)
+        pair_edge_rank1<true>(st, tab, e, l, chunk, g.e_chunks, st.raw_pending != 0);
+    else
+        pair_edge_rank1<false>(st, tab, e, l, chunk, g.e_chunks, false);
 }
 
 // 1 / ||column|| of every stored right factor (after initialisation or an
@@ -3331,9 +3341,13 @@ cudaError_t launch_persistent(const DevState& st, const int* tab, const Tile* ro
 // Asks the bounds check about one range inside the parameter section and one that ends a float past
 // it; nothing is read or written.  The checked build raises the bounds bit for the second range.
 __global__ void bounds_probe_kernel(DevState st) {
+#ifdef PG_BOUNDS_CHECK
     const float* last = reinterpret_cast<const float*>(st.sec_hi[kSecX]) - 4;
     if (PG_OOB(st, kSecX, last, 4)) atomicOr(st.status, 1 << kStatusTimeout);     // must not happen
     (void)PG_OOB(st, kSecX, last, 5);
+#else
+    (void)st;
+#endif
 }
 
 cudaError_t launch_bounds_probe(const DevState& st, cudaStream_t stream) {
