@@ -980,6 +980,11 @@ int pg_create(const pg_topology* topo, const float* W_host, const pg_layer_shape
     st.rank = rank;
     st.n_workers = c->topo.n_workers;
     st.max_degree = lay.max_degree;
+    st.f_chunk_max = st.f_rows_max = 0;
+    for (const LayerGeom& g : lay.layers) {
+        st.f_chunk_max = std::max(st.f_chunk_max, g.f_chunk);
+        st.f_rows_max = std::max(st.f_rows_max, g.f_rows);
+    }
     st.tab = lay.tab;
 #ifdef PG_BOUNDS_CHECK
     {   // section bounds for the bounds-checked build

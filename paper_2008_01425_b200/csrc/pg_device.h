@@ -130,6 +130,7 @@ struct DevState {
     int e_total;
     long long x_stride, q_stride, y_stride, ph_stride, z_stride, up_stride, sp_stride;
     int n_layers, rank, n_workers, max_degree;
+    int f_chunk_max, f_rows_max;   // widest column chunk and tallest tile of the row-oriented sweeps over all layers
     TabLayout tab;
 #ifdef PG_BOUNDS_CHECK
     const char* sec_lo[kSecCount];   // first byte and one past the last byte of every workspace section

@@ -44,8 +44,12 @@ constexpr long long kBarrierSpinLimit = 1LL << 23;   // polls before a grid barr
 
 // Rows a warp of the row sweep works on at once, per number of vectors S.
 constexpr int kRowsPerWarp1 = 4, kRowsPerWarp2 = 4, kRowsPerWarp4 = 2, kRowsPerWarp8 = 2;
-// Resident CTAs per SM the row sweep is compiled for (caps its registers).
-constexpr int kRowMinBlocks = 4;
+// Resident CTAs per SM the row sweep is compiled for (caps its registers), per number of vectors S.
+__host__ __device__ constexpr int row_min_blocks(int s) { return s <= 2 ? 4 : (s == 4 ? 3 : 2); }
+// Stages of the row sweep's ring of rows in shared memory (see row_tile): 3 stages of 4 rows (128 bytes in
+// flight per thread, 48 KB per CTA) or 4 stages of 2 rows (96 bytes, 32 KB).
+__host__ __device__ constexpr int row_stages(int s, int rt) { return rt >= 4 ? 3 : 4; }
+constexpr size_t row_ring_bytes(int s, int rt) { return (size_t)row_stages(s, rt) * rt * 256 * sizeof(float4); }
 
 __device__ __forceinline__ float4 ld_stream(const float* p) {
     float4 v;
@@ -59,6 +63,20 @@ __device__ __forceinline__ void st_stream(float* p, const float4& v) {
     asm volatile("st.global.L1::no_allocate.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y),
                  "f"(v.z), "f"(v.w)
                  : "memory");
+}
+
+// Asynchronous 16-byte copies from global to shared memory (past L1), in groups a thread commits and
+// later waits for: the bytes in flight cost no registers.  A thread reads back only what it copied
+// itself, so no barrier is involved.
+__device__ __forceinline__ void copy_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void copy_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void copy_async_wait() {      // all but the N most recent groups have landed
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
 // Programmatic dependent launch.  Every kernel of a round starts with this pair:
@@ -135,11 +153,122 @@ struct RowShared {
     int nu, nf;
 };
 
+// The work of one float4 column step on RT rows of a row-oriented sweep, the rows' values in x:
+// the pending corrections (and the gradient step) applied and stored, then the products' partial sums.
+// QS: the vectors of the tile's column chunk are staged in shared memory (uqs / fqs: one vector every
+// `cmax` floats, `cs` = this step's first column within the chunk) instead of read through L1.
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD, bool QS = false>
+__device__ __forceinline__ void row_columns(const RowShared<S>& sh, const int nu, const int nf, float4 (&x)[RT],
+                                            const float (&a)[RT][S], float (&acc)[RT][S], const int c,
+                                            const int rb, const int r1, const float* const (&xrow)[RT],
+                                            const float* __restrict__ X, float* Xw,
+                                            const float* __restrict__ Gw, const float eta, const int m,
+                                            const int ld, const float* uqs = nullptr, const float* fqs = nullptr,
+                                            const int cmax = 0, const int cs = 0) {
+    if (UPDATE && SAME) {
+        // slot order: first every correction, then every product, as in the general case
+        float4 q[S];
+#pragma unroll
+        for (int v = 0; v < S; ++v) {
+            if (v < nu) {
+                q[v] = QS ? *reinterpret_cast<const float4*>(uqs + v * cmax + cs) : ld_vec<COH>(sh.uq[v] + c);
+#pragma unroll
+                for (int t = 0; t < RT; ++t) {
+                    x[t].x = fmaf(-a[t][v], q[v].x, x[t].x);
+                    x[t].y = fmaf(-a[t][v], q[v].y, x[t].y);
+                    x[t].z = fmaf(-a[t][v], q[v].z, x[t].z);
+                    x[t].w = fmaf(-a[t][v], q[v].w, x[t].w);
+                }
+            }
+        }
+        if (GRAD) {
+#pragma unroll
+            for (int t = 0; t < RT; ++t) {
+                float4 gv = ld_stream(Gw + (xrow[t] - X) + c);
+                // columns past the matrix are padding: X keeps zeros there whatever G holds
+                if (c + 1 >= m) gv.y = 0.0f;
+                if (c + 2 >= m) gv.z = 0.0f;
+                if (c + 3 >= m) gv.w = 0.0f;
+                x[t].x = fmaf(-eta, gv.x, x[t].x); x[t].y = fmaf(-eta, gv.y, x[t].y);
+                x[t].z = fmaf(-eta, gv.z, x[t].z); x[t].w = fmaf(-eta, gv.w, x[t].w);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < RT; ++t)
+            if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
+#pragma unroll
+        for (int v = 0; v < S; ++v) {
+            if (v < nu) {
+#pragma unroll
+                for (int t = 0; t < RT; ++t) {
+                    acc[t][v] = fmaf(x[t].x, q[v].x, acc[t][v]);
+                    acc[t][v] = fmaf(x[t].y, q[v].y, acc[t][v]);
+                    acc[t][v] = fmaf(x[t].z, q[v].z, acc[t][v]);
+                    acc[t][v] = fmaf(x[t].w, q[v].w, acc[t][v]);
+                }
+            }
+        }
+    } else if (UPDATE) {
+#pragma unroll
+        for (int v = 0; v < S; ++v) {
+            if (v < nu) {
+                const float4 q = QS ? *reinterpret_cast<const float4*>(uqs + v * cmax + cs) : ld_vec<COH>(sh.uq[v] + c);
+#pragma unroll
+                for (int t = 0; t < RT; ++t) {
+                    x[t].x = fmaf(-a[t][v], q.x, x[t].x);
+                    x[t].y = fmaf(-a[t][v], q.y, x[t].y);
+                    x[t].z = fmaf(-a[t][v], q.z, x[t].z);
+                    x[t].w = fmaf(-a[t][v], q.w, x[t].w);
+                }
+            }
+        }
+        if (GRAD) {
+#pragma unroll
+            for (int t = 0; t < RT; ++t) {
+                float4 gv = ld_stream(Gw + (xrow[t] - X) + c);
+                // columns past the matrix are padding: X keeps zeros there whatever G holds
+                if (c + 1 >= m) gv.y = 0.0f;
+                if (c + 2 >= m) gv.z = 0.0f;
+                if (c + 3 >= m) gv.w = 0.0f;
+                x[t].x = fmaf(-eta, gv.x, x[t].x); x[t].y = fmaf(-eta, gv.y, x[t].y);
+                x[t].z = fmaf(-eta, gv.z, x[t].z); x[t].w = fmaf(-eta, gv.w, x[t].w);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < RT; ++t)
+            if (rb + t < r1) {
+                // the update-only sweep may write to the other copy of the stack
+                float* dst = FORWARD ? const_cast<float*>(xrow[t]) : Xw + (long long)(rb + t) * ld;
+                st_stream(dst + c, x[t]);
+            }
+    }
+    if (FORWARD && !(UPDATE && SAME)) {
+#pragma unroll
+        for (int v = 0; v < S; ++v) {
+            if (v < nf) {
+                const float4 q = QS ? *reinterpret_cast<const float4*>(fqs + v * cmax + cs) : ld_vec<COH>(sh.fq[v] + c);
+#pragma unroll
+                for (int t = 0; t < RT; ++t) {
+                    acc[t][v] = fmaf(x[t].x, q.x, acc[t][v]);
+                    acc[t][v] = fmaf(x[t].y, q.y, acc[t][v]);
+                    acc[t][v] = fmaf(x[t].z, q.z, acc[t][v]);
+                    acc[t][v] = fmaf(x[t].w, q.w, acc[t][v]);
+                }
+            }
+        }
+    }
+}
+
 // GRAD: the update also subtracts eta * G (Algorithm 1, line 6), G laid out like X.
-template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD = false>
+// ST > 0: the rows of X arrive through a ring of ST stages in shared memory, `ring` = ST x RT x 256
+// float4, each thread copying ahead (copy_async16) what it will work on itself: a warp has ST - 1
+// column steps of RT rows in flight while it works on one, across the row batches of the tile.
+// ST = 0: plain loads, one column step in flight (the cooperative kernel, which has no room for a ring).
+// Either way a row's sum is taken over the same columns in the same order.
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD = false, int ST = 0>
 __device__ __forceinline__ void row_tile(const DevState& st, const int* __restrict__ tab_u,
                                          const int* __restrict__ tab_f, const Tile tile,
-                                         RowShared<S>& sh) {
+                                         RowShared<S>& sh, float4* ring = nullptr) {
     const LayerGeom g = st.layers[tile.layer];
     const int w = tile.worker;
     const int rank = st.rank;
@@ -147,6 +276,41 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
     float* Xw = st.Xw + (long long)w * st.x_stride + g.x_off;
     const float* __restrict__ Gw = GRAD ? st.G + (long long)w * st.x_stride + g.x_off : nullptr;
     const float eta = GRAD ? st.eta : 0.0f;
+
+    const int r0 = tile.rtile * g.f_rows;
+    const int r1 = min(g.n, r0 + g.f_rows);
+    const int c0 = tile.ctile * g.f_chunk;
+    const int c1 = min(g.ld, c0 + g.f_chunk);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ld = g.ld;
+    // ring of rows (ST > 0): the first stages are on their way before the tables are read
+    const int nc = (c1 - c0 + 127) >> 7;                       // column steps of a row batch
+    const int first = r0 + warp * RT;
+    const int nb = first < r1 ? (r1 - first + 8 * RT - 1) / (8 * RT) : 0;   // row batches of this warp
+    const int cl = c0 + lane * 4;
+    float4* const mine = ring + threadIdx.x;                   // slot (stage, t) at mine[(stage * RT + t) * 256]
+    int ib = 0, ic = 0, ig = 0;      // the next step to fetch, (batch ib, column step ic), goes to stage ig
+    auto issue = [&]() {
+        if (ib < nb) {
+            const int c = cl + (ic << 7);
+            if (c < c1) {
+                const int rb = first + ib * 8 * RT;
+#pragma unroll
+                for (int t = 0; t < RT; ++t)
+                    copy_async16(mine + (ig * RT + t) * 256, X + (long long)min(rb + t, r1 - 1) * ld + c);
+            }
+            if (++ic == nc) { ic = 0; ++ib; }
+            if (++ig == ST) ig = 0;
+        }
+        copy_async_commit();
+    };
+    if constexpr (ST > 0) {
+        if (r1 > r0 && c1 > c0 &&
+            PG_OOB(st, kSecX, X + (long long)r0 * ld + c0, (long long)(r1 - 1 - r0) * ld + (c1 - c0)))
+            return;                  // (checked build; the same for every thread)
+#pragma unroll
+        for (int s = 0; s < ST - 1; ++s) issue();
+    }
 
     if (threadIdx.x < S) {
         const int v = threadIdx.x;
@@ -180,12 +344,6 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
     const int nu = UPDATE ? sh.nu : 0;
     const int nf = FORWARD ? sh.nf : 0;
 
-    const int r0 = tile.rtile * g.f_rows;
-    const int r1 = min(g.n, r0 + g.f_rows);
-    const int c0 = tile.ctile * g.f_chunk;
-    const int c1 = min(g.ld, c0 + g.f_chunk);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ld = g.ld;
     if (r1 > r0 && c1 > c0) {      // (checked build) everything this tile touches; the same for every thread
         const long long span = (long long)(r1 - 1 - r0) * ld + (c1 - c0);
         bool bad = PG_OOB(st, kSecX, X + (long long)r0 * ld + c0, span);
@@ -199,128 +357,107 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
         if (bad) return;
     }
 
-    for (int rb = r0 + warp * RT; rb < r1; rb += 8 * RT) {
-        float a[RT][S];
-        float acc[RT][S];
-        const float* xrow[RT];
-#pragma unroll
-        for (int t = 0; t < RT; ++t) {
-            const int r = min(rb + t, r1 - 1);  // rows past the tile repeat the last one; never stored
-            xrow[t] = X + (long long)r * ld;
-#pragma unroll
-            for (int v = 0; v < S; ++v) {
-                acc[t][v] = 0.0f;
-                a[t][v] = 0.0f;
-                if (UPDATE && v < nu && rb + t < r1) a[t][v] = sh.uc[v] * ld_f<COH>(sh.up[v] + r);
+    if constexpr (ST > 0) {
+        // the vectors of this tile's column chunk and the rows' coefficients, staged once for all warps
+        const int cmax = st.f_chunk_max;
+        float* const uqs = reinterpret_cast<float*>(ring + ST * RT * 256);
+        float* const fqs = uqs + ((UPDATE && !SAME) || !FORWARD ? S * cmax : 0);
+        float* const as = fqs + (FORWARD ? S * cmax : 0);          // [S][f_rows_max]
+        const int amax = st.f_rows_max;
+        if (UPDATE) {
+            for (int v = 0; v < nu; ++v)
+                for (int i = threadIdx.x * 4; i < c1 - c0; i += 1024) copy_async16(uqs + v * cmax + i, sh.uq[v] + c0 + i);
+            for (int i = threadIdx.x; i < nu * amax; i += 256) {
+                const int v = i / amax, rr = i - v * amax;
+                as[i] = r0 + rr < r1 ? sh.uc[v] * ld_f<COH>(sh.up[v] + r0 + rr) : 0.0f;
             }
         }
-        for (int c = c0 + lane * 4; c < c1; c += 128) {
-            float4 x[RT];
+        if (FORWARD && !(UPDATE && SAME))
+            for (int v = 0; v < nf; ++v)
+                for (int i = threadIdx.x * 4; i < c1 - c0; i += 1024) copy_async16(fqs + v * cmax + i, sh.fq[v] + c0 + i);
+        copy_async_commit();
+        copy_async_wait<0>();
+        __syncthreads();
+        int stage = 0;
+        for (int b = 0; b < nb; ++b) {
+            const int rb = first + b * 8 * RT;
+            float a[RT][S];
+            float acc[RT][S];
+            const float* xrow[RT];
 #pragma unroll
-            for (int t = 0; t < RT; ++t) x[t] = ld_stream(xrow[t] + c);
-            if (UPDATE && SAME) {
-                // slot order: first every correction, then every product, as in the general case
-                float4 q[S];
-#pragma unroll
-                for (int v = 0; v < S; ++v) {
-                    if (v < nu) {
-                        q[v] = ld_vec<COH>(sh.uq[v] + c);
-#pragma unroll
-                        for (int t = 0; t < RT; ++t) {
-                            x[t].x = fmaf(-a[t][v], q[v].x, x[t].x);
-                            x[t].y = fmaf(-a[t][v], q[v].y, x[t].y);
-                            x[t].z = fmaf(-a[t][v], q[v].z, x[t].z);
-                            x[t].w = fmaf(-a[t][v], q[v].w, x[t].w);
-                        }
-                    }
-                }
-                if (GRAD) {
-#pragma unroll
-                    for (int t = 0; t < RT; ++t) {
-                        float4 gv = ld_stream(Gw + (xrow[t] - X) + c);
-                        // columns past the matrix are padding: X keeps zeros there whatever G holds
-                        if (c + 1 >= g.m) gv.y = 0.0f;
-                        if (c + 2 >= g.m) gv.z = 0.0f;
-                        if (c + 3 >= g.m) gv.w = 0.0f;
-                        x[t].x = fmaf(-eta, gv.x, x[t].x); x[t].y = fmaf(-eta, gv.y, x[t].y);
-                        x[t].z = fmaf(-eta, gv.z, x[t].z); x[t].w = fmaf(-eta, gv.w, x[t].w);
-                    }
-                }
-#pragma unroll
-                for (int t = 0; t < RT; ++t)
-                    if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
+            for (int t = 0; t < RT; ++t) {
+                const int r = min(rb + t, r1 - 1);  // rows past the tile repeat the last one; never stored
+                xrow[t] = X + (long long)r * ld;
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
-                    if (v < nu) {
-#pragma unroll
-                        for (int t = 0; t < RT; ++t) {
-                            acc[t][v] = fmaf(x[t].x, q[v].x, acc[t][v]);
-                            acc[t][v] = fmaf(x[t].y, q[v].y, acc[t][v]);
-                            acc[t][v] = fmaf(x[t].z, q[v].z, acc[t][v]);
-                            acc[t][v] = fmaf(x[t].w, q[v].w, acc[t][v]);
-                        }
-                    }
+                    acc[t][v] = 0.0f;
+                    a[t][v] = 0.0f;
+                    if (UPDATE && v < nu && rb + t < r1) a[t][v] = as[v * amax + r - r0];
                 }
-            } else if (UPDATE) {
-#pragma unroll
-                for (int v = 0; v < S; ++v) {
-                    if (v < nu) {
-                        const float4 q = ld_vec<COH>(sh.uq[v] + c);
-#pragma unroll
-                        for (int t = 0; t < RT; ++t) {
-                            x[t].x = fmaf(-a[t][v], q.x, x[t].x);
-                            x[t].y = fmaf(-a[t][v], q.y, x[t].y);
-                            x[t].z = fmaf(-a[t][v], q.z, x[t].z);
-                            x[t].w = fmaf(-a[t][v], q.w, x[t].w);
-                        }
-                    }
-                }
-                if (GRAD) {
-#pragma unroll
-                    for (int t = 0; t < RT; ++t) {
-                        float4 gv = ld_stream(Gw + (xrow[t] - X) + c);
-                        // columns past the matrix are padding: X keeps zeros there whatever G holds
-                        if (c + 1 >= g.m) gv.y = 0.0f;
-                        if (c + 2 >= g.m) gv.z = 0.0f;
-                        if (c + 3 >= g.m) gv.w = 0.0f;
-                        x[t].x = fmaf(-eta, gv.x, x[t].x); x[t].y = fmaf(-eta, gv.y, x[t].y);
-                        x[t].z = fmaf(-eta, gv.z, x[t].z); x[t].w = fmaf(-eta, gv.w, x[t].w);
-                    }
-                }
-#pragma unroll
-                for (int t = 0; t < RT; ++t)
-                    if (rb + t < r1) {
-                        // the update-only sweep may write to the other copy of the stack
-                        float* dst = FORWARD ? const_cast<float*>(xrow[t]) : Xw + (long long)(rb + t) * ld;
-                        st_stream(dst + c, x[t]);
-                    }
             }
-            if (FORWARD && !(UPDATE && SAME)) {
+            for (int c = cl, k = 0; k < nc; ++k, c += 128) {
+                issue();
+                copy_async_wait<ST - 1>();
+                if (c < c1) {
+                    float4 x[RT];
+#pragma unroll
+                    for (int t = 0; t < RT; ++t) x[t] = mine[(stage * RT + t) * 256];
+                    row_columns<S, UPDATE, FORWARD, SAME, RT, COH, GRAD, true>(sh, nu, nf, x, a, acc, c, rb, r1, xrow, X,
+                                                                               Xw, Gw, eta, g.m, ld, uqs, fqs, cmax,
+                                                                               c - c0);
+                }
+                if (++stage == ST) stage = 0;
+            }
+            if (FORWARD) {
+                float* __restrict__ Y = st.Y + (long long)w * st.y_stride + g.y_off;
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nf) {
-                        const float4 q = ld_vec<COH>(sh.fq[v] + c);
 #pragma unroll
                         for (int t = 0; t < RT; ++t) {
-                            acc[t][v] = fmaf(x[t].x, q.x, acc[t][v]);
-                            acc[t][v] = fmaf(x[t].y, q.y, acc[t][v]);
-                            acc[t][v] = fmaf(x[t].z, q.z, acc[t][v]);
-                            acc[t][v] = fmaf(x[t].w, q.w, acc[t][v]);
+                            const float s = warp_sum(acc[t][v]);
+                            if (lane == 0 && rb + t < r1)
+                                Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * sh.fs[v];
                         }
                     }
                 }
             }
         }
-        if (FORWARD) {
-            float* __restrict__ Y = st.Y + (long long)w * st.y_stride + g.y_off;
+        copy_async_wait<0>();
+    } else {
+        for (int rb = r0 + warp * RT; rb < r1; rb += 8 * RT) {
+            float a[RT][S];
+            float acc[RT][S];
+            const float* xrow[RT];
 #pragma unroll
-            for (int v = 0; v < S; ++v) {
-                if (v < nf) {
+            for (int t = 0; t < RT; ++t) {
+                const int r = min(rb + t, r1 - 1);  // rows past the tile repeat the last one; never stored
+                xrow[t] = X + (long long)r * ld;
 #pragma unroll
-                    for (int t = 0; t < RT; ++t) {
-                        const float s = warp_sum(acc[t][v]);
-                        if (lane == 0 && rb + t < r1)
-                            Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * sh.fs[v];
+                for (int v = 0; v < S; ++v) {
+                    acc[t][v] = 0.0f;
+                    a[t][v] = 0.0f;
+                    if (UPDATE && v < nu && rb + t < r1) a[t][v] = sh.uc[v] * ld_f<COH>(sh.up[v] + r);
+                }
+            }
+            for (int c = c0 + lane * 4; c < c1; c += 128) {
+                float4 x[RT];
+#pragma unroll
+                for (int t = 0; t < RT; ++t) x[t] = ld_stream(xrow[t] + c);
+                row_columns<S, UPDATE, FORWARD, SAME, RT, COH, GRAD>(sh, nu, nf, x, a, acc, c, rb, r1, xrow, X, Xw, Gw, eta,
+                                                                     g.m, ld);
+            }
+            if (FORWARD) {
+                float* __restrict__ Y = st.Y + (long long)w * st.y_stride + g.y_off;
+#pragma unroll
+                for (int v = 0; v < S; ++v) {
+                    if (v < nf) {
+#pragma unroll
+                        for (int t = 0; t < RT; ++t) {
+                            const float s = warp_sum(acc[t][v]);
+                            if (lane == 0 && rb + t < r1)
+                                Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * sh.fs[v];
+                        }
                     }
                 }
             }
@@ -329,12 +466,14 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
 }
 
 template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool GRAD = false>
-__global__ void __launch_bounds__(256, kRowMinBlocks)
+__global__ void __launch_bounds__(256, row_min_blocks(S))
 row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restrict__ tab_f,
                  const Tile* __restrict__ tiles) {
     grid_dependency_sync();
     __shared__ RowShared<S> sh;
-    row_tile<S, UPDATE, FORWARD, SAME, RT, false, GRAD>(st, tab_u, tab_f, tiles[blockIdx.x], sh);
+    extern __shared__ float4 row_ring[];
+    row_tile<S, UPDATE, FORWARD, SAME, RT, false, GRAD, row_stages(S, RT)>(st, tab_u, tab_f, tiles[blockIdx.x], sh,
+                                                                        row_ring);
 }
 
 // --------------------------------------------------------------------------
@@ -2916,31 +3055,36 @@ cudaError_t launch_dep(int allowed, void (*kernel)(Params...), dim3 grid, dim3 b
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
 }
 
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool GRAD>
+cudaError_t launch_row_t(const DevState& st, const int* tab_u, const int* tab_f, const Tile* tiles, int n_tiles,
+                         cudaStream_t stream) {
+    const size_t smem = row_ring_bytes(S, RT) +
+                        sizeof(float) * S * ((size_t)st.f_chunk_max * (UPDATE && FORWARD && !SAME ? 2 : 1) + st.f_rows_max);
+    cudaError_t rc = cudaFuncSetAttribute(row_sweep_kernel<S, UPDATE, FORWARD, SAME, RT, GRAD>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (rc != cudaSuccess) return rc;
+    launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<S, UPDATE, FORWARD, SAME, RT, GRAD>, dim3(n_tiles),
+               dim3(256), smem, stream, st, tab_u, tab_f, tiles);
+    return cudaGetLastError();
+}
+
+template <bool UPDATE, bool FORWARD, bool SAME, bool GRAD>
+cudaError_t launch_row_s(const DevState& st, const int* tab_u, const int* tab_f, const Tile* tiles, int n_tiles,
+                         cudaStream_t stream) {
+    const int slots = st.max_degree * st.rank;
+    if (slots <= 1) return launch_row_t<1, UPDATE, FORWARD, SAME, kRowsPerWarp1, GRAD>(st, tab_u, tab_f, tiles, n_tiles, stream);
+    if (slots <= 2) return launch_row_t<2, UPDATE, FORWARD, SAME, kRowsPerWarp2, GRAD>(st, tab_u, tab_f, tiles, n_tiles, stream);
+    if (slots <= 4) return launch_row_t<4, UPDATE, FORWARD, SAME, kRowsPerWarp4, GRAD>(st, tab_u, tab_f, tiles, n_tiles, stream);
+    return launch_row_t<8, UPDATE, FORWARD, SAME, kRowsPerWarp8, GRAD>(st, tab_u, tab_f, tiles, n_tiles, stream);
+}
+
 template <bool UPDATE, bool FORWARD, bool SAME>
 cudaError_t launch_row(const DevState& st, const int* tab_u, const int* tab_f, const Tile* tiles,
                        int n_tiles, cudaStream_t stream) {
     if (n_tiles <= 0) return cudaSuccess;
-    const int slots = st.max_degree * st.rank;
-    if (UPDATE && st.G) {     // the update also takes the caller's gradient step
-        if (slots <= 1)
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, kRowsPerWarp1, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-        else if (slots <= 2)
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, kRowsPerWarp2, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-        else if (slots <= 4)
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, kRowsPerWarp4, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-        else
-            launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, kRowsPerWarp8, UPDATE>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-        return cudaGetLastError();
-    }
-    if (slots <= 1)
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<1, UPDATE, FORWARD, SAME, kRowsPerWarp1>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-    else if (slots <= 2)
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<2, UPDATE, FORWARD, SAME, kRowsPerWarp2>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-    else if (slots <= 4)
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<4, UPDATE, FORWARD, SAME, kRowsPerWarp4>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-    else
-        launch_dep(st.dep_launch & kDepSweep, row_sweep_kernel<8, UPDATE, FORWARD, SAME, kRowsPerWarp8>, dim3(n_tiles), dim3(256), 0, stream, st, tab_u, tab_f, tiles);
-    return cudaGetLastError();
+    if (UPDATE && st.G)      // the update also takes the caller's gradient step
+        return launch_row_s<UPDATE, FORWARD, SAME, UPDATE>(st, tab_u, tab_f, tiles, n_tiles, stream);
+    return launch_row_s<UPDATE, FORWARD, SAME, false>(st, tab_u, tab_f, tiles, n_tiles, stream);
 }
 
 }  // namespace
