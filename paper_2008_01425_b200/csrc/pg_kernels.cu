@@ -137,6 +137,36 @@ __device__ double block_sum(double v, double* scratch /* >= 33 doubles of shared
     return scratch[32];
 }
 
+// Packed fp32 arithmetic (fma.rn.f32x2: two IEEE fused multiply-adds per instruction, each
+// lane rounded exactly like fmaf).  The row sweeps with four or more vectors and the two-column
+// pair sweep are bound by instruction issue, and most of their instructions are these.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// x += a * v
+__device__ __forceinline__ void fma4(float4& x, float a, const float4& v) {
+    const unsigned long long aa = pack2(a, a);
+    unpack2(fma2(aa, pack2(v.x, v.y), pack2(x.x, x.y)), x.x, x.y);
+    unpack2(fma2(aa, pack2(v.z, v.w), pack2(x.z, x.w)), x.z, x.w);
+}
+// acc (two partial sums) += d * v, lane by lane
+__device__ __forceinline__ void dot4(float2& acc, const float4& d, const float4& v) {
+    unsigned long long t = pack2(acc.x, acc.y);
+    t = fma2(pack2(d.x, d.y), pack2(v.x, v.y), t);
+    t = fma2(pack2(d.z, d.w), pack2(v.z, v.w), t);
+    unpack2(t, acc.x, acc.y);
+}
+
 // --------------------------------------------------------------------------
 // Row-oriented sweep: optional rank-r update of X, optional forward product.
 // A warp owns RT rows at a time; its lanes walk the columns with float4 loads.
@@ -153,13 +183,36 @@ struct RowShared {
     int nu, nf;
 };
 
+// x += a * v and acc += x . v of one float4: packed (two lanes per instruction) where the sweep carries four or
+// more vectors and is bound by instruction issue, plain where it waits on memory and the packed form's
+// extra registers would spill.  The packed dot keeps even and odd column pairs in two partial sums.
+template <int S>
+__device__ __forceinline__ void row_axpy(float4& x, float a, const float4& v) {
+    if (S >= 4) {
+        fma4(x, a, v);
+    } else {
+        x.x = fmaf(a, v.x, x.x); x.y = fmaf(a, v.y, x.y); x.z = fmaf(a, v.z, x.z); x.w = fmaf(a, v.w, x.w);
+    }
+}
+template <int S>
+__device__ __forceinline__ void row_dot(float2& acc, const float4& x, const float4& v) {
+    if (S >= 4) {
+        dot4(acc, x, v);
+    } else {
+        acc.x = fmaf(x.x, v.x, acc.x); acc.x = fmaf(x.y, v.y, acc.x);
+        acc.x = fmaf(x.z, v.z, acc.x); acc.x = fmaf(x.w, v.w, acc.x);
+    }
+}
+
 // The work of one float4 column step on RT rows of a row-oriented sweep, the rows' values in x:
 // the pending corrections (and the gradient step) applied and stored, then the products' partial sums.
 // QS: the vectors of the tile's column chunk are staged in shared memory (uqs / fqs: one vector every
 // `cmax` floats, `cs` = this step's first column within the chunk) instead of read through L1.
-template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD, bool QS = false>
+// FULL: every row and column step of the tile is inside it and all S vectors are worked on (those a
+// worker does not have are zeros with zero coefficients), so nothing in the step is conditional.
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD, bool QS = false, bool FULL = false>
 __device__ __forceinline__ void row_columns(const RowShared<S>& sh, const int nu, const int nf, float4 (&x)[RT],
-                                            const float (&a)[RT][S], float (&acc)[RT][S], const int c,
+                                            const float (&a)[RT][S], float2 (&acc)[RT][S], const int c,
                                             const int rb, const int r1, const float* const (&xrow)[RT],
                                             const float* __restrict__ X, float* Xw,
                                             const float* __restrict__ Gw, const float eta, const int m,
@@ -170,14 +223,11 @@ __device__ __forceinline__ void row_columns(const RowShared<S>& sh, const int nu
         float4 q[S];
 #pragma unroll
         for (int v = 0; v < S; ++v) {
-            if (v < nu) {
+            if (FULL || v < nu) {
                 q[v] = QS ? *reinterpret_cast<const float4*>(uqs + v * cmax + cs) : ld_vec<COH>(sh.uq[v] + c);
 #pragma unroll
                 for (int t = 0; t < RT; ++t) {
-                    x[t].x = fmaf(-a[t][v], q[v].x, x[t].x);
-                    x[t].y = fmaf(-a[t][v], q[v].y, x[t].y);
-                    x[t].z = fmaf(-a[t][v], q[v].z, x[t].z);
-                    x[t].w = fmaf(-a[t][v], q[v].w, x[t].w);
+                    row_axpy<S>(x[t], -a[t][v], q[v]);
                 }
             }
         }
@@ -195,30 +245,24 @@ __device__ __forceinline__ void row_columns(const RowShared<S>& sh, const int nu
         }
 #pragma unroll
         for (int t = 0; t < RT; ++t)
-            if (rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
+            if (FULL || rb + t < r1) st_stream(const_cast<float*>(xrow[t]) + c, x[t]);
 #pragma unroll
         for (int v = 0; v < S; ++v) {
-            if (v < nu) {
+            if (FULL || v < nu) {
 #pragma unroll
                 for (int t = 0; t < RT; ++t) {
-                    acc[t][v] = fmaf(x[t].x, q[v].x, acc[t][v]);
-                    acc[t][v] = fmaf(x[t].y, q[v].y, acc[t][v]);
-                    acc[t][v] = fmaf(x[t].z, q[v].z, acc[t][v]);
-                    acc[t][v] = fmaf(x[t].w, q[v].w, acc[t][v]);
+                    row_dot<S>(acc[t][v], x[t], q[v]);
                 }
             }
         }
     } else if (UPDATE) {
 #pragma unroll
         for (int v = 0; v < S; ++v) {
-            if (v < nu) {
+            if (FULL || v < nu) {
                 const float4 q = QS ? *reinterpret_cast<const float4*>(uqs + v * cmax + cs) : ld_vec<COH>(sh.uq[v] + c);
 #pragma unroll
                 for (int t = 0; t < RT; ++t) {
-                    x[t].x = fmaf(-a[t][v], q.x, x[t].x);
-                    x[t].y = fmaf(-a[t][v], q.y, x[t].y);
-                    x[t].z = fmaf(-a[t][v], q.z, x[t].z);
-                    x[t].w = fmaf(-a[t][v], q.w, x[t].w);
+                    row_axpy<S>(x[t], -a[t][v], q);
                 }
             }
         }
@@ -236,7 +280,7 @@ __device__ __forceinline__ void row_columns(const RowShared<S>& sh, const int nu
         }
 #pragma unroll
         for (int t = 0; t < RT; ++t)
-            if (rb + t < r1) {
+            if (FULL || rb + t < r1) {
                 // the update-only sweep may write to the other copy of the stack
                 float* dst = FORWARD ? const_cast<float*>(xrow[t]) : Xw + (long long)(rb + t) * ld;
                 st_stream(dst + c, x[t]);
@@ -245,14 +289,11 @@ __device__ __forceinline__ void row_columns(const RowShared<S>& sh, const int nu
     if (FORWARD && !(UPDATE && SAME)) {
 #pragma unroll
         for (int v = 0; v < S; ++v) {
-            if (v < nf) {
+            if (FULL || v < nf) {
                 const float4 q = QS ? *reinterpret_cast<const float4*>(fqs + v * cmax + cs) : ld_vec<COH>(sh.fq[v] + c);
 #pragma unroll
                 for (int t = 0; t < RT; ++t) {
-                    acc[t][v] = fmaf(x[t].x, q.x, acc[t][v]);
-                    acc[t][v] = fmaf(x[t].y, q.y, acc[t][v]);
-                    acc[t][v] = fmaf(x[t].z, q.z, acc[t][v]);
-                    acc[t][v] = fmaf(x[t].w, q.w, acc[t][v]);
+                    row_dot<S>(acc[t][v], x[t], q);
                 }
             }
         }
@@ -265,7 +306,8 @@ __device__ __forceinline__ void row_columns(const RowShared<S>& sh, const int nu
 // column steps of RT rows in flight while it works on one, across the row batches of the tile.
 // ST = 0: plain loads, one column step in flight (the cooperative kernel, which has no room for a ring).
 // Either way a row's sum is taken over the same columns in the same order.
-template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD = false, int ST = 0>
+// FULL (ST > 0 only): the tile's rows are whole batches of 8 RT and its columns whole steps of 128.
+template <int S, bool UPDATE, bool FORWARD, bool SAME, int RT, bool COH, bool GRAD = false, int ST = 0, bool FULL = false>
 __device__ __forceinline__ void row_tile(const DevState& st, const int* __restrict__ tab_u,
                                          const int* __restrict__ tab_f, const Tile tile,
                                          RowShared<S>& sh, float4* ring = nullptr) {
@@ -364,6 +406,7 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
         float* const fqs = uqs + ((UPDATE && !SAME) || !FORWARD ? S * cmax : 0);
         float* const as = fqs + (FORWARD ? S * cmax : 0);          // [S][f_rows_max]
         const int amax = st.f_rows_max;
+        const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
         if (UPDATE) {
             for (int v = 0; v < nu; ++v)
                 for (int i = threadIdx.x * 4; i < c1 - c0; i += 1024) copy_async16(uqs + v * cmax + i, sh.uq[v] + c0 + i);
@@ -371,10 +414,19 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                 const int v = i / amax, rr = i - v * amax;
                 as[i] = r0 + rr < r1 ? sh.uc[v] * ld_f<COH>(sh.up[v] + r0 + rr) : 0.0f;
             }
+            if (FULL) {      // vectors this worker does not have: zeros with zero coefficients, worked on like the rest
+                for (int v = nu; v < S; ++v)
+                    for (int i = threadIdx.x * 4; i < c1 - c0; i += 1024) *reinterpret_cast<float4*>(uqs + v * cmax + i) = zero4;
+                for (int i = nu * amax + threadIdx.x; i < S * amax; i += 256) as[i] = 0.0f;
+            }
         }
-        if (FORWARD && !(UPDATE && SAME))
+        if (FORWARD && !(UPDATE && SAME)) {
             for (int v = 0; v < nf; ++v)
                 for (int i = threadIdx.x * 4; i < c1 - c0; i += 1024) copy_async16(fqs + v * cmax + i, sh.fq[v] + c0 + i);
+            if (FULL)
+                for (int v = nf; v < S; ++v)
+                    for (int i = threadIdx.x * 4; i < c1 - c0; i += 1024) *reinterpret_cast<float4*>(fqs + v * cmax + i) = zero4;
+        }
         copy_async_commit();
         copy_async_wait<0>();
         __syncthreads();
@@ -382,27 +434,27 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
         for (int b = 0; b < nb; ++b) {
             const int rb = first + b * 8 * RT;
             float a[RT][S];
-            float acc[RT][S];
+            float2 acc[RT][S];      // even and odd column pairs apart until the row's sum
             const float* xrow[RT];
 #pragma unroll
             for (int t = 0; t < RT; ++t) {
-                const int r = min(rb + t, r1 - 1);  // rows past the tile repeat the last one; never stored
+                const int r = FULL ? rb + t : min(rb + t, r1 - 1);  // rows past the tile repeat the last one; never stored
                 xrow[t] = X + (long long)r * ld;
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
-                    acc[t][v] = 0.0f;
+                    acc[t][v] = make_float2(0.f, 0.f);
                     a[t][v] = 0.0f;
-                    if (UPDATE && v < nu && rb + t < r1) a[t][v] = as[v * amax + r - r0];
+                    if (UPDATE && (FULL || (v < nu && rb + t < r1))) a[t][v] = as[v * amax + r - r0];
                 }
             }
             for (int c = cl, k = 0; k < nc; ++k, c += 128) {
                 issue();
                 copy_async_wait<ST - 1>();
-                if (c < c1) {
+                if (FULL || c < c1) {
                     float4 x[RT];
 #pragma unroll
                     for (int t = 0; t < RT; ++t) x[t] = mine[(stage * RT + t) * 256];
-                    row_columns<S, UPDATE, FORWARD, SAME, RT, COH, GRAD, true>(sh, nu, nf, x, a, acc, c, rb, r1, xrow, X,
+                    row_columns<S, UPDATE, FORWARD, SAME, RT, COH, GRAD, true, FULL>(sh, nu, nf, x, a, acc, c, rb, r1, xrow, X,
                                                                                Xw, Gw, eta, g.m, ld, uqs, fqs, cmax,
                                                                                c - c0);
                 }
@@ -415,8 +467,8 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                     if (v < nf) {
 #pragma unroll
                         for (int t = 0; t < RT; ++t) {
-                            const float s = warp_sum(acc[t][v]);
-                            if (lane == 0 && rb + t < r1)
+                            const float s = warp_sum(acc[t][v].x + acc[t][v].y);
+                            if (lane == 0 && (FULL || rb + t < r1))
                                 Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * sh.fs[v];
                         }
                     }
@@ -427,7 +479,7 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
     } else {
         for (int rb = r0 + warp * RT; rb < r1; rb += 8 * RT) {
             float a[RT][S];
-            float acc[RT][S];
+            float2 acc[RT][S];      // even and odd column pairs apart until the row's sum
             const float* xrow[RT];
 #pragma unroll
             for (int t = 0; t < RT; ++t) {
@@ -435,7 +487,7 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                 xrow[t] = X + (long long)r * ld;
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
-                    acc[t][v] = 0.0f;
+                    acc[t][v] = make_float2(0.f, 0.f);
                     a[t][v] = 0.0f;
                     if (UPDATE && v < nu && rb + t < r1) a[t][v] = sh.uc[v] * ld_f<COH>(sh.up[v] + r);
                 }
@@ -454,7 +506,7 @@ __device__ __forceinline__ void row_tile(const DevState& st, const int* __restri
                     if (v < nf) {
 #pragma unroll
                         for (int t = 0; t < RT; ++t) {
-                            const float s = warp_sum(acc[t][v]);
+                            const float s = warp_sum(acc[t][v].x + acc[t][v].y);
                             if (lane == 0 && rb + t < r1)
                                 Y[((long long)v * g.f_csplit + tile.ctile) * g.npad + rb + t] = s * sh.fs[v];
                         }
@@ -472,8 +524,15 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
     grid_dependency_sync();
     __shared__ RowShared<S> sh;
     extern __shared__ float4 row_ring[];
-    row_tile<S, UPDATE, FORWARD, SAME, RT, false, GRAD, row_stages(S, RT)>(st, tab_u, tab_f, tiles[blockIdx.x], sh,
-                                                                        row_ring);
+    const Tile tile = tiles[blockIdx.x];
+    const LayerGeom& g = st.layers[tile.layer];
+    // a tile of whole row batches and whole column steps takes the form without conditions
+    const int rows = min(g.n, (tile.rtile + 1) * g.f_rows) - tile.rtile * g.f_rows;
+    const int cols = min(g.ld, (tile.ctile + 1) * g.f_chunk) - tile.ctile * g.f_chunk;
+    if (rows % (8 * RT) == 0 && cols % 128 == 0)
+        row_tile<S, UPDATE, FORWARD, SAME, RT, false, GRAD, row_stages(S, RT), true>(st, tab_u, tab_f, tile, sh, row_ring);
+    else
+        row_tile<S, UPDATE, FORWARD, SAME, RT, false, GRAD, row_stages(S, RT), false>(st, tab_u, tab_f, tile, sh, row_ring);
 }
 
 // --------------------------------------------------------------------------
@@ -2080,28 +2139,6 @@ pair_sweep_mid_bulk_kernel(DevState st, const int* __restrict__ tab_prev, const 
 constexpr int kMid2Threads = 384;
 __host__ __device__ constexpr int mid2_rows(int nvm) { return nvm <= 3 ? 2 : 1; }
 
-// Packed fp32 arithmetic (fma.rn.f32x2: two IEEE fused multiply-adds per instruction, each
-// lane rounded exactly like fmaf).  The two-column sweep is bound by instruction issue, and
-// most of its instructions are these.
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
-    unsigned long long d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-// x += a * v
-__device__ __forceinline__ void fma4(float4& x, float a, const float4& v) {
-    const unsigned long long aa = pack2(a, a);
-    unpack2(fma2(aa, pack2(v.x, v.y), pack2(x.x, x.y)), x.x, x.y);
-    unpack2(fma2(aa, pack2(v.z, v.w), pack2(x.z, x.w)), x.z, x.w);
-}
 // a - b (as fma(b, -1, a): the same rounding as the subtraction)
 __device__ __forceinline__ float4 sub4(const float4& a, const float4& b) {
     const unsigned long long m = pack2(-1.0f, -1.0f);
@@ -2110,14 +2147,6 @@ __device__ __forceinline__ float4 sub4(const float4& a, const float4& b) {
     unpack2(fma2(pack2(b.z, b.w), m, pack2(a.z, a.w)), d.z, d.w);
     return d;
 }
-// acc (two partial sums) += d * v, lane by lane
-__device__ __forceinline__ void dot4(float2& acc, const float4& d, const float4& v) {
-    unsigned long long t = pack2(acc.x, acc.y);
-    t = fma2(pack2(d.x, d.y), pack2(v.x, v.y), t);
-    t = fma2(pack2(d.z, d.w), pack2(v.z, v.w), t);
-    unpack2(t, acc.x, acc.y);
-}
-
 template <int NVM, bool UPDATE>
 __global__ void __launch_bounds__(kMid2Threads, 1)
 pair_sweep_mid2_kernel(DevState st, const int* __restrict__ tab, const Tile* __restrict__ tiles, int ld_pad,
@@ -2585,15 +2614,19 @@ pair_sweep_mid2_raw_kernel(DevState st, const int* __restrict__ tab, const Tile*
             issue(it + n_stage);
             issued = it + n_stage + 1;
         }
+        // the warps' shares of the RS x R row products: lane (t, c) of every warp adds one up in warp order,
+        // the others take it from there
+        float lane_sum = 0.0f;
+        if (lane < RS * R) {
+            const float* sh_w = &s_warp[it & 1][0][0][0] + lane * (NT / 32);
+#pragma unroll
+            for (int w8 = 0; w8 < NT / 32; ++w8) lane_sum += sh_w[w8];
+        }
 #pragma unroll
         for (int t = 0; t < RS; ++t) {
             float p[R];
 #pragma unroll
-            for (int c = 0; c < R; ++c) {
-                p[c] = 0.0f;
-#pragma unroll
-                for (int w8 = 0; w8 < NT / 32; ++w8) p[c] += s_warp[it & 1][t][c][w8];
-            }
+            for (int c = 0; c < R; ++c) p[c] = __shfl_sync(0xffffffffu, lane_sum, t * R + c);
             const int rr = min(r + t, r1 - 1) - r0;
             p[0] = p[0] * qinv0 - s_corr[rr];        // the products with the unit columns, less the pending terms' part
             p[1] = p[1] * qinv1 - s_corr[rows_pad + rr];
