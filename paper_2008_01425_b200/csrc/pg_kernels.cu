@@ -541,7 +541,10 @@ row_sweep_kernel(DevState st, const int* __restrict__ tab_u, const int* __restri
 // --------------------------------------------------------------------------
 template <int S>
 struct ColShared {
-    float p[S][kColTileRowsMax];
+    // P-hat of the tile's rows; up to four vectors each value twice, the operand of a packed FMA (eight
+    // vectors would not leave room in the cooperative kernel's static shared memory)
+    static constexpr int kDup = S <= 4 ? 2 : 1;
+    float p[S][kColTileRowsMax][kDup];
     float a[S][kColTileRowsMax];   // UPDATE: coefficient of the pending correction per row
     float4 red[3][S][64];
 };
@@ -595,7 +598,8 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
         } else if (UPDATE) {
             sh.a[v][rr] = 0.0f;
         }
-        sh.p[v][rr] = val;
+#pragma unroll
+        for (int d2 = 0; d2 < ColShared<S>::kDup; ++d2) sh.p[v][rr][d2] = val;
     }
     __syncthreads();
 
@@ -619,7 +623,36 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
             }
         }
     }
-    if (c < ld) {
+    if (!UPDATE && S <= 4 && c < ld && (r1 - r0) % 16 == 0) {
+        // whole groups of 16 rows: nothing in the step is conditional.  Vectors the worker does not have were
+        // staged as zeros and are worked on like the rest (their sums are never stored); packed FMAs, each
+        // lane the same fused multiply-add as in the general form below.
+        unsigned long long a2[S][2];
+#pragma unroll
+        for (int v = 0; v < S; ++v) a2[v][0] = a2[v][1] = 0ull;
+        const float* xp = X + (long long)(r0 + ty) * ld + c;
+        const long long step4 = 4LL * ld;
+        for (int ro = ty; ro < r1 - r0; ro += 16, xp += 4 * step4) {
+            float4 x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) x[u] = ld_stream(xp + u * step4);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const unsigned long long xlo = pack2(x[u].x, x[u].y), xhi = pack2(x[u].z, x[u].w);
+#pragma unroll
+                for (int v = 0; v < S; ++v) {
+                    const unsigned long long pp = *reinterpret_cast<const unsigned long long*>(&sh.p[v][ro + 4 * u][0]);
+                    a2[v][0] = fma2(pp, xlo, a2[v][0]);
+                    a2[v][1] = fma2(pp, xhi, a2[v][1]);
+                }
+            }
+        }
+#pragma unroll
+        for (int v = 0; v < S; ++v) {
+            unpack2(a2[v][0], acc[v].x, acc[v].y);
+            unpack2(a2[v][1], acc[v].z, acc[v].w);
+        }
+    } else if (c < ld) {
         const float* xc = X + c;
         for (int r = r0 + ty; r < r1; r += 16) {
             float4 x[4];
@@ -647,7 +680,7 @@ __device__ __forceinline__ void col_tile(const DevState& st, const int* __restri
 #pragma unroll
                 for (int v = 0; v < S; ++v) {
                     if (v < nv) {
-                        const float p = in ? sh.p[v][ro] : 0.0f;
+                        const float p = in ? sh.p[v][ro][0] : 0.0f;
                         acc[v].x = fmaf(p, x[u].x, acc[v].x);
                         acc[v].y = fmaf(p, x[u].y, acc[v].y);
                         acc[v].z = fmaf(p, x[u].z, acc[v].z);
