@@ -253,6 +253,17 @@ def test_graph_variants(kind):
     _run(w, rounds=4)
 
 
+@pytest.mark.parametrize("rank", [1, 2])
+def test_whole_tiles_on_workers_with_fewer_edges_than_slots(rank):
+    """A star with a tail: degrees 3, 1, 1, 2, 1 under kernels built for four (rank 1) or eight (rank 2)
+    vectors, on matrices whose tiles are whole row batches and column steps, so the sweeps take their
+    forms without conditions and work on the vectors a worker lacks as zeros."""
+    w = wl.Workload("t", 9, 5, wl.CUSTOM, 0, 0, wl.W_METROPOLIS, None, ((64, 256), (32, 128), (128, 384)), rank, 2, 6, 5,
+                    "normal1", custom_edges=((0, 1), (0, 2), (0, 3), (3, 4)))
+    _run(w, rebased=True)
+    _run(w, rounds=3)
+
+
 def test_identical_workers_stay_bit_identical():
     """Consensus is a fixed point (Section 4.1): nothing moves, nothing is NaN."""
     w = wl.Workload("same", 9, 6, wl.RING, 0, 0, wl.W_UNIFORM, None, ((33, 70),), 2, 2, 3, 5, "normal1")
