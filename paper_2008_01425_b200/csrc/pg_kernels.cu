@@ -23,7 +23,7 @@ namespace {
 
 constexpr int kStatusNumeric = 6;  // PG_ERR_NUMERIC
 constexpr int kStatusTimeout = 5;  // PG_ERR_TIMEOUT
-constexpr int kStatusBounds = 8;   // PG_ERR_BOUNDS
+[[maybe_unused]] constexpr int kStatusBounds = 8;   // PG_ERR_BOUNDS (raised by the checked build only)
 
 // Bounds-checked build (-DPG_BOUNDS_CHECK; the stand-in for a memory checker): PG_OOB(st, section,
 // pointer, count) is true, and raises the bounds bit of the status word, if the `count` elements at
@@ -38,7 +38,7 @@ __device__ __noinline__ bool pg_out_of_bounds(const DevState& st, int sec, const
 }
 #define PG_OOB(st, sec, ptr, count) pg_out_of_bounds(st, sec, ptr, (long long)(count) * (long long)sizeof(*(ptr)))
 #else
-#define PG_OOB(st, sec, ptr, count) false
+#define PG_OOB(st, sec, ptr, count) ((void)sizeof(ptr), (void)sizeof(count), false)   // names its operands, evaluates nothing
 #endif
 constexpr long long kBarrierSpinLimit = 1LL << 23;   // polls before a grid barrier gives up (a few seconds)
 
